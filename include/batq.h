@@ -1,0 +1,164 @@
+/* batq -- the inference-time W4A4 linear layer of BATQuant on one B200 (sm_100a).
+ *
+ * Y ~= Q(X P) * Q(P^-1 W^T)   (the paper's arg-min objective, Sec. 3.1)
+ *
+ *   X [s x n] bf16 activations, W [m x n] bf16 weights, n = k * 32.
+ *   P = diag(P_1..P_k) is block diagonal on the 32-element MX groups (Eq. 1)
+ *   and every block is a Kronecker product P_j = L_j (x) R_j (Eq. 2; the paper
+ *   writes B_i (x) A).  A block x of 32 channels is the matrix V[r][c],
+ *   element index e = r*gc + c (Algorithm 1's reshape [-1, k, g2, g1]), and
+ *   x P_j  <=>  L_j^T V R_j  (the vec identity after Eq. 2).
+ *   Q is MXFP4: E2M1 elements, one UE8M0 scale per 32 elements (Sec. 2),
+ *   round-to-nearest-even, OCP scale rule e = floor(log2 amax) - 2.
+ *
+ * Conventions.  Every pointer says "dev" (device memory of the current CUDA
+ * device, owned by the caller) or "host".  Calls validate on the host and
+ * return a status; nothing throws or aborts.  Kernel launches are asynchronous
+ * on the given stream (a cudaStream_t passed as void*; NULL = default stream).
+ * The library allocates device memory only in batq_transform_create; every
+ * other buffer is the caller's.  Device-side waits are bounded: a kernel that
+ * gives up records BATQ_ERR_TIMEOUT, read back by batq_last_device_status.
+ */
+#ifndef BATQ_H_
+#define BATQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  BATQ_OK = 0,
+  BATQ_ERR_NULL = 1,        /* a required pointer is NULL                          */
+  BATQ_ERR_SHAPE = 2,       /* n % 32 != 0, a size <= 0, ld < n, sizes too large   */
+  BATQ_ERR_ALIGN = 3,       /* pointer not 16-byte aligned, ld % 8 != 0            */
+  BATQ_ERR_UNSUPPORTED = 4, /* factor sizes other than (4,8), dtype, layout, arch  */
+  BATQ_ERR_WORKSPACE = 5,   /* workspace smaller than batq_linear_workspace_bytes  */
+  BATQ_ERR_SINGULAR = 6,    /* a transform factor is not invertible                */
+  BATQ_ERR_CUDA = 7,        /* a CUDA runtime / driver call failed                 */
+  BATQ_ERR_TIMEOUT = 8      /* a bounded device-side wait ran out                  */
+} batq_status;
+
+enum { BATQ_SF_ROWMAJOR = 0, BATQ_SF_MMA = 1 };  /* scale-byte layouts, see batq_sf_bytes */
+enum { BATQ_F32 = 0, BATQ_BF16 = 1 };            /* output dtypes of the GEMM             */
+
+typedef struct batq_transform batq_transform; /* Theta of one layer: factors + clip ratios */
+typedef struct batq_weight batq_weight;       /* one prepared (transformed, quantized) W   */
+
+const char* batq_status_string(batq_status s);
+int batq_version(void);
+
+/* Theta = {A, {B_i}, {alpha_i}} of the paper's algorithm flow ("Store Theta for
+ * online activation transformation"), as two Kronecker factors and clip ratios.
+ *   n            channels, n % 32 == 0, k = n / 32 blocks.
+ *   gr, gc       factor sizes, gr * gc == 32; only (4, 8) is implemented.
+ *   left         host fp32, row-major gr x gr matrices: one if left_stride == 0
+ *                (shared by all blocks) else k of them, left_stride (= gr*gr)
+ *                floats apart.  Acts on the slow index r of a block.
+ *   right        host fp32, gc x gc, same rule with right_stride; acts on the
+ *                contiguous index c.  The paper's default GPK is left = B_i
+ *                (private 4x4), right = A (shared 8x8).
+ *   clip_lo/hi   host fp32 [k] post-sigmoid ratios of Eq. 4, or both NULL for no
+ *                clipping.
+ * The arrays are copied (host copy for the inverse, device copy for the
+ * kernels); the handle belongs to the CUDA device current at creation. */
+batq_status batq_transform_create(batq_transform** out, int32_t n, int32_t gr, int32_t gc,
+                                  const float* left, int64_t left_stride,
+                                  const float* right, int64_t right_stride,
+                                  const float* clip_lo, const float* clip_hi);
+batq_status batq_transform_destroy(batq_transform* t);
+
+/* Size in bytes of a scale-byte buffer for a [rows x n] tensor.
+ *   BATQ_SF_ROWMAJOR: rows * k bytes, byte (row, j) at row*k + j.
+ *   BATQ_SF_MMA: the layout the block-scaled tensor-core instruction reads.
+ *     The tensor is cut into atoms of 128 rows x 4 blocks = 512 bytes; with
+ *     KA = 2*ceil(k/8) atoms per 128-row tile, byte (row, j) is at
+ *       ((row/128)*KA + j/4)*512 + (row%32)*16 + ((row%128)/32)*4 + j%4.
+ *     rows are padded to a multiple of 128 and blocks to a multiple of 8.
+ * Returns 0 for invalid arguments. */
+size_t batq_sf_bytes(int64_t rows, int64_t n, int32_t layout);
+
+/* Stages 1+2 of the path: x~ = x P (Eq. 1-2), block clip (Eq. 3-4), MXFP4
+ * quantisation (Sec. 2), in that order (transform, clip, quantise: the paper's
+ * algorithm flow).
+ *   t        transform or NULL (identity, no clip: plain MXFP4 of X).
+ *   x_bf16   dev, [s x n] bf16, row stride ld elements (ld >= n, ld % 8 == 0),
+ *            16-byte aligned.
+ *   n        channels (must equal t's n when t is given).
+ *   codes    dev, s * n/2 bytes row-major; element 2i in bits 0-3 of byte i,
+ *            element 2i+1 in bits 4-7; bit 3 of a code is the sign.
+ *   scales   dev, batq_sf_bytes(s, n, scale_layout) bytes of E8M0 (e + 127).
+ * s == 0 is a no-op.  Errors: NULL / SHAPE / ALIGN / UNSUPPORTED / CUDA. */
+batq_status batq_quantize_act(const batq_transform* t, const void* x_bf16, int64_t s, int64_t n,
+                              int64_t ld, void* codes, void* scales, int32_t scale_layout,
+                              void* stream);
+
+/* Test hook: the exact fp32 values the quantiser rounds (after transform and
+ * clip, before scaling), out dev fp32 [s x n] row-major. */
+batq_status batq_debug_transform_clip_f32(const batq_transform* t, const void* x_bf16, int64_t s,
+                                          int64_t n, int64_t ld, float* out, void* stream);
+
+/* Offline weight fusion ("Offline Fusion for Deployment" in the paper's
+ * algorithm flow): W~ = W P^-T per 32-block of each weight row, optional block
+ * clip (Eq. 3-4 applied to weights), MXFP4 quantisation, written in the GEMM's
+ * layout into a caller-provided buffer.  Computed in fp64 (inverse factors by
+ * Gauss-Jordan on the host); not on the timed path.
+ *   t            transform or NULL (identity).
+ *   w_bf16       dev [m x n] bf16, row stride ld.
+ *   w_clip_lo/hi dev fp32 [m * k] ratios per (row, block), or both NULL.
+ *   weight_buf   dev, batq_weight_bytes(m, n) bytes, 1024-byte aligned; holds
+ *                codes [m x n/2] row-major then scales in BATQ_SF_MMA layout.
+ *                Must outlive the handle.
+ * The call synchronises the stream (it is offline).  SINGULAR if a factor has
+ * no inverse. */
+size_t batq_weight_bytes(int64_t m, int64_t n);
+batq_status batq_prepare_weight(const batq_transform* t, const void* w_bf16, int64_t m, int64_t n,
+                                int64_t ld, const float* w_clip_lo, const float* w_clip_hi,
+                                void* weight_buf, batq_weight** out, void* stream);
+batq_status batq_weight_destroy(batq_weight* w);
+/* Copies a prepared weight out as row-major packed codes [m x n/2] and row-major
+ * scale bytes [m x k] (dev buffers), for inspection and tests. */
+batq_status batq_weight_export(const batq_weight* w, void* codes_rowmajor, void* scales_rowmajor,
+                               void* stream);
+
+/* Stage 3 alone: Y[s, m] = sum_j 2^(ex[s,j] + ew[m,j]) * sum_{i<32} qx[s,j,i] * qw[m,j,i]
+ * (the low-bit matrix multiplication of Sec. 3.2) on the block-scaled FP4
+ * tensor cores, fp32 accumulation.
+ *   x_codes       dev [s x n/2], 16-byte aligned, as written by batq_quantize_act.
+ *   x_scales_mma  dev, BATQ_SF_MMA layout for [s x n].
+ *   y             dev [s x m] row-major with row stride ldy elements, fp32 or bf16
+ *                 (bf16 = round-to-nearest-even of the fp32 accumulator).
+ * s == 0 is a no-op. */
+batq_status batq_gemm_mxfp4(const void* x_codes, const void* x_scales_mma, const batq_weight* w,
+                            int64_t s, void* y, int32_t y_dtype, int64_t ldy, void* stream);
+
+/* The whole layer, stages 1+2+3: quantise X into the workspace, then the GEMM.
+ *   workspace  dev, at least batq_linear_workspace_bytes(w, s) bytes, 1024-byte
+ *              aligned; overwritten by every call (calls sharing a workspace
+ *              must be ordered on one stream). */
+size_t batq_linear_workspace_bytes(const batq_weight* w, int64_t s);
+batq_status batq_linear_w4a4(const batq_transform* t, const batq_weight* w, const void* x_bf16,
+                             int64_t s, int64_t ld, void* y, int32_t y_dtype, int64_t ldy,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* Same layer with HOST input and output: copies x_host (pinned or pageable host
+ * memory, [s x n] bf16 dense) to x_stage_dev, runs batq_linear_w4a4, copies the
+ * result from y_stage_dev to y_host, all on `stream`; returns after the stream
+ * has drained.  x_stage_dev (s*n*2 bytes) and y_stage_dev (s*m*{4,2} bytes) are
+ * caller-provided device staging buffers. */
+batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w, const void* x_host,
+                                  int64_t s, void* y_host, int32_t y_dtype, void* x_stage_dev,
+                                  void* y_stage_dev, void* workspace, size_t workspace_bytes,
+                                  void* stream);
+
+/* Synchronises `stream` and returns BATQ_ERR_TIMEOUT if any kernel of this
+ * library gave up a bounded wait since the last query (the record is cleared),
+ * BATQ_ERR_CUDA if the stream reports an error, else BATQ_OK. */
+batq_status batq_last_device_status(void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BATQ_H_ */

@@ -1,0 +1,223 @@
+"""ctypes binding of the batq C-ABI (include/batq.h): argument marshalling only.
+
+Every function has the name of the C entry point it calls.  Tensors are
+torch tensors used purely as device (or host) buffers; all arithmetic of the
+path runs in the library's CUDA kernels.  There is no CPU fallback: loading
+fails loudly when the shared library is missing.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+BATQ_OK = 0
+SF_ROWMAJOR, SF_MMA = 0, 1
+F32, BF16 = 0, 1
+STATUS_NAMES = {0: "OK", 1: "ERR_NULL", 2: "ERR_SHAPE", 3: "ERR_ALIGN", 4: "ERR_UNSUPPORTED",
+                5: "ERR_WORKSPACE", 6: "ERR_SINGULAR", 7: "ERR_CUDA", 8: "ERR_TIMEOUT"}
+
+_LIB = None
+_P, _I64, _I32, _SZ = C.c_void_p, C.c_int64, C.c_int32, C.c_size_t
+
+# name -> (restype, argtypes); must list every symbol include/batq.h declares
+SIGNATURES = {
+    "batq_status_string": (C.c_char_p, [C.c_int]),
+    "batq_version": (C.c_int, []),
+    "batq_transform_create": (C.c_int, [C.POINTER(_P), _I32, _I32, _I32, _P, _I64, _P, _I64, _P, _P]),
+    "batq_transform_destroy": (C.c_int, [_P]),
+    "batq_sf_bytes": (_SZ, [_I64, _I64, _I32]),
+    "batq_quantize_act": (C.c_int, [_P, _P, _I64, _I64, _I64, _P, _P, _I32, _P]),
+    "batq_debug_transform_clip_f32": (C.c_int, [_P, _P, _I64, _I64, _I64, _P, _P]),
+    "batq_weight_bytes": (_SZ, [_I64, _I64]),
+    "batq_prepare_weight": (C.c_int, [_P, _P, _I64, _I64, _I64, _P, _P, _P, C.POINTER(_P), _P]),
+    "batq_weight_destroy": (C.c_int, [_P]),
+    "batq_weight_export": (C.c_int, [_P, _P, _P, _P]),
+    "batq_gemm_mxfp4": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _I64, _P]),
+    "batq_linear_workspace_bytes": (_SZ, [_P, _I64]),
+    "batq_linear_w4a4": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P, _SZ, _P]),
+    "batq_linear_w4a4_host": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _P, _P, _P, _SZ, _P]),
+    "batq_last_device_status": (C.c_int, [_P]),
+}
+
+
+class BatqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: BATQ_{STATUS_NAMES.get(status, status)}")
+
+
+def lib_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbatq.so")
+
+
+def load():
+    """Loads libbatq.so (built in-tree by build.py); raises if it is missing."""
+    global _LIB
+    if _LIB is None:
+        path = lib_path()
+        if not os.path.exists(path):
+            raise FileNotFoundError(f"{path} not found: run `python -m paper_2603_16590_b200.build`")
+        lib = C.CDLL(path)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _LIB = lib
+    return _LIB
+
+
+def _check(status: int, where: str):
+    if status != BATQ_OK:
+        raise BatqError(status, where)
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, torch.Tensor):
+        return t.data_ptr()
+    return int(t)
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _f32(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.float32)
+
+
+class Transform:
+    """Owns a batq_transform handle."""
+
+    def __init__(self, n, left, right, clip_lo=None, clip_hi=None, gr=4, gc=8):
+        left, right, clip_lo, clip_hi = _f32(left), _f32(right), _f32(clip_lo), _f32(clip_hi)
+        self._keep = (left, right, clip_lo, clip_hi)
+        h = _P()
+        ls = 0 if left.shape[0] == 1 else gr * gr
+        rs = 0 if right.shape[0] == 1 else gc * gc
+        st = load().batq_transform_create(
+            C.byref(h), n, gr, gc, left.ctypes.data, ls, right.ctypes.data, rs,
+            None if clip_lo is None else clip_lo.ctypes.data, None if clip_hi is None else clip_hi.ctypes.data)
+        _check(st, "batq_transform_create")
+        self.handle, self.n = h, n
+
+    def close(self):
+        if self.handle:
+            load().batq_transform_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def batq_transform_create(n, left, right, clip_lo=None, clip_hi=None, gr=4, gc=8) -> Transform:
+    return Transform(n, left, right, clip_lo, clip_hi, gr, gc)
+
+
+def batq_sf_bytes(rows, n, layout) -> int:
+    return load().batq_sf_bytes(rows, n, layout)
+
+
+def batq_weight_bytes(m, n) -> int:
+    return load().batq_weight_bytes(m, n)
+
+
+def batq_quantize_act(t, x, codes, scales, scale_layout=SF_ROWMAJOR, ld=None, s=None, n=None):
+    """x: bf16 (or int16 bit-pattern) CUDA tensor [s, n]; codes / scales: uint8 CUDA buffers."""
+    s = x.shape[0] if s is None else s
+    n = x.shape[1] if n is None else n
+    ld = x.stride(0) if ld is None else ld
+    st = load().batq_quantize_act(t.handle if t else None, _ptr(x), s, n, ld, _ptr(codes), _ptr(scales),
+                                  scale_layout, _stream())
+    _check(st, "batq_quantize_act")
+
+
+def batq_debug_transform_clip_f32(t, x, out):
+    st = load().batq_debug_transform_clip_f32(t.handle if t else None, _ptr(x), x.shape[0], x.shape[1],
+                                              x.stride(0), _ptr(out), _stream())
+    _check(st, "batq_debug_transform_clip_f32")
+
+
+class Weight:
+    """Owns a batq_weight handle and the device buffer behind it."""
+
+    def __init__(self, t, w, clip_lo=None, clip_hi=None):
+        m, n = w.shape
+        self.m, self.n = m, n
+        self.buf = torch.empty(batq_weight_bytes(m, n) + 1024, dtype=torch.uint8, device=w.device)
+        off = (-self.buf.data_ptr()) % 1024
+        self._base = self.buf.data_ptr() + off
+        h = _P()
+        st = load().batq_prepare_weight(t.handle if t else None, _ptr(w), m, n, w.stride(0), _ptr(clip_lo),
+                                        _ptr(clip_hi), self._base, C.byref(h), _stream())
+        _check(st, "batq_prepare_weight")
+        self.handle = h
+
+    def close(self):
+        if self.handle:
+            load().batq_weight_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def batq_prepare_weight(t, w, clip_lo=None, clip_hi=None) -> Weight:
+    return Weight(t, w, clip_lo, clip_hi)
+
+
+def batq_weight_export(w: Weight):
+    codes = torch.empty((w.m, w.n // 2), dtype=torch.uint8, device=w.buf.device)
+    scales = torch.empty((w.m, w.n // 32), dtype=torch.uint8, device=w.buf.device)
+    _check(load().batq_weight_export(w.handle, _ptr(codes), _ptr(scales), _stream()), "batq_weight_export")
+    return codes, scales
+
+
+def batq_gemm_mxfp4(x_codes, x_scales_mma, w: Weight, s, y, ldy=None):
+    dt = F32 if y.dtype == torch.float32 else BF16
+    st = load().batq_gemm_mxfp4(_ptr(x_codes), _ptr(x_scales_mma), w.handle, s, _ptr(y), dt,
+                                y.stride(0) if ldy is None else ldy, _stream())
+    _check(st, "batq_gemm_mxfp4")
+
+
+def batq_linear_workspace_bytes(w: Weight, s) -> int:
+    return load().batq_linear_workspace_bytes(w.handle, s)
+
+
+def aligned_workspace(nbytes, device="cuda"):
+    """A uint8 CUDA buffer whose returned view starts on a 1024-byte boundary."""
+    buf = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
+    off = (-buf.data_ptr()) % 1024
+    return buf[off:off + nbytes]
+
+
+def batq_linear_w4a4(t, w: Weight, x, y, workspace):
+    dt = F32 if y.dtype == torch.float32 else BF16
+    st = load().batq_linear_w4a4(t.handle if t else None, w.handle, _ptr(x), x.shape[0], x.stride(0), _ptr(y), dt,
+                                 y.stride(0), _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "batq_linear_w4a4")
+
+
+def batq_linear_w4a4_host(t, w: Weight, x_host, y_host, x_stage, y_stage, workspace):
+    dt = F32 if y_host.dtype == torch.float32 else BF16
+    st = load().batq_linear_w4a4_host(t.handle if t else None, w.handle, _ptr(x_host), x_host.shape[0], _ptr(y_host),
+                                      dt, _ptr(x_stage), _ptr(y_stage), _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "batq_linear_w4a4_host")
+
+
+def batq_last_device_status() -> int:
+    return load().batq_last_device_status(_stream())
+
+
+def bits_to_cuda_bf16(bits: np.ndarray) -> torch.Tensor:
+    """uint16 bf16 bit patterns (host) -> CUDA bf16 tensor (a copy, no arithmetic)."""
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)

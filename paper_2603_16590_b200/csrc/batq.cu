@@ -1,0 +1,541 @@
+// C-ABI of the batq library: host-side validation, handles and kernel launches.
+// The whole library is this one translation unit.
+#include "batq.h"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "gemm_mxfp4.cuh"
+#include "prepare_weight.cuh"
+#include "quantize_act.cuh"
+
+using namespace batq;
+
+// ------------------------------------------------------------------------------------
+// handles
+// ------------------------------------------------------------------------------------
+struct batq_transform {
+  int device;
+  int32_t n, k, gr, gc;
+  int32_t left_stride, right_stride;  // 0 = shared
+  bool has_clip;
+  std::vector<float> left, right;     // host copies (for the inverse)
+  float* d_left;                      // device copies (for the kernels)
+  float* d_right;
+  float* d_clip_lo;
+  float* d_clip_hi;
+};
+
+struct batq_weight {
+  int device;
+  int64_t m, n;
+  int32_t k, katoms;
+  uint8_t* codes;   // [m x n/2]
+  uint8_t* scales;  // BATQ_SF_MMA
+  CUtensorMap tmap_b256;
+  CUtensorMap tmap_b128;
+};
+
+namespace {
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int32_t katoms_of(int64_t k) { return static_cast<int32_t>(2 * ((k + 7) / 8)); }
+
+constexpr int kMaxDevices = 64;
+
+struct DeviceInfo {
+  bool ready = false;
+  int sm_count = 0;
+  int cc_major = 0;
+};
+DeviceInfo g_dev[kMaxDevices];
+std::mutex g_mutex;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode_tiled = nullptr;
+
+template <typename K>
+cudaError_t set_smem(K kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
+// Per-device one-time setup: properties, opt-in shared memory sizes, driver entry point.
+batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BATQ_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceInfo& d = g_dev[dev];
+  if (!d.ready) {
+    if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return BATQ_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return BATQ_ERR_CUDA;
+    if (d.cc_major != 10) return BATQ_ERR_UNSUPPORTED;
+    cudaError_t e = cudaSuccess;
+    e = e ? e : set_smem(quantize_act_kernel<true, true, false>, kQaSmemBytes);
+    e = e ? e : set_smem(quantize_act_kernel<true, false, false>, kQaSmemBytes);
+    e = e ? e : set_smem(quantize_act_kernel<false, false, false>, kQaSmemBytes);
+    e = e ? e : set_smem(quantize_act_kernel<true, true, true>, kQaSmemBytes);
+    e = e ? e : set_smem(quantize_act_kernel<true, false, true>, kQaSmemBytes);
+    e = e ? e : set_smem(quantize_act_kernel<false, false, true>, kQaSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_kernel<256, false>, GemmCfg<256>::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_kernel<256, true>, GemmCfg<256>::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_kernel<128, false>, GemmCfg<128>::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_kernel<128, true>, GemmCfg<128>::kSmemBytes);
+    if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+    if (g_encode_tiled == nullptr) {
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+          qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+        cudaGetLastError();
+        return BATQ_ERR_CUDA;
+      }
+      g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    d.ready = true;
+  }
+  if (device_out) *device_out = dev;
+  if (info_out) *info_out = &d;
+  return BATQ_OK;
+}
+
+// Tensor map over packed codes [rows x row_bytes] (uint8), box = 128 bytes x box_rows, 128-byte swizzle.
+batq_status make_codes_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t row_bytes, int box_rows) {
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(row_bytes), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(row_bytes)};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBKBytes), static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides,
+                                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? BATQ_OK : BATQ_ERR_CUDA;
+}
+
+// Gauss-Jordan inverse with partial pivoting of a small dense matrix, fp64.
+bool invert_small(const double* a, int n, double* inv) {
+  std::vector<double> w(static_cast<size_t>(n) * 2 * n);
+  for (int r = 0; r < n; ++r)
+    for (int c = 0; c < n; ++c) {
+      w[r * 2 * n + c] = a[r * n + c];
+      w[r * 2 * n + n + c] = (r == c) ? 1.0 : 0.0;
+    }
+  for (int col = 0; col < n; ++col) {
+    int piv = col;
+    for (int r = col + 1; r < n; ++r)
+      if (std::fabs(w[r * 2 * n + col]) > std::fabs(w[piv * 2 * n + col])) piv = r;
+    const double pv = w[piv * 2 * n + col];
+    if (!(std::fabs(pv) > 1e-300) || !std::isfinite(pv)) return false;
+    if (piv != col)
+      for (int c = 0; c < 2 * n; ++c) std::swap(w[col * 2 * n + c], w[piv * 2 * n + c]);
+    for (int c = 0; c < 2 * n; ++c) w[col * 2 * n + c] /= pv;
+    for (int r = 0; r < n; ++r) {
+      if (r == col) continue;
+      const double f = w[r * 2 * n + col];
+      if (f == 0.0) continue;
+      for (int c = 0; c < 2 * n; ++c) w[r * 2 * n + c] -= f * w[col * 2 * n + c];
+    }
+  }
+  for (int r = 0; r < n; ++r)
+    for (int c = 0; c < n; ++c) inv[r * n + c] = w[r * 2 * n + n + c];
+  return true;
+}
+
+batq_status check_x(const void* x, int64_t s, int64_t n, int64_t ld) {
+  if (s < 0 || n <= 0 || n % 32 != 0 || ld < n || n > (int64_t(1) << 24) || s > (int64_t(1) << 30)) return BATQ_ERR_SHAPE;
+  if (s > 0 && x == nullptr) return BATQ_ERR_NULL;
+  if (ld % 8 != 0 || !aligned(x, 16)) return BATQ_ERR_ALIGN;
+  return BATQ_OK;
+}
+
+batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, int64_t n, int64_t ld, void* codes,
+                            void* scales, int32_t layout, float* debug_out, cudaStream_t stream) {
+  int dev;
+  const DeviceInfo* info;
+  batq_status st = device_setup(&dev, &info);
+  if (st != BATQ_OK) return st;
+  if (t != nullptr && t->device != dev) return BATQ_ERR_CUDA;
+  QuantActParams p{};
+  p.x = static_cast<const uint16_t*>(x);
+  p.ld = ld;
+  p.s = s;
+  p.n = static_cast<int32_t>(n);
+  p.k = static_cast<int32_t>(n / 32);
+  int gs = 32;
+  while (p.k % gs != 0) gs >>= 1;
+  p.gs = gs;
+  p.rows_per_tile = kQaConsumers / gs;
+  p.n_row_tiles = (s + p.rows_per_tile - 1) / p.rows_per_tile;
+  p.n_units = (p.k / gs) * p.n_row_tiles;
+  if (t != nullptr) {
+    p.left = t->d_left; p.right = t->d_right;
+    p.left_stride = t->left_stride; p.right_stride = t->right_stride;
+    p.clip_lo = t->d_clip_lo; p.clip_hi = t->d_clip_hi;
+  }
+  p.clip_row_stride = 0;
+  p.codes = static_cast<uint8_t*>(codes);
+  p.scales = static_cast<uint8_t*>(scales);
+  p.sf_layout = layout;
+  p.sf_katoms = katoms_of(p.k);
+  p.debug_out = debug_out;
+  const int grid = static_cast<int>(std::min<int64_t>(info->sm_count, p.n_units));
+  const bool xf = t != nullptr, cl = t != nullptr && t->has_clip, dbg = debug_out != nullptr;
+#define BATQ_QA(XF, CL, DB) quantize_act_kernel<XF, CL, DB><<<grid, kQaThreads, kQaSmemBytes, stream>>>(p)
+  if (xf && cl && !dbg) BATQ_QA(true, true, false);
+  else if (xf && !cl && !dbg) BATQ_QA(true, false, false);
+  else if (!xf && !dbg) BATQ_QA(false, false, false);
+  else if (xf && cl && dbg) BATQ_QA(true, true, true);
+  else if (xf && !cl && dbg) BATQ_QA(true, false, true);
+  else BATQ_QA(false, false, true);
+#undef BATQ_QA
+  return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
+}
+
+// Tile width: the wider tile halves shared-memory traffic per flop; the narrower one has two
+// accumulators (epilogue overlapped with the next tile) and finer wave granularity.
+int pick_bn(int64_t s, int64_t m, int sm_count) {
+  const int64_t mt = (s + kBM - 1) / kBM;
+  auto waves_eff = [&](int bn) {
+    const int64_t tiles = mt * ((m + bn - 1) / bn);
+    const int64_t waves = (tiles + sm_count - 1) / sm_count;
+    return static_cast<double>(tiles) / static_cast<double>(waves * sm_count);
+  };
+  if (m <= 128) return 128;
+  return waves_eff(256) >= 0.92 * waves_eff(128) ? 256 : 128;
+}
+
+batq_status launch_gemm(const void* x_codes, const void* x_sf, const batq_weight* w, int64_t s, void* y,
+                        int32_t y_dtype, int64_t ldy, cudaStream_t stream) {
+  int dev;
+  const DeviceInfo* info;
+  batq_status st = device_setup(&dev, &info);
+  if (st != BATQ_OK) return st;
+  if (w->device != dev) return BATQ_ERR_CUDA;
+  CUtensorMap tmap_a;
+  st = make_codes_tmap(&tmap_a, x_codes, s, w->n / 2, kBM);
+  if (st != BATQ_OK) return st;
+  const int bn = pick_bn(s, w->m, info->sm_count);
+  GemmParams p{};
+  p.sfa = static_cast<const uint8_t*>(x_sf);
+  p.sfb = w->scales;
+  p.y = y;
+  p.ldy = ldy;
+  p.s = static_cast<int32_t>(s);
+  p.m = static_cast<int32_t>(w->m);
+  p.k_bytes = static_cast<int32_t>(w->n / 2);
+  p.katoms = w->katoms;
+  p.k_steps = static_cast<int32_t>((w->n + 255) / 256);
+  p.m_tiles = static_cast<int32_t>((s + kBM - 1) / kBM);
+  p.n_tiles = static_cast<int32_t>((w->m + bn - 1) / bn);
+  p.sfa_row_tiles = p.m_tiles;
+  p.sfb_row_tiles = static_cast<int32_t>((w->m + 127) / 128);
+  const int grid = std::min(info->sm_count, p.m_tiles * p.n_tiles);
+  const bool bf = y_dtype == BATQ_BF16;
+  if (bn == 256) {
+    if (bf) gemm_mxfp4_kernel<256, true><<<grid, kGemmThreads, GemmCfg<256>::kSmemBytes, stream>>>(tmap_a, w->tmap_b256, p);
+    else gemm_mxfp4_kernel<256, false><<<grid, kGemmThreads, GemmCfg<256>::kSmemBytes, stream>>>(tmap_a, w->tmap_b256, p);
+  } else {
+    if (bf) gemm_mxfp4_kernel<128, true><<<grid, kGemmThreads, GemmCfg<128>::kSmemBytes, stream>>>(tmap_a, w->tmap_b128, p);
+    else gemm_mxfp4_kernel<128, false><<<grid, kGemmThreads, GemmCfg<128>::kSmemBytes, stream>>>(tmap_a, w->tmap_b128, p);
+  }
+  return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
+}
+
+batq_status check_y(const void* y, int32_t y_dtype, int64_t ldy, int64_t m) {
+  if (y_dtype != BATQ_F32 && y_dtype != BATQ_BF16) return BATQ_ERR_UNSUPPORTED;
+  if (ldy < m) return BATQ_ERR_SHAPE;
+  if (!aligned(y, 16) || ldy % (y_dtype == BATQ_F32 ? 4 : 8) != 0) return BATQ_ERR_ALIGN;
+  return BATQ_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------
+// exported functions
+// ------------------------------------------------------------------------------------
+extern "C" {
+
+const char* batq_status_string(batq_status s) {
+  switch (s) {
+    case BATQ_OK: return "ok";
+    case BATQ_ERR_NULL: return "null pointer";
+    case BATQ_ERR_SHAPE: return "bad shape";
+    case BATQ_ERR_ALIGN: return "bad alignment";
+    case BATQ_ERR_UNSUPPORTED: return "unsupported";
+    case BATQ_ERR_WORKSPACE: return "workspace too small";
+    case BATQ_ERR_SINGULAR: return "singular transform factor";
+    case BATQ_ERR_CUDA: return "CUDA error";
+    case BATQ_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+int batq_version(void) { return 100; }
+
+batq_status batq_transform_create(batq_transform** out, int32_t n, int32_t gr, int32_t gc, const float* left,
+                                  int64_t left_stride, const float* right, int64_t right_stride,
+                                  const float* clip_lo, const float* clip_hi) {
+  if (out == nullptr) return BATQ_ERR_NULL;
+  *out = nullptr;
+  if (left == nullptr || right == nullptr) return BATQ_ERR_NULL;
+  if ((clip_lo == nullptr) != (clip_hi == nullptr)) return BATQ_ERR_NULL;
+  if (n <= 0 || n % 32 != 0 || gr <= 0 || gc <= 0 || gr * gc != 32) return BATQ_ERR_SHAPE;
+  if (gr != 4 || gc != 8) return BATQ_ERR_UNSUPPORTED;
+  if ((left_stride != 0 && left_stride != gr * gr) || (right_stride != 0 && right_stride != gc * gc)) return BATQ_ERR_SHAPE;
+  int dev;
+  batq_status st = device_setup(&dev, nullptr);
+  if (st != BATQ_OK) return st;
+  batq_transform* t = new (std::nothrow) batq_transform();
+  if (t == nullptr) return BATQ_ERR_CUDA;
+  t->device = dev;
+  t->n = n; t->k = n / 32; t->gr = gr; t->gc = gc;
+  t->left_stride = static_cast<int32_t>(left_stride);
+  t->right_stride = static_cast<int32_t>(right_stride);
+  t->has_clip = clip_lo != nullptr;
+  const size_t nl = left_stride ? static_cast<size_t>(t->k) * 16 : 16;
+  const size_t nr = right_stride ? static_cast<size_t>(t->k) * 64 : 64;
+  t->left.assign(left, left + nl);
+  t->right.assign(right, right + nr);
+  t->d_left = t->d_right = t->d_clip_lo = t->d_clip_hi = nullptr;
+  cudaError_t e = cudaMalloc(&t->d_left, nl * sizeof(float));
+  e = e ? e : cudaMalloc(&t->d_right, nr * sizeof(float));
+  e = e ? e : cudaMemcpy(t->d_left, left, nl * sizeof(float), cudaMemcpyHostToDevice);
+  e = e ? e : cudaMemcpy(t->d_right, right, nr * sizeof(float), cudaMemcpyHostToDevice);
+  if (t->has_clip) {
+    e = e ? e : cudaMalloc(&t->d_clip_lo, t->k * sizeof(float));
+    e = e ? e : cudaMalloc(&t->d_clip_hi, t->k * sizeof(float));
+    e = e ? e : cudaMemcpy(t->d_clip_lo, clip_lo, t->k * sizeof(float), cudaMemcpyHostToDevice);
+    e = e ? e : cudaMemcpy(t->d_clip_hi, clip_hi, t->k * sizeof(float), cudaMemcpyHostToDevice);
+  }
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    batq_transform_destroy(t);
+    return BATQ_ERR_CUDA;
+  }
+  *out = t;
+  return BATQ_OK;
+}
+
+batq_status batq_transform_destroy(batq_transform* t) {
+  if (t == nullptr) return BATQ_OK;
+  cudaFree(t->d_left);
+  cudaFree(t->d_right);
+  cudaFree(t->d_clip_lo);
+  cudaFree(t->d_clip_hi);
+  delete t;
+  return BATQ_OK;
+}
+
+size_t batq_sf_bytes(int64_t rows, int64_t n, int32_t layout) {
+  if (rows < 0 || n <= 0 || n % 32 != 0) return 0;
+  const int64_t k = n / 32;
+  if (layout == BATQ_SF_ROWMAJOR) return static_cast<size_t>(rows * k);
+  if (layout == BATQ_SF_MMA) return static_cast<size_t>((rows + 127) / 128) * katoms_of(k) * 512;
+  return 0;
+}
+
+batq_status batq_quantize_act(const batq_transform* t, const void* x_bf16, int64_t s, int64_t n, int64_t ld,
+                              void* codes, void* scales, int32_t scale_layout, void* stream) {
+  batq_status st = check_x(x_bf16, s, n, ld);
+  if (st != BATQ_OK) return st;
+  if (t != nullptr && t->n != n) return BATQ_ERR_SHAPE;
+  if (scale_layout != BATQ_SF_ROWMAJOR && scale_layout != BATQ_SF_MMA) return BATQ_ERR_UNSUPPORTED;
+  if (s == 0) return BATQ_OK;
+  if (codes == nullptr || scales == nullptr) return BATQ_ERR_NULL;
+  if (!aligned(codes, 16)) return BATQ_ERR_ALIGN;
+  return launch_quantize(t, x_bf16, s, n, ld, codes, scales, scale_layout, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+batq_status batq_debug_transform_clip_f32(const batq_transform* t, const void* x_bf16, int64_t s, int64_t n,
+                                          int64_t ld, float* out, void* stream) {
+  batq_status st = check_x(x_bf16, s, n, ld);
+  if (st != BATQ_OK) return st;
+  if (t != nullptr && t->n != n) return BATQ_ERR_SHAPE;
+  if (s == 0) return BATQ_OK;
+  if (out == nullptr) return BATQ_ERR_NULL;
+  if (!aligned(out, 16)) return BATQ_ERR_ALIGN;
+  return launch_quantize(t, x_bf16, s, n, ld, nullptr, nullptr, BATQ_SF_ROWMAJOR, out, static_cast<cudaStream_t>(stream));
+}
+
+size_t batq_weight_bytes(int64_t m, int64_t n) {
+  if (m <= 0 || n <= 0 || n % 32 != 0) return 0;
+  return round_up(static_cast<size_t>(m * (n / 2)), 1024) + batq_sf_bytes(m, n, BATQ_SF_MMA);
+}
+
+batq_status batq_prepare_weight(const batq_transform* t, const void* w_bf16, int64_t m, int64_t n, int64_t ld,
+                                const float* w_clip_lo, const float* w_clip_hi, void* weight_buf, batq_weight** out,
+                                void* stream) {
+  if (out == nullptr) return BATQ_ERR_NULL;
+  *out = nullptr;
+  if (m <= 0 || m > (int64_t(1) << 24)) return BATQ_ERR_SHAPE;
+  batq_status st = check_x(w_bf16, m, n, ld);
+  if (st != BATQ_OK) return st;
+  if (weight_buf == nullptr) return BATQ_ERR_NULL;
+  if ((w_clip_lo == nullptr) != (w_clip_hi == nullptr)) return BATQ_ERR_NULL;
+  if (!aligned(weight_buf, 1024)) return BATQ_ERR_ALIGN;
+  if (t != nullptr && t->n != n) return BATQ_ERR_SHAPE;
+  int dev;
+  st = device_setup(&dev, nullptr);
+  if (st != BATQ_OK) return st;
+  if (t != nullptr && t->device != dev) return BATQ_ERR_CUDA;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const int32_t k = static_cast<int32_t>(n / 32);
+
+  // L' = L^-T and R' = R^-T in fp64: W~_blk = L^-1 Wv R^-T = L'^T Wv R'.
+  double* d_fac = nullptr;
+  size_t nl = 0, nr = 0;
+  if (t != nullptr) {
+    const size_t cl = t->left_stride ? k : 1, cr = t->right_stride ? k : 1;
+    nl = cl * 16; nr = cr * 64;
+    std::vector<double> fac(nl + nr);
+    double a[64], inv[64];
+    for (size_t i = 0; i < cl; ++i) {
+      for (int e = 0; e < 16; ++e) a[e] = t->left[i * 16 + e];
+      if (!invert_small(a, 4, inv)) return BATQ_ERR_SINGULAR;
+      for (int r = 0; r < 4; ++r)
+        for (int c = 0; c < 4; ++c) fac[i * 16 + r * 4 + c] = inv[c * 4 + r];
+    }
+    for (size_t i = 0; i < cr; ++i) {
+      for (int e = 0; e < 64; ++e) a[e] = t->right[i * 64 + e];
+      if (!invert_small(a, 8, inv)) return BATQ_ERR_SINGULAR;
+      for (int r = 0; r < 8; ++r)
+        for (int c = 0; c < 8; ++c) fac[nl + i * 64 + r * 8 + c] = inv[c * 8 + r];
+    }
+    if (cudaMalloc(&d_fac, fac.size() * sizeof(double)) != cudaSuccess ||
+        cudaMemcpyAsync(d_fac, fac.data(), fac.size() * sizeof(double), cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+        cudaStreamSynchronize(cs) != cudaSuccess) {
+      cudaGetLastError();
+      cudaFree(d_fac);
+      return BATQ_ERR_CUDA;
+    }
+  }
+  batq_weight* w = new (std::nothrow) batq_weight();
+  if (w == nullptr) { cudaFree(d_fac); return BATQ_ERR_CUDA; }
+  w->device = dev;
+  w->m = m; w->n = n; w->k = k; w->katoms = katoms_of(k);
+  w->codes = static_cast<uint8_t*>(weight_buf);
+  w->scales = w->codes + round_up(static_cast<size_t>(m * (n / 2)), 1024);
+
+  PrepWeightParams p{};
+  p.w = static_cast<const uint16_t*>(w_bf16);
+  p.ld = ld; p.m = m; p.n = static_cast<int32_t>(n); p.k = k;
+  if (t != nullptr) {
+    p.left = d_fac; p.right = d_fac + nl;
+    p.left_stride = t->left_stride; p.right_stride = t->right_stride;
+  }
+  p.clip_lo = w_clip_lo; p.clip_hi = w_clip_hi;
+  p.codes = w->codes; p.scales = w->scales; p.katoms = w->katoms;
+  const int64_t items = m * k;
+  prepare_weight_kernel<<<static_cast<unsigned>((items + 127) / 128), 128, 0, cs>>>(p);
+  cudaError_t e = cudaGetLastError();
+  e = e ? e : cudaStreamSynchronize(cs);
+  cudaFree(d_fac);
+  if (e != cudaSuccess) { cudaGetLastError(); delete w; return BATQ_ERR_CUDA; }
+  st = make_codes_tmap(&w->tmap_b256, w->codes, m, n / 2, 256);
+  if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b128, w->codes, m, n / 2, 128);
+  if (st != BATQ_OK) { delete w; return st; }
+  *out = w;
+  return BATQ_OK;
+}
+
+batq_status batq_weight_destroy(batq_weight* w) {
+  delete w;
+  return BATQ_OK;
+}
+
+batq_status batq_weight_export(const batq_weight* w, void* codes_rowmajor, void* scales_rowmajor, void* stream) {
+  if (w == nullptr || codes_rowmajor == nullptr || scales_rowmajor == nullptr) return BATQ_ERR_NULL;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(codes_rowmajor, w->codes, static_cast<size_t>(w->m * (w->n / 2)), cudaMemcpyDeviceToDevice, cs) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return BATQ_ERR_CUDA;
+  }
+  const int64_t items = w->m * w->k;
+  export_scales_kernel<<<static_cast<unsigned>((items + 255) / 256), 256, 0, cs>>>(
+      w->scales, static_cast<uint8_t*>(scales_rowmajor), w->m, w->k, w->katoms);
+  return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
+}
+
+batq_status batq_gemm_mxfp4(const void* x_codes, const void* x_scales_mma, const batq_weight* w, int64_t s, void* y,
+                            int32_t y_dtype, int64_t ldy, void* stream) {
+  if (w == nullptr) return BATQ_ERR_NULL;
+  if (s < 0 || s > (int64_t(1) << 30)) return BATQ_ERR_SHAPE;
+  if (s == 0) return BATQ_OK;
+  if (x_codes == nullptr || x_scales_mma == nullptr || y == nullptr) return BATQ_ERR_NULL;
+  if (!aligned(x_codes, 16) || !aligned(x_scales_mma, 16)) return BATQ_ERR_ALIGN;
+  batq_status st = check_y(y, y_dtype, ldy, w->m);
+  if (st != BATQ_OK) return st;
+  return launch_gemm(x_codes, x_scales_mma, w, s, y, y_dtype, ldy, static_cast<cudaStream_t>(stream));
+}
+
+size_t batq_linear_workspace_bytes(const batq_weight* w, int64_t s) {
+  if (w == nullptr || s < 0) return 0;
+  return round_up(static_cast<size_t>(s * (w->n / 2)), 1024) + batq_sf_bytes(s, w->n, BATQ_SF_MMA);
+}
+
+batq_status batq_linear_w4a4(const batq_transform* t, const batq_weight* w, const void* x_bf16, int64_t s, int64_t ld,
+                             void* y, int32_t y_dtype, int64_t ldy, void* workspace, size_t workspace_bytes,
+                             void* stream) {
+  if (w == nullptr) return BATQ_ERR_NULL;
+  batq_status st = check_x(x_bf16, s, w->n, ld);
+  if (st != BATQ_OK) return st;
+  if (t != nullptr && t->n != w->n) return BATQ_ERR_SHAPE;
+  if (s == 0) return BATQ_OK;
+  if (y == nullptr || workspace == nullptr) return BATQ_ERR_NULL;
+  st = check_y(y, y_dtype, ldy, w->m);
+  if (st != BATQ_OK) return st;
+  if (!aligned(workspace, 1024)) return BATQ_ERR_ALIGN;
+  if (workspace_bytes < batq_linear_workspace_bytes(w, s)) return BATQ_ERR_WORKSPACE;
+  uint8_t* codes = static_cast<uint8_t*>(workspace);
+  uint8_t* sf = codes + round_up(static_cast<size_t>(s * (w->n / 2)), 1024);
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  st = launch_quantize(t, x_bf16, s, w->n, ld, codes, sf, BATQ_SF_MMA, nullptr, cs);
+  if (st != BATQ_OK) return st;
+  return launch_gemm(codes, sf, w, s, y, y_dtype, ldy, cs);
+}
+
+batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w, const void* x_host, int64_t s,
+                                  void* y_host, int32_t y_dtype, void* x_stage_dev, void* y_stage_dev, void* workspace,
+                                  size_t workspace_bytes, void* stream) {
+  if (w == nullptr) return BATQ_ERR_NULL;
+  if (s < 0) return BATQ_ERR_SHAPE;
+  if (s == 0) return BATQ_OK;
+  if (x_host == nullptr || y_host == nullptr || x_stage_dev == nullptr || y_stage_dev == nullptr) return BATQ_ERR_NULL;
+  if (y_dtype != BATQ_F32 && y_dtype != BATQ_BF16) return BATQ_ERR_UNSUPPORTED;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const size_t xb = static_cast<size_t>(s * w->n) * 2;
+  const size_t yb = static_cast<size_t>(s * w->m) * (y_dtype == BATQ_F32 ? 4 : 2);
+  if (cudaMemcpyAsync(x_stage_dev, x_host, xb, cudaMemcpyHostToDevice, cs) != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+  batq_status st = batq_linear_w4a4(t, w, x_stage_dev, s, w->n, y_stage_dev, y_dtype, w->m, workspace, workspace_bytes, stream);
+  if (st != BATQ_OK) return st;
+  if (cudaMemcpyAsync(y_host, y_stage_dev, yb, cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
+      cudaStreamSynchronize(cs) != cudaSuccess) {
+    cudaGetLastError();
+    return BATQ_ERR_CUDA;
+  }
+  return BATQ_OK;
+}
+
+batq_status batq_last_device_status(void* stream) {
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+  int flag = 0;
+  if (cudaMemcpyFromSymbol(&flag, g_device_error, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+  if (flag != 0) {
+    const int zero = 0;
+    cudaMemcpyToSymbol(g_device_error, &zero, sizeof(int));
+    return BATQ_ERR_TIMEOUT;
+  }
+  return BATQ_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,308 @@
+"""Parity of the CUDA path against the CPU oracle, through the C-ABI.  GPU only."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import batq_oracle as O
+from paper_2603_16590_b200 import synth
+from tests.helpers import near_rounding_boundary, sf_mma_to_rowmajor
+
+pytestmark = pytest.mark.gpu
+
+# a-priori bound on the fp32 transform error relative to the block's magnitude:
+# 12 fused multiply-adds per output plus the bf16->fp32 input (exact), each 2^-24
+FP32_REL = 16 * 2.0 ** -24
+
+
+def _mk_transform(batq, t):
+    return batq.batq_transform_create(t.n, t.left, t.right, t.clip_lo, t.clip_hi)
+
+
+def _gpu_quantize(batq, tr, xb, layout=0, ld=None):
+    S, N = xb.shape
+    x = batq.bits_to_cuda_bf16(xb)
+    if ld is not None:
+        xp = torch.zeros((S, ld), dtype=torch.bfloat16, device="cuda")
+        xp[:, :N] = x
+        x = xp[:, :N]
+    codes = torch.full((S * N // 2 + 64,), 0xEE, dtype=torch.uint8, device="cuda")
+    nsf = batq.batq_sf_bytes(S, N, layout)
+    scales = torch.full((nsf + 64,), 0xEE, dtype=torch.uint8, device="cuda")
+    batq.batq_quantize_act(tr, x, codes, scales, layout)
+    assert batq.batq_last_device_status() == 0
+    torch.cuda.synchronize()
+    c, s = codes.cpu().numpy(), scales.cpu().numpy()
+    assert (c[S * N // 2:] == 0xEE).all() and (s[nsf:] == 0xEE).all(), "wrote past the output buffers"
+    c = O.unpack_codes(c[:S * N // 2].reshape(S, N // 2))
+    s = s[:nsf]
+    s = s.reshape(S, N // 32) if layout == 0 else sf_mma_to_rowmajor(s, S, N // 32)
+    return c, s
+
+
+SHAPES = [(1, 32), (3, 96), (128, 1024), (77, 3584), (300, 4096), (257, 2048 + 32)]
+
+
+@pytest.mark.parametrize("S,N", SHAPES)
+@pytest.mark.parametrize("geometry", ["baseline", "paper"])
+def test_quantizer_bit_exact_on_identical_transformed_input(batq, S, N, geometry):
+    """Feed the oracle's Q(.) the GPU's own fp32 transformed+clipped values:
+    codes and scale bytes must match exactly, every element."""
+    xb = synth.make_activations(S, N, 100 + S)
+    t = synth.make_transform(N, 7, geometry)
+    tr = _mk_transform(batq, t)
+    x = batq.bits_to_cuda_bf16(xb)
+    vhat = torch.empty((S, N), dtype=torch.float32, device="cuda")
+    batq.batq_debug_transform_clip_f32(tr, x, vhat)
+    gc, gs = _gpu_quantize(batq, tr, xb)
+    oc, os_ = O.mxfp4_quantize(vhat.cpu().numpy().astype(np.float64))
+    assert np.array_equal(gs, os_)
+    assert np.array_equal(gc, oc)
+
+
+@pytest.mark.parametrize("S,N", SHAPES)
+@pytest.mark.parametrize("geometry,clip", [("baseline", True), ("paper", True), ("naive", False)])
+def test_quantizer_end_to_end_vs_oracle(batq, S, N, geometry, clip):
+    xb = synth.make_activations(S, N, 200 + S)
+    t = synth.make_transform(N, 8, geometry, clip=clip)
+    tr = _mk_transform(batq, t)
+    gc, gs = _gpu_quantize(batq, tr, xb)
+    V = O.transform_clip(xb, t.left, t.right, t.clip_lo, t.clip_hi)
+    oc, os_ = O.mxfp4_quantize(V)
+    # the fp32 transform output vs the fp64 one
+    vhat = torch.empty((S, N), dtype=torch.float32, device="cuda")
+    batq.batq_debug_transform_clip_f32(tr, batq.bits_to_cuda_bf16(xb), vhat)
+    X = np.abs(O.bf16_bits_to_f64(xb)).reshape(S, N // 32, 32)
+    P = np.abs(O.block_matrices(t.left, t.right, N // 32))
+    bound = FP32_REL * np.einsum("sje,jef->sjf", X, P).reshape(S, N)
+    assert np.all(np.abs(vhat.cpu().numpy().astype(np.float64) - V) <= bound + 1e-300)
+    # scale bytes: bit-exact, except blocks whose amax sits within the fp32 error of a power of two
+    sdiff = gs != os_
+    if sdiff.any():
+        amax = np.abs(V).reshape(S, N // 32, 32).max(axis=2)
+        frac = amax / np.exp2(np.floor(np.log2(amax)))
+        tol = bound.reshape(S, N // 32, 32).max(axis=2) / amax
+        assert np.all((np.minimum(frac - 1, 2 - frac) <= 2 * tol)[sdiff])
+        assert sdiff.mean() <= 1e-5
+    # codes: mismatches only next to a rounding boundary, at most 1e-4 of the elements
+    same_scale = np.repeat(~sdiff, 32, axis=1)
+    cdiff = (gc != oc) & same_scale
+    assert cdiff.mean() <= 1e-4
+    if cdiff.any():
+        scale = np.repeat(np.exp2(os_.astype(np.float64) - 127), 32, axis=1)
+        u = np.abs(V) / scale
+        rel = 2 * bound / np.maximum(np.abs(V), 1e-300)
+        strict = near_rounding_boundary(u[cdiff], 2.0 ** -22)      # ~ 1 fp32 ulp of the threshold
+        loose = np.array([near_rounding_boundary(np.array([uu]), rr)[0] for uu, rr in zip(u[cdiff], rel[cdiff])])
+        assert np.all(strict | loose)
+        # a mismatching code is always the neighbouring code
+        assert np.all(np.abs((gc[cdiff] & 7).astype(int) - (oc[cdiff] & 7).astype(int)) <= 1)
+
+
+@pytest.mark.parametrize("S,N", SHAPES)
+def test_identity_transform_is_bit_exact_plain_mxfp4(batq, S, N):
+    xb = synth.make_activations(S, N, 300 + S)
+    gc, gs = _gpu_quantize(batq, None, xb)
+    oc, os_ = O.quantize_act(xb, None, None)
+    assert np.array_equal(gs, os_) and np.array_equal(gc, oc)
+    # identity *factors* through the transform kernel give the same bits
+    t = synth.make_transform(N, 1, identity=True, clip=False)
+    gc2, gs2 = _gpu_quantize(batq, _mk_transform(batq, t), xb)
+    assert np.array_equal(gs2, os_) and np.array_equal(gc2, oc)
+
+
+def test_quantizer_special_values(batq):
+    """Zero blocks, signed zeros, ties, saturation, tiny and huge magnitudes."""
+    N = 256
+    X = np.zeros((4, N), np.float32)
+    X[0, 32:64] = np.array([6, 5, 3.5, 2.5, 1.75, 1.25, 0.75, 0.25, -0.25, -7, 0.1, -0.1, 7, 7.5, 4, 3] * 2, np.float32)
+    X[1, :32] = -0.0
+    X[1, 64:96] = np.linspace(-1, 1, 32) * 2.0 ** -120
+    X[2, :] = np.random.default_rng(0).standard_normal(N).astype(np.float32) * 2.0 ** 100
+    X[3, 96:128] = 2.0 ** -133   # below the normal range: flushes into the clamped scale
+    xb = synth.f32_to_bf16_bits(X)
+    gc, gs = _gpu_quantize(batq, None, xb)
+    oc, os_ = O.quantize_act(xb, None, None)
+    assert np.array_equal(gs, os_) and np.array_equal(gc, oc)
+    assert gs[0, 0] == 0 and gc[1, 0] == 8
+
+
+@pytest.mark.parametrize("S,N", [(5, 96), (130, 1024), (257, 3584)])
+def test_scale_layout_mma_matches_rowmajor(batq, S, N):
+    xb = synth.make_activations(S, N, 400 + S)
+    tr = _mk_transform(batq, synth.make_transform(N, 9, "baseline"))
+    c0, s0 = _gpu_quantize(batq, tr, xb, layout=0)
+    c1, s1 = _gpu_quantize(batq, tr, xb, layout=1)
+    assert np.array_equal(c0, c1) and np.array_equal(s0, s1)
+
+
+def test_quantizer_row_stride_and_determinism(batq):
+    S, N = 70, 1024
+    xb = synth.make_activations(S, N, 55)
+    tr = _mk_transform(batq, synth.make_transform(N, 9, "baseline"))
+    a = _gpu_quantize(batq, tr, xb)
+    b = _gpu_quantize(batq, tr, xb, ld=N + 72)
+    c = _gpu_quantize(batq, tr, xb)
+    for u, v, w in zip(a, b, c):
+        assert np.array_equal(u, v) and np.array_equal(u, w)
+
+
+# ---------------------------------------------------------------------------- weights
+def _weight_mismatch_ok(gc, gs, oc, os_, Wt):
+    sdiff = gs != os_
+    assert sdiff.mean() <= 1e-6
+    cdiff = (gc != oc) & np.repeat(~sdiff, 32, axis=1)
+    assert cdiff.mean() <= 1e-5
+    if cdiff.any():  # fp64 on both sides: only exact-tie neighbourhoods may differ
+        scale = np.repeat(np.exp2(os_.astype(np.float64) - 127), 32, axis=1)
+        assert np.all(near_rounding_boundary((np.abs(Wt) / scale)[cdiff], 1e-9))
+
+
+@pytest.mark.parametrize("M,N,geometry", [(1024, 1024, "baseline"), (200, 96, "paper"), (129, 3584, "baseline"),
+                                          (64, 256, None)])
+def test_prepare_weight_vs_oracle(batq, M, N, geometry):
+    wb = synth.make_weight(M, N, 500 + M)
+    t = synth.make_transform(N, 10, geometry, clip=False) if geometry else None
+    tr = _mk_transform(batq, t) if t else None
+    w = batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(wb))
+    codes, scales = batq.batq_weight_export(w)
+    torch.cuda.synchronize()
+    gc, gs = O.unpack_codes(codes.cpu().numpy()), scales.cpu().numpy()
+    Wt = O.transform_weight(wb, t.left if t else None, t.right if t else None)
+    oc, os_ = O.mxfp4_quantize(Wt)
+    _weight_mismatch_ok(gc, gs, oc, os_, Wt)
+
+
+def test_prepare_weight_with_clip(batq):
+    M, N = 96, 512
+    wb = synth.make_weight(M, N, 77)
+    t = synth.make_transform(N, 11, "baseline", clip=False)
+    rng = np.random.default_rng(5)
+    lo = rng.uniform(0.7, 1.0, (M, N // 32)).astype(np.float32)
+    hi = rng.uniform(0.7, 1.0, (M, N // 32)).astype(np.float32)
+    w = batq.batq_prepare_weight(_mk_transform(batq, t), batq.bits_to_cuda_bf16(wb),
+                                 torch.from_numpy(lo).cuda(), torch.from_numpy(hi).cuda())
+    codes, scales = batq.batq_weight_export(w)
+    gc, gs = O.unpack_codes(codes.cpu().numpy()), scales.cpu().numpy()
+    Wt = O.block_clip(O.transform_weight(wb, t.left, t.right), lo, hi)
+    oc, os_ = O.mxfp4_quantize(Wt)
+    _weight_mismatch_ok(gc, gs, oc, os_, Wt)
+
+
+def test_singular_factor_is_reported(batq):
+    N = 64
+    t = synth.make_transform(N, 3, "baseline", clip=False)
+    t.left[0][:, 1] = t.left[0][:, 0]
+    tr = _mk_transform(batq, t)
+    with pytest.raises(batq.BatqError) as e:
+        batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(synth.make_weight(8, N, 1)))
+    assert e.value.status == 6
+
+
+# ---------------------------------------------------------------------------- GEMM
+def _gemm_case(batq, S, M, N, seed, xb=None, wb=None, out_dtype=torch.float32):
+    """Quantise X and W on the GPU (identity transform), run the GEMM on those
+    codes, and compare with the oracle GEMM fed the *same* codes and scales."""
+    xb = synth.make_activations(S, N, seed) if xb is None else xb
+    wb = synth.make_weight(M, N, seed) if wb is None else wb
+    x = batq.bits_to_cuda_bf16(xb)
+    w = batq.batq_prepare_weight(None, batq.bits_to_cuda_bf16(wb))
+    codes = torch.empty((S, N // 2), dtype=torch.uint8, device="cuda")
+    sf = torch.empty(batq.batq_sf_bytes(S, N, 1), dtype=torch.uint8, device="cuda")
+    batq.batq_quantize_act(None, x, codes, sf, 1)
+    ldy = M + (-M) % 8
+    y = torch.full((S + 1, ldy), float("nan"), dtype=out_dtype, device="cuda")
+    batq.batq_gemm_mxfp4(codes, sf, w, S, y)
+    assert batq.batq_last_device_status() == 0
+    torch.cuda.synchronize()
+    yh = y.float().cpu().numpy()
+    assert np.isnan(yh[S]).all() and np.isnan(yh[:S, M:]).all(), "wrote outside [S x M]"
+    xc = O.unpack_codes(codes.cpu().numpy())
+    xs = sf_mma_to_rowmajor(sf.cpu().numpy(), S, N // 32)
+    wc, ws = batq.batq_weight_export(w)
+    Y, Sabs = O.gemm_mxfp4(xc, xs, O.unpack_codes(wc.cpu().numpy()), ws.cpu().numpy())
+    return yh[:S, :M].astype(np.float64), Y, Sabs
+
+
+GEMM_SHAPES = [(128, 1024, 1024), (128, 128, 256), (1, 8, 32), (77, 200, 96), (300, 520, 3584), (16, 4096, 4096),
+               (260, 384, 512), (129, 257, 2048 + 32)]
+
+
+@pytest.mark.parametrize("S,M,N", GEMM_SHAPES)
+def test_gemm_vs_oracle_same_codes(batq, S, M, N):
+    got, Y, Sabs = _gemm_case(batq, S, M, N, 600 + S)
+    assert np.all(np.isfinite(got))
+    assert np.all(np.abs(got - Y) <= 1e-3 * Sabs + 1e-30)
+    # fp32 accumulation of exact products: in fact far tighter than the stated tolerance
+    assert np.max(np.abs(got - Y) / (Sabs + 1e-30)) < 1e-5
+
+
+def test_gemm_scale_layout_localising_case(batq):
+    """All codes = 4.0 and a distinct power-of-two scale per (row, block): any
+    mistake in the scale layout or in the operand/scale pairing shows up as a
+    wrong power of two in a specific output."""
+    S, M, N = 200, 300, 1024
+    k = N // 32
+    ex = ((np.arange(S)[:, None] * 7 + np.arange(k)[None, :] * 3) % 21) - 10
+    ew = ((np.arange(M)[:, None] * 5 + np.arange(k)[None, :] * 11) % 21) - 10
+    X = np.repeat(4.0 * np.exp2(ex), 32, axis=1).astype(np.float32)
+    W = np.repeat(4.0 * np.exp2(ew), 32, axis=1).astype(np.float32)
+    got, Y, Sabs = _gemm_case(batq, S, M, N, 0, synth.f32_to_bf16_bits(X), synth.f32_to_bf16_bits(W))
+    want = 32 * 16.0 * (np.exp2(ex.astype(np.float64)) @ np.exp2(ew.astype(np.float64)).T)
+    assert np.array_equal(Y, want)
+    assert np.all(np.abs(got - want) <= 1e-6 * want)
+
+
+def test_gemm_bf16_output_is_rounded_fp32(batq):
+    S, M, N = 130, 264, 1024
+    a, _, _ = _gemm_case(batq, S, M, N, 42, out_dtype=torch.float32)
+    b, _, _ = _gemm_case(batq, S, M, N, 42, out_dtype=torch.bfloat16)
+    want = torch.from_numpy(a.astype(np.float32)).bfloat16().float().numpy()
+    assert np.array_equal(b.astype(np.float32), want)
+
+
+# ---------------------------------------------------------------------------- whole layer
+@pytest.mark.parametrize("S,M,N,geometry", [(128, 1024, 1024, "baseline"), (128, 1024, 1024, "paper"),
+                                            (50, 136, 544, "baseline"), (4, 1024, 1024, "baseline")])
+def test_linear_w4a4_vs_oracle(batq, S, M, N, geometry):
+    xb = synth.make_activations(S, N, synth.BASE_SEED)
+    wb = synth.make_weight(M, N, synth.BASE_SEED)
+    t = synth.make_transform(N, synth.BASE_SEED, geometry)
+    tr = _mk_transform(batq, t)
+    w = batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(wb))
+    ws = batq.aligned_workspace(batq.batq_linear_workspace_bytes(w, S))
+    y = torch.empty((S, M), dtype=torch.float32, device="cuda")
+    batq.batq_linear_w4a4(tr, w, batq.bits_to_cuda_bf16(xb), y, ws)
+    assert batq.batq_last_device_status() == 0
+    got = y.cpu().numpy().astype(np.float64)
+    Y, Sabs, (oc, os_), _ = O.linear_w4a4(xb, wb, t.left, t.right, t.clip_lo, t.clip_hi)
+    # a few activation codes may legitimately differ (fp32 vs fp64 transform); each shifts an
+    # output by at most one grid step of one element, far inside 1e-3 * Sabs unless K is tiny
+    frac_bad = np.mean(np.abs(got - Y) > 1e-3 * Sabs + 1e-30)
+    assert frac_bad <= 1e-3
+    assert np.linalg.norm(got - Y) <= 1e-4 * np.linalg.norm(Sabs)
+    # and the quantised layer tracks the full-precision one
+    ref = O.bf16_bits_to_f64(xb) @ O.bf16_bits_to_f64(wb).T
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) < 0.5
+
+
+def test_linear_host_entry_point_matches_device_entry_point(batq):
+    S, M, N = 96, 256, 512
+    xb = synth.make_activations(S, N, 5)
+    t = synth.make_transform(N, 5, "baseline")
+    tr = _mk_transform(batq, t)
+    w = batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(synth.make_weight(M, N, 5)))
+    ws = batq.aligned_workspace(batq.batq_linear_workspace_bytes(w, S))
+    y = torch.empty((S, M), dtype=torch.float32, device="cuda")
+    batq.batq_linear_w4a4(tr, w, batq.bits_to_cuda_bf16(xb), y, ws)
+    xh = torch.from_numpy(xb.view(np.int16)).pin_memory()
+    yh = torch.empty((S, M), dtype=torch.float32).pin_memory()
+    xs = torch.empty((S, N), dtype=torch.bfloat16, device="cuda")
+    ys = torch.empty((S, M), dtype=torch.float32, device="cuda")
+    batq.batq_linear_w4a4_host(tr, w, xh, yh, xs, ys, ws)
+    assert torch.equal(yh, y.cpu())
+
+
+def test_empty_input_is_a_noop(batq):
+    tr = _mk_transform(batq, synth.make_transform(64, 1, "baseline"))
+    x = torch.empty((0, 64), dtype=torch.bfloat16, device="cuda")
+    batq.batq_quantize_act(tr, x, None, None, 0, ld=64, s=0, n=64)
