@@ -31,6 +31,10 @@ WORKLOADS = {
     "cfg1_llama8b_prefill": (2048, synth.LLAMA8B_PREFILL, 0.0, 0.01),
     "cfg3_qwen2vl7b_prefill": (8192, synth.QWEN2VL7B_PREFILL, 0.75, 0.005),
     "cfg0_single_layer": (128, [("lin", 1024, 1024)], 0.0, 0.01),
+    # single-kernel cases for profiler captures (m = 0: quantiser only, input larger than L2)
+    "profile_gemm_gate_up": (2048, [("gate_up", 4096, 28672)], 0.0, 0.01),
+    "profile_gemm_down": (2048, [("down", 14336, 4096)], 0.0, 0.01),
+    "profile_quant_32768x4096": (32768, [("quant", 4096, 0)], 0.0, 0.01),
 }
 FP4_OVER_BF16 = 4.0  # nominal dense peak ratio 9 / 2.25 PFLOP/s
 
@@ -179,13 +183,15 @@ def run_ours(args):
     projs = WORKLOADS[args.workload][1]
     for L in layers:
         L["tr"] = B.batq_transform_create(L["n"], L["t"].left, L["t"].right, L["t"].clip_lo, L["t"].clip_hi)
+        L["x"] = B.bits_to_cuda_bf16(L["x_bits"])
+        L["codes"] = torch.empty((S, L["n"] // 2), dtype=torch.uint8, device="cuda")
+        L["sf"] = torch.empty(B.batq_sf_bytes(S, L["n"], B.SF_MMA), dtype=torch.uint8, device="cuda")
+        if L["m"] == 0:
+            continue
         wdev = B.bits_to_cuda_bf16(synth.make_weight(L["m"], L["n"], L["w_seed"]))
         L["w"] = B.batq_prepare_weight(L["tr"], wdev)
         del wdev
-        L["x"] = B.bits_to_cuda_bf16(L["x_bits"])
         L["y"] = torch.empty((S, L["m"]), dtype=torch.bfloat16, device="cuda")
-        L["codes"] = torch.empty((S, L["n"] // 2), dtype=torch.uint8, device="cuda")
-        L["sf"] = torch.empty(B.batq_sf_bytes(S, L["n"], B.SF_MMA), dtype=torch.uint8, device="cuda")
         L["ws"] = B.aligned_workspace(B.batq_linear_workspace_bytes(L["w"], S))
         L["x_host"] = torch.from_numpy(L["x_bits"].view(np.int16)).pin_memory()
         L["y_host"] = torch.empty((S, L["m"]), dtype=torch.bfloat16).pin_memory()
@@ -216,7 +222,8 @@ def run_ours(args):
             B.batq_quantize_act(L["tr"], L["x"], L["codes"], L["sf"], B.SF_MMA)
             if m is not None:
                 m[i][1].record()
-            B.batq_gemm_mxfp4(L["codes"], L["sf"], L["w"], S, L["y"])
+            if L["m"]:
+                B.batq_gemm_mxfp4(L["codes"], L["sf"], L["w"], S, L["y"])
             if m is not None:
                 m[i][2].record()
 
@@ -243,6 +250,8 @@ def run_ours(args):
     # ---- end-to-end arm: host buffers in, host buffers out, through the C-ABI host entry point
     def step_host():
         for L in layers:
+            if L["m"] == 0:
+                continue
             B.batq_linear_w4a4_host(L["tr"], L["w"], L["x_host"], L["y_host"], L["x"], L["y"], L["ws"])
 
     e2e_steps = max(1, min(args.steps, 5))
@@ -265,7 +274,7 @@ def run_ours(args):
     value = flops_step * args.steps * world / (ms * 1e-3) / 1e12
     fp4_peak = peaks["bf16_tflops_sustained"] * FP4_OVER_BF16
     gemm_flops = [2.0 * S * L["n"] * L["m"] for L in layers]
-    gemm_achieved = sum(gemm_flops) / (g_ms.sum() * 1e-3) / 1e12
+    gemm_achieved = sum(gemm_flops) / (max(g_ms.sum(), 1e-9) * 1e-3) / 1e12
     q_bytes = [S * L["n"] * 2.53125 for L in layers]
     quant_gbs = sum(q_bytes) / (q_ms.sum() * 1e-3) / 1e9
     cpu_val, cpu_dt, cpu_desc = time_oracle(args.workload, synth.BASE_SEED, 256, 1024, 3, 1)
@@ -284,7 +293,7 @@ def run_ours(args):
                       "unit": "GB/s", "frac": quant_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"]},
         "kernels": [{"name": L["name"], "n": L["n"], "m": L["m"], "quant_us": float(q_ms[i] * 1e3),
                      "quant_gbs": q_bytes[i] / (q_ms[i] * 1e-3) / 1e9, "gemm_us": float(g_ms[i] * 1e3),
-                     "gemm_tflops": gemm_flops[i] / (g_ms[i] * 1e-3) / 1e12} for i, L in enumerate(layers)],
+                     "gemm_tflops": gemm_flops[i] / (max(g_ms[i], 1e-9) * 1e-3) / 1e12} for i, L in enumerate(layers)],
         "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
                          "sample": cpu_desc},
         "e2e": {"value": flops_step * e2e_steps * world / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
