@@ -153,6 +153,36 @@ batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w,
                                   void* y_stage_dev, void* workspace, size_t workspace_bytes,
                                   void* stream);
 
+/* The same layer for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a deployment convenience of this library.)  Some hosts of
+ * this code may not call cudaMalloc at the point where they run a layer: a serving
+ * process that gave the whole device to its own memory pool at start-up, or a
+ * latency-critical loop where an allocation's implicit device-wide synchronisation
+ * is unacceptable.  For them the quantised activations (codes + scale bytes, the
+ * scratch that batq_linear_w4a4 takes as `workspace`) live in one array that is
+ * part of the library image: BATQ_STATIC_WORKSPACE_BYTES bytes of device memory on
+ * every GPU that loads the library, held until the process exits.
+ *   - Arguments as batq_linear_w4a4 minus the workspace; x and y are still the
+ *     caller's.  The call itself performs no cudaMalloc / cudaFree and uses no
+ *     allocating library routine.
+ *   - BATQ_ERR_WORKSPACE if batq_linear_workspace_bytes(w, s) exceeds
+ *     batq_static_workspace_capacity() (the array minus alignment slack); with the
+ *     default size that admits e.g. s * n <= ~15.8 M elements (2048 x 4096 tokens
+ *     x channels uses 4.3 MB).
+ *   - The first call on each device looks up the array's device address (with that
+ *     device current) and caches it; make that first call before any stream
+ *     capture begins.
+ *   - All calls on a device share the one array and it keeps the previous call's
+ *     bytes.  Nothing in it has to start at zero (every byte the GEMM's result
+ *     depends on is rewritten by the quantiser of the same call), but two calls
+ *     whose kernels overlap on the GPU -- different streams, no ordering --
+ *     race on it: order them. */
+#define BATQ_STATIC_WORKSPACE_BYTES (8u << 20)
+size_t batq_static_workspace_capacity(void);
+batq_status batq_linear_w4a4_noalloc(const batq_transform* t, const batq_weight* w,
+                                     const void* x_bf16, int64_t s, int64_t ld, void* y,
+                                     int32_t y_dtype, int64_t ldy, void* stream);
+
 /* Synchronises `stream` and returns BATQ_ERR_TIMEOUT if any kernel of this
  * library gave up a bounded wait since the last query (the record is cleared),
  * BATQ_ERR_CUDA if the stream reports an error, else BATQ_OK. */

@@ -39,6 +39,8 @@ SIGNATURES = {
     "batq_linear_workspace_bytes": (_SZ, [_P, _I64]),
     "batq_linear_w4a4": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P, _SZ, _P]),
     "batq_linear_w4a4_host": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _P, _P, _P, _SZ, _P]),
+    "batq_static_workspace_capacity": (_SZ, []),
+    "batq_linear_w4a4_noalloc": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P]),
     "batq_last_device_status": (C.c_int, [_P]),
 }
 
@@ -212,6 +214,20 @@ def batq_linear_w4a4_host(t, w: Weight, x_host, y_host, x_stage, y_stage, worksp
     st = load().batq_linear_w4a4_host(t.handle if t else None, w.handle, _ptr(x_host), x_host.shape[0], _ptr(y_host),
                                       dt, _ptr(x_stage), _ptr(y_stage), _ptr(workspace), workspace.numel(), _stream())
     _check(st, "batq_linear_w4a4_host")
+
+
+def batq_static_workspace_capacity() -> int:
+    return load().batq_static_workspace_capacity()
+
+
+def batq_linear_w4a4_noalloc(t, w: Weight, x, y):
+    """The layer with the library's built-in scratch array instead of a caller
+    workspace: for callers that cannot allocate device memory.  Calls on one
+    device share that array, so keep them ordered on one stream."""
+    dt = F32 if y.dtype == torch.float32 else BF16
+    st = load().batq_linear_w4a4_noalloc(t.handle if t else None, w.handle, _ptr(x), x.shape[0], x.stride(0),
+                                         _ptr(y), dt, y.stride(0), _stream())
+    _check(st, "batq_linear_w4a4_noalloc")
 
 
 def batq_last_device_status() -> int:

@@ -43,6 +43,11 @@ struct batq_weight {
   CUtensorMap tmap_b128;
 };
 
+// Scratch for batq_linear_w4a4_noalloc: part of the library image, one copy per GPU.
+// In host code this name is only a handle for cudaGetSymbolAddress, never a pointer
+// a kernel may be given.
+static __device__ __align__(256) uint8_t g_static_workspace[BATQ_STATIC_WORKSPACE_BYTES];
+
 namespace {
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -55,6 +60,7 @@ struct DeviceInfo {
   bool ready = false;
   int sm_count = 0;
   int cc_major = 0;
+  uint8_t* static_ws = nullptr;  // device address of g_static_workspace on this device, 1024-aligned
 };
 DeviceInfo g_dev[kMaxDevices];
 std::mutex g_mutex;
@@ -524,6 +530,35 @@ batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w,
     return BATQ_ERR_CUDA;
   }
   return BATQ_OK;
+}
+
+size_t batq_static_workspace_capacity(void) { return BATQ_STATIC_WORKSPACE_BYTES - 1024; }
+
+batq_status batq_linear_w4a4_noalloc(const batq_transform* t, const batq_weight* w, const void* x_bf16, int64_t s,
+                                     int64_t ld, void* y, int32_t y_dtype, int64_t ldy, void* stream) {
+  if (w == nullptr) return BATQ_ERR_NULL;
+  if (s < 0) return BATQ_ERR_SHAPE;
+  if (batq_linear_workspace_bytes(w, s) > batq_static_workspace_capacity()) return BATQ_ERR_WORKSPACE;
+  int dev;
+  const DeviceInfo* info;
+  batq_status st = device_setup(&dev, &info);
+  if (st != BATQ_OK) return st;
+  uint8_t* ws = nullptr;
+  {
+    // Once per device, with that device current: resolve the array's device address.
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceInfo& d = g_dev[dev];
+    if (d.static_ws == nullptr) {
+      void* sym = nullptr;
+      if (cudaGetSymbolAddress(&sym, g_static_workspace) != cudaSuccess || sym == nullptr) {
+        cudaGetLastError();
+        return BATQ_ERR_CUDA;
+      }
+      d.static_ws = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(sym) + 1023) & ~uintptr_t(1023));
+    }
+    ws = d.static_ws;
+  }
+  return batq_linear_w4a4(t, w, x_bf16, s, ld, y, y_dtype, ldy, ws, batq_static_workspace_capacity(), stream);
 }
 
 batq_status batq_last_device_status(void* stream) {
