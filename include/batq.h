@@ -134,6 +134,14 @@ batq_status batq_weight_export(const batq_weight* w, void* codes_rowmajor, void*
 batq_status batq_gemm_mxfp4(const void* x_codes, const void* x_scales_mma, const batq_weight* w,
                             int64_t s, void* y, int32_t y_dtype, int64_t ldy, void* stream);
 
+/* Test / tuning hook: forces the GEMM's output-tile width to 128, 192 or 256 columns for all
+ * later calls in this process; any other value restores the automatic choice. */
+void batq_debug_force_tile_width(int32_t bn);
+/* Timing experiments only (results become meaningless): bit 0 = the GEMM's producer stops
+ * reloading shared-memory stages after the first fill, bit 1 = scale factors are copied to
+ * tensor memory only for the first stages.  Isolates load-bound from issue-bound behaviour. */
+void batq_debug_set_gemm_flags(int32_t flags);
+
 /* The whole layer, stages 1+2+3: quantise X into the workspace, then the GEMM.
  *   workspace  dev, at least batq_linear_workspace_bytes(w, s) bytes, 1024-byte
  *              aligned; overwritten by every call (calls sharing a workspace

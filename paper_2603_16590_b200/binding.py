@@ -36,6 +36,8 @@ SIGNATURES = {
     "batq_weight_destroy": (C.c_int, [_P]),
     "batq_weight_export": (C.c_int, [_P, _P, _P, _P]),
     "batq_gemm_mxfp4": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _I64, _P]),
+    "batq_debug_force_tile_width": (None, [_I32]),
+    "batq_debug_set_gemm_flags": (None, [_I32]),
     "batq_linear_workspace_bytes": (_SZ, [_P, _I64]),
     "batq_linear_w4a4": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P, _SZ, _P]),
     "batq_linear_w4a4_host": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _P, _P, _P, _SZ, _P]),
@@ -189,6 +191,14 @@ def batq_gemm_mxfp4(x_codes, x_scales_mma, w: Weight, s, y, ldy=None):
     st = load().batq_gemm_mxfp4(_ptr(x_codes), _ptr(x_scales_mma), w.handle, s, _ptr(y), dt,
                                 y.stride(0) if ldy is None else ldy, _stream())
     _check(st, "batq_gemm_mxfp4")
+
+
+def batq_debug_force_tile_width(bn: int):
+    load().batq_debug_force_tile_width(bn)
+
+
+def batq_debug_set_gemm_flags(flags: int):
+    load().batq_debug_set_gemm_flags(flags)
 
 
 def batq_linear_workspace_bytes(w: Weight, s) -> int:

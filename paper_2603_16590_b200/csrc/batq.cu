@@ -39,7 +39,8 @@ struct batq_weight {
   int32_t k, katoms;
   uint8_t* codes;   // [m x n/2]
   uint8_t* scales;  // BATQ_SF_MMA
-  CUtensorMap tmap_b256;
+  CUtensorMap tmap_b256;  // boxes of 256 / 192 / 128 weight rows x 128 bytes
+  CUtensorMap tmap_b192;
   CUtensorMap tmap_b128;
 };
 
@@ -95,6 +96,8 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(quantize_act_kernel<false, false, true>, kQaSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<256, false>, GemmCfg<256>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<256, true>, GemmCfg<256>::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_kernel<192, false>, GemmCfg<192>::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_kernel<192, true>, GemmCfg<192>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<128, false>, GemmCfg<128>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<128, true>, GemmCfg<128>::kSmemBytes);
     if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
@@ -206,17 +209,39 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
   return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
 }
 
-// Tile width: the wider tile halves shared-memory traffic per flop; the narrower one has two
-// accumulators (epilogue overlapped with the next tile) and finer wave granularity.
-int pick_bn(int64_t s, int64_t m, int sm_count) {
+// Tensor map over a row-major output [rows x cols], box = 128 bytes x 32 rows, 128-byte swizzle.
+batq_status make_y_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, bool bf16) {
+  const int esz = bf16 ? 2 : 4;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld * esz)};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / esz), 32};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = g_encode_tiled(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                                    const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? BATQ_OK : BATQ_ERR_CUDA;
+}
+
+// Tile width.  192 and 128 keep two accumulators in tensor memory (the epilogue of a tile
+// overlaps the main loop of the next); 256 has the highest flop per byte staged but a single
+// accumulator.  Pick by modelled time: waves x (main loop + exposed epilogue), with the main
+// loop proportional to the tile width.
+int g_force_bn = 0;  // test hook: 0 = automatic
+int g_gemm_debug_flags = 0;
+int pick_bn(int64_t s, int64_t m, int64_t n, int sm_count) {
+  if (g_force_bn == 128 || g_force_bn == 192 || g_force_bn == 256) return g_force_bn;
   const int64_t mt = (s + kBM - 1) / kBM;
-  auto waves_eff = [&](int bn) {
+  const double k_steps = static_cast<double>((n + 255) / 256);
+  auto cost = [&](int bn, double exposed_epilogue) {
     const int64_t tiles = mt * ((m + bn - 1) / bn);
     const int64_t waves = (tiles + sm_count - 1) / sm_count;
-    return static_cast<double>(tiles) / static_cast<double>(waves * sm_count);
+    return static_cast<double>(waves) * (k_steps * bn / 256.0 + exposed_epilogue * bn / 256.0);
   };
+  const double c256 = cost(256, 3.0), c192 = cost(192, 0.3), c128 = cost(128, 0.3) * 1.08;
   if (m <= 128) return 128;
-  return waves_eff(256) >= 0.92 * waves_eff(128) ? 256 : 128;
+  if (c192 <= c256 && c192 <= c128) return 192;
+  return c256 <= c128 ? 256 : 128;
 }
 
 batq_status launch_gemm(const void* x_codes, const void* x_sf, const batq_weight* w, int64_t s, void* y,
@@ -226,33 +251,35 @@ batq_status launch_gemm(const void* x_codes, const void* x_sf, const batq_weight
   batq_status st = device_setup(&dev, &info);
   if (st != BATQ_OK) return st;
   if (w->device != dev) return BATQ_ERR_CUDA;
-  CUtensorMap tmap_a;
+  const bool bf = y_dtype == BATQ_BF16;
+  CUtensorMap tmap_a, tmap_y;
+  std::memset(&tmap_y, 0, sizeof(tmap_y));
   st = make_codes_tmap(&tmap_a, x_codes, s, w->n / 2, kBM);
+  const int64_t m16 = w->m / (bf ? 8 : 4) * (bf ? 8 : 4);
+  if (st == BATQ_OK && m16 > 0) st = make_y_tmap(&tmap_y, y, s, m16, ldy, bf);
   if (st != BATQ_OK) return st;
-  const int bn = pick_bn(s, w->m, info->sm_count);
+  const int bn = pick_bn(s, w->m, w->n, info->sm_count);
   GemmParams p{};
   p.sfa = static_cast<const uint8_t*>(x_sf);
   p.sfb = w->scales;
-  p.y = y;
-  p.ldy = ldy;
   p.s = static_cast<int32_t>(s);
   p.m = static_cast<int32_t>(w->m);
-  p.k_bytes = static_cast<int32_t>(w->n / 2);
   p.katoms = w->katoms;
   p.k_steps = static_cast<int32_t>((w->n + 255) / 256);
   p.m_tiles = static_cast<int32_t>((s + kBM - 1) / kBM);
   p.n_tiles = static_cast<int32_t>((w->m + bn - 1) / bn);
-  p.sfa_row_tiles = p.m_tiles;
   p.sfb_row_tiles = static_cast<int32_t>((w->m + 127) / 128);
+  p.m16 = static_cast<int32_t>(m16);
+  p.y = y;
+  p.ldy = ldy;
+  p.debug_flags = g_gemm_debug_flags;
   const int grid = std::min(info->sm_count, p.m_tiles * p.n_tiles);
-  const bool bf = y_dtype == BATQ_BF16;
-  if (bn == 256) {
-    if (bf) gemm_mxfp4_kernel<256, true><<<grid, kGemmThreads, GemmCfg<256>::kSmemBytes, stream>>>(tmap_a, w->tmap_b256, p);
-    else gemm_mxfp4_kernel<256, false><<<grid, kGemmThreads, GemmCfg<256>::kSmemBytes, stream>>>(tmap_a, w->tmap_b256, p);
-  } else {
-    if (bf) gemm_mxfp4_kernel<128, true><<<grid, kGemmThreads, GemmCfg<128>::kSmemBytes, stream>>>(tmap_a, w->tmap_b128, p);
-    else gemm_mxfp4_kernel<128, false><<<grid, kGemmThreads, GemmCfg<128>::kSmemBytes, stream>>>(tmap_a, w->tmap_b128, p);
-  }
+#define BATQ_GEMM(BN, BF, TB) \
+  gemm_mxfp4_kernel<BN, BF><<<grid, kGemmThreads, GemmCfg<BN>::kSmemBytes, stream>>>(tmap_a, TB, tmap_y, p)
+  if (bn == 256) { if (bf) BATQ_GEMM(256, true, w->tmap_b256); else BATQ_GEMM(256, false, w->tmap_b256); }
+  else if (bn == 192) { if (bf) BATQ_GEMM(192, true, w->tmap_b192); else BATQ_GEMM(192, false, w->tmap_b192); }
+  else { if (bf) BATQ_GEMM(128, true, w->tmap_b128); else BATQ_GEMM(128, false, w->tmap_b128); }
+#undef BATQ_GEMM
   return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
 }
 
@@ -447,6 +474,7 @@ batq_status batq_prepare_weight(const batq_transform* t, const void* w_bf16, int
   cudaFree(d_fac);
   if (e != cudaSuccess) { cudaGetLastError(); delete w; return BATQ_ERR_CUDA; }
   st = make_codes_tmap(&w->tmap_b256, w->codes, m, n / 2, 256);
+  if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b192, w->codes, m, n / 2, 192);
   if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b128, w->codes, m, n / 2, 128);
   if (st != BATQ_OK) { delete w; return st; }
   *out = w;
@@ -531,6 +559,9 @@ batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w,
   }
   return BATQ_OK;
 }
+
+void batq_debug_force_tile_width(int32_t bn) { g_force_bn = bn; }
+void batq_debug_set_gemm_flags(int32_t flags) { g_gemm_debug_flags = flags; }
 
 size_t batq_static_workspace_capacity(void) { return BATQ_STATIC_WORKSPACE_BYTES - 1024; }
 

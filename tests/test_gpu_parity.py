@@ -236,6 +236,29 @@ def test_gemm_vs_oracle_same_codes(batq, S, M, N):
     assert np.max(np.abs(got - Y) / (Sabs + 1e-30)) < 1e-5
 
 
+@pytest.mark.parametrize("bn", [128, 192, 256])
+@pytest.mark.parametrize("S,M,N", [(300, 520, 3584), (129, 257, 2048 + 32), (260, 1000, 512)])
+def test_gemm_every_tile_width(batq, bn, S, M, N):
+    batq.batq_debug_force_tile_width(bn)
+    try:
+        got, Y, Sabs = _gemm_case(batq, S, M, N, 700 + S)
+        got16, _, _ = _gemm_case(batq, S, M, N, 700 + S, out_dtype=torch.bfloat16)
+    finally:
+        batq.batq_debug_force_tile_width(0)
+    assert np.max(np.abs(got - Y) / (Sabs + 1e-30)) < 1e-5
+    want16 = torch.from_numpy(got.astype(np.float32)).bfloat16().float().numpy()
+    assert np.array_equal(got16.astype(np.float32), want16)
+
+
+@pytest.mark.parametrize("bn", [128, 192, 256])
+def test_gemm_scale_layout_localising_case_every_tile_width(batq, bn):
+    batq.batq_debug_force_tile_width(bn)
+    try:
+        test_gemm_scale_layout_localising_case(batq)
+    finally:
+        batq.batq_debug_force_tile_width(0)
+
+
 def test_gemm_scale_layout_localising_case(batq):
     """All codes = 4.0 and a distinct power-of-two scale per (row, block): any
     mistake in the scale layout or in the operand/scale pairing shows up as a
