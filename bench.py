@@ -188,6 +188,7 @@ def run_ours(args):
     B.load()
     B.batq_debug_force_tile_width(args.tile_width)
     B.batq_debug_set_gemm_flags(args.gemm_debug_flags)
+    B.batq_debug_force_quantizer(args.quantizer)
     peaks = load_peaks()
 
     # weak scaling: every rank runs the same workload on its own seeded batch, no exchange step
@@ -326,6 +327,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg1_llama8b_prefill", choices=sorted(WORKLOADS))
     ap.add_argument("--gemm-debug-flags", type=int, default=0, help="timing experiments only; results invalid")
+    ap.add_argument("--quantizer", type=int, default=0, help="0 auto, 1 ALU kernel, 2 tensor-core kernel (tuning)")
     ap.add_argument("--tile-width", type=int, default=0, help="force the GEMM tile width (tuning); 0 = automatic")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

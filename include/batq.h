@@ -137,6 +137,10 @@ batq_status batq_gemm_mxfp4(const void* x_codes, const void* x_scales_mma, const
 /* Test / tuning hook: forces the GEMM's output-tile width to 128, 192 or 256 columns for all
  * later calls in this process; any other value restores the automatic choice. */
 void batq_debug_force_tile_width(int32_t bn);
+/* Test / tuning hook: which activation quantiser later calls use.  0 = automatic (tensor-core
+ * dense-block kernel for s >= 64 tokens, ALU Kronecker-form kernel below that and for the
+ * identity transform), 1 = always the ALU kernel, 2 = always the tensor-core kernel. */
+void batq_debug_force_quantizer(int32_t which);
 /* Timing experiments only (results become meaningless): bit 0 = the GEMM's producer stops
  * reloading shared-memory stages after the first fill, bit 1 = scale factors are copied to
  * tensor memory only for the first stages.  Isolates load-bound from issue-bound behaviour. */

@@ -38,6 +38,7 @@ SIGNATURES = {
     "batq_gemm_mxfp4": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _I64, _P]),
     "batq_debug_force_tile_width": (None, [_I32]),
     "batq_debug_set_gemm_flags": (None, [_I32]),
+    "batq_debug_force_quantizer": (None, [_I32]),
     "batq_linear_workspace_bytes": (_SZ, [_P, _I64]),
     "batq_linear_w4a4": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P, _SZ, _P]),
     "batq_linear_w4a4_host": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _P, _P, _P, _SZ, _P]),
@@ -195,6 +196,10 @@ def batq_gemm_mxfp4(x_codes, x_scales_mma, w: Weight, s, y, ldy=None):
 
 def batq_debug_force_tile_width(bn: int):
     load().batq_debug_force_tile_width(bn)
+
+
+def batq_debug_force_quantizer(which: int):
+    load().batq_debug_force_quantizer(which)
 
 
 def batq_debug_set_gemm_flags(flags: int):

@@ -15,6 +15,7 @@
 #include "gemm_mxfp4.cuh"
 #include "prepare_weight.cuh"
 #include "quantize_act.cuh"
+#include "quantize_act_tc.cuh"
 
 using namespace batq;
 
@@ -31,6 +32,7 @@ struct batq_transform {
   float* d_right;
   float* d_clip_lo;
   float* d_clip_hi;
+  uint8_t* d_pimg;                    // [k][3][2048]: dense P_j^T as three bf16 terms, tensor-core operand layout
 };
 
 struct batq_weight {
@@ -94,6 +96,10 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(quantize_act_kernel<true, true, true>, kQaSmemBytes);
     e = e ? e : set_smem(quantize_act_kernel<true, false, true>, kQaSmemBytes);
     e = e ? e : set_smem(quantize_act_kernel<false, false, true>, kQaSmemBytes);
+    e = e ? e : set_smem(quantize_act_tc_kernel<true, false>, kQtSmemBytes);
+    e = e ? e : set_smem(quantize_act_tc_kernel<false, false>, kQtSmemBytes);
+    e = e ? e : set_smem(quantize_act_tc_kernel<true, true>, kQtSmemBytes);
+    e = e ? e : set_smem(quantize_act_tc_kernel<false, true>, kQtSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<256, false>, GemmCfg<256>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<256, true>, GemmCfg<256>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<192, false>, GemmCfg<192>::kSmemBytes);
@@ -128,6 +134,59 @@ batq_status make_codes_tmap(CUtensorMap* map, const void* base, int64_t rows, in
                                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? BATQ_OK : BATQ_ERR_CUDA;
+}
+
+batq_status make_tmap_2d(CUtensorMap* map, CUtensorMapDataType dt, int esz, const void* base, int64_t cols,
+                         int64_t rows, int64_t ld_bytes, int box_cols, int box_rows, CUtensorMapSwizzle sw) {
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld_bytes)};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1, 1};
+  (void)esz;
+  const CUresult r = g_encode_tiled(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
+                                    CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? BATQ_OK : BATQ_ERR_CUDA;
+}
+
+// fp32 -> bf16 bits, round to nearest even (finite inputs).
+inline uint16_t bf16_rn(float f) {
+  uint32_t b;
+  std::memcpy(&b, &f, 4);
+  b += 0x7FFFu + ((b >> 16) & 1u);
+  return static_cast<uint16_t>(b >> 16);
+}
+inline float bf16_to_f32(uint16_t h) {
+  const uint32_t b = static_cast<uint32_t>(h) << 16;
+  float f;
+  std::memcpy(&f, &b, 4);
+  return f;
+}
+
+// Dense block matrices P_j = L_j (x) R_j (Eq. 2), P[(r,c),(r',c')] = L[r][r'] R[c][c'], rounded to
+// fp32 and split into three bf16 terms, laid out as the tensor-core B operand (rows = output
+// channel f, K = input channel e, no-swizzle K-major: 8 x 16-byte core matrices, K chunks 128
+// bytes apart, 8-row groups 512 bytes apart).
+void build_block_images(const batq_transform* t, std::vector<uint8_t>* out) {
+  out->assign(static_cast<size_t>(t->k) * kQtImageBytes, 0);
+  for (int j = 0; j < t->k; ++j) {
+    const float* L = t->left.data() + (t->left_stride ? static_cast<size_t>(j) * 16 : 0);
+    const float* R = t->right.data() + (t->right_stride ? static_cast<size_t>(j) * 64 : 0);
+    uint8_t* img = out->data() + static_cast<size_t>(j) * kQtImageBytes;
+    for (int e = 0; e < 32; ++e)
+      for (int f = 0; f < 32; ++f) {
+        const float pv = static_cast<float>(static_cast<double>(L[(e >> 3) * 4 + (f >> 3)]) *
+                                            static_cast<double>(R[(e & 7) * 8 + (f & 7)]));
+        const uint16_t hi = bf16_rn(pv);
+        const float r1 = pv - bf16_to_f32(hi);
+        const uint16_t mid = bf16_rn(r1);
+        const float r2 = r1 - bf16_to_f32(mid);
+        const uint16_t lo = bf16_rn(r2);
+        const size_t off = static_cast<size_t>(((f >> 3) * 4 + (e >> 3)) * 128 + (f & 7) * 16 + (e & 7) * 2);
+        const uint16_t terms[3] = {hi, mid, lo};
+        for (int term = 0; term < 3; ++term) std::memcpy(img + term * kQtTermBytes + off, &terms[term], 2);
+      }
+  }
 }
 
 // Gauss-Jordan inverse with partial pivoting of a small dense matrix, fp64.
@@ -166,6 +225,48 @@ batq_status check_x(const void* x, int64_t s, int64_t n, int64_t ld) {
   return BATQ_OK;
 }
 
+int g_force_quantizer = 0;  // tuning hook: 0 = automatic, 1 = ALU (Kronecker form), 2 = tensor cores (dense form)
+
+// Tensor-core version: 128-token x 4-block units.
+batq_status launch_quantize_tc(const batq_transform* t, const void* x, int64_t s, int64_t n, int64_t ld, void* codes,
+                               void* scales, int32_t layout, float* debug_out, cudaStream_t stream, int sm_count) {
+  QuantTcParams p{};
+  p.s = s;
+  p.n = static_cast<int32_t>(n);
+  p.k = static_cast<int32_t>(n / 32);
+  p.n_strips = (p.k + kQtGroups - 1) / kQtGroups;
+  p.n_row_tiles = (s + kQtRows - 1) / kQtRows;
+  p.n_units = p.n_strips * p.n_row_tiles;
+  p.pimg = t->d_pimg;
+  p.clip_lo = t->d_clip_lo;
+  p.clip_hi = t->d_clip_hi;
+  p.scales = static_cast<uint8_t*>(scales);
+  p.sf_layout = layout;
+  p.sf_katoms = katoms_of(p.k);
+  p.debug_out = debug_out;
+  CUtensorMap tmap_x, tmap_codes;
+  std::memset(&tmap_codes, 0, sizeof(tmap_codes));
+  batq_status st = make_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x, n, s, ld * 2, 64, kQtRows,
+                                CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st == BATQ_OK && debug_out == nullptr)
+    st = make_tmap_2d(&tmap_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, n / 2, s, n / 2, 16, 32,
+                      CU_TENSOR_MAP_SWIZZLE_NONE);
+  if (st != BATQ_OK) return st;
+  if (debug_out == nullptr && layout == BATQ_SF_MMA && p.sf_katoms > p.n_strips) {
+    // an odd number of 4-block atoms: keep the padding atom finite
+    if (cudaMemsetAsync(scales, 0, batq_sf_bytes(s, n, BATQ_SF_MMA), stream) != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+  }
+  const int grid = static_cast<int>(std::min<int64_t>(sm_count, p.n_units));
+  const bool cl = t->has_clip, dbg = debug_out != nullptr;
+#define BATQ_QT(CL, DB) quantize_act_tc_kernel<CL, DB><<<grid, kQtThreads, kQtSmemBytes, stream>>>(tmap_x, tmap_codes, p)
+  if (cl && !dbg) BATQ_QT(true, false);
+  else if (!cl && !dbg) BATQ_QT(false, false);
+  else if (cl && dbg) BATQ_QT(true, true);
+  else BATQ_QT(false, true);
+#undef BATQ_QT
+  return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
+}
+
 batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, int64_t n, int64_t ld, void* codes,
                             void* scales, int32_t layout, float* debug_out, cudaStream_t stream) {
   int dev;
@@ -173,6 +274,10 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
   batq_status st = device_setup(&dev, &info);
   if (st != BATQ_OK) return st;
   if (t != nullptr && t->device != dev) return BATQ_ERR_CUDA;
+  // The dense-block tensor-core kernel works on 128-token tiles; tiny batches (decode) and the
+  // identity transform stay on the ALU kernel.
+  const bool use_tc = t != nullptr && (g_force_quantizer == 2 || (g_force_quantizer == 0 && s >= 64));
+  if (use_tc) return launch_quantize_tc(t, x, s, n, ld, codes, scales, layout, debug_out, stream, info->sm_count);
   QuantActParams p{};
   p.x = static_cast<const uint16_t*>(x);
   p.ld = ld;
@@ -339,7 +444,12 @@ batq_status batq_transform_create(batq_transform** out, int32_t n, int32_t gr, i
   t->left.assign(left, left + nl);
   t->right.assign(right, right + nr);
   t->d_left = t->d_right = t->d_clip_lo = t->d_clip_hi = nullptr;
+  t->d_pimg = nullptr;
+  std::vector<uint8_t> pimg;
+  build_block_images(t, &pimg);
   cudaError_t e = cudaMalloc(&t->d_left, nl * sizeof(float));
+  e = e ? e : cudaMalloc(&t->d_pimg, pimg.size());
+  e = e ? e : cudaMemcpy(t->d_pimg, pimg.data(), pimg.size(), cudaMemcpyHostToDevice);
   e = e ? e : cudaMalloc(&t->d_right, nr * sizeof(float));
   e = e ? e : cudaMemcpy(t->d_left, left, nl * sizeof(float), cudaMemcpyHostToDevice);
   e = e ? e : cudaMemcpy(t->d_right, right, nr * sizeof(float), cudaMemcpyHostToDevice);
@@ -364,6 +474,7 @@ batq_status batq_transform_destroy(batq_transform* t) {
   cudaFree(t->d_right);
   cudaFree(t->d_clip_lo);
   cudaFree(t->d_clip_hi);
+  cudaFree(t->d_pimg);
   delete t;
   return BATQ_OK;
 }
@@ -561,6 +672,7 @@ batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w,
 }
 
 void batq_debug_force_tile_width(int32_t bn) { g_force_bn = bn; }
+void batq_debug_force_quantizer(int32_t which) { g_force_quantizer = which; }
 void batq_debug_set_gemm_flags(int32_t flags) { g_gemm_debug_flags = flags; }
 
 size_t batq_static_workspace_capacity(void) { return BATQ_STATIC_WORKSPACE_BYTES - 1024; }
