@@ -134,6 +134,20 @@ batq_status batq_weight_export(const batq_weight* w, void* codes_rowmajor, void*
 batq_status batq_gemm_mxfp4(const void* x_codes, const void* x_scales_mma, const batq_weight* w,
                             int64_t s, void* y, int32_t y_dtype, int64_t ldy, void* stream);
 
+/* Stage 3 alone for a handful of tokens (decode), s <= 64: the same contraction as
+ * batq_gemm_mxfp4, organised for the case where streaming the weights from HBM once is the
+ * whole cost.  The weights are the 128-row tensor-core operand and the tokens the narrow one;
+ * the grid is (128-row weight tiles) x (K splits), and the partial sums of the splits meet in
+ * `scratch` (added in split order, so results are deterministic).
+ *   scratch        dev, batq_gemm_small_s_scratch_bytes(w, s) bytes, 1024-byte aligned; contents
+ *                  need not be initialised; calls sharing it must be ordered on one stream.
+ *   y              dev [s x m], fp32 or bf16, row stride ldy.
+ * Errors as batq_gemm_mxfp4, plus SHAPE for s > 64 and WORKSPACE for a short scratch. */
+size_t batq_gemm_small_s_scratch_bytes(const batq_weight* w, int64_t s);
+batq_status batq_gemm_mxfp4_small_s(const void* x_codes, const void* x_scales_mma, const batq_weight* w,
+                                    int64_t s, void* y, int32_t y_dtype, int64_t ldy, void* scratch,
+                                    size_t scratch_bytes, void* stream);
+
 /* Test / tuning hook: forces the GEMM's output-tile width to 128, 192 or 256 columns for all
  * later calls in this process; any other value restores the automatic choice. */
 void batq_debug_force_tile_width(int32_t bn);
@@ -141,12 +155,16 @@ void batq_debug_force_tile_width(int32_t bn);
  * dense-block kernel for s >= 64 tokens, ALU Kronecker-form kernel below that and for the
  * identity transform), 1 = always the ALU kernel, 2 = always the tensor-core kernel. */
 void batq_debug_force_quantizer(int32_t which);
+/* Test / tuning hook: number of K splits of the small-s GEMM (clamped to the number of
+ * 256-element K steps and to 32); 0 restores the automatic choice.  Scratch sizes follow it. */
+void batq_debug_force_small_s_splits(int32_t splits);
 /* Timing experiments only (results become meaningless): bit 0 = the GEMM's producer stops
  * reloading shared-memory stages after the first fill, bit 1 = scale factors are copied to
  * tensor memory only for the first stages.  Isolates load-bound from issue-bound behaviour. */
 void batq_debug_set_gemm_flags(int32_t flags);
 
-/* The whole layer, stages 1+2+3: quantise X into the workspace, then the GEMM.
+/* The whole layer, stages 1+2+3: quantise X into the workspace, then the GEMM.  Up to 64
+ * tokens take the small-s GEMM, launched so that its weight stream overlaps the quantiser.
  *   workspace  dev, at least batq_linear_workspace_bytes(w, s) bytes, 1024-byte
  *              aligned; overwritten by every call (calls sharing a workspace
  *              must be ordered on one stream). */

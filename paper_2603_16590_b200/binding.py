@@ -36,6 +36,9 @@ SIGNATURES = {
     "batq_weight_destroy": (C.c_int, [_P]),
     "batq_weight_export": (C.c_int, [_P, _P, _P, _P]),
     "batq_gemm_mxfp4": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _I64, _P]),
+    "batq_gemm_small_s_scratch_bytes": (_SZ, [_P, _I64]),
+    "batq_gemm_mxfp4_small_s": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _I64, _P, _SZ, _P]),
+    "batq_debug_force_small_s_splits": (None, [_I32]),
     "batq_debug_force_tile_width": (None, [_I32]),
     "batq_debug_set_gemm_flags": (None, [_I32]),
     "batq_debug_force_quantizer": (None, [_I32]),
@@ -192,6 +195,21 @@ def batq_gemm_mxfp4(x_codes, x_scales_mma, w: Weight, s, y, ldy=None):
     st = load().batq_gemm_mxfp4(_ptr(x_codes), _ptr(x_scales_mma), w.handle, s, _ptr(y), dt,
                                 y.stride(0) if ldy is None else ldy, _stream())
     _check(st, "batq_gemm_mxfp4")
+
+
+def batq_gemm_small_s_scratch_bytes(w: Weight, s) -> int:
+    return load().batq_gemm_small_s_scratch_bytes(w.handle, s)
+
+
+def batq_gemm_mxfp4_small_s(x_codes, x_scales_mma, w: Weight, s, y, scratch, ldy=None):
+    dt = F32 if y.dtype == torch.float32 else BF16
+    st = load().batq_gemm_mxfp4_small_s(_ptr(x_codes), _ptr(x_scales_mma), w.handle, s, _ptr(y), dt,
+                                        y.stride(0) if ldy is None else ldy, _ptr(scratch), scratch.numel(), _stream())
+    _check(st, "batq_gemm_mxfp4_small_s")
+
+
+def batq_debug_force_small_s_splits(splits: int):
+    load().batq_debug_force_small_s_splits(splits)
 
 
 def batq_debug_force_tile_width(bn: int):

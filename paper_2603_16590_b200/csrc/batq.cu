@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "gemm_mxfp4.cuh"
+#include "gemm_small_s.cuh"
 #include "prepare_weight.cuh"
 #include "quantize_act.cuh"
 #include "quantize_act_tc.cuh"
@@ -39,6 +40,7 @@ struct batq_weight {
   int device;
   int64_t m, n;
   int32_t k, katoms;
+  int32_t sm_count;  // of the device the weight lives on (sizes the small-s split-K scratch)
   uint8_t* codes;   // [m x n/2]
   uint8_t* scales;  // BATQ_SF_MMA
   CUtensorMap tmap_b256;  // boxes of 256 / 192 / 128 weight rows x 128 bytes
@@ -106,6 +108,12 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(gemm_mxfp4_kernel<192, true>, GemmCfg<192>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<128, false>, GemmCfg<128>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<128, true>, GemmCfg<128>::kSmemBytes);
+    e = e ? e : set_smem(gemm_small_s_kernel<16, false>, SmallCfg<16>::kSmemBytes);
+    e = e ? e : set_smem(gemm_small_s_kernel<16, true>, SmallCfg<16>::kSmemBytes);
+    e = e ? e : set_smem(gemm_small_s_kernel<32, false>, SmallCfg<32>::kSmemBytes);
+    e = e ? e : set_smem(gemm_small_s_kernel<32, true>, SmallCfg<32>::kSmemBytes);
+    e = e ? e : set_smem(gemm_small_s_kernel<64, false>, SmallCfg<64>::kSmemBytes);
+    e = e ? e : set_smem(gemm_small_s_kernel<64, true>, SmallCfg<64>::kSmemBytes);
     if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
     if (g_encode_tiled == nullptr) {
       void* fn = nullptr;
@@ -225,6 +233,7 @@ batq_status check_x(const void* x, int64_t s, int64_t n, int64_t ld) {
   return BATQ_OK;
 }
 
+constexpr int64_t kSmallSMax = 64;  // token counts up to this take the swapped-operand split-K GEMM
 int g_force_quantizer = 0;  // tuning hook: 0 = automatic, 1 = ALU (Kronecker form), 2 = tensor cores (dense form)
 
 // Tensor-core version: 128-token x 4-block units.
@@ -268,7 +277,8 @@ batq_status launch_quantize_tc(const batq_transform* t, const void* x, int64_t s
 }
 
 batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, int64_t n, int64_t ld, void* codes,
-                            void* scales, int32_t layout, float* debug_out, cudaStream_t stream) {
+                            void* scales, int32_t layout, float* debug_out, cudaStream_t stream,
+                            uint32_t* zero_words = nullptr, int32_t n_zero_words = 0) {
   int dev;
   const DeviceInfo* info;
   batq_status st = device_setup(&dev, &info);
@@ -276,7 +286,8 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
   if (t != nullptr && t->device != dev) return BATQ_ERR_CUDA;
   // The dense-block tensor-core kernel works on 128-token tiles; tiny batches (decode) and the
   // identity transform stay on the ALU kernel.
-  const bool use_tc = t != nullptr && (g_force_quantizer == 2 || (g_force_quantizer == 0 && s >= 64));
+  const bool use_tc = n_zero_words == 0 && t != nullptr &&
+                      (g_force_quantizer == 2 || (g_force_quantizer == 0 && s > kSmallSMax));
   if (use_tc) return launch_quantize_tc(t, x, s, n, ld, codes, scales, layout, debug_out, stream, info->sm_count);
   QuantActParams p{};
   p.x = static_cast<const uint16_t*>(x);
@@ -301,6 +312,8 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
   p.sf_layout = layout;
   p.sf_katoms = katoms_of(p.k);
   p.debug_out = debug_out;
+  p.zero_words = zero_words;
+  p.n_zero_words = n_zero_words;
   const int grid = static_cast<int>(std::min<int64_t>(info->sm_count, p.n_units));
   const bool xf = t != nullptr, cl = t != nullptr && t->has_clip, dbg = debug_out != nullptr;
 #define BATQ_QA(XF, CL, DB) quantize_act_kernel<XF, CL, DB><<<grid, kQaThreads, kQaSmemBytes, stream>>>(p)
@@ -386,6 +399,100 @@ batq_status launch_gemm(const void* x_codes, const void* x_sf, const batq_weight
   else { if (bf) BATQ_GEMM(128, true, w->tmap_b128); else BATQ_GEMM(128, false, w->tmap_b128); }
 #undef BATQ_GEMM
   return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
+}
+
+// ---- small-s (decode) GEMM: split choice, scratch layout, launch -------------------------------
+int g_force_splits = 0;  // tuning hook: 0 = automatic
+constexpr int kMaxSplits = 32;
+
+inline int small_ntok(int64_t s) { return s <= 16 ? 16 : (s <= 32 ? 32 : 64); }
+
+// Number of K splits: the grid is (row tiles) x (splits) CTAs, two resident per SM.  Modelled
+// time = waves x (K-steps per CTA + fixed cost) + a reduction term that grows with the splits.
+int pick_splits(int64_t m, int64_t n, int sm_count) {
+  const int k_steps = static_cast<int>((n + 255) / 256);
+  if (g_force_splits > 0) return std::min(std::min(g_force_splits, k_steps), kMaxSplits);
+  const int64_t tiles = (m + 127) / 128;
+  const int64_t slots = 2 * static_cast<int64_t>(sm_count > 0 ? sm_count : 148);
+  int best = 1;
+  double best_cost = 1e30;
+  for (int sp = 1; sp <= std::min(k_steps, kMaxSplits); ++sp) {
+    const int64_t waves = (tiles * sp + slots - 1) / slots;
+    const double cost = static_cast<double>(waves) * ((k_steps + sp - 1) / sp + 3.0) + 0.15 * sp;
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = sp; }
+  }
+  return best;
+}
+
+// Scratch of the small-s GEMM: split-K partial tiles, then one ticket word per row tile.
+struct SmallScratch {
+  size_t partial_bytes, ticket_bytes;
+  int splits, ntok;
+  int64_t tiles;
+  size_t total() const { return partial_bytes + ticket_bytes; }
+};
+SmallScratch small_scratch(const batq_weight* w, int64_t s) {
+  SmallScratch sc{};
+  sc.ntok = small_ntok(s);
+  sc.splits = pick_splits(w->m, w->n, w->sm_count);
+  sc.tiles = (w->m + 127) / 128;
+  sc.partial_bytes = sc.splits > 1 ? round_up(static_cast<size_t>(sc.tiles) * sc.splits * sc.ntok * 128 * 4, 1024) : 0;
+  sc.ticket_bytes = round_up(static_cast<size_t>(sc.tiles) * 4, 1024);
+  return sc;
+}
+
+template <int NTOK, bool BF>
+cudaError_t launch_small_kernel(dim3 grid, cudaStream_t stream, bool dependent, const CUtensorMap& tw,
+                                const CUtensorMap& tx, const SmallParams& p) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kSmallThreads);
+  cfg.dynamicSmemBytes = SmallCfg<NTOK>::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = dependent ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, gemm_small_s_kernel<NTOK, BF>, tw, tx, p);
+}
+
+// `dependent`: the kernel directly before this one on the stream is the activation quantiser
+// (which releases its dependents early); the weight stream then starts while it still runs.
+batq_status launch_gemm_small(const void* x_codes, const void* x_sf, const batq_weight* w, int64_t s, void* y,
+                              int32_t y_dtype, int64_t ldy, uint8_t* scratch, const SmallScratch& sc,
+                              cudaStream_t stream, bool dependent) {
+  int dev;
+  const DeviceInfo* info;
+  batq_status st = device_setup(&dev, &info);
+  if (st != BATQ_OK) return st;
+  if (w->device != dev) return BATQ_ERR_CUDA;
+  CUtensorMap tmap_x;
+  st = make_codes_tmap(&tmap_x, x_codes, s, w->n / 2, sc.ntok);
+  if (st != BATQ_OK) return st;
+  SmallParams p{};
+  p.sfx = static_cast<const uint8_t*>(x_sf);
+  p.sfw = w->scales;
+  p.s = static_cast<int32_t>(s);
+  p.m = static_cast<int32_t>(w->m);
+  p.katoms = w->katoms;
+  p.k_steps = static_cast<int32_t>((w->n + 255) / 256);
+  p.splits = sc.splits;
+  p.y = y;
+  p.ldy = ldy;
+  p.partial = reinterpret_cast<float*>(scratch);
+  p.tickets = reinterpret_cast<uint32_t*>(scratch + sc.partial_bytes);
+  const dim3 grid(static_cast<unsigned>(sc.tiles), static_cast<unsigned>(sc.splits));
+  const bool bf = y_dtype == BATQ_BF16;
+  cudaError_t e;
+#define BATQ_SMALL(NT) (bf ? launch_small_kernel<NT, true>(grid, stream, dependent, w->tmap_b128, tmap_x, p) \
+                           : launch_small_kernel<NT, false>(grid, stream, dependent, w->tmap_b128, tmap_x, p))
+  if (sc.ntok == 16) e = BATQ_SMALL(16);
+  else if (sc.ntok == 32) e = BATQ_SMALL(32);
+  else e = BATQ_SMALL(64);
+#undef BATQ_SMALL
+  if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+  return BATQ_OK;
 }
 
 batq_status check_y(const void* y, int32_t y_dtype, int64_t ldy, int64_t m) {
@@ -528,7 +635,8 @@ batq_status batq_prepare_weight(const batq_transform* t, const void* w_bf16, int
   if (!aligned(weight_buf, 1024)) return BATQ_ERR_ALIGN;
   if (t != nullptr && t->n != n) return BATQ_ERR_SHAPE;
   int dev;
-  st = device_setup(&dev, nullptr);
+  const DeviceInfo* dinfo;
+  st = device_setup(&dev, &dinfo);
   if (st != BATQ_OK) return st;
   if (t != nullptr && t->device != dev) return BATQ_ERR_CUDA;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
@@ -566,6 +674,7 @@ batq_status batq_prepare_weight(const batq_transform* t, const void* w_bf16, int
   if (w == nullptr) { cudaFree(d_fac); return BATQ_ERR_CUDA; }
   w->device = dev;
   w->m = m; w->n = n; w->k = k; w->katoms = katoms_of(k);
+  w->sm_count = dinfo->sm_count;
   w->codes = static_cast<uint8_t*>(weight_buf);
   w->scales = w->codes + round_up(static_cast<size_t>(m * (n / 2)), 1024);
 
@@ -623,9 +732,33 @@ batq_status batq_gemm_mxfp4(const void* x_codes, const void* x_scales_mma, const
   return launch_gemm(x_codes, x_scales_mma, w, s, y, y_dtype, ldy, static_cast<cudaStream_t>(stream));
 }
 
+size_t batq_gemm_small_s_scratch_bytes(const batq_weight* w, int64_t s) {
+  if (w == nullptr || s <= 0 || s > kSmallSMax) return 0;
+  return small_scratch(w, s).total();
+}
+
+batq_status batq_gemm_mxfp4_small_s(const void* x_codes, const void* x_scales_mma, const batq_weight* w, int64_t s,
+                                    void* y, int32_t y_dtype, int64_t ldy, void* scratch, size_t scratch_bytes,
+                                    void* stream) {
+  if (w == nullptr) return BATQ_ERR_NULL;
+  if (s < 0 || s > kSmallSMax) return BATQ_ERR_SHAPE;
+  if (s == 0) return BATQ_OK;
+  if (x_codes == nullptr || x_scales_mma == nullptr || y == nullptr || scratch == nullptr) return BATQ_ERR_NULL;
+  if (!aligned(x_codes, 16) || !aligned(x_scales_mma, 16) || !aligned(scratch, 1024)) return BATQ_ERR_ALIGN;
+  batq_status st = check_y(y, y_dtype, ldy, w->m);
+  if (st != BATQ_OK) return st;
+  const SmallScratch sc = small_scratch(w, s);
+  if (scratch_bytes < sc.total()) return BATQ_ERR_WORKSPACE;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  uint8_t* sp = static_cast<uint8_t*>(scratch);
+  if (cudaMemsetAsync(sp + sc.partial_bytes, 0, sc.ticket_bytes, cs) != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+  return launch_gemm_small(x_codes, x_scales_mma, w, s, y, y_dtype, ldy, sp, sc, cs, false);
+}
+
 size_t batq_linear_workspace_bytes(const batq_weight* w, int64_t s) {
   if (w == nullptr || s < 0) return 0;
-  return round_up(static_cast<size_t>(s * (w->n / 2)), 1024) + batq_sf_bytes(s, w->n, BATQ_SF_MMA);
+  const size_t q = round_up(static_cast<size_t>(s * (w->n / 2)), 1024) + round_up(batq_sf_bytes(s, w->n, BATQ_SF_MMA), 1024);
+  return q + (s > 0 && s <= kSmallSMax ? small_scratch(w, s).total() : 0);
 }
 
 batq_status batq_linear_w4a4(const batq_transform* t, const batq_weight* w, const void* x_bf16, int64_t s, int64_t ld,
@@ -644,6 +777,16 @@ batq_status batq_linear_w4a4(const batq_transform* t, const batq_weight* w, cons
   uint8_t* codes = static_cast<uint8_t*>(workspace);
   uint8_t* sf = codes + round_up(static_cast<size_t>(s * (w->n / 2)), 1024);
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (s <= kSmallSMax) {
+    // A handful of tokens: the quantiser also clears the split-K tickets, and the GEMM is launched
+    // as its programmatic dependent so that the weight stream starts while it still runs.
+    uint8_t* scratch = sf + round_up(batq_sf_bytes(s, w->n, BATQ_SF_MMA), 1024);
+    const SmallScratch sc = small_scratch(w, s);
+    st = launch_quantize(t, x_bf16, s, w->n, ld, codes, sf, BATQ_SF_MMA, nullptr, cs,
+                         reinterpret_cast<uint32_t*>(scratch + sc.partial_bytes), static_cast<int32_t>(sc.tiles));
+    if (st != BATQ_OK) return st;
+    return launch_gemm_small(codes, sf, w, s, y, y_dtype, ldy, scratch, sc, cs, true);
+  }
   st = launch_quantize(t, x_bf16, s, w->n, ld, codes, sf, BATQ_SF_MMA, nullptr, cs);
   if (st != BATQ_OK) return st;
   return launch_gemm(codes, sf, w, s, y, y_dtype, ldy, cs);
@@ -674,6 +817,7 @@ batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w,
 void batq_debug_force_tile_width(int32_t bn) { g_force_bn = bn; }
 void batq_debug_force_quantizer(int32_t which) { g_force_quantizer = which; }
 void batq_debug_set_gemm_flags(int32_t flags) { g_gemm_debug_flags = flags; }
+void batq_debug_force_small_s_splits(int32_t splits) { g_force_splits = splits; }
 
 size_t batq_static_workspace_capacity(void) { return BATQ_STATIC_WORKSPACE_BYTES - 1024; }
 

@@ -44,6 +44,8 @@ struct QuantActParams {
   int32_t sf_layout;     // BATQ_SF_ROWMAJOR / BATQ_SF_MMA
   int32_t sf_katoms;     // KA = 2*ceil(k/8), atoms per 128-row tile
   float* debug_out;      // [s x n] fp32 when the kernel is built with DEBUG_OUT
+  uint32_t* zero_words;  // optional: n_zero_words 32-bit words set to zero (tickets of the kernel that follows)
+  int32_t n_zero_words;
 };
 
 // Two floats -> one byte holding two E2M1 codes (hi in bits 4-7, lo in bits 0-3),
@@ -75,6 +77,11 @@ __global__ void __launch_bounds__(kQaThreads, 1) quantize_act_kernel(const Quant
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
   const int lane = tid & 31;
+  // A kernel launched as a programmatic dependent of this one may start its own prologue now;
+  // it still waits for this grid to finish before it reads anything written here.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (p.n_zero_words > 0 && blockIdx.x == 0)
+    for (int i = tid; i < p.n_zero_words; i += kQaThreads) p.zero_words[i] = 0u;
   // 128-byte aligned base of the ring
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(qa_smem) + 127) & ~uintptr_t(127));
 

@@ -298,9 +298,79 @@ def test_gemm_bf16_output_is_rounded_fp32(batq):
     assert np.array_equal(b.astype(np.float32), want)
 
 
+# ---------------------------------------------------------------------------- small-s (decode) GEMM
+def _small_case(batq, S, M, N, seed, out_dtype=torch.float32, splits=0):
+    """Quantise X and W on the GPU (identity transform), run the small-s GEMM on those codes and
+    compare with the oracle GEMM fed the same codes and scales."""
+    xb = synth.make_activations(S, N, seed)
+    wb = synth.make_weight(M, N, seed)
+    w = batq.batq_prepare_weight(None, batq.bits_to_cuda_bf16(wb))
+    codes = torch.empty((S, N // 2), dtype=torch.uint8, device="cuda")
+    sf = torch.full((batq.batq_sf_bytes(S, N, 1),), 0xFF, dtype=torch.uint8, device="cuda")  # NaN scales in the padding
+    batq.batq_quantize_act(None, batq.bits_to_cuda_bf16(xb), codes, sf, 1)
+    batq.batq_debug_force_small_s_splits(splits)
+    try:
+        scratch = batq.aligned_workspace(batq.batq_gemm_small_s_scratch_bytes(w, S))
+        scratch.fill_(0xA5)
+        ldy = M + (-M) % 8
+        ys = []
+        for _ in range(2):   # twice: the tickets must be back at zero after a call
+            y = torch.full((S + 1, ldy), float("nan"), dtype=out_dtype, device="cuda")
+            batq.batq_gemm_mxfp4_small_s(codes, sf, w, S, y, scratch)
+            ys.append(y)
+        assert batq.batq_last_device_status() == 0
+    finally:
+        batq.batq_debug_force_small_s_splits(0)
+    torch.cuda.synchronize()
+    assert torch.equal(ys[0][:S, :M], ys[1][:S, :M]), "not deterministic"
+    yh = ys[0].float().cpu().numpy()
+    assert np.isnan(yh[S]).all() and np.isnan(yh[:S, M:]).all(), "wrote outside [S x M]"
+    xc = O.unpack_codes(codes.cpu().numpy())
+    xs = sf_mma_to_rowmajor(sf.cpu().numpy(), S, N // 32)
+    wc, ws = batq.batq_weight_export(w)
+    Y, Sabs = O.gemm_mxfp4(xc, xs, O.unpack_codes(wc.cpu().numpy()), ws.cpu().numpy())
+    return yh[:S, :M].astype(np.float64), Y, Sabs
+
+
+SMALL_SHAPES = [(1, 8, 32), (1, 1024, 1024), (4, 300, 544), (16, 4096, 4096), (17, 257, 2048 + 32), (32, 520, 3584),
+                (33, 128, 256), (64, 1000, 1024)]
+
+
+@pytest.mark.parametrize("S,M,N", SMALL_SHAPES)
+@pytest.mark.parametrize("splits", [0, 1, 3])
+def test_gemm_small_s_vs_oracle_same_codes(batq, S, M, N, splits):
+    got, Y, Sabs = _small_case(batq, S, M, N, 800 + S, splits=splits)
+    assert np.all(np.isfinite(got))
+    assert np.all(np.abs(got - Y) <= 1e-3 * Sabs + 1e-30)
+    assert np.max(np.abs(got - Y) / (Sabs + 1e-30)) < 1e-5
+
+
+def test_gemm_small_s_many_splits_and_bf16(batq):
+    S, M, N = 16, 264, 14336
+    a, Y, Sabs = _small_case(batq, S, M, N, 900, splits=32)
+    assert np.max(np.abs(a - Y) / (Sabs + 1e-30)) < 1e-5
+    b, _, _ = _small_case(batq, S, M, N, 900, out_dtype=torch.bfloat16, splits=32)
+    want = torch.from_numpy(a.astype(np.float32)).bfloat16().float().numpy()
+    assert np.array_equal(b.astype(np.float32), want)
+
+
+def test_gemm_small_s_rejects_large_s_and_short_scratch(batq):
+    w = batq.batq_prepare_weight(None, batq.bits_to_cuda_bf16(synth.make_weight(128, 256, 1)))
+    z = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    y = torch.empty((65, 128), dtype=torch.float32, device="cuda")
+    with pytest.raises(batq.BatqError) as e:
+        batq.batq_gemm_mxfp4_small_s(z, z, w, 65, y, batq.aligned_workspace(4096))
+    assert e.value.status == 2
+    with pytest.raises(batq.BatqError) as e:
+        batq.batq_gemm_mxfp4_small_s(z, z, w, 8, y, batq.aligned_workspace(4096)[:512])
+    assert e.value.status == 5
+
+
 # ---------------------------------------------------------------------------- whole layer
 @pytest.mark.parametrize("S,M,N,geometry", [(128, 1024, 1024, "baseline"), (128, 1024, 1024, "paper"),
-                                            (50, 136, 544, "baseline"), (4, 1024, 1024, "baseline")])
+                                            (50, 136, 544, "baseline"), (4, 1024, 1024, "baseline"),
+                                            (1, 4096, 4096, "baseline"), (16, 6144, 4096, "paper"),
+                                            (64, 520, 1024, "baseline"), (65, 520, 1024, "baseline")])
 def test_linear_w4a4_vs_oracle(batq, qmode, S, M, N, geometry):
     xb = synth.make_activations(S, N, synth.BASE_SEED)
     wb = synth.make_weight(M, N, synth.BASE_SEED)
