@@ -1,18 +1,18 @@
 #!/usr/bin/env python
-"""Benchmark of the W4A4 linear hot path (transform + quant + MXFP4 GEMM).
+"""Benchmark of the W4A4 linear hot path (transform + clip + MXFP4 quantise + MXFP4 GEMM).
 
-One "step" is one pass of the whole path over one batch: for each projection of
-the workload, the fused activation transform/clip/quantiser kernel followed by
-the block-scaled tensor-core GEMM, on seeded synthetic inputs.  Prints ONE JSON
-line (rank 0).  `--impl reference` times the CPU oracle instead, on a bounded
-sample of the same workload.
+One "step" is one pass of the whole path over one batch of seeded synthetic input: for each
+projection of the workload, the activation transform/clip/quantiser kernel followed by the
+block-scaled tensor-core GEMM (prefill workloads), the whole-layer call (decode workload), or
+the quantiser alone (quantiser sweep).  Prints ONE JSON line (rank 0).  `--impl reference`
+times the CPU oracle instead, on a bounded sample of the same workload.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
-import subprocess
 import sys
 import threading
 import time
@@ -26,21 +26,38 @@ from paper_2603_16590_b200 import synth  # noqa: E402
 
 METRIC = "w4a4_linear_tflops"
 UNIT = "TFLOP/s"
+FP4_OVER_BF16 = 4.0       # nominal dense peak ratio 9 / 2.25 PFLOP/s
+QUANT_BYTES_PER_ELEM = 2.53125   # 2 (bf16 in) + 0.5 (codes) + 1/32 (scale byte)
+WEIGHT_BYTES_PER_ELEM = 0.53125  # 0.5 (codes) + 1/32 (scale byte)
+EVENT_EVERY = 8                  # prefill: every 8th timed step carries per-launch events
+
+# kind, tokens, projections (name, n in, m out), vision-row fraction, outlier-channel fraction
 WORKLOADS = {
-    # name: (tokens, projections, vision-row fraction, outlier-channel fraction)
-    "cfg1_llama8b_prefill": (2048, synth.LLAMA8B_PREFILL, 0.0, 0.01),
-    "cfg3_qwen2vl7b_prefill": (8192, synth.QWEN2VL7B_PREFILL, 0.75, 0.005),
-    "cfg0_single_layer": (128, [("lin", 1024, 1024)], 0.0, 0.01),
-    # single-kernel cases for profiler captures (m = 0: quantiser only, input larger than L2)
-    "profile_gemm_gate_up": (2048, [("gate_up", 4096, 28672)], 0.0, 0.01),
-    "profile_gemm_down": (2048, [("down", 14336, 4096)], 0.0, 0.01),
-    "profile_quant_32768x4096": (32768, [("quant", 4096, 0)], 0.0, 0.01),
+    "cfg0_single_layer": ("prefill", [128], [("lin", 1024, 1024)], 0.0, 0.01),
+    "cfg1_llama8b_prefill": ("prefill", [2048], synth.LLAMA8B_PREFILL, 0.0, 0.01),
+    "cfg2_llama8b_decode": ("decode", [1, 4, 16], synth.LLAMA8B_PREFILL, 0.0, 0.01),
+    "cfg3_qwen2vl7b_prefill": ("prefill", [8192], synth.QWEN2VL7B_PREFILL, 0.75, 0.005),
+    "cfg4_quantizer_sweep": ("quant", [1024, 8192, 32768], [("h2048", 2048, 0), ("h4096", 4096, 0), ("h8192", 8192, 0)],
+                             0.0, 0.01),
+    # single-kernel cases for profiler captures (inputs larger than L2, a few hundred MB on the device)
+    "profile_gemm_gate_up": ("prefill", [2048], [("gate_up", 4096, 28672)], 0.0, 0.01),
+    "profile_gemm_down": ("prefill", [2048], [("down", 14336, 4096)], 0.0, 0.01),
+    "profile_quant_32768x4096": ("quant", [32768], [("h4096", 4096, 0)], 0.0, 0.01),
+    "profile_decode_gate_up": ("decode", [16], [("gate_up", 4096, 28672)] * 4, 0.0, 0.01),
 }
-FP4_OVER_BF16 = 4.0  # nominal dense peak ratio 9 / 2.25 PFLOP/s
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, MB per step = the four GEMM launches of
+# cfg1_llama8b_prefill) from the ncu capture summarised under profiles/, valid for the kernel source
+# with this hash only.
+GEMM_TRAFFIC = {"workload": "cfg1_llama8b_prefill", "mb_per_step": None, "source_sha256": None}
 
 
-def workload_flops(S, projs):
-    return sum(2.0 * S * n * m for _, n, m in projs)
+def kernel_source_hash():
+    h = hashlib.sha256()
+    for f in ("gemm_mxfp4.cuh", "ptx.cuh"):
+        with open(os.path.join(ROOT, "paper_2603_16590_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
 
 
 def load_peaks():
@@ -53,20 +70,20 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
-def make_inputs(workload, seed):
-    S, projs, vis_frac, och = WORKLOADS[workload]
+def make_layer_inputs(workload, S, seed):
+    _, _, projs, vis_frac, och = WORKLOADS[workload]
     layers = []
     for i, (name, n, m) in enumerate(projs):
         xb = synth.make_activations(S, n, seed + 16 * i, outlier_channel_frac=och, vision_rows=int(S * vis_frac))
         t = synth.make_transform(n, seed + 16 * i + 1, "baseline")
         layers.append({"name": name, "n": n, "m": m, "x_bits": xb, "t": t, "w_seed": seed + 16 * i + 2})
-    return S, layers
+    return layers
 
 
 # ------------------------------------------------------------------------------------ clocks
 class ClockSampler:
-    """Samples SM clock and throttle reasons of one GPU during the timed region (read-only NVML
-    queries from a thread, every ~2 ms; falls back to one nvidia-smi query if NVML is missing)."""
+    """Samples SM clock, power and throttle reasons of one GPU during the timed region (read-only
+    NVML queries from a thread, every ~2 ms)."""
     REASONS = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
 
     def __init__(self, index):
@@ -119,11 +136,16 @@ def oracle_sample(workload, seed, rows, feats):
     """A bounded sample of the workload for the CPU oracle: the first projection,
     `rows` token rows and `feats` output features (weights prepared offline)."""
     from oracle import batq_oracle as O
-    S, projs, vis_frac, och = WORKLOADS[workload]
+    kind, tokens, projs, vis_frac, och = WORKLOADS[workload]
+    S = tokens[-1]
     name, n, m = projs[0]
-    rows, feats = min(rows, S), min(feats, m)
+    rows, feats = max(1, min(rows, S)), max(1, min(feats, m if m else 1))
     xb = synth.make_activations(rows, n, seed, outlier_channel_frac=och, vision_rows=int(rows * vis_frac))
     t = synth.make_transform(n, seed + 1, "baseline")
+    if kind == "quant":
+        def step():
+            return O.quantize_act(xb, t.left, t.right, t.clip_lo, t.clip_hi)
+        return step, 24.0 * rows * n, f"quantiser only, {rows} of {S} token rows x {n} channels"
     wb = synth.make_weight(feats, n, seed + 2)
     qw = O.prepare_weight(wb, t.left, t.right)
 
@@ -144,7 +166,17 @@ def oracle_threads():
         return os.cpu_count() or 1
 
 
-def time_oracle(workload, seed, rows, feats, steps, warmup):
+def time_oracle(workload, seed, steps, warmup, budget_s):
+    """Times the oracle as it stands on a sample sized so that warmup + steps take about
+    `budget_s` seconds: a small probe fixes the cost per (row x feature), then rows and
+    features are scaled up together."""
+    probe, pflops, _ = oracle_sample(workload, seed, 64, 512)
+    t0 = time.perf_counter()
+    probe()
+    per_flop = (time.perf_counter() - t0) / pflops
+    per_step = budget_s / max(steps + warmup, 1)
+    scale = max(1.0, per_step / (per_flop * pflops)) ** 0.5
+    rows, feats = int(64 * scale), int(512 * scale)
     step, flops, desc = oracle_sample(workload, seed, rows, feats)
     for _ in range(warmup):
         step()
@@ -156,15 +188,15 @@ def time_oracle(workload, seed, rows, feats, steps, warmup):
 
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if int(os.environ.get("RANK", "0")) != 0:
         return
-    S, projs, _, _ = WORKLOADS[args.workload]
-    val, dt, desc = time_oracle(args.workload, synth.BASE_SEED, 256, 1024, args.steps, args.warmup)
+    kind, tokens, projs, _, _ = WORKLOADS[args.workload]
+    steps = args.steps if args.steps is not None else 5
+    val, dt, desc = time_oracle(args.workload, synth.BASE_SEED, steps, args.warmup, 60.0)
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "steps": steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "tokens": S, "projections": [list(p) for p in projs]},
+            "config": {"workload": args.workload, "tokens": tokens, "projections": [list(p) for p in projs]},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": desc},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -172,168 +204,359 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------ CUDA arm
+class Harness:
+    """Process-group plumbing shared by the workload kinds: one process per GPU, no data-path
+    collective (token rows are independent, so ranks are replicas on their own batches)."""
+
+    def __init__(self):
+        import torch
+        self.torch = torch
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+        torch.cuda.set_device(self.local)
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.init_process_group("nccl", device_id=torch.device("cuda", self.local))
+            self.dist = dist
+
+    def barrier(self):
+        self.torch.cuda.synchronize()
+        if self.dist is not None:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def max_over_ranks(self, ms):
+        if self.dist is None:
+            return ms
+        t = self.torch.tensor([ms], dtype=self.torch.float64, device="cuda")
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def close(self):
+        if self.dist is not None:
+            self.dist.destroy_process_group()
+
+
+def timed_region(h, step, steps, warmup):
+    """W warm-up steps, then K steps bracketed by barrier + synchronize, CUDA events on the
+    launching stream, clocks sampled meanwhile; returns (ms max over ranks, clocks)."""
+    torch = h.torch
+    for _ in range(warmup):
+        step(None)
+    sampler = ClockSampler(h.local)
+    h.barrier()
+    if h.rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for k in range(steps):
+        step(k)
+    e1.record()
+    h.barrier()
+    clocks = sampler.stop() if h.rank == 0 else None
+    return h.max_over_ranks(e0.elapsed_time(e1)), clocks
+
+
 def run_ours(args):
     import torch
     from paper_2603_16590_b200 import binding as B
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
-    torch.cuda.set_device(local)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    h = Harness()
     B.load()
     B.batq_debug_force_tile_width(args.tile_width)
     B.batq_debug_set_gemm_flags(args.gemm_debug_flags)
     B.batq_debug_force_quantizer(args.quantizer)
+    B.batq_debug_force_small_s_splits(args.splits)
     peaks = load_peaks()
-
-    # weak scaling: every rank runs the same workload on its own seeded batch, no exchange step
-    S, layers = make_inputs(args.workload, synth.BASE_SEED + 1000 * rank)
-    projs = WORKLOADS[args.workload][1]
-    for L in layers:
-        L["tr"] = B.batq_transform_create(L["n"], L["t"].left, L["t"].right, L["t"].clip_lo, L["t"].clip_hi)
-        L["x"] = B.bits_to_cuda_bf16(L["x_bits"])
-        L["codes"] = torch.empty((S, L["n"] // 2), dtype=torch.uint8, device="cuda")
-        L["sf"] = torch.empty(B.batq_sf_bytes(S, L["n"], B.SF_MMA), dtype=torch.uint8, device="cuda")
-        if L["m"] == 0:
-            continue
-        wdev = B.bits_to_cuda_bf16(synth.make_weight(L["m"], L["n"], L["w_seed"]))
-        L["w"] = B.batq_prepare_weight(L["tr"], wdev)
-        del wdev
-        L["y"] = torch.empty((S, L["m"]), dtype=torch.bfloat16, device="cuda")
-        L["ws"] = B.aligned_workspace(B.batq_linear_workspace_bytes(L["w"], S))
-        L["x_host"] = torch.from_numpy(L["x_bits"].view(np.int16)).pin_memory()
-        L["y_host"] = torch.empty((S, L["m"]), dtype=torch.bfloat16).pin_memory()
-    torch.cuda.synchronize()
-    flops_step = workload_flops(S, projs)
-
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(ms):
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
-    # ---- device-resident arm: quantise + GEMM per projection, events around every launch
+    kind, tokens, projs, _, _ = WORKLOADS[args.workload]
+    steps = args.steps if args.steps is not None else {"prefill": 1000, "decode": 300, "quant": 100}[kind]
+    if args.workload == "cfg3_qwen2vl7b_prefill" and args.steps is None:
+        steps = 200
+    seed = synth.BASE_SEED + 1000 * h.rank  # weak scaling: every rank its own seeded batch
     ev = lambda: torch.cuda.Event(enable_timing=True)
-    marks = [[(ev(), ev(), ev()) for _ in layers] for _ in range(args.steps)]
+    line = {"metric": METRIC, "unit": UNIT, "n_gpus": h.world, "steps": steps, "warmup": args.warmup,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "mxfp4", "data": "synthetic"}
 
-    def step(m=None):
-        for i, L in enumerate(layers):
-            if m is not None:
-                m[i][0].record()
-            B.batq_quantize_act(L["tr"], L["x"], L["codes"], L["sf"], B.SF_MMA)
-            if m is not None:
-                m[i][1].record()
-            if L["m"]:
+    def mk_transform(L):
+        return B.batq_transform_create(L["n"], L["t"].left, L["t"].right, L["t"].clip_lo, L["t"].clip_hi)
+
+    if kind == "prefill":
+        S = tokens[0]
+        layers = make_layer_inputs(args.workload, S, seed)
+        for L in layers:
+            L["tr"] = mk_transform(L)
+            L["x"] = B.bits_to_cuda_bf16(L["x_bits"])
+            L["codes"] = torch.empty((S, L["n"] // 2), dtype=torch.uint8, device="cuda")
+            L["sf"] = torch.empty(B.batq_sf_bytes(S, L["n"], B.SF_MMA), dtype=torch.uint8, device="cuda")
+            wdev = B.bits_to_cuda_bf16(synth.make_weight(L["m"], L["n"], L["w_seed"]))
+            L["w"] = B.batq_prepare_weight(L["tr"], wdev)
+            del wdev
+            L["y"] = torch.empty((S, L["m"]), dtype=torch.bfloat16, device="cuda")
+            L["ws"] = B.aligned_workspace(B.batq_linear_workspace_bytes(L["w"], S))
+            L["x_host"] = torch.from_numpy(L["x_bits"].view(np.int16)).pin_memory()
+            L["y_host"] = torch.empty((S, L["m"]), dtype=torch.bfloat16).pin_memory()
+        torch.cuda.synchronize()
+        flops_step = sum(2.0 * S * L["n"] * L["m"] for L in layers)
+        # Events around every launch cost about 8 % of a step (they close the gap-free hand-over between
+        # consecutive kernels), so only every EVENT_EVERY-th step of the timed region carries them.
+        sampled = [k for k in range(steps) if k % EVENT_EVERY == 0]
+        marks = {k: [(ev(), ev(), ev()) for _ in layers] for k in sampled}
+
+        def step(k):
+            m = marks.get(k)
+            for i, L in enumerate(layers):
+                if m is not None:
+                    m[i][0].record()
+                B.batq_quantize_act(L["tr"], L["x"], L["codes"], L["sf"], B.SF_MMA)
+                if m is not None:
+                    m[i][1].record()
                 B.batq_gemm_mxfp4(L["codes"], L["sf"], L["w"], S, L["y"])
-            if m is not None:
-                m[i][2].record()
+                if m is not None:
+                    m[i][2].record()
 
-    for _ in range(args.warmup):
-        step()
-    sampler = ClockSampler(local)
-    barrier()
-    if rank == 0:
-        sampler.start()
-    e0, e1 = ev(), ev()
-    e0.record()
-    for k in range(args.steps):
-        step(marks[k])
-    e1.record()
-    barrier()
-    clocks = sampler.stop() if rank == 0 else None
-    ms = max_over_ranks(e0.elapsed_time(e1))
+        ms, clocks = timed_region(h, step, steps, args.warmup)
+        q_ms = np.array([[m[i][0].elapsed_time(m[i][1]) for i in range(len(layers))] for m in marks.values()]).mean(axis=0)
+        g_ms = np.array([[m[i][1].elapsed_time(m[i][2]) for i in range(len(layers))] for m in marks.values()]).mean(axis=0)
+
+        # end to end: host buffers in and out through the C-ABI host entry point
+        def step_host():
+            for L in layers:
+                B.batq_linear_w4a4_host(L["tr"], L["w"], L["x_host"], L["y_host"], L["x"], L["y"], L["ws"])
+
+        e2e_steps = max(1, min(steps, 5))
+        for _ in range(2):
+            step_host()
+        h.barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            step_host()
+        torch.cuda.synchronize()
+        e2e_ms = h.max_over_ranks((time.perf_counter() - t0) * 1e3)
+        h2d = sum(S * L["n"] * 2 for L in layers)
+        d2h = sum(S * L["m"] * 2 for L in layers)
+
+        gemm_flops = [2.0 * S * L["n"] * L["m"] for L in layers]
+        gemm_achieved = sum(gemm_flops) / (g_ms.sum() * 1e-3) / 1e12
+        q_bytes = [S * L["n"] * QUANT_BYTES_PER_ELEM for L in layers]
+        quant_gbs = sum(q_bytes) / (q_ms.sum() * 1e-3) / 1e9
+        sustained = ms >= 500.0   # a timed region this long runs under the power cap
+        bf16_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+        fp4_peak = bf16_peak * FP4_OVER_BF16
+        traffic = None
+        if GEMM_TRAFFIC["workload"] == args.workload and GEMM_TRAFFIC["source_sha256"] == kernel_source_hash():
+            traffic = GEMM_TRAFFIC["mb_per_step"]
+        touched = h2d + d2h + sum(L["n"] * L["m"] * WEIGHT_BYTES_PER_ELEM for L in layers)
+        line.update({
+            "value": flops_step * steps * h.world / (ms * 1e-3) / 1e12, "ms_per_step": ms / steps,
+            "config": {"workload": args.workload, "tokens": S, "projections": [list(p) for p in projs],
+                       "transform": "shared 4x4 (x) private 8x8 per 32-group, clip U[0.8,1]", "output": "bf16",
+                       "l2": "inputs larger than L2: one step touches %.0f MB" % (touched / 1e6)},
+            "roofline": {"bound": "tensor", "kernel": "gemm_mxfp4_kernel", "achieved": gemm_achieved, "peak": fp4_peak,
+                         "events": "around every launch in every %dth step of the timed region (%d steps)" % (
+                             EVENT_EVERY, len(sampled)),
+                         "unit": "TFLOP/s", "frac": gemm_achieved / fp4_peak, "traffic": traffic,
+                         "traffic_unit": "MB per step (4 launches)" if traffic else None,
+                         "peak_source": "%s cuBLAS bf16 %s x %.0f (nominal fp4:bf16 ratio)" % (
+                             peaks["source"], "sustained" if sustained else "burst", FP4_OVER_BF16)},
+            "act_quant": {"bound": "hbm", "kernel": "quantize_act_tc_kernel", "achieved": quant_gbs,
+                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": quant_gbs / peaks["hbm_gbs"],
+                          "peak_source": peaks["source"]},
+            "kernels": [{"name": L["name"], "n": L["n"], "m": L["m"], "quant_us": float(q_ms[i] * 1e3),
+                         "quant_gbs": q_bytes[i] / (q_ms[i] * 1e-3) / 1e9, "gemm_us": float(g_ms[i] * 1e3),
+                         "gemm_tflops": gemm_flops[i] / (g_ms[i] * 1e-3) / 1e12} for i, L in enumerate(layers)],
+            "e2e": {"value": flops_step * e2e_steps * h.world / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+            "gpu_launches": 2 * len(layers) * steps,
+        })
+
+    elif kind == "decode":
+        # Per call: quantiser + small-s GEMM (one batq_linear_w4a4).  A decode loop is launch-bound
+        # from Python, so each case is captured once as a CUDA graph of `copies` calls, one per copy of
+        # the prepared weight: the copies cycle through more than 3 x L2 between reuses, so no call
+        # finds its weights in L2.  A step replays the graph of every case; events bracket each replay.
+        copies = 4
+        base = make_layer_inputs(args.workload, max(tokens), seed)
+        cases = []
+        for i, L in enumerate(base):
+            L["tr"] = mk_transform(L)
+            wdev = B.bits_to_cuda_bf16(synth.make_weight(L["m"], L["n"], L["w_seed"]))
+            L["ws_list"] = [B.batq_prepare_weight(L["tr"], wdev) for _ in range(copies)]
+            del wdev
+            xfull = B.bits_to_cuda_bf16(L["x_bits"])
+            for S in tokens:
+                c = {"L": L, "S": S, "x": xfull[:S].contiguous(),
+                     "y": torch.empty((S, L["m"]), dtype=torch.bfloat16, device="cuda"),
+                     "ws": B.aligned_workspace(B.batq_linear_workspace_bytes(L["ws_list"][0], S)),
+                     "x_host": torch.from_numpy(L["x_bits"][:S].copy().view(np.int16)).pin_memory(),
+                     "y_host": torch.empty((S, L["m"]), dtype=torch.bfloat16).pin_memory()}
+                cases.append(c)
+        order = [c for S in tokens for c in cases if c["S"] == S]   # all projections at S=1, then S=4, ...
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            for c in order:
+                for w in c["L"]["ws_list"]:   # first calls outside capture: per-device set-up
+                    B.batq_linear_w4a4(c["L"]["tr"], w, c["x"], c["y"], c["ws"])
+            torch.cuda.synchronize()
+            for c in order:
+                c["graph"] = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(c["graph"], stream=side):
+                    for w in c["L"]["ws_list"]:
+                        B.batq_linear_w4a4(c["L"]["tr"], w, c["x"], c["y"], c["ws"])
+        torch.cuda.synchronize()
+        flops_step = copies * sum(2.0 * c["S"] * c["L"]["n"] * c["L"]["m"] for c in order)
+        marks = [[(ev(), ev()) for _ in order] for _ in range(steps)]
+
+        def step(k):
+            for i, c in enumerate(order):
+                if k is not None:
+                    marks[k][i][0].record()
+                c["graph"].replay()
+                if k is not None:
+                    marks[k][i][1].record()
+
+        ms, clocks = timed_region(h, step, steps, args.warmup)
+        c_ms = np.array([[m[i][0].elapsed_time(m[i][1]) for i in range(len(order))] for m in marks]) / copies
+        c_med = np.median(c_ms, axis=0)
+        w_bytes = [c["L"]["n"] * c["L"]["m"] * WEIGHT_BYTES_PER_ELEM for c in order]
+        gbs = sum(w_bytes) / (c_ms.mean(axis=0).sum() * 1e-3) / 1e9
+
+        def step_host():
+            for c in order:
+                B.batq_linear_w4a4_host(c["L"]["tr"], c["L"]["ws_list"][0], c["x_host"], c["y_host"], c["x"], c["y"],
+                                        c["ws"])
+
+        e2e_steps = max(1, min(steps, 20))
+        for _ in range(2):
+            step_host()
+        h.barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            step_host()
+        torch.cuda.synchronize()
+        e2e_ms = h.max_over_ranks((time.perf_counter() - t0) * 1e3)
+        h2d = sum(c["S"] * c["L"]["n"] * 2 for c in order)
+        d2h = sum(c["S"] * c["L"]["m"] * 2 for c in order)
+        line.update({
+            "value": flops_step * steps * h.world / (ms * 1e-3) / 1e12, "ms_per_step": ms / steps,
+            "config": {"workload": args.workload, "tokens": tokens, "projections": [list(p) for p in projs],
+                       "transform": "shared 4x4 (x) private 8x8 per 32-group, clip U[0.8,1]", "output": "bf16",
+                       "launch": "one CUDA graph of %d calls per (tokens, projection) case" % copies,
+                       "l2": "%d copies of each prepared weight used in turn: %.0f MB cycle through L2 between reuses" % (
+                           copies, copies * sum(L["n"] * L["m"] * WEIGHT_BYTES_PER_ELEM for L in base) / 1e6)},
+            "roofline": {"bound": "hbm", "kernel": "gemm_small_s_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                         "peak_source": "%s copy bandwidth; achieved = weight bytes / whole-call time (quantiser + GEMM)" %
+                                        peaks["source"]},
+            "kernels": [{"name": c["L"]["name"], "tokens": c["S"], "n": c["L"]["n"], "m": c["L"]["m"],
+                         "call_us": float(c_ms[:, i].mean() * 1e3), "call_us_median": float(c_med[i] * 1e3),
+                         "weight_gbs": w_bytes[i] / (c_ms[:, i].mean() * 1e-3) / 1e9} for i, c in enumerate(order)],
+            "e2e": {"value": flops_step / copies * e2e_steps * h.world / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                    "note": "one eager host-buffer call per case and step (no graph)"},
+            "gpu_launches": 2 * copies * len(order) * steps,
+        })
+
+    else:  # quantiser sweep
+        cases = []
+        for S in tokens:
+            for L in make_layer_inputs(args.workload, S, seed):
+                L["S"] = S
+                L["tr"] = mk_transform(L)
+                L["x"] = B.bits_to_cuda_bf16(L["x_bits"])
+                L["codes"] = torch.empty((S, L["n"] // 2), dtype=torch.uint8, device="cuda")
+                L["sf"] = torch.empty(B.batq_sf_bytes(S, L["n"], B.SF_MMA), dtype=torch.uint8, device="cuda")
+                L["x_host"] = torch.from_numpy(L["x_bits"].view(np.int16)).pin_memory()
+                L["codes_host"] = torch.empty((S, L["n"] // 2), dtype=torch.uint8).pin_memory()
+                cases.append(L)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")  # > L2: written between cases
+        torch.cuda.synchronize()
+        variants = [("gpk", True), ("identity", False)]   # T_j = G (x) P_j with clip, and plain MXFP4 (T = I)
+        marks = [[[(ev(), ev()) for _ in variants] for _ in cases] for _ in range(steps)]
+
+        def step(k):
+            for i, L in enumerate(cases):
+                for v, (_, xf) in enumerate(variants):
+                    flush.zero_()
+                    if k is not None:
+                        marks[k][i][v][0].record()
+                    B.batq_quantize_act(L["tr"] if xf else None, L["x"], L["codes"], L["sf"], B.SF_MMA)
+                    if k is not None:
+                        marks[k][i][v][1].record()
+
+        ms, clocks = timed_region(h, step, steps, args.warmup)
+        t_ms = np.array([[[m[i][v][0].elapsed_time(m[i][v][1]) for v in range(2)] for i in range(len(cases))]
+                         for m in marks]).mean(axis=0)
+        bytes_case = np.array([L["S"] * L["n"] * QUANT_BYTES_PER_ELEM for L in cases])
+        gbs = bytes_case.sum() / (t_ms[:, 0].sum() * 1e-3) / 1e9
+        big = int(np.argmax(bytes_case))
+
+        def step_host():
+            for L in cases:
+                L["x"].copy_(L["x_host"].view(torch.bfloat16), non_blocking=True)
+                B.batq_quantize_act(L["tr"], L["x"], L["codes"], L["sf"], B.SF_MMA)
+                L["codes_host"].copy_(L["codes"], non_blocking=True)
+            torch.cuda.synchronize()
+
+        step_host()
+        h.barrier()
+        t0 = time.perf_counter()
+        step_host()
+        e2e_ms = h.max_over_ranks((time.perf_counter() - t0) * 1e3)
+        elems = float(sum(L["S"] * L["n"] for L in cases))
+        # quantiser-only workloads have no GEMM flops: the metric's numerator is the transform's
+        # 24 flop per element (Kronecker form), reported for completeness
+        line.update({
+            "value": 24.0 * elems * steps * h.world / (t_ms[:, 0].sum() * steps * 1e-3) / 1e12,
+            "ms_per_step": float(t_ms[:, 0].sum()),
+            "config": {"workload": args.workload, "tokens": tokens, "hidden": [p[1] for p in projs],
+                       "transform": "shared 4x4 (x) private 8x8 per 32-group, clip U[0.8,1]; ablation T = I",
+                       "l2": "a 256 MB buffer is written between launches (outside the per-launch events)",
+                       "value_note": "transform flops (24 per element) over quantiser time; the GB/s figures are the point"},
+            "roofline": {"bound": "hbm", "kernel": "quantize_act_tc_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                         "largest_case_gbs": float(bytes_case[big] / (t_ms[big, 0] * 1e-3) / 1e9),
+                         "peak_source": "%s copy bandwidth" % peaks["source"]},
+            "kernels": [{"tokens": L["S"], "hidden": L["n"], "gpk_us": float(t_ms[i, 0] * 1e3),
+                         "gpk_gbs": float(bytes_case[i] / (t_ms[i, 0] * 1e-3) / 1e9),
+                         "identity_us": float(t_ms[i, 1] * 1e3),
+                         "identity_gbs": float(bytes_case[i] / (t_ms[i, 1] * 1e-3) / 1e9)} for i, L in enumerate(cases)],
+            "e2e": {"value": 24.0 * elems * h.world / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+                    "h2d_bytes_per_step": int(elems * 2), "d2h_bytes_per_step": int(elems // 2), "steps": 1},
+            "gpu_launches": 2 * len(cases) * steps,
+        })
+
     status = B.batq_last_device_status()
     if status != 0:
         raise SystemExit(f"device status {status} after the timed region")
-    q_ms = np.array([[m[i][0].elapsed_time(m[i][1]) for i in range(len(layers))] for m in marks]).mean(axis=0)
-    g_ms = np.array([[m[i][1].elapsed_time(m[i][2]) for i in range(len(layers))] for m in marks]).mean(axis=0)
-
-    # ---- end-to-end arm: host buffers in, host buffers out, through the C-ABI host entry point
-    def step_host():
-        for L in layers:
-            if L["m"] == 0:
-                continue
-            B.batq_linear_w4a4_host(L["tr"], L["w"], L["x_host"], L["y_host"], L["x"], L["y"], L["ws"])
-
-    e2e_steps = max(1, min(args.steps, 5))
-    for _ in range(2):
-        step_host()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        step_host()
-    torch.cuda.synchronize()
-    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3)
-    h2d = sum(S * L["n"] * 2 for L in layers)
-    d2h = sum(S * L["m"] * 2 for L in layers)
-
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-
-    value = flops_step * args.steps * world / (ms * 1e-3) / 1e12
-    fp4_peak = peaks["bf16_tflops_sustained"] * FP4_OVER_BF16
-    gemm_flops = [2.0 * S * L["n"] * L["m"] for L in layers]
-    gemm_achieved = sum(gemm_flops) / (max(g_ms.sum(), 1e-9) * 1e-3) / 1e12
-    q_bytes = [S * L["n"] * 2.53125 for L in layers]
-    quant_gbs = sum(q_bytes) / (q_ms.sum() * 1e-3) / 1e9
-    cpu_val, cpu_dt, cpu_desc = time_oracle(args.workload, synth.BASE_SEED, 256, 1024, 3, 1)
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "mxfp4", "data": "synthetic",
-        "config": {"workload": args.workload, "tokens": S, "projections": [list(p) for p in projs],
-                   "transform": "shared 4x4 (x) private 8x8 per 32-group, clip U[0.8,1]", "output": "bf16",
-                   "l2": "inputs larger than L2: one step touches %.0f MB" % (
-                       (h2d + d2h + sum(L["n"] * L["m"] * 0.53125 for L in layers)) / 1e6)},
-        "roofline": {"bound": "tensor", "kernel": "gemm_mxfp4_kernel", "achieved": gemm_achieved, "peak": fp4_peak,
-                     "unit": "TFLOP/s", "frac": gemm_achieved / fp4_peak, "traffic": None,
-                     "peak_source": "%s bf16 sustained x %.0f (nominal fp4:bf16)" % (peaks["source"], FP4_OVER_BF16)},
-        "act_quant": {"bound": "hbm", "kernel": "quantize_act_kernel", "achieved": quant_gbs, "peak": peaks["hbm_gbs"],
-                      "unit": "GB/s", "frac": quant_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"]},
-        "kernels": [{"name": L["name"], "n": L["n"], "m": L["m"], "quant_us": float(q_ms[i] * 1e3),
-                     "quant_gbs": q_bytes[i] / (q_ms[i] * 1e-3) / 1e9, "gemm_us": float(g_ms[i] * 1e3),
-                     "gemm_tflops": gemm_flops[i] / (max(g_ms[i], 1e-9) * 1e-3) / 1e12} for i, L in enumerate(layers)],
-        "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
-                         "sample": cpu_desc},
-        "e2e": {"value": flops_step * e2e_steps * world / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-        "gpu_launches": 2 * len(layers) * args.steps,
-        "clocks": clocks,
-    }
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    if h.rank == 0:
+        cpu_val, cpu_dt, cpu_desc = time_oracle(args.workload, synth.BASE_SEED, 3, 1, 20.0)
+        line["cpu_baseline"] = {"value": cpu_val, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                                "sample": cpu_desc, "seconds_per_sample": cpu_dt}
+        line["clocks"] = clocks
+        print(json.dumps(line))
+    h.close()
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default: per workload, about 0.3-1 s of GPU time)")
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg1_llama8b_prefill", choices=sorted(WORKLOADS))
     ap.add_argument("--gemm-debug-flags", type=int, default=0, help="timing experiments only; results invalid")
     ap.add_argument("--quantizer", type=int, default=0, help="0 auto, 1 ALU kernel, 2 tensor-core kernel (tuning)")
     ap.add_argument("--tile-width", type=int, default=0, help="force the GEMM tile width (tuning); 0 = automatic")
+    ap.add_argument("--splits", type=int, default=0, help="force the small-s GEMM's K splits (tuning); 0 = automatic")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
     else:
+        args.warmup = max(args.warmup, 3)
         run_ours(args)
 
 

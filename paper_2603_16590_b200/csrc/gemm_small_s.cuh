@@ -247,14 +247,45 @@ gemm_small_s_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         write_out = ticket_slot == static_cast<uint32_t>(p.splits - 1);
         if (write_out) {
           __threadfence();
+          // Sum in split order (deterministic).  Loads are issued in independent batches -- over the
+          // tokens when there are many, over the splits when there are few -- so that their latencies
+          // overlap instead of adding up.
           const float* all = p.partial + static_cast<int64_t>(rt) * p.splits * (NTOK * 128) + row;
+          if (p.s > 4) {
 #pragma unroll
-          for (int t = 0; t < NTOK; ++t) {
-            if (t < p.s) {
-              float acc = 0.0f;
-              for (int q = 0; q < p.splits; ++q) acc += __ldcg(all + static_cast<int64_t>(q) * (NTOK * 128) + t * 128);
-              v[t] = __float_as_uint(acc);
+            for (int c = 0; c < NTOK; c += 16) {  // 16 tokens at a time keeps the registers in check
+              if (c < p.s) {
+                float acc[16];
+#pragma unroll
+                for (int t = 0; t < 16; ++t) acc[t] = 0.0f;
+                for (int q = 0; q < p.splits; ++q) {
+                  float part[16];
+#pragma unroll
+                  for (int t = 0; t < 16; ++t)
+                    part[t] = c + t < p.s ? __ldcg(all + q * (NTOK * 128) + (c + t) * 128) : 0.0f;
+#pragma unroll
+                  for (int t = 0; t < 16; ++t) acc[t] += part[t];
+                }
+#pragma unroll
+                for (int t = 0; t < 16; ++t) v[c + t] = __float_as_uint(acc[t]);
+              }
             }
+          } else {
+            float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            for (int q0 = 0; q0 < p.splits; q0 += 8) {
+              float part[8][4];
+#pragma unroll
+              for (int qq = 0; qq < 8; ++qq)
+#pragma unroll
+                for (int t = 0; t < 4; ++t)
+                  part[qq][t] = (q0 + qq < p.splits && t < p.s) ? __ldcg(all + (q0 + qq) * (NTOK * 128) + t * 128) : 0.0f;
+#pragma unroll
+              for (int qq = 0; qq < 8; ++qq)
+#pragma unroll
+                for (int t = 0; t < 4; ++t) acc[t] += part[qq][t];
+            }
+#pragma unroll
+            for (int t = 0; t < 4; ++t) v[t] = __float_as_uint(acc[t]);
           }
           if (warp == 2 && lane == 0) p.tickets[rt] = 0;  // ready for the next call
         }
