@@ -54,7 +54,7 @@ GEMM_TRAFFIC = {"workload": "cfg1_llama8b_prefill", "mb_per_step": 210.7, "sourc
 
 def kernel_source_hash():
     h = hashlib.sha256()
-    for f in ("gemm_mxfp4.cuh", "ptx.cuh"):
+    for f in ("gemm_mxfp4.cuh", "gemm_mxfp4_pair.cuh", "ptx.cuh"):
         with open(os.path.join(ROOT, "paper_2603_16590_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -270,6 +270,7 @@ def run_ours(args):
     B.batq_debug_force_tile_width(args.tile_width)
     B.batq_debug_set_gemm_flags(args.gemm_debug_flags)
     B.batq_debug_force_quantizer(args.quantizer)
+    B.batq_debug_force_gemm_kernel(args.gemm_kernel)
     B.batq_debug_force_small_s_splits(args.splits)
     peaks = load_peaks()
     kind, tokens, projs, _, _ = WORKLOADS[args.workload]
@@ -550,6 +551,7 @@ def main():
     ap.add_argument("--workload", default="cfg1_llama8b_prefill", choices=sorted(WORKLOADS))
     ap.add_argument("--gemm-debug-flags", type=int, default=0, help="timing experiments only; results invalid")
     ap.add_argument("--quantizer", type=int, default=0, help="0 auto, 1 ALU kernel, 2 tensor-core kernel (tuning)")
+    ap.add_argument("--gemm-kernel", type=int, default=0, help="0 auto, 1 one CTA per tile, 2 CTA pairs (tuning)")
     ap.add_argument("--tile-width", type=int, default=0, help="force the GEMM tile width (tuning); 0 = automatic")
     ap.add_argument("--splits", type=int, default=0, help="force the small-s GEMM's K splits (tuning); 0 = automatic")
     args = ap.parse_args()

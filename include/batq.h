@@ -151,6 +151,10 @@ batq_status batq_gemm_mxfp4_small_s(const void* x_codes, const void* x_scales_mm
 /* Test / tuning hook: forces the GEMM's output-tile width to 128, 192 or 256 columns for all
  * later calls in this process; any other value restores the automatic choice. */
 void batq_debug_force_tile_width(int32_t bn);
+/* Test / tuning hook: which prefill GEMM kernel later calls use.  0 = automatic (CTA pairs sharing a
+ * 256-token tile for s > 128, one CTA per 128-token tile otherwise), 1 = always one CTA per tile,
+ * 2 = always CTA pairs (tile widths 192 and 256 only). */
+void batq_debug_force_gemm_kernel(int32_t which);
 /* Test / tuning hook: which activation quantiser later calls use.  0 = automatic (tensor-core
  * dense-block kernel for s >= 64 tokens, ALU Kronecker-form kernel below that and for the
  * identity transform), 1 = always the ALU kernel, 2 = always the tensor-core kernel. */

@@ -40,6 +40,7 @@ SIGNATURES = {
     "batq_gemm_mxfp4_small_s": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _I64, _P, _SZ, _P]),
     "batq_debug_force_small_s_splits": (None, [_I32]),
     "batq_debug_force_tile_width": (None, [_I32]),
+    "batq_debug_force_gemm_kernel": (None, [_I32]),
     "batq_debug_set_gemm_flags": (None, [_I32]),
     "batq_debug_force_quantizer": (None, [_I32]),
     "batq_linear_workspace_bytes": (_SZ, [_P, _I64]),
@@ -214,6 +215,10 @@ def batq_debug_force_small_s_splits(splits: int):
 
 def batq_debug_force_tile_width(bn: int):
     load().batq_debug_force_tile_width(bn)
+
+
+def batq_debug_force_gemm_kernel(which: int):
+    load().batq_debug_force_gemm_kernel(which)
 
 
 def batq_debug_force_quantizer(which: int):

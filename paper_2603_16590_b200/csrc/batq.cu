@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "gemm_mxfp4.cuh"
+#include "gemm_mxfp4_pair.cuh"
 #include "gemm_small_s.cuh"
 #include "prepare_weight.cuh"
 #include "quantize_act.cuh"
@@ -43,9 +44,11 @@ struct batq_weight {
   int32_t sm_count;  // of the device the weight lives on (sizes the small-s split-K scratch)
   uint8_t* codes;   // [m x n/2]
   uint8_t* scales;  // BATQ_SF_MMA
-  CUtensorMap tmap_b256;  // boxes of 256 / 192 / 128 weight rows x 128 bytes
+  CUtensorMap tmap_b256;  // boxes of 256 / 192 / 128 / 96 weight rows x 128 bytes
   CUtensorMap tmap_b192;
   CUtensorMap tmap_b128;
+  CUtensorMap tmap_b96;
+  CUtensorMap tmap_sf;    // scale atoms: [row tiles x KA] rows of 512 bytes, boxes of two atoms
 };
 
 // Scratch for batq_linear_w4a4_noalloc: part of the library image, one copy per GPU.
@@ -108,6 +111,10 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(gemm_mxfp4_kernel<192, true>, GemmCfg<192>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<128, false>, GemmCfg<128>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<128, true>, GemmCfg<128>::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_pair_kernel<192, false>, PairCfg<192>::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_pair_kernel<192, true>, PairCfg<192>::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_pair_kernel<256, false>, PairCfg<256>::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_pair_kernel<256, true>, PairCfg<256>::kSmemBytes);
     e = e ? e : set_smem(gemm_small_s_kernel<16, false>, SmallCfg<16>::kSmemBytes);
     e = e ? e : set_smem(gemm_small_s_kernel<16, true>, SmallCfg<16>::kSmemBytes);
     e = e ? e : set_smem(gemm_small_s_kernel<32, false>, SmallCfg<32>::kSmemBytes);
@@ -155,6 +162,13 @@ batq_status make_tmap_2d(CUtensorMap* map, CUtensorMapDataType dt, int esz, cons
                                     CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? BATQ_OK : BATQ_ERR_CUDA;
+}
+
+// Tensor map over scale bytes in the BATQ_SF_MMA layout: one row per 512-byte atom (128 uint32),
+// boxes of two consecutive atoms = the 8 blocks of one K step; rows past the buffer read as zero.
+batq_status make_sf_tmap(CUtensorMap* map, const void* base, int64_t row_tiles, int64_t katoms) {
+  return make_tmap_2d(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, base, 128, row_tiles * katoms, 512, 128, 2,
+                      CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 
 // fp32 -> bf16 bits, round to nearest even (finite inputs).
@@ -362,6 +376,69 @@ int pick_bn(int64_t s, int64_t m, int64_t n, int sm_count) {
   return c256 <= c128 ? 256 : 128;
 }
 
+int g_force_gemm_kernel = 0;  // tuning hook: 0 = automatic, 1 = one CTA per tile, 2 = CTA pairs
+
+// CTA-pair kernel: tile width by the same wave model, over sm_count / 2 pairs.
+int pick_bn_pair(int64_t s, int64_t m, int64_t n, int sm_count) {
+  if (g_force_bn == 192 || g_force_bn == 256) return g_force_bn;
+  const int64_t mp = (s + 255) / 256;
+  const double k_steps = static_cast<double>((n + 255) / 256);
+  const int pairs = std::max(1, sm_count / 2);
+  auto cost = [&](int bn, double exposed_epilogue) {
+    const int64_t tiles = mp * ((m + bn - 1) / bn);
+    const int64_t waves = (tiles + pairs - 1) / pairs;
+    return static_cast<double>(waves) * (k_steps + exposed_epilogue) * bn / 256.0;
+  };
+  return cost(192, 0.3) <= cost(256, 3.0) ? 192 : 256;
+}
+
+template <int BN, bool BF>
+cudaError_t launch_pair_kernel(int grid, cudaStream_t stream, const CUtensorMap& ta, const CUtensorMap& tb,
+                               const CUtensorMap& tsfa, const CUtensorMap& tsfb, const CUtensorMap& ty,
+                               const PairParams& p) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(grid));
+  cfg.blockDim = dim3(kPairThreads);
+  cfg.dynamicSmemBytes = PairCfg<BN>::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_mxfp4_pair_kernel<BN, BF>, ta, tb, tsfa, tsfb, ty, p);
+}
+
+batq_status launch_gemm_pair(const void* x_codes, const void* x_sf, const batq_weight* w, int64_t s, void* y,
+                             bool bf, int64_t ldy, cudaStream_t stream, int sm_count, const CUtensorMap& tmap_a,
+                             const CUtensorMap& tmap_y, int64_t m16) {
+  (void)x_codes;
+  CUtensorMap tmap_sfa;
+  batq_status st = make_sf_tmap(&tmap_sfa, x_sf, (s + 127) / 128, w->katoms);
+  if (st != BATQ_OK) return st;
+  const int bn = pick_bn_pair(s, w->m, w->n, sm_count);
+  PairParams p{};
+  p.s = static_cast<int32_t>(s);
+  p.m = static_cast<int32_t>(w->m);
+  p.katoms = w->katoms;
+  p.k_steps = static_cast<int32_t>((w->n + 255) / 256);
+  p.m_pairs = static_cast<int32_t>((s + 255) / 256);
+  p.n_tiles = static_cast<int32_t>((w->m + bn - 1) / bn);
+  p.m16 = static_cast<int32_t>(m16);
+  p.y = y;
+  p.ldy = ldy;
+  const int grid = 2 * std::min(sm_count / 2, p.m_pairs * p.n_tiles);
+  cudaError_t e;
+  if (bn == 256) e = bf ? launch_pair_kernel<256, true>(grid, stream, tmap_a, w->tmap_b128, tmap_sfa, w->tmap_sf, tmap_y, p)
+                        : launch_pair_kernel<256, false>(grid, stream, tmap_a, w->tmap_b128, tmap_sfa, w->tmap_sf, tmap_y, p);
+  else e = bf ? launch_pair_kernel<192, true>(grid, stream, tmap_a, w->tmap_b96, tmap_sfa, w->tmap_sf, tmap_y, p)
+              : launch_pair_kernel<192, false>(grid, stream, tmap_a, w->tmap_b96, tmap_sfa, w->tmap_sf, tmap_y, p);
+  if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+  return BATQ_OK;
+}
+
 batq_status launch_gemm(const void* x_codes, const void* x_sf, const batq_weight* w, int64_t s, void* y,
                         int32_t y_dtype, int64_t ldy, cudaStream_t stream) {
   int dev;
@@ -376,6 +453,9 @@ batq_status launch_gemm(const void* x_codes, const void* x_sf, const batq_weight
   const int64_t m16 = w->m / (bf ? 8 : 4) * (bf ? 8 : 4);
   if (st == BATQ_OK && m16 > 0) st = make_y_tmap(&tmap_y, y, s, m16, ldy, bf);
   if (st != BATQ_OK) return st;
+  // CTA pairs need at least two 128-token tiles to pay, and wide enough a layer for their tiles.
+  const bool use_pair = g_force_gemm_kernel == 2 || (g_force_gemm_kernel == 0 && s > 128 && w->m >= 192);
+  if (use_pair) return launch_gemm_pair(x_codes, x_sf, w, s, y, bf, ldy, stream, info->sm_count, tmap_a, tmap_y, m16);
   const int bn = pick_bn(s, w->m, w->n, info->sm_count);
   GemmParams p{};
   p.sfa = static_cast<const uint8_t*>(x_sf);
@@ -696,6 +776,8 @@ batq_status batq_prepare_weight(const batq_transform* t, const void* w_bf16, int
   st = make_codes_tmap(&w->tmap_b256, w->codes, m, n / 2, 256);
   if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b192, w->codes, m, n / 2, 192);
   if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b128, w->codes, m, n / 2, 128);
+  if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b96, w->codes, m, n / 2, 96);
+  if (st == BATQ_OK) st = make_sf_tmap(&w->tmap_sf, w->scales, (m + 127) / 128, w->katoms);
   if (st != BATQ_OK) { delete w; return st; }
   *out = w;
   return BATQ_OK;
@@ -816,6 +898,7 @@ batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w,
 
 void batq_debug_force_tile_width(int32_t bn) { g_force_bn = bn; }
 void batq_debug_force_quantizer(int32_t which) { g_force_quantizer = which; }
+void batq_debug_force_gemm_kernel(int32_t which) { g_force_gemm_kernel = which; }
 void batq_debug_set_gemm_flags(int32_t flags) { g_gemm_debug_flags = flags; }
 void batq_debug_force_small_s_splits(int32_t splits) { g_force_splits = splits; }
 

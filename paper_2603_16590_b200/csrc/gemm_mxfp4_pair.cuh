@@ -1,0 +1,313 @@
+// MXFP4 x MXFP4 block-scaled GEMM on CTA pairs (stage 3, prefill shapes).
+//
+//   Y[s, m] = sum_j 2^(ex[s,j] + ew[m,j]) * sum_{i<32} qx[s,j,i] * qw[m,j,i]
+//
+// the low-bit matrix multiplication Q(XP) Q(P^-1 W^T) of the paper's Sec. 3.
+//
+// Same pipeline as gemm_mxfp4.cuh, but two CTAs on the two SMs of a pair (a cluster of 2) share
+// one 256 x BN output tile: each CTA owns 128 token rows (its A tile, its accumulator rows in
+// its own tensor memory) and stages only half of the BN weight rows; one thread of the leader
+// CTA issues tcgen05.mma.cta_group::2, which reads A and the two halves of B from both shared
+// memories.  Per CTA and K-step that is 16 KiB + BN/2 * 128 B instead of 16 KiB + BN * 128 B:
+// less traffic from L2, less shared-memory read bandwidth per MMA, and room for a deeper ring.
+//
+//   leader (cluster rank 0): rows [m0, m0+128),      weight rows [n0, n0+BN/2)
+//   peer   (cluster rank 1): rows [m0+128, m0+256),  weight rows [n0+BN/2, n0+BN)
+//
+// Barriers.  full[stage] lives in the leader and counts the bytes of both CTAs' loads (the
+// peer's TMA loads name the leader's barrier); empty[stage] and acc_full[] exist in both CTAs
+// and are signalled by the leader's tcgen05.commit with a CTA mask; acc_empty[] lives in the
+// leader and collects the epilogue warps of both CTAs.  No load carries a multicast qualifier.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "gemm_mxfp4.cuh"
+#include "ptx.cuh"
+
+namespace batq {
+
+constexpr int kPairThreads = 192;
+
+template <int BN>
+struct PairCfg {
+  static constexpr int kABytes = kBM * kBKBytes;          // 16 KiB: this CTA's 128 token rows
+  static constexpr int kBBytes = (BN / 2) * kBKBytes;     // this CTA's half of the weight rows
+  static constexpr int kSfaBytes = 1024;                  // 128 rows x 8 blocks
+  static constexpr int kSfbAtoms = 2;                     // 128-row scale tiles a BN-wide tile can touch
+  static constexpr int kSfbBytes = kSfbAtoms * 1024;
+  static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
+  static constexpr int kStages = 5;
+  static constexpr int kAccStages = (BN == 256) ? 1 : 2;
+  static constexpr int kAccCols = BN * kAccStages;
+  static constexpr int kSfColsPerStage = 8 + 2 * 4 * kSfbAtoms;
+  static constexpr int kTmemCols = 512;
+  static constexpr int kStagingBufs = (BN == 256) ? 1 : 2;
+  static constexpr int kStagingBytes = 4 * kStagingBufs * 4096;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kStagingBytes + 1024;
+  static_assert(BN == 192 || BN == 256, "tile width");
+  static_assert(kAccCols + kStages * kSfColsPerStage <= kTmemCols, "tensor memory budget");
+  static_assert(kSmemBytes <= 232448, "shared memory budget");
+  static_assert(kStageBytes % 1024 == 0, "stage alignment");
+};
+
+struct PairParams {
+  int32_t s;            // rows of X (tokens)
+  int32_t m;            // rows of W (output features)
+  int32_t katoms;       // KA = 2*ceil(k/8): 512-byte scale atoms per 128-row tile
+  int32_t k_steps;      // ceil(n / 256)
+  int32_t m_pairs;      // ceil(s / 256)
+  int32_t n_tiles;      // ceil(m / BN)
+  int32_t m16;          // as in GemmParams: columns covered by the TMA store
+  void* y;
+  int64_t ldy;
+};
+
+template <int BN, bool OUT_BF16>
+__global__ void __launch_bounds__(kPairThreads, 1)
+gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                       const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfb,
+                       const __grid_constant__ CUtensorMap tmap_y, const PairParams p) {
+  using Cfg = PairCfg<BN>;
+  extern __shared__ uint8_t pair_smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[Cfg::kStages];   // used in the leader only
+  __shared__ __align__(8) uint64_t empty_bar[Cfg::kStages];  // one set per CTA
+  __shared__ __align__(8) uint64_t acc_full_bar[2];          // one set per CTA
+  __shared__ __align__(8) uint64_t acc_empty_bar[2];         // used in the leader only
+  __shared__ __align__(8) uint64_t drain_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int tid = threadIdx.x;
+  const int warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0);
+  const int lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();          // 0 = leader
+  const int pair = blockIdx.x >> 1;
+  const int n_pairs = gridDim.x >> 1;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(pair_smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* staging = smem + Cfg::kStages * Cfg::kStageBytes;
+
+  if (tid == 0) {
+    for (int i = 0; i < Cfg::kStages; ++i) {
+      mbar_init(smem_u32(&full_bar[i]), 1);
+      mbar_init(smem_u32(&empty_bar[i]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&acc_full_bar[i]), 1);
+      mbar_init(smem_u32(&acc_empty_bar[i]), 8);  // 4 epilogue warps of each CTA
+    }
+    mbar_init(smem_u32(&drain_bar), 1);
+    abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmap_a);
+    tma_prefetch_desc(&tmap_b);
+    tma_prefetch_desc(&tmap_sfa);
+    tma_prefetch_desc(&tmap_sfb);
+    tma_prefetch_desc(&tmap_y);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(&tmem_base_slot), Cfg::kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();  // the other CTA's barriers are initialised before anything signals them
+  tc_fence_after_sync();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  const int total_tiles = p.m_pairs * p.n_tiles;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer (both CTAs)
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t full0_leader = map_to_cta(smem_u32(&full_bar[0]), 0);
+    for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
+      const int mp = tile % p.m_pairs;
+      const int nt = tile / p.m_pairs;
+      const int m0 = mp * 256 + static_cast<int>(rank) * kBM;
+      const int n0 = nt * BN;
+      const int nb0 = n0 + static_cast<int>(rank) * (BN / 2);
+      const int sfa_row0 = (m0 >> 7) * p.katoms;
+      const int sfb_row0 = (n0 >> 7) * p.katoms;
+      for (int kt = 0; kt < p.k_steps; ++kt) {
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag));
+        if (!ok) break;
+        if (elect_one()) {
+          const uint32_t st = smem_base + stage * Cfg::kStageBytes;
+          const uint32_t bar = full0_leader + 8u * stage;
+          if (rank == 0) mbar_arrive_expect_tx(smem_u32(&full_bar[stage]), 2u * Cfg::kStageBytes);
+          tma_load_2d_pair(st, &tmap_a, kt * kBKBytes, m0, bar);
+          tma_load_2d_pair(st + Cfg::kABytes, &tmap_b, kt * kBKBytes, nb0, bar);
+          tma_load_2d_pair(st + Cfg::kABytes + Cfg::kBBytes, &tmap_sfa, 0, sfa_row0 + 2 * kt, bar);
+#pragma unroll
+          for (int rt = 0; rt < Cfg::kSfbAtoms; ++rt)
+            tma_load_2d_pair(st + Cfg::kABytes + Cfg::kBBytes + Cfg::kSfaBytes + rt * 1024, &tmap_sfb, 0,
+                             sfb_row0 + rt * p.katoms + 2 * kt, bar);
+        }
+        if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+      }
+    }
+    if (!ok && lane == 0) {
+      // Given up: the loads of both CTAs are counted on the leader's barriers, so neither CTA can
+      // wait for its own; give the copies already in flight ample time to land instead.
+      const uint64_t t0 = global_timer_ns();
+      while (global_timer_ns() - t0 < 1000000ull) {}
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer (leader CTA only)
+    if (rank == 0) {
+      constexpr uint32_t idesc0 = mxf4_idesc(256, BN);
+      constexpr uint32_t idesc1 = idesc0 | (2u << 29) | (2u << 4);
+      const uint32_t smem_base = smem_u32(smem);
+      const uint64_t ab_desc0 = make_smem_desc(smem_base, 16, 1024, 2);
+      const uint64_t sf_desc0 = make_smem_desc(smem_base + Cfg::kABytes + Cfg::kBBytes, 0, 128, 0);
+      const uint32_t sf_tmem0 = tmem_base + Cfg::kAccCols;
+      const uint32_t full0 = smem_u32(&full_bar[0]);
+      const uint32_t empty0 = smem_u32(&empty_bar[0]);
+
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++it) {
+        const int nt = tile / p.m_pairs;
+        const uint32_t sfb_sub = static_cast<uint32_t>((nt * BN) & 127) >> 5;
+        const int acc = it % Cfg::kAccStages;
+        const uint32_t acc_phase = (it / Cfg::kAccStages) & 1u;
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&acc_empty_bar[acc]), acc_phase ^ 1u, &abort_flag));
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kt = 0; kt < p.k_steps; ++kt) {
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(full0 + 8u * stage, phase, &abort_flag));
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t soff = static_cast<uint32_t>(stage * (Cfg::kStageBytes >> 4));
+          const uint64_t adesc = ab_desc0 + soff;
+          const uint64_t bdesc = adesc + (Cfg::kABytes >> 4);
+          const uint64_t sfd = sf_desc0 + soff;
+          const uint32_t sfa_col = sf_tmem0 + stage * Cfg::kSfColsPerStage;
+          const uint32_t sfb_col = sfa_col + 8 + sfb_sub;
+          if (elect_one()) {
+            tc_cp_32x128b_warpx4_pair(sfa_col, sfd);
+            tc_cp_32x128b_warpx4_pair(sfa_col + 4, sfd + 32);
+#pragma unroll
+            for (int rt = 0; rt < Cfg::kSfbAtoms; ++rt)
+#pragma unroll
+              for (int c = 0; c < 2; ++c)
+                tc_cp_32x128b_warpx4_pair(sfa_col + 8 + c * 4 * Cfg::kSfbAtoms + 4 * rt,
+                                          sfd + ((Cfg::kSfaBytes + rt * 1024 + c * 512) >> 4));
+#pragma unroll
+            for (int kb = 0; kb < 4; ++kb) {
+              const uint32_t c = kb >> 1;
+              const uint32_t sfid = (kb & 1) * 2;
+              tc_mma_mxf4_pair(d_tmem, adesc + 2 * kb, bdesc + 2 * kb, (kb & 1) ? idesc1 : idesc0,
+                               (sfa_col + 4 * c) | (sfid << 30), (sfb_col + c * 4 * Cfg::kSfbAtoms) | (sfid << 30),
+                               (kt | kb) != 0 ? 1u : 0u);
+            }
+            tc_commit_pair(empty0 + 8u * stage, 3);  // frees the stage in both CTAs
+          }
+          if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        if (elect_one()) tc_commit_pair(smem_u32(&acc_full_bar[acc]), 3);
+      }
+      if (lane == 0) {
+        tc_commit_pair_local(smem_u32(&drain_bar));
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(smem_u32(&drain_bar), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
+      }
+      __syncwarp();
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue warps (both CTAs)
+    const int quad = warp & 3;
+    uint8_t* my_staging = staging + quad * (Cfg::kStagingBufs * 4096);
+    constexpr int kChunkCols = OUT_BF16 ? 64 : 32;
+    const uint32_t acc_empty0_leader = map_to_cta(smem_u32(&acc_empty_bar[0]), 0);
+    int buf = 0;
+    int it = 0;
+    for (int tile = pair; tile < total_tiles; tile += n_pairs, ++it) {
+      const int mp = tile % p.m_pairs;
+      const int nt = tile / p.m_pairs;
+      const int acc = it % Cfg::kAccStages;
+      const uint32_t acc_phase = (it / Cfg::kAccStages) & 1u;
+      bool ok = mbar_wait(smem_u32(&acc_full_bar[acc]), acc_phase, &abort_flag);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const int row0 = mp * 256 + static_cast<int>(rank) * kBM + quad * 32;
+      const uint32_t taddr = tmem_base + acc * BN + (static_cast<uint32_t>(quad * 32) << 16);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += kChunkCols) {
+        uint32_t w[32];
+        if (OUT_BF16) {
+          uint32_t r0[32], r1[32];
+          tmem_ld_32x32b_x32(taddr + c0, r0);
+          tmem_ld_32x32b_x32(taddr + c0 + 32, r1);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const __nv_bfloat162 a = __floats2bfloat162_rn(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]));
+            const __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(r1[2 * i]), __uint_as_float(r1[2 * i + 1]));
+            w[i] = *reinterpret_cast<const uint32_t*>(&a);
+            w[16 + i] = *reinterpret_cast<const uint32_t*>(&b);
+          }
+        } else {
+          tmem_ld_32x32b_x32(taddr + c0, w);
+          tmem_ld_wait();
+        }
+        const int col0 = nt * BN + c0;
+        if (p.m16 < p.m && col0 < p.m && col0 + kChunkCols > p.m16 && row0 + lane < p.s) {
+          if (OUT_BF16) {
+            __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(p.y) + static_cast<int64_t>(row0 + lane) * p.ldy + col0;
+#pragma unroll
+            for (int i = 0; i < kChunkCols; ++i)
+              if (col0 + i >= p.m16 && col0 + i < p.m) {
+                const uint32_t word = w[((i >> 5) << 4) + ((i & 31) >> 1)];
+                const uint16_t hv = static_cast<uint16_t>((i & 1) ? (word >> 16) : (word & 0xFFFFu));
+                yp[i] = *reinterpret_cast<const __nv_bfloat16*>(&hv);
+              }
+          } else {
+            float* yp = reinterpret_cast<float*>(p.y) + static_cast<int64_t>(row0 + lane) * p.ldy + col0;
+#pragma unroll
+            for (int i = 0; i < kChunkCols; ++i)
+              if (col0 + i >= p.m16 && col0 + i < p.m) yp[i] = __uint_as_float(w[i]);
+          }
+        }
+        if (lane == 0) bulk_wait_group_read<Cfg::kStagingBufs - 1>();
+        __syncwarp();
+        uint8_t* sb = my_staging + buf * 4096 + lane * 128;
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          *reinterpret_cast<uint4*>(sb + ((q ^ (lane & 7)) << 4)) = make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          if (row0 < p.s && col0 < p.m16) tma_store_2d(&tmap_y, col0, row0, smem_u32(my_staging + buf * 4096));
+          bulk_commit_group();
+        }
+        buf = (buf + 1) % Cfg::kStagingBufs;
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(acc_empty0_leader + 8u * acc);
+    }
+    if (lane == 0) bulk_wait_group<0>();
+  }
+
+  // Neither CTA may leave (or release tensor memory) while the other can still read its shared
+  // memory or signal its barriers.
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, Cfg::kTmemCols);
+  }
+}
+
+}  // namespace batq

@@ -24,6 +24,14 @@ def qmode(request, batq):
     batq.batq_debug_force_quantizer(0)
 
 
+@pytest.fixture(params=[1, 2], ids=["cta", "ctapair"])
+def gkernel(request, batq):
+    """Runs a test once per prefill GEMM kernel (one CTA per tile / CTA pairs)."""
+    batq.batq_debug_force_gemm_kernel(request.param)
+    yield request.param
+    batq.batq_debug_force_gemm_kernel(0)
+
+
 def _mk_transform(batq, t):
     return batq.batq_transform_create(t.n, t.left, t.right, t.clip_lo, t.clip_hi)
 
@@ -239,11 +247,11 @@ def _gemm_case(batq, S, M, N, seed, xb=None, wb=None, out_dtype=torch.float32):
 
 
 GEMM_SHAPES = [(128, 1024, 1024), (128, 128, 256), (1, 8, 32), (77, 200, 96), (300, 520, 3584), (16, 4096, 4096),
-               (260, 384, 512), (129, 257, 2048 + 32)]
+               (260, 384, 512), (129, 257, 2048 + 32), (1000, 1100, 768)]
 
 
 @pytest.mark.parametrize("S,M,N", GEMM_SHAPES)
-def test_gemm_vs_oracle_same_codes(batq, S, M, N):
+def test_gemm_vs_oracle_same_codes(batq, gkernel, S, M, N):
     got, Y, Sabs = _gemm_case(batq, S, M, N, 600 + S)
     assert np.all(np.isfinite(got))
     assert np.all(np.abs(got - Y) <= 1e-3 * Sabs + 1e-30)
@@ -253,7 +261,9 @@ def test_gemm_vs_oracle_same_codes(batq, S, M, N):
 
 @pytest.mark.parametrize("bn", [128, 192, 256])
 @pytest.mark.parametrize("S,M,N", [(300, 520, 3584), (129, 257, 2048 + 32), (260, 1000, 512)])
-def test_gemm_every_tile_width(batq, bn, S, M, N):
+def test_gemm_every_tile_width(batq, gkernel, bn, S, M, N):
+    if gkernel == 2 and bn == 128:
+        pytest.skip("CTA pairs have tile widths 192 and 256")
     batq.batq_debug_force_tile_width(bn)
     try:
         got, Y, Sabs = _gemm_case(batq, S, M, N, 700 + S)
@@ -266,7 +276,7 @@ def test_gemm_every_tile_width(batq, bn, S, M, N):
 
 
 @pytest.mark.parametrize("bn", [128, 192, 256])
-def test_gemm_scale_layout_localising_case_every_tile_width(batq, bn):
+def test_gemm_scale_layout_localising_case_every_tile_width(batq, gkernel, bn):
     batq.batq_debug_force_tile_width(bn)
     try:
         test_gemm_scale_layout_localising_case(batq)
@@ -370,8 +380,10 @@ def test_gemm_small_s_rejects_large_s_and_short_scratch(batq):
 @pytest.mark.parametrize("S,M,N,geometry", [(128, 1024, 1024, "baseline"), (128, 1024, 1024, "paper"),
                                             (50, 136, 544, "baseline"), (4, 1024, 1024, "baseline"),
                                             (1, 4096, 4096, "baseline"), (16, 6144, 4096, "paper"),
-                                            (64, 520, 1024, "baseline"), (65, 520, 1024, "baseline")])
+                                            (64, 520, 1024, "baseline"), (65, 520, 1024, "baseline"),
+                                            (520, 1032, 1024, "baseline")])
 def test_linear_w4a4_vs_oracle(batq, qmode, S, M, N, geometry):
+    # automatic kernel choice: the small-s GEMM up to 64 tokens, one CTA per tile up to 128, CTA pairs above
     xb = synth.make_activations(S, N, synth.BASE_SEED)
     wb = synth.make_weight(M, N, synth.BASE_SEED)
     t = synth.make_transform(N, synth.BASE_SEED, geometry)
