@@ -162,10 +162,6 @@ void batq_debug_force_quantizer(int32_t which);
 /* Test / tuning hook: number of K splits of the small-s GEMM (clamped to the number of
  * 256-element K steps and to 32); 0 restores the automatic choice.  Scratch sizes follow it. */
 void batq_debug_force_small_s_splits(int32_t splits);
-/* Timing experiments only (results become meaningless): bit 0 = the GEMM's producer stops
- * reloading shared-memory stages after the first fill, bit 1 = scale factors are copied to
- * tensor memory only for the first stages.  Isolates load-bound from issue-bound behaviour. */
-void batq_debug_set_gemm_flags(int32_t flags);
 
 /* The whole layer, stages 1+2+3: quantise X into the workspace, then the GEMM.  Up to 64
  * tokens take the small-s GEMM, launched so that its weight stream overlaps the quantiser.

@@ -41,7 +41,6 @@ SIGNATURES = {
     "batq_debug_force_small_s_splits": (None, [_I32]),
     "batq_debug_force_tile_width": (None, [_I32]),
     "batq_debug_force_gemm_kernel": (None, [_I32]),
-    "batq_debug_set_gemm_flags": (None, [_I32]),
     "batq_debug_force_quantizer": (None, [_I32]),
     "batq_linear_workspace_bytes": (_SZ, [_P, _I64]),
     "batq_linear_w4a4": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P, _SZ, _P]),
@@ -223,10 +222,6 @@ def batq_debug_force_gemm_kernel(which: int):
 
 def batq_debug_force_quantizer(which: int):
     load().batq_debug_force_quantizer(which)
-
-
-def batq_debug_set_gemm_flags(flags: int):
-    load().batq_debug_set_gemm_flags(flags)
 
 
 def batq_linear_workspace_bytes(w: Weight, s) -> int:

@@ -360,7 +360,6 @@ batq_status make_y_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_
 // accumulator.  Pick by modelled time: waves x (main loop + exposed epilogue), with the main
 // loop proportional to the tile width.
 int g_force_bn = 0;  // test hook: 0 = automatic
-int g_gemm_debug_flags = 0;
 int pick_bn(int64_t s, int64_t m, int64_t n, int sm_count) {
   if (g_force_bn == 128 || g_force_bn == 192 || g_force_bn == 256) return g_force_bn;
   const int64_t mt = (s + kBM - 1) / kBM;
@@ -393,7 +392,7 @@ int pick_bn_pair(int64_t s, int64_t m, int64_t n, int sm_count) {
 }
 
 template <int BN, bool BF>
-cudaError_t launch_pair_kernel(int grid, cudaStream_t stream, const CUtensorMap& ta, const CUtensorMap& tb,
+cudaError_t launch_pair_kernel(int grid, cudaStream_t stream, bool dependent, const CUtensorMap& ta, const CUtensorMap& tb,
                                const CUtensorMap& tsfa, const CUtensorMap& tsfb, const CUtensorMap& ty,
                                const PairParams& p) {
   cudaLaunchConfig_t cfg{};
@@ -401,19 +400,21 @@ cudaError_t launch_pair_kernel(int grid, cudaStream_t stream, const CUtensorMap&
   cfg.blockDim = dim3(kPairThreads);
   cfg.dynamicSmemBytes = PairCfg<BN>::kSmemBytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = dependent ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, gemm_mxfp4_pair_kernel<BN, BF>, ta, tb, tsfa, tsfb, ty, p);
 }
 
 batq_status launch_gemm_pair(const void* x_codes, const void* x_sf, const batq_weight* w, int64_t s, void* y,
                              bool bf, int64_t ldy, cudaStream_t stream, int sm_count, const CUtensorMap& tmap_a,
-                             const CUtensorMap& tmap_y, int64_t m16) {
+                             const CUtensorMap& tmap_y, int64_t m16, bool dependent) {
   (void)x_codes;
   CUtensorMap tmap_sfa;
   batq_status st = make_sf_tmap(&tmap_sfa, x_sf, (s + 127) / 128, w->katoms);
@@ -431,16 +432,18 @@ batq_status launch_gemm_pair(const void* x_codes, const void* x_sf, const batq_w
   p.ldy = ldy;
   const int grid = 2 * std::min(sm_count / 2, p.m_pairs * p.n_tiles);
   cudaError_t e;
-  if (bn == 256) e = bf ? launch_pair_kernel<256, true>(grid, stream, tmap_a, w->tmap_b128, tmap_sfa, w->tmap_sf, tmap_y, p)
-                        : launch_pair_kernel<256, false>(grid, stream, tmap_a, w->tmap_b128, tmap_sfa, w->tmap_sf, tmap_y, p);
-  else e = bf ? launch_pair_kernel<192, true>(grid, stream, tmap_a, w->tmap_b96, tmap_sfa, w->tmap_sf, tmap_y, p)
-              : launch_pair_kernel<192, false>(grid, stream, tmap_a, w->tmap_b96, tmap_sfa, w->tmap_sf, tmap_y, p);
+  if (bn == 256) e = bf ? launch_pair_kernel<256, true>(grid, stream, dependent, tmap_a, w->tmap_b128, tmap_sfa, w->tmap_sf, tmap_y, p)
+                        : launch_pair_kernel<256, false>(grid, stream, dependent, tmap_a, w->tmap_b128, tmap_sfa, w->tmap_sf, tmap_y, p);
+  else e = bf ? launch_pair_kernel<192, true>(grid, stream, dependent, tmap_a, w->tmap_b96, tmap_sfa, w->tmap_sf, tmap_y, p)
+              : launch_pair_kernel<192, false>(grid, stream, dependent, tmap_a, w->tmap_b96, tmap_sfa, w->tmap_sf, tmap_y, p);
   if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
   return BATQ_OK;
 }
 
+// `dependent`: the kernel directly before this one on the stream is the activation quantiser of
+// the same layer; the GEMM is then launched as its programmatic dependent.
 batq_status launch_gemm(const void* x_codes, const void* x_sf, const batq_weight* w, int64_t s, void* y,
-                        int32_t y_dtype, int64_t ldy, cudaStream_t stream) {
+                        int32_t y_dtype, int64_t ldy, cudaStream_t stream, bool dependent = false) {
   int dev;
   const DeviceInfo* info;
   batq_status st = device_setup(&dev, &info);
@@ -455,7 +458,7 @@ batq_status launch_gemm(const void* x_codes, const void* x_sf, const batq_weight
   if (st != BATQ_OK) return st;
   // CTA pairs need at least two 128-token tiles to pay, and wide enough a layer for their tiles.
   const bool use_pair = g_force_gemm_kernel == 2 || (g_force_gemm_kernel == 0 && s > 128 && w->m >= 192);
-  if (use_pair) return launch_gemm_pair(x_codes, x_sf, w, s, y, bf, ldy, stream, info->sm_count, tmap_a, tmap_y, m16);
+  if (use_pair) return launch_gemm_pair(x_codes, x_sf, w, s, y, bf, ldy, stream, info->sm_count, tmap_a, tmap_y, m16, dependent);
   const int bn = pick_bn(s, w->m, w->n, info->sm_count);
   GemmParams p{};
   p.sfa = static_cast<const uint8_t*>(x_sf);
@@ -470,15 +473,25 @@ batq_status launch_gemm(const void* x_codes, const void* x_sf, const batq_weight
   p.m16 = static_cast<int32_t>(m16);
   p.y = y;
   p.ldy = ldy;
-  p.debug_flags = g_gemm_debug_flags;
   const int grid = std::min(info->sm_count, p.m_tiles * p.n_tiles);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(grid));
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = dependent ? 1 : 0;
+  cudaError_t e;
 #define BATQ_GEMM(BN, BF, TB) \
-  gemm_mxfp4_kernel<BN, BF><<<grid, kGemmThreads, GemmCfg<BN>::kSmemBytes, stream>>>(tmap_a, TB, tmap_y, p)
-  if (bn == 256) { if (bf) BATQ_GEMM(256, true, w->tmap_b256); else BATQ_GEMM(256, false, w->tmap_b256); }
-  else if (bn == 192) { if (bf) BATQ_GEMM(192, true, w->tmap_b192); else BATQ_GEMM(192, false, w->tmap_b192); }
-  else { if (bf) BATQ_GEMM(128, true, w->tmap_b128); else BATQ_GEMM(128, false, w->tmap_b128); }
+  (cfg.dynamicSmemBytes = GemmCfg<BN>::kSmemBytes, cudaLaunchKernelEx(&cfg, gemm_mxfp4_kernel<BN, BF>, tmap_a, TB, tmap_y, p))
+  if (bn == 256) e = bf ? BATQ_GEMM(256, true, w->tmap_b256) : BATQ_GEMM(256, false, w->tmap_b256);
+  else if (bn == 192) e = bf ? BATQ_GEMM(192, true, w->tmap_b192) : BATQ_GEMM(192, false, w->tmap_b192);
+  else e = bf ? BATQ_GEMM(128, true, w->tmap_b128) : BATQ_GEMM(128, false, w->tmap_b128);
 #undef BATQ_GEMM
-  return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
+  if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+  return BATQ_OK;
 }
 
 // ---- small-s (decode) GEMM: split choice, scratch layout, launch -------------------------------
@@ -871,7 +884,7 @@ batq_status batq_linear_w4a4(const batq_transform* t, const batq_weight* w, cons
   }
   st = launch_quantize(t, x_bf16, s, w->n, ld, codes, sf, BATQ_SF_MMA, nullptr, cs);
   if (st != BATQ_OK) return st;
-  return launch_gemm(codes, sf, w, s, y, y_dtype, ldy, cs);
+  return launch_gemm(codes, sf, w, s, y, y_dtype, ldy, cs, true);
 }
 
 batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w, const void* x_host, int64_t s,
@@ -899,7 +912,6 @@ batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w,
 void batq_debug_force_tile_width(int32_t bn) { g_force_bn = bn; }
 void batq_debug_force_quantizer(int32_t which) { g_force_quantizer = which; }
 void batq_debug_force_gemm_kernel(int32_t which) { g_force_gemm_kernel = which; }
-void batq_debug_set_gemm_flags(int32_t flags) { g_gemm_debug_flags = flags; }
 void batq_debug_force_small_s_splits(int32_t splits) { g_force_splits = splits; }
 
 size_t batq_static_workspace_capacity(void) { return BATQ_STATIC_WORKSPACE_BYTES - 1024; }

@@ -64,7 +64,6 @@ struct GemmParams {
   int32_t m16;
   void* y;
   int64_t ldy;
-  int32_t debug_flags;  // timing experiments only: 1 = reuse resident stages (no reloads), 2 = skip scale copies
 };
 
 // Instruction descriptor of tcgen05.mma kind::mxf4.block_scale:
@@ -133,6 +132,7 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     int issued = 0;
     bool ok = true;
     const uint32_t smem_base = smem_u32(smem);
+    grid_dependency_wait();  // the quantised activations come from the kernel before this one
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int mt = tile % p.m_tiles;
       const int nt = tile / p.m_tiles;
@@ -145,9 +145,7 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         if (!ok) break;
         const uint32_t st = smem_base + stage * Cfg::kStageBytes;
         const uint32_t bar = smem_u32(&full_bar[0]) + 8u * stage;
-        if ((p.debug_flags & 1) && issued >= Cfg::kStages) {  // timing experiment: stage already resident
-          if (elect_one()) mbar_arrive(bar);
-        } else if (elect_one()) {
+        if (elect_one()) {
           mbar_arrive_expect_tx(bar, Cfg::kTxBytes);
           tma_load_2d(st, &tmap_a, kt * kBKBytes, m0, bar);
           tma_load_2d(st + Cfg::kABytes, &tmap_b, kt * kBKBytes, n0, bar);
@@ -205,8 +203,6 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     uint32_t phase = 0;
     int it = 0;
     bool ok = true;
-    const bool skip_sf = (p.debug_flags & 2) != 0;
-    int64_t step = 0;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
       const int nt = tile / p.m_tiles;
       const uint32_t sfb_sub = static_cast<uint32_t>((nt * BN) & 127) >> 5;  // tile starts mid-atom (BN = 192)
@@ -216,11 +212,11 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t d_tmem = tmem_base + acc * BN;
-      for (int kt = 0; kt < p.k_steps; ++kt, ++step) {
+      for (int kt = 0; kt < p.k_steps; ++kt) {
         ok = __all_sync(0xFFFFFFFFu, mbar_wait(full0 + 8u * stage, phase, &abort_flag));
         if (!ok) break;
         tc_fence_after_sync();
-        if (!skip_sf || step < Cfg::kStages) copy_scales(stage);
+        copy_scales(stage);
         const uint32_t soff = static_cast<uint32_t>(stage * (Cfg::kStageBytes >> 4));
         const uint64_t adesc = ab_desc0 + soff;
         const uint64_t bdesc = adesc + (Cfg::kABytes >> 4);

@@ -119,36 +119,54 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer (both CTAs)
-    int stage = 0;
-    uint32_t phase = 0;
     bool ok = true;
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t full0_leader = map_to_cta(smem_u32(&full_bar[0]), 0);
-    for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
+    const int my_tiles = pair < total_tiles ? (total_tiles - pair + n_pairs - 1) / n_pairs : 0;
+    const int my_steps = my_tiles * p.k_steps;
+    // Step g of this pair = K-step g % k_steps of its tile number g / k_steps.  `what`: 1 = the
+    // weight side (B tile half, weight scales; the leader also arms the barrier), 2 = the
+    // activation side (A tile, activation scales), 3 = both.
+    auto issue = [&](int g, int stage, int what) {
+      const int tile = pair + (g / p.k_steps) * n_pairs;
+      const int kt = g % p.k_steps;
       const int mp = tile % p.m_pairs;
       const int nt = tile / p.m_pairs;
       const int m0 = mp * 256 + static_cast<int>(rank) * kBM;
       const int n0 = nt * BN;
-      const int nb0 = n0 + static_cast<int>(rank) * (BN / 2);
-      const int sfa_row0 = (m0 >> 7) * p.katoms;
-      const int sfb_row0 = (n0 >> 7) * p.katoms;
-      for (int kt = 0; kt < p.k_steps; ++kt) {
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag));
-        if (!ok) break;
-        if (elect_one()) {
-          const uint32_t st = smem_base + stage * Cfg::kStageBytes;
-          const uint32_t bar = full0_leader + 8u * stage;
-          if (rank == 0) mbar_arrive_expect_tx(smem_u32(&full_bar[stage]), 2u * Cfg::kStageBytes);
-          tma_load_2d_pair(st, &tmap_a, kt * kBKBytes, m0, bar);
-          tma_load_2d_pair(st + Cfg::kABytes, &tmap_b, kt * kBKBytes, nb0, bar);
-          tma_load_2d_pair(st + Cfg::kABytes + Cfg::kBBytes, &tmap_sfa, 0, sfa_row0 + 2 * kt, bar);
+      const uint32_t st = smem_base + stage * Cfg::kStageBytes;
+      const uint32_t bar = full0_leader + 8u * stage;
+      if (what & 1) {
+        if (rank == 0) mbar_arrive_expect_tx(smem_u32(&full_bar[stage]), 2u * Cfg::kStageBytes);
+        tma_load_2d_pair(st + Cfg::kABytes, &tmap_b, kt * kBKBytes, n0 + static_cast<int>(rank) * (BN / 2), bar);
 #pragma unroll
-          for (int rt = 0; rt < Cfg::kSfbAtoms; ++rt)
-            tma_load_2d_pair(st + Cfg::kABytes + Cfg::kBBytes + Cfg::kSfaBytes + rt * 1024, &tmap_sfb, 0,
-                             sfb_row0 + rt * p.katoms + 2 * kt, bar);
-        }
-        if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+        for (int rt = 0; rt < Cfg::kSfbAtoms; ++rt)
+          tma_load_2d_pair(st + Cfg::kABytes + Cfg::kBBytes + Cfg::kSfaBytes + rt * 1024, &tmap_sfb, 0,
+                           ((n0 >> 7) + rt) * p.katoms + 2 * kt, bar);
       }
+      if (what & 2) {
+        tma_load_2d_pair(st, &tmap_a, kt * kBKBytes, m0, bar);
+        tma_load_2d_pair(st + Cfg::kABytes + Cfg::kBBytes, &tmap_sfa, 0, (m0 >> 7) * p.katoms + 2 * kt, bar);
+      }
+    };
+    // The weights do not depend on the kernel that quantises the activations: fill the ring's
+    // weight side first, then wait for that kernel (programmatic dependent launch; an ordinary
+    // launch does not wait here), then add the activation side.
+    const int prefill = min(my_steps, Cfg::kStages);
+    if (elect_one())
+      for (int g = 0; g < prefill; ++g) issue(g, g, 1);
+    __syncwarp();
+    grid_dependency_wait();
+    if (elect_one())
+      for (int g = 0; g < prefill; ++g) issue(g, g, 2);
+    __syncwarp();
+    int stage = prefill % Cfg::kStages;
+    uint32_t phase = (prefill == Cfg::kStages) ? 1u : 0u;
+    for (int g = prefill; g < my_steps; ++g) {
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag));
+      if (!ok) break;
+      if (elect_one()) issue(g, stage, 3);
+      if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
     }
     if (!ok && lane == 0) {
       // Given up: the loads of both CTAs are counted on the leader's barriers, so neither CTA can

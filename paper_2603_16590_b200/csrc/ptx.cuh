@@ -20,6 +20,13 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 
+// ------------------------------------------------------------------ programmatic dependent launch
+// wait: blocks until the grid this one was launched as a dependent of has completed and its
+// memory is visible (returns at once for an ordinary launch).  launch_dependents: lets the
+// dependent grid start being scheduled before this one has finished.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ------------------------------------------------------------------ mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
@@ -46,26 +53,40 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
+// Same test, but the hardware may park the warp for up to `hint_ns` while the phase is
+// incomplete (it resumes as soon as the phase completes), so a waiting warp does not compete
+// for issue slots and shared-memory bandwidth with the warps that do the work.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
+
 // Bounded wait.  Returns false when the wait was given up: either another
 // thread of the CTA already raised *abort_flag (shared memory), or this wait
 // exceeded kWaitLimitNs, in which case it raises the flag and records the
 // error for the host.  Callers leave their loops and fall through to the
 // kernel's common exit, so tensor memory is always released.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s: ~1000x the longest kernel here
+constexpr uint32_t kParkNs = 20000u;              // longest single park; the limits are checked between parks
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   uint64_t t0 = 0;
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 63u) == 0) {
-      if (*abort_flag) return false;
-      uint64_t now = global_timer_ns();
-      if (t0 == 0) t0 = now;
-      if (now - t0 > kWaitLimitNs) {
-        *abort_flag = 1;
-        atomicExch(&g_device_error, 1);
-        return false;
-      }
+  for (;;) {
+    if (mbar_try_wait_parked(bar, parity, kParkNs)) return true;
+    if (*abort_flag) return false;
+    const uint64_t now = global_timer_ns();
+    if (t0 == 0) t0 = now;
+    if (now - t0 > kWaitLimitNs) {
+      *abort_flag = 1;
+      atomicExch(&g_device_error, 1);
+      return false;
     }
   }
 }

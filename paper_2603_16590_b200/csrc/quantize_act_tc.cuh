@@ -103,6 +103,10 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
   const int tid = threadIdx.x;
   const int warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0);
   const int lane = tid & 31;
+  // A kernel launched as a programmatic dependent of this one (the GEMM of the same layer) may
+  // take over each SM as soon as this grid's CTA there has finished; it still waits for the whole
+  // grid before it reads the codes and scales written here.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(qt_smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* const x_smem = smem;                                             // kQtStages x 32 KiB
   uint8_t* const img_smem = smem + kQtStages * kQtStageBytes;               // 2 x 24 KiB
