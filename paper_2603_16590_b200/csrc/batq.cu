@@ -272,8 +272,8 @@ batq_status launch_quantize_tc(const batq_transform* t, const void* x, int64_t s
   batq_status st = make_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x, n, s, ld * 2, 64, kQtRows,
                                 CU_TENSOR_MAP_SWIZZLE_128B);
   if (st == BATQ_OK && debug_out == nullptr)
-    st = make_tmap_2d(&tmap_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, n / 2, s, n / 2, 16, 32,
-                      CU_TENSOR_MAP_SWIZZLE_NONE);
+    st = make_tmap_2d(&tmap_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, n / 2, s, n / 2, 64, kQtRows,
+                      CU_TENSOR_MAP_SWIZZLE_64B);
   if (st != BATQ_OK) return st;
   if (debug_out == nullptr && layout == BATQ_SF_MMA && p.sf_katoms > p.n_strips) {
     // an odd number of 4-block atoms: keep the padding atom finite
@@ -695,7 +695,7 @@ batq_status batq_quantize_act(const batq_transform* t, const void* x_bf16, int64
   if (scale_layout != BATQ_SF_ROWMAJOR && scale_layout != BATQ_SF_MMA) return BATQ_ERR_UNSUPPORTED;
   if (s == 0) return BATQ_OK;
   if (codes == nullptr || scales == nullptr) return BATQ_ERR_NULL;
-  if (!aligned(codes, 16)) return BATQ_ERR_ALIGN;
+  if (!aligned(codes, 16) || (scale_layout == BATQ_SF_MMA && !aligned(scales, 16))) return BATQ_ERR_ALIGN;
   return launch_quantize(t, x_bf16, s, n, ld, codes, scales, scale_layout, nullptr, static_cast<cudaStream_t>(stream));
 }
 

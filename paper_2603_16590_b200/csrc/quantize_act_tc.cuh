@@ -32,7 +32,8 @@ constexpr int kQtImageBytes = 3 * kQtTermBytes;            // per block
 constexpr int kQtStripImageBytes = kQtGroups * kQtImageBytes;  // 24 KiB
 constexpr int kQtQuantWarps = 16;
 constexpr int kQtThreads = (2 + kQtQuantWarps) * 32;
-constexpr int kQtStagingBytes = kQtQuantWarps * 2 * 512;    // per warp: 2 x (32 rows x 16 bytes)
+constexpr int kQtCodeTileBytes = kQtRows * kQtGroups * 16;  // codes of one unit: 128 rows x 64 bytes
+constexpr int kQtStagingBytes = 2 * kQtCodeTileBytes + 2 * 512;  // two code tiles, two scale atoms
 constexpr int kQtSmemBytes = kQtStages * kQtStageBytes + 2 * kQtStripImageBytes + kQtStagingBytes + 1024;
 constexpr int kQtTmemCols = 256;              // 2 buffers x 4 blocks x 32 columns
 
@@ -74,6 +75,10 @@ __device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src_smem, uint32_t 
                : "memory");
 }
 
+__device__ __forceinline__ void qt_named_barrier_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 __device__ __forceinline__ float fmin3(float a, float b, float c) {
   float d;
   asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -93,6 +98,7 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
   __shared__ __align__(8) uint64_t bars[2 * kQtStages + 8];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
+  __shared__ int go_slot;
   uint64_t* const x_full = bars;                     // [kQtStages]
   uint64_t* const x_empty = bars + kQtStages;        // [kQtStages]
   uint64_t* const p_full = bars + 2 * kQtStages;     // [2]
@@ -110,7 +116,7 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(qt_smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* const x_smem = smem;                                             // kQtStages x 32 KiB
   uint8_t* const img_smem = smem + kQtStages * kQtStageBytes;               // 2 x 24 KiB
-  uint8_t* const staging = img_smem + 2 * kQtStripImageBytes;               // 8 warps x 2 KiB
+  uint8_t* const staging = img_smem + 2 * kQtStripImageBytes;               // 1024-aligned: code tiles, scale atoms
 
   if (tid == 0) {
     for (int i = 0; i < kQtStages; ++i) {
@@ -244,8 +250,6 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
     const int qw = warp - 2;            // 0..15
     const int quad = warp & 3;          // tensor-memory lanes [32 quad, 32 quad + 32)
     const int g = qw >> 2;              // block of the unit this warp quantises
-    uint8_t* my_staging = staging + qw * 1024;
-    int sbuf = 0;
     int it = 0;
     for (int64_t u = u0; u < u1; ++u, ++it) {
       const int64_t strip = u / p.n_row_tiles;
@@ -253,7 +257,9 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
       const int buf = it & 1;
       bool ok = mbar_wait(smem_u32(&d_full[buf]), (it >> 1) & 1u, &abort_flag);
       ok = __all_sync(0xFFFFFFFFu, ok);
-      if (!ok) break;
+      // A warp whose wait gave up may not leave on its own: the sixteen quantiser warps meet at
+      // named barriers below, so they leave together (see `go_slot`).  The debug build has no barriers.
+      if (DEBUG_OUT && !ok) break;
       tc_fence_after_sync();
       const int64_t row = row_tile * kQtRows + quad * 32 + lane;
       const int j = static_cast<int>(strip) * kQtGroups + g;
@@ -314,26 +320,36 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         for (int c = 0; c < 8; ++c) uu[c] = o[8 * r + c] * inv;
         cw[r] = e2m1x8_pack(uu);
       }
-      // codes: 32 rows x 16 bytes per warp -> staging -> TMA store (clips ragged edges)
-      if (lane == 0) bulk_wait_group_read<1>();
-      __syncwarp();
-      *reinterpret_cast<uint4*>(my_staging + sbuf * 512 + lane * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+      // Codes and scale bytes of the whole unit meet in shared memory (128 rows x 64 bytes of codes,
+      // one 512-byte scale atom) and leave as one TMA store and one bulk copy: full 32-byte sectors
+      // instead of 16-byte and 1-byte pieces.
+      const int sb = it & 1;
+      if (qw == 0 && lane == 0) {
+        bulk_wait_group_read<1>();  // the stores of two units ago have read buffer sb
+        go_slot = *static_cast<volatile int*>(&abort_flag) == 0;  // one thread decides for all, published by the barrier
+      }
+      qt_named_barrier_sync(1, kQtQuantWarps * 32);
+      if (!go_slot) break;
+      const int trow = quad * 32 + lane;
+      *reinterpret_cast<uint4*>(staging + sb * kQtCodeTileBytes + trow * 64 + ((g ^ ((trow >> 1) & 3)) << 4)) =
+          make_uint4(cw[0], cw[1], cw[2], cw[3]);
+      const uint8_t sbv = static_cast<uint8_t>(j < p.k ? sbyte : 0);
+      if (p.sf_layout == 0) {
+        if (row < p.s && j < p.k) p.scales[row * p.k + j] = sbv;
+      } else {
+        staging[2 * kQtCodeTileBytes + sb * 512 + lane * 16 + quad * 4 + g] = sbv;
+      }
       fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) {
-        const int yrow = static_cast<int>(row_tile) * kQtRows + quad * 32;
-        if (yrow < p.s && j < p.k) tma_store_2d(&tmap_codes, j * 16, yrow, smem_u32(my_staging + sbuf * 512));
+      qt_named_barrier_sync(1, kQtQuantWarps * 32);
+      if (qw == 0 && lane == 0) {
+        const int yrow = static_cast<int>(row_tile) * kQtRows;
+        tma_store_2d(&tmap_codes, static_cast<int>(strip) * (kQtGroups * 16), yrow, smem_u32(staging + sb * kQtCodeTileBytes));
+        if (p.sf_layout != 0)
+          bulk_s2g(p.scales + (row_tile * p.sf_katoms + strip) * 512, smem_u32(staging + 2 * kQtCodeTileBytes + sb * 512), 512);
         bulk_commit_group();
       }
-      sbuf ^= 1;
-      // scale byte (rows past s are padding of the 128-row atom: harmless, and kept finite)
-      if (p.sf_layout == 0) {
-        if (row < p.s && j < p.k) p.scales[row * p.k + j] = static_cast<uint8_t>(sbyte);
-      } else {
-        p.scales[sf_mma_offset(row, j, p.sf_katoms)] = static_cast<uint8_t>(sbyte);
-      }
     }
-    if (lane == 0) bulk_wait_group<0>();
+    if (qw == 0 && lane == 0) bulk_wait_group<0>();
   }
 
   tc_fence_before_sync();
