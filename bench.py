@@ -206,35 +206,54 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------ CUDA arm
 class Harness:
     """Process-group plumbing shared by the workload kinds: one process per GPU, no data-path
-    collective (token rows are independent, so ranks are replicas on their own batches)."""
+    collective (token rows are independent, so ranks are replicas on their own batches).  The
+    benchmark always uses NCCL on CUDA devices; the "gloo" backend exists so that this plumbing
+    (rank seeds, barrier, max-over-ranks, whole-job aggregation) can be tested on CPU ranks."""
 
-    def __init__(self):
+    def __init__(self, backend="nccl"):
         import torch
         self.torch = torch
         self.rank = int(os.environ.get("RANK", "0"))
         self.world = int(os.environ.get("WORLD_SIZE", "1"))
         self.local = int(os.environ.get("LOCAL_RANK", "0"))
-        if not torch.cuda.is_available():
-            raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
-        torch.cuda.set_device(self.local)
+        self.cuda = backend == "nccl"
+        if self.cuda:
+            if not torch.cuda.is_available():
+                raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+            torch.cuda.set_device(self.local)
+        self.device = torch.device("cuda", self.local) if self.cuda else torch.device("cpu")
         self.dist = None
         if self.world > 1:
             import torch.distributed as dist
-            dist.init_process_group("nccl", device_id=torch.device("cuda", self.local))
+            if self.cuda:
+                dist.init_process_group("nccl", device_id=self.device)
+            else:
+                dist.init_process_group("gloo")
             self.dist = dist
 
+    def rank_seed(self, base):
+        """Weak scaling: every rank draws its own batch."""
+        return base + 1000 * self.rank
+
     def barrier(self):
-        self.torch.cuda.synchronize()
+        if self.cuda:
+            self.torch.cuda.synchronize()
         if self.dist is not None:
             self.dist.barrier()
-        self.torch.cuda.synchronize()
+        if self.cuda:
+            self.torch.cuda.synchronize()
 
     def max_over_ranks(self, ms):
         if self.dist is None:
             return ms
-        t = self.torch.tensor([ms], dtype=self.torch.float64, device="cuda")
+        t = self.torch.tensor([ms], dtype=self.torch.float64, device=self.device)
         self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
         return float(t.item())
+
+    def whole_job_rate(self, units_per_rank_step, steps, ms):
+        """Units all ranks processed per second: every rank did `steps` steps of
+        `units_per_rank_step`, in the max-over-ranks time `ms`."""
+        return units_per_rank_step * steps * self.world / (ms * 1e-3)
 
     def close(self):
         if self.dist is not None:
@@ -277,7 +296,7 @@ def run_ours(args):
     steps = args.steps if args.steps is not None else {"prefill": 5000, "decode": 300, "quant": 100}[kind]
     if args.workload == "cfg3_qwen2vl7b_prefill" and args.steps is None:
         steps = 1200
-    seed = synth.BASE_SEED + 1000 * h.rank  # weak scaling: every rank its own seeded batch
+    seed = h.rank_seed(synth.BASE_SEED)
     ev = lambda: torch.cuda.Event(enable_timing=True)
     line = {"metric": METRIC, "unit": UNIT, "n_gpus": h.world, "steps": steps, "warmup": args.warmup,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "mxfp4", "data": "synthetic"}
@@ -354,7 +373,7 @@ def run_ours(args):
             traffic = GEMM_TRAFFIC["mb_per_step"]
         touched = h2d + d2h + sum(L["n"] * L["m"] * WEIGHT_BYTES_PER_ELEM for L in layers)
         line.update({
-            "value": flops_step * steps * h.world / (ms * 1e-3) / 1e12, "ms_per_step": ms / steps,
+            "value": h.whole_job_rate(flops_step, steps, ms) / 1e12, "ms_per_step": ms / steps,
             "config": {"workload": args.workload, "tokens": S, "projections": [list(p) for p in projs],
                        "transform": "shared 4x4 (x) private 8x8 per 32-group, clip U[0.8,1]", "output": "bf16",
                        "l2": "inputs larger than L2: one step touches %.0f MB" % (touched / 1e6)},
@@ -444,7 +463,7 @@ def run_ours(args):
         h2d = sum(c["S"] * c["L"]["n"] * 2 for c in order)
         d2h = sum(c["S"] * c["L"]["m"] * 2 for c in order)
         line.update({
-            "value": flops_step * steps * h.world / (ms * 1e-3) / 1e12, "ms_per_step": ms / steps,
+            "value": h.whole_job_rate(flops_step, steps, ms) / 1e12, "ms_per_step": ms / steps,
             "config": {"workload": args.workload, "tokens": tokens, "projections": [list(p) for p in projs],
                        "transform": "shared 4x4 (x) private 8x8 per 32-group, clip U[0.8,1]", "output": "bf16",
                        "launch": "one CUDA graph of %d calls per (tokens, projection) case" % copies,
