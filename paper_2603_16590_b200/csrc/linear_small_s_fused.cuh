@@ -1,0 +1,394 @@
+// The whole layer in ONE kernel for a handful of tokens (decode, s <= 16): activation transform
+// + block clip + MXFP4 quantisation fused into the prologue of the small-s GEMM.
+//
+//   x~ = x P (Eq. 1-2, Kronecker form V~ = L^T V R of Algorithm 1), block clip (Eq. 3-4), MXFP4
+//   (Sec. 2), then Y[s, m] = sum_j 2^(ex[s,j] + ew[m,j]) * sum_{i<32} qx[s,j,i] * qw[m,j,i]
+//   (the low-bit matrix multiplication of Sec. 3.2).
+//
+// At these sizes a call is a chain of latencies, not of bandwidths: two kernels (quantiser, GEMM)
+// cost two launches, two prologues and a round trip of the codes through global memory.  Here a
+// CTA owns 128 weight rows and a slice of at most 8 K-steps (2048 channels); while its TMA
+// producer streams the weight slice, the four warps that will later run the epilogue quantise
+// the matching slice of the s activation rows straight into shared memory, in the operand
+// layout the MMA reads (the activations are tiny: every CTA of a K split redoes the same few
+// blocks).  The K splits of a row tile form a thread-block cluster; their partial tiles meet in
+// the leader's view of distributed shared memory and are added in rank order (deterministic; no
+// scratch in global memory, no atomics).
+//
+// Warp roles: warp 0 = TMA producer (weights), warp 1 = MMA issuer and tensor-memory owner,
+// warps 2..5 = activation quantisers, then epilogue.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "gemm_small_s.cuh"
+#include "ptx.cuh"
+#include "quantize_act.cuh"
+
+namespace batq {
+
+constexpr int kFusedThreads = 192;
+constexpr int kFusedTok = 16;        // MMA N: tokens padded to 16
+constexpr int kFusedMaxSteps = 8;    // K-steps per CTA (the slice of X it quantises)
+constexpr int kFusedMaxSplits = 8;   // cluster size (portable limit)
+
+struct FusedCfg {
+  static constexpr int kWBytes = 128 * kBKBytes;            // 16 KiB of weight codes per K-step
+  static constexpr int kSfBytes = 1024;                     // two 512-byte scale atoms (8 blocks)
+  static constexpr int kStageBytes = kWBytes + kSfBytes;    // ring stage: weights only
+  static constexpr int kStages = 5;
+  static constexpr int kXStepBytes = kFusedTok * kBKBytes;  // 2 KiB of activation codes per K-step
+  static constexpr int kXBytes = kFusedMaxSteps * kXStepBytes;
+  static constexpr int kXSfBytes = kFusedMaxSteps * kSfBytes;
+  static constexpr int kSfColsPerStage = 16;                // W: 2 atoms x 4 columns, X: 2 atoms x 4 columns
+  static constexpr int kTmemCols = 128;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kXBytes + kXSfBytes + 1024;
+  static_assert(kFusedTok + kStages * kSfColsPerStage <= kTmemCols, "tensor memory budget");
+  static_assert(2 * (kSmemBytes + 2048) <= 232448, "two CTAs per SM");
+  static_assert(kStageBytes % 1024 == 0, "stage alignment");
+  static_assert(kXBytes >= kFusedTok * 128 * 4, "the partial tile reuses the activation-code region");
+};
+
+struct FusedParams {
+  const uint16_t* x;     // bf16 bits [s x n], row stride ld
+  int64_t ld;
+  int32_t s;             // tokens (<= 16)
+  int32_t n;
+  int32_t k;             // n / 32
+  const float* left;     // [.][16], left_stride floats apart (0 = shared); NULL = identity transform
+  const float* right;    // [.][64]
+  int32_t left_stride;
+  int32_t right_stride;
+  const float* clip_lo;  // [k] or NULL
+  const float* clip_hi;
+  const uint8_t* sfw;    // weight scales, BATQ_SF_MMA layout
+  int32_t m;             // weight rows = output features
+  int32_t katoms;        // 2*ceil(k/8)
+  int32_t k_steps;       // ceil(n / 256)
+  int32_t splits;        // gridDim.y = cluster size along y
+  void* y;               // [s x m] fp32 or bf16, row stride ldy
+  int64_t ldy;
+};
+
+__device__ __forceinline__ float ld_shared_cluster_f32(uint32_t cluster_addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
+  return v;
+}
+
+// One (token, block): 32 bf16 values -> transformed, clipped, quantised: 16 code bytes + scale byte.
+// Same arithmetic as quantize_act_kernel (fp32 fused multiply-adds over the Kronecker form).
+__device__ __forceinline__ void fused_quant_item(const uint16_t* xp, const float* L, const float* R, bool clip,
+                                                 float c_lo, float c_hi, uint32_t (&cw)[4], uint32_t& sbyte) {
+  // All loads of the item first (x: 4 x 16 bytes, R: 16 x 16 bytes, L: 4 x 16 bytes), so that their
+  // latencies overlap: at this size the kernel is a chain of latencies.
+  uint4 q[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) q[i] = __ldg(reinterpret_cast<const uint4*>(xp) + i);
+  float Rr[64], Lr[16];
+  if (L != nullptr) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float4 t = __ldg(reinterpret_cast<const float4*>(R) + i);
+      Rr[4 * i] = t.x; Rr[4 * i + 1] = t.y; Rr[4 * i + 2] = t.z; Rr[4 * i + 3] = t.w;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float4 t = __ldg(reinterpret_cast<const float4*>(L) + i);
+      Lr[4 * i] = t.x; Lr[4 * i + 1] = t.y; Lr[4 * i + 2] = t.z; Lr[4 * i + 3] = t.w;
+    }
+  }
+  float v[4][8];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t w[4] = {q[i].x, q[i].y, q[i].z, q[i].w};
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+      v[i][2 * h] = __uint_as_float(w[h] << 16);
+      v[i][2 * h + 1] = __uint_as_float(w[h] & 0xFFFF0000u);
+    }
+  }
+  float o[4][8];
+  if (L != nullptr) {
+    float U[4][8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        float acc = v[i][0] * Rr[c];
+#pragma unroll
+        for (int cc = 1; cc < 8; ++cc) acc = fmaf(v[i][cc], Rr[cc * 8 + c], acc);
+        U[i][c] = acc;
+      }
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        float acc = Lr[r] * U[0][c];
+#pragma unroll
+        for (int i = 1; i < 4; ++i) acc = fmaf(Lr[4 * i + r], U[i][c], acc);
+        o[r][c] = acc;
+      }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int c = 0; c < 8; ++c) o[i][c] = v[i][c];
+  }
+  float mn = o[0][0], mx = o[0][0];
+#pragma unroll
+  for (int r = 0; r < 4; ++r)
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      mn = fminf(mn, o[r][c]);
+      mx = fmaxf(mx, o[r][c]);
+    }
+  float amax;
+  if (clip) {
+    const float lo = c_lo * mn, hi = c_hi * mx;
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < 8; ++c) o[r][c] = fminf(fmaxf(o[r][c], lo), hi);
+    amax = fmaxf(fabsf(fminf(fmaxf(mn, lo), hi)), fabsf(fminf(fmaxf(mx, lo), hi)));
+  } else {
+    amax = fmaxf(fabsf(mn), fabsf(mx));
+  }
+  // shared scale: byte = max(biased_exponent(amax) - 2, 0) = clamp(floor(log2 amax) - 2) + 127
+  const int ef = static_cast<int>(__float_as_uint(amax) >> 23);
+  const int sb = max(ef - 2, 0);
+  const float inv = __uint_as_float(static_cast<uint32_t>(254 - sb) << 23);
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    float uu[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) uu[c] = o[r][c] * inv;
+    cw[r] = e2m1x8_pack(uu);
+  }
+  sbyte = static_cast<uint32_t>(sb);
+}
+
+template <bool OUT_BF16>
+__global__ void __launch_bounds__(kFusedThreads, 2)
+linear_small_s_fused_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams p) {
+  using Cfg = FusedCfg;
+  extern __shared__ uint8_t fused_smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[Cfg::kStages];
+  __shared__ __align__(8) uint64_t empty_bar[Cfg::kStages];
+  __shared__ __align__(8) uint64_t x_ready_bar;
+  __shared__ __align__(8) uint64_t acc_full_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int tid = threadIdx.x;
+  const int warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0);
+  const int lane = tid & 31;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(fused_smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* const x_codes = smem + Cfg::kStages * Cfg::kStageBytes;  // [step][16 rows x 128 B], 128-byte swizzle
+  uint8_t* const x_sf = x_codes + Cfg::kXBytes;                     // [step][2 atoms x 512 B]
+
+  if (tid == 0) {
+    for (int i = 0; i < Cfg::kStages; ++i) {
+      mbar_init(smem_u32(&full_bar[i]), 1);
+      mbar_init(smem_u32(&empty_bar[i]), 1);
+    }
+    mbar_init(smem_u32(&x_ready_bar), 4);
+    mbar_init(smem_u32(&acc_full_bar), 1);
+    abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmap_w);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_base_slot), Cfg::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  const int rt = blockIdx.x;   // 128-row tile of W
+  const int sp = blockIdx.y;   // K split = rank in the cluster
+  const int kt0 = static_cast<int>(static_cast<int64_t>(p.k_steps) * sp / p.splits);
+  const int kt1 = static_cast<int>(static_cast<int64_t>(p.k_steps) * (sp + 1) / p.splits);
+  const int n_steps = kt1 - kt0;  // 1..kFusedMaxSteps: the host chooses the splits accordingly
+  bool epi_ok = false;
+  uint32_t v[kFusedTok];
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer (weights)
+    const uint32_t smem_base = smem_u32(smem);
+    const uint8_t* sfw_src = p.sfw + static_cast<int64_t>(rt) * p.katoms * 512;
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    int issued = 0;
+    for (int i = 0; i < n_steps; ++i) {
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag));
+      if (!ok) break;
+      if (elect_one()) {
+        const uint32_t st = smem_base + stage * Cfg::kStageBytes;
+        const uint32_t bar = smem_u32(&full_bar[stage]);
+        mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
+        tma_load_2d(st, &tmap_w, (kt0 + i) * kBKBytes, rt * 128, bar);
+        bulk_g2s(st + Cfg::kWBytes, sfw_src + static_cast<int64_t>(kt0 + i) * 1024, 1024, bar);
+      }
+      ++issued;
+      if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+    }
+    if (!ok && lane == 0) {
+      // Given up: let the copies already in flight land before the CTA exits.
+      const int pending = min(issued, Cfg::kStages);
+      for (int i = 0; i < pending; ++i) {
+        if (--stage < 0) { stage = Cfg::kStages - 1; phase ^= 1u; }
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(smem_u32(&full_bar[stage]), phase) && global_timer_ns() - t0 < 100000000ull) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    constexpr uint32_t idesc0 = mxf4_idesc(128, kFusedTok);
+    constexpr uint32_t idesc1 = idesc0 | (2u << 29) | (2u << 4);  // scale byte pair 2 instead of 0
+    const uint32_t smem_base = smem_u32(smem);
+    const uint64_t w_desc0 = make_smem_desc(smem_base, 16, 1024, 2);
+    const uint64_t wsf_desc0 = make_smem_desc(smem_base + Cfg::kWBytes, 0, 128, 0);
+    const uint64_t x_desc0 = make_smem_desc(smem_u32(x_codes), 16, 1024, 2);
+    const uint64_t xsf_desc0 = make_smem_desc(smem_u32(x_sf), 0, 128, 0);
+    const uint32_t sf_tmem0 = tmem_base + kFusedTok;
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&x_ready_bar), 0, &abort_flag));
+    for (int i = 0; i < n_steps && ok; ++i) {
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&full_bar[stage]), phase, &abort_flag));
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint64_t wdesc = w_desc0 + static_cast<uint32_t>(stage * (Cfg::kStageBytes >> 4));
+      const uint64_t wsfd = wsf_desc0 + static_cast<uint32_t>(stage * (Cfg::kStageBytes >> 4));
+      const uint64_t xdesc = x_desc0 + static_cast<uint32_t>(i * (Cfg::kXStepBytes >> 4));
+      const uint64_t xsfd = xsf_desc0 + static_cast<uint32_t>(i * (Cfg::kSfBytes >> 4));
+      const uint32_t sfw_col = sf_tmem0 + stage * Cfg::kSfColsPerStage;
+      const uint32_t sfx_col = sfw_col + 8;
+      if (elect_one()) {
+        tc_cp_32x128b_warpx4(sfw_col, wsfd);
+        tc_cp_32x128b_warpx4(sfw_col + 4, wsfd + 32);
+        tc_cp_32x128b_warpx4(sfx_col, xsfd);
+        tc_cp_32x128b_warpx4(sfx_col + 4, xsfd + 32);
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+          const uint32_t c = kb >> 1;
+          const uint32_t sfid = (kb & 1) * 2;
+          tc_mma_mxf4(tmem_base, wdesc + 2 * kb, xdesc + 2 * kb, (kb & 1) ? idesc1 : idesc0,
+                      (sfw_col + 4 * c) | (sfid << 30), (sfx_col + 4 * c) | (sfid << 30), (i | kb) != 0 ? 1u : 0u);
+        }
+        tc_commit(smem_u32(&empty_bar[stage]));
+      }
+      if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+    }
+    if (lane == 0) {
+      // Arrives when every MMA issued above is done -- also on the give-up path, so that the
+      // tensor memory is idle before it is released.
+      tc_commit(smem_u32(&acc_full_bar));
+      if (!ok) {
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(smem_u32(&acc_full_bar), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---------------------------------------------------------------- activation quantisers, then epilogue
+    const int qt = tid - 64;                 // 0..127
+    const int nb = n_steps * 8;              // blocks of this CTA's K slice
+    const bool clip = p.clip_lo != nullptr;
+    for (int item = qt; item < p.s * nb; item += 128) {
+      const int t = item / nb;
+      const int jj = item - t * nb;
+      const int j = kt0 * 8 + jj;
+      uint32_t cw[4] = {0u, 0u, 0u, 0u};
+      uint32_t sbyte = 0u;                   // blocks past the last channel: zero codes, finite scale
+      if (j < p.k) {
+        const float* L = p.left ? p.left + static_cast<int64_t>(j) * p.left_stride : nullptr;
+        const float* R = p.left ? p.right + static_cast<int64_t>(j) * p.right_stride : nullptr;
+        fused_quant_item(p.x + t * p.ld + static_cast<int64_t>(j) * 32, L, R, clip, clip ? __ldg(p.clip_lo + j) : 1.0f,
+                         clip ? __ldg(p.clip_hi + j) : 1.0f, cw, sbyte);
+      }
+      const int step = jj >> 3, c = jj & 7;
+      *reinterpret_cast<uint4*>(x_codes + step * Cfg::kXStepBytes + t * 128 + ((c ^ (t & 7)) << 4)) =
+          make_uint4(cw[0], cw[1], cw[2], cw[3]);
+      x_sf[step * Cfg::kSfBytes + (c >> 2) * 512 + t * 16 + (c & 3)] = static_cast<uint8_t>(sbyte);
+    }
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&x_ready_bar));
+
+    mbar_wait(smem_u32(&acc_full_bar), 0, &abort_flag);
+    // A wait that gave up has raised abort_flag before this barrier, so the four warps agree.
+    named_barrier_sync(1, 128);
+    epi_ok = *static_cast<volatile int*>(&abort_flag) == 0;
+    if (epi_ok) {
+      tc_fence_after_sync();
+      const int quad = warp & 3;  // tensor-memory lanes [32*quad, 32*quad + 32)
+      tmem_ld_32x32b_x16(tmem_base + (static_cast<uint32_t>(quad * 32) << 16), v);
+      tmem_ld_wait();
+      tc_fence_before_sync();
+      if (p.splits > 1) {
+        // every MMA has completed: the activation-code region is free and takes the partial tile
+        float* part = reinterpret_cast<float*>(x_codes);
+        const int row = quad * 32 + lane;
+#pragma unroll
+        for (int t = 0; t < kFusedTok; ++t)
+          if (t < p.s) part[t * 128 + row] = __uint_as_float(v[t]);
+      }
+    }
+  }
+
+  // The K splits of this row tile (one cluster) exchange their partial tiles.  Every thread of
+  // every CTA takes both barriers, whatever happened above, so none can wait for ever.
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp >= 2 && sp == 0 && epi_ok) {
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;
+    const int64_t mrow = static_cast<int64_t>(rt) * 128 + row;
+    if (p.splits > 1) {
+      const uint32_t mine = smem_u32(x_codes) + row * 4;
+#pragma unroll
+      for (int t0 = 0; t0 < kFusedTok; t0 += 4) {
+        if (t0 < p.s) {
+          float part[kFusedMaxSplits - 1][4];
+#pragma unroll
+          for (int q = 1; q < kFusedMaxSplits; ++q)
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+              part[q - 1][t] = (q < p.splits && t0 + t < p.s)
+                                   ? ld_shared_cluster_f32(map_to_cta(mine + (t0 + t) * 512, q)) : 0.0f;
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            float acc = __uint_as_float(v[t0 + t]);  // rank 0's own part, then ranks 1.. in order
+#pragma unroll
+            for (int q = 1; q < kFusedMaxSplits; ++q) acc += part[q - 1][t];
+            v[t0 + t] = __float_as_uint(acc);
+          }
+        }
+      }
+    }
+    if (mrow < p.m) {
+#pragma unroll
+      for (int t = 0; t < kFusedTok; ++t) {
+        if (t < p.s) {
+          if (OUT_BF16)
+            reinterpret_cast<__nv_bfloat16*>(p.y)[t * p.ldy + mrow] = __float2bfloat16_rn(__uint_as_float(v[t]));
+          else
+            reinterpret_cast<float*>(p.y)[t * p.ldy + mrow] = __uint_as_float(v[t]);
+        }
+      }
+    }
+  }
+  cluster_sync_all();  // the leader has read everybody's shared memory
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, Cfg::kTmemCols);
+  }
+}
+
+}  // namespace batq

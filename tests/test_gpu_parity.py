@@ -405,6 +405,47 @@ def test_linear_w4a4_vs_oracle(batq, qmode, S, M, N, geometry):
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) < 0.5
 
 
+@pytest.mark.parametrize("S,M,N,geometry", [(1, 4096, 4096, "baseline"), (4, 6144, 4096, "paper"), (16, 1032, 2048, "baseline"),
+                                            (3, 136, 544, "naive"), (2, 264, 14336, "baseline"), (5, 520, 1024, None)])
+@pytest.mark.parametrize("splits", [0, 2])
+def test_linear_fused_small_s_vs_oracle(batq, S, M, N, geometry, splits):
+    """The single-kernel path (activations quantised inside the GEMM kernel) against the oracle
+    and against the two-kernel path."""
+    xb = synth.make_activations(S, N, synth.BASE_SEED + S)
+    wb = synth.make_weight(M, N, synth.BASE_SEED + S)
+    t = synth.make_transform(N, synth.BASE_SEED + S, geometry) if geometry else None
+    tr = _mk_transform(batq, t) if t else None
+    w = batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(wb))
+    x = batq.bits_to_cuda_bf16(xb)
+    outs = {}
+    batq.batq_debug_force_small_s_splits(splits)
+    try:
+        for path in (1, 2):
+            batq.batq_debug_force_small_s_path(path)
+            ws = batq.aligned_workspace(batq.batq_linear_workspace_bytes(w, S))
+            y = torch.full((S + 1, M + 8), float("nan"), dtype=torch.float32, device="cuda")
+            for _ in range(2):
+                batq.batq_linear_w4a4(tr, w, x, y[:S, :M], ws)
+            yb = torch.empty((S, M), dtype=torch.bfloat16, device="cuda")
+            batq.batq_linear_w4a4(tr, w, x, yb, ws)
+            assert batq.batq_last_device_status() == 0
+            yh = y.cpu().numpy()
+            assert np.isnan(yh[S]).all() and np.isnan(yh[:S, M:]).all(), "wrote outside [S x M]"
+            outs[path] = yh[:S, :M].astype(np.float64)
+            assert torch.equal(yb, y[:S, :M].bfloat16())
+    finally:
+        batq.batq_debug_force_small_s_path(0)
+        batq.batq_debug_force_small_s_splits(0)
+    L, R = (t.left, t.right) if t else (None, None)
+    Y, Sabs, _, _ = O.linear_w4a4(xb, wb, L, R, t.clip_lo if t else None, t.clip_hi if t else None)
+    for got in outs.values():
+        assert np.all(np.isfinite(got))
+        assert np.mean(np.abs(got - Y) > 1e-3 * Sabs + 1e-30) <= 1e-3
+        assert np.linalg.norm(got - Y) <= 1e-4 * np.linalg.norm(Sabs)
+    # the two paths round the same fp32 arithmetic; at most a few boundary codes may differ
+    assert np.linalg.norm(outs[1] - outs[2]) <= 1e-4 * np.linalg.norm(Sabs)
+
+
 def test_linear_host_entry_point_matches_device_entry_point(batq):
     S, M, N = 96, 256, 512
     xb = synth.make_activations(S, N, 5)
