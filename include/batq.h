@@ -162,16 +162,18 @@ void batq_debug_force_quantizer(int32_t which);
 /* Test / tuning hook: number of K splits of the small-s GEMM (clamped to the number of
  * 256-element K steps and to 32); 0 restores the automatic choice.  Scratch sizes follow it. */
 void batq_debug_force_small_s_splits(int32_t splits);
-/* Test / tuning hook: how batq_linear_w4a4 runs a handful of tokens.  0 = automatic (up to 4 tokens
- * one fused kernel that quantises the activations inside the GEMM, above that the quantiser
- * kernel followed by the small-s GEMM), 1 = always the two kernels, 2 = the fused kernel up to 16
- * tokens.  The fused kernel needs n <= 16384; other shapes take the two kernels. */
+/* Test / tuning hook: how batq_linear_w4a4 runs a handful of tokens.  0 = automatic (one fused
+ * kernel that quantises the activations inside the GEMM where that is the faster one -- tokens x
+ * K-steps per CTA <= 8 and a grid of one wave --, else the quantiser kernel followed by the small-s
+ * GEMM), 1 = always the two kernels, 2 = the fused kernel up to 16 tokens.  The fused kernel needs
+ * n <= 16384; other shapes take the two kernels. */
 void batq_debug_force_small_s_path(int32_t which);
 
 /* The whole layer, stages 1+2+3: quantise X into the workspace, then the GEMM.  Up to 64
- * tokens take the small-s GEMM, launched so that its weight stream overlaps the quantiser; up to
- * 4 tokens take a single kernel that quantises the activations inside the GEMM (no workspace
- * traffic at all).
+ * tokens take the small-s GEMM, launched so that its weight stream overlaps the quantiser; the
+ * smallest cases take a single kernel that quantises the activations inside the GEMM (no
+ * workspace traffic at all).  Above 64 tokens the GEMM is launched as a programmatic dependent of
+ * the quantiser as well.
  *   workspace  dev, at least batq_linear_workspace_bytes(w, s) bytes, 1024-byte
  *              aligned; overwritten by every call (calls sharing a workspace
  *              must be ordered on one stream). */
