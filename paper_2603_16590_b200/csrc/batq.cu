@@ -391,7 +391,7 @@ int pick_bn_pair(int64_t s, int64_t m, int64_t n, int sm_count) {
     const int64_t waves = (tiles + pairs - 1) / pairs;
     return static_cast<double>(waves) * (k_steps + exposed_epilogue) * bn / 256.0;
   };
-  return cost(192, 0.3) <= cost(256, 3.0) ? 192 : 256;
+  return cost(192, 0.3) <= cost(256, 2.0) ? 192 : 256;
 }
 
 template <int BN, bool BF>
