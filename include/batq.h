@@ -34,7 +34,7 @@ typedef enum {
   BATQ_ERR_NULL = 1,        /* a required pointer is NULL                          */
   BATQ_ERR_SHAPE = 2,       /* n % 32 != 0, a size <= 0, ld < n, sizes too large   */
   BATQ_ERR_ALIGN = 3,       /* pointer not 16-byte aligned, ld % 8 != 0            */
-  BATQ_ERR_UNSUPPORTED = 4, /* factor sizes other than (4,8), dtype, layout, arch  */
+  BATQ_ERR_UNSUPPORTED = 4, /* dtype, layout, architecture                         */
   BATQ_ERR_WORKSPACE = 5,   /* workspace smaller than batq_linear_workspace_bytes  */
   BATQ_ERR_SINGULAR = 6,    /* a transform factor is not invertible                */
   BATQ_ERR_CUDA = 7,        /* a CUDA runtime / driver call failed                 */
@@ -53,7 +53,10 @@ int batq_version(void);
 /* Theta = {A, {B_i}, {alpha_i}} of the paper's algorithm flow ("Store Theta for
  * online activation transformation"), as two Kronecker factors and clip ratios.
  *   n            channels, n % 32 == 0, k = n / 32 blocks.
- *   gr, gc       factor sizes, gr * gc == 32; only (4, 8) is implemented.
+ *   gr, gc       factor sizes, gr * gc == 32: (4, 8) is the paper's default (g2 = 4, g1 = 8);
+ *                (1, 32), (2, 16), (8, 4), (16, 2), (32, 1) cover its ablation of the shared
+ *                factor's size and, as (1, 32) with private right factors, the undecomposed
+ *                32 x 32 block matrices of Table 1's "w/o" row.
  *   left         host fp32, row-major gr x gr matrices: one if left_stride == 0
  *                (shared by all blocks) else k of them, left_stride (= gr*gr)
  *                floats apart.  Acts on the slow index r of a block.

@@ -195,13 +195,14 @@ inline float bf16_to_f32(uint16_t h) {
 void build_block_images(const batq_transform* t, std::vector<uint8_t>* out) {
   out->assign(static_cast<size_t>(t->k) * kQtImageBytes, 0);
   for (int j = 0; j < t->k; ++j) {
-    const float* L = t->left.data() + (t->left_stride ? static_cast<size_t>(j) * 16 : 0);
-    const float* R = t->right.data() + (t->right_stride ? static_cast<size_t>(j) * 64 : 0);
+    const int gr = t->gr, gc = t->gc;
+    const float* L = t->left.data() + (t->left_stride ? static_cast<size_t>(j) * gr * gr : 0);
+    const float* R = t->right.data() + (t->right_stride ? static_cast<size_t>(j) * gc * gc : 0);
     uint8_t* img = out->data() + static_cast<size_t>(j) * kQtImageBytes;
     for (int e = 0; e < 32; ++e)
       for (int f = 0; f < 32; ++f) {
-        const float pv = static_cast<float>(static_cast<double>(L[(e >> 3) * 4 + (f >> 3)]) *
-                                            static_cast<double>(R[(e & 7) * 8 + (f & 7)]));
+        const float pv = static_cast<float>(static_cast<double>(L[(e / gc) * gr + (f / gc)]) *
+                                            static_cast<double>(R[(e % gc) * gc + (f % gc)]));
         const uint16_t hi = bf16_rn(pv);
         const float r1 = pv - bf16_to_f32(hi);
         const uint16_t mid = bf16_rn(r1);
@@ -303,9 +304,19 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
   if (t != nullptr && t->device != dev) return BATQ_ERR_CUDA;
   // The dense-block tensor-core kernel works on 128-token tiles; tiny batches (decode) and the
   // identity transform stay on the ALU kernel.
-  const bool use_tc = n_zero_words == 0 && t != nullptr &&
-                      (g_force_quantizer == 2 || (g_force_quantizer == 0 && s > kSmallSMax));
-  if (use_tc) return launch_quantize_tc(t, x, s, n, ld, codes, scales, layout, debug_out, stream, info->sm_count);
+  // The ALU kernel is written for 4 x 8 factors; every other factorisation of 32 goes through the
+  // tensor-core kernel, which only sees the dense block matrices.
+  const bool only_tc = t != nullptr && (t->gr != 4 || t->gc != 8);
+  const bool use_tc = only_tc || (n_zero_words == 0 && t != nullptr &&
+                                  (g_force_quantizer == 2 || (g_force_quantizer == 0 && s > kSmallSMax)));
+  if (use_tc) {
+    if (n_zero_words > 0 &&
+        cudaMemsetAsync(zero_words, 0, static_cast<size_t>(n_zero_words) * 4, stream) != cudaSuccess) {
+      cudaGetLastError();
+      return BATQ_ERR_CUDA;
+    }
+    return launch_quantize_tc(t, x, s, n, ld, codes, scales, layout, debug_out, stream, info->sm_count);
+  }
   QuantActParams p{};
   p.x = static_cast<const uint16_t*>(x);
   p.ld = ld;
@@ -616,8 +627,9 @@ int pick_fused_splits(int64_t m, int64_t n, int sm_count) {
 // Automatic choice: every CTA of a K split requantises its slice of the activations, which is only
 // hidden behind the weight stream while that is a few items per thread (tokens x K-steps <= 8) and
 // the grid fits the SMs in one wave; measured, the fused kernel then saves 10-20 % of a call.
-bool use_fused_small(const batq_weight* w, int64_t s) {
+bool use_fused_small(const batq_transform* t, const batq_weight* w, int64_t s) {
   if (g_force_small_path == 1 || s > kFusedTok) return false;
+  if (t != nullptr && (t->gr != 4 || t->gc != 8)) return false;  // its in-kernel quantiser is the 4 x 8 form
   const int sp = pick_fused_splits(w->m, w->n, w->sm_count);
   if (sp == 0) return false;
   if (g_force_small_path == 2) return true;
@@ -709,7 +721,6 @@ batq_status batq_transform_create(batq_transform** out, int32_t n, int32_t gr, i
   if (left == nullptr || right == nullptr) return BATQ_ERR_NULL;
   if ((clip_lo == nullptr) != (clip_hi == nullptr)) return BATQ_ERR_NULL;
   if (n <= 0 || n % 32 != 0 || gr <= 0 || gc <= 0 || gr * gc != 32) return BATQ_ERR_SHAPE;
-  if (gr != 4 || gc != 8) return BATQ_ERR_UNSUPPORTED;
   if ((left_stride != 0 && left_stride != gr * gr) || (right_stride != 0 && right_stride != gc * gc)) return BATQ_ERR_SHAPE;
   int dev;
   batq_status st = device_setup(&dev, nullptr);
@@ -721,8 +732,8 @@ batq_status batq_transform_create(batq_transform** out, int32_t n, int32_t gr, i
   t->left_stride = static_cast<int32_t>(left_stride);
   t->right_stride = static_cast<int32_t>(right_stride);
   t->has_clip = clip_lo != nullptr;
-  const size_t nl = left_stride ? static_cast<size_t>(t->k) * 16 : 16;
-  const size_t nr = right_stride ? static_cast<size_t>(t->k) * 64 : 64;
+  const size_t nl = static_cast<size_t>(left_stride ? t->k : 1) * gr * gr;
+  const size_t nr = static_cast<size_t>(right_stride ? t->k : 1) * gc * gc;
   t->left.assign(left, left + nl);
   t->right.assign(right, right + nr);
   t->d_left = t->d_right = t->d_clip_lo = t->d_clip_hi = nullptr;
@@ -822,20 +833,21 @@ batq_status batq_prepare_weight(const batq_transform* t, const void* w_bf16, int
   size_t nl = 0, nr = 0;
   if (t != nullptr) {
     const size_t cl = t->left_stride ? k : 1, cr = t->right_stride ? k : 1;
-    nl = cl * 16; nr = cr * 64;
+    const int gr = t->gr, gc = t->gc;
+    nl = cl * gr * gr; nr = cr * gc * gc;
     std::vector<double> fac(nl + nr);
-    double a[64], inv[64];
+    double a[1024], inv[1024];
     for (size_t i = 0; i < cl; ++i) {
-      for (int e = 0; e < 16; ++e) a[e] = t->left[i * 16 + e];
-      if (!invert_small(a, 4, inv)) return BATQ_ERR_SINGULAR;
-      for (int r = 0; r < 4; ++r)
-        for (int c = 0; c < 4; ++c) fac[i * 16 + r * 4 + c] = inv[c * 4 + r];
+      for (int e = 0; e < gr * gr; ++e) a[e] = t->left[i * gr * gr + e];
+      if (!invert_small(a, gr, inv)) return BATQ_ERR_SINGULAR;
+      for (int r = 0; r < gr; ++r)
+        for (int c = 0; c < gr; ++c) fac[i * gr * gr + r * gr + c] = inv[c * gr + r];
     }
     for (size_t i = 0; i < cr; ++i) {
-      for (int e = 0; e < 64; ++e) a[e] = t->right[i * 64 + e];
-      if (!invert_small(a, 8, inv)) return BATQ_ERR_SINGULAR;
-      for (int r = 0; r < 8; ++r)
-        for (int c = 0; c < 8; ++c) fac[nl + i * 64 + r * 8 + c] = inv[c * 8 + r];
+      for (int e = 0; e < gc * gc; ++e) a[e] = t->right[i * gc * gc + e];
+      if (!invert_small(a, gc, inv)) return BATQ_ERR_SINGULAR;
+      for (int r = 0; r < gc; ++r)
+        for (int c = 0; c < gc; ++c) fac[nl + i * gc * gc + r * gc + c] = inv[c * gc + r];
     }
     if (cudaMalloc(&d_fac, fac.size() * sizeof(double)) != cudaSuccess ||
         cudaMemcpyAsync(d_fac, fac.data(), fac.size() * sizeof(double), cudaMemcpyHostToDevice, cs) != cudaSuccess ||
@@ -859,6 +871,7 @@ batq_status batq_prepare_weight(const batq_transform* t, const void* w_bf16, int
   if (t != nullptr) {
     p.left = d_fac; p.right = d_fac + nl;
     p.left_stride = t->left_stride; p.right_stride = t->right_stride;
+    p.gr = t->gr; p.gc = t->gc;
   }
   p.clip_lo = w_clip_lo; p.clip_hi = w_clip_hi;
   p.codes = w->codes; p.scales = w->scales; p.katoms = w->katoms;
@@ -954,7 +967,7 @@ batq_status batq_linear_w4a4(const batq_transform* t, const batq_weight* w, cons
   uint8_t* codes = static_cast<uint8_t*>(workspace);
   uint8_t* sf = codes + round_up(static_cast<size_t>(s * (w->n / 2)), 1024);
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  if (use_fused_small(w, s)) return launch_linear_fused(t, w, x_bf16, s, ld, y, y_dtype, ldy, cs);
+  if (use_fused_small(t, w, s)) return launch_linear_fused(t, w, x_bf16, s, ld, y, y_dtype, ldy, cs);
   if (s <= kSmallSMax) {
     // A handful of tokens: the quantiser also clears the split-K tickets, and the GEMM is launched
     // as its programmatic dependent so that the weight stream starts while it still runs.

@@ -18,6 +18,7 @@ struct PrepWeightParams {
   const double* right;  // R' = R^-T: [.][64]
   int32_t left_stride;
   int32_t right_stride;
+  int32_t gr, gc;        // factor sizes, gr * gc == 32 (set when left != NULL)
   const float* clip_lo;  // [m x k] or NULL
   const float* clip_hi;
   uint8_t* codes;   // [m x n/2]
@@ -45,46 +46,41 @@ __global__ void __launch_bounds__(128) prepare_weight_kernel(const PrepWeightPar
   const int64_t row = item / p.k;
   const int j = static_cast<int>(item - row * p.k);
   const uint16_t* src = p.w + row * p.ld + static_cast<int64_t>(j) * 32;
-  double v[4][8];
-  for (int r = 0; r < 4; ++r)
-    for (int c = 0; c < 8; ++c)
-      v[r][c] = static_cast<double>(__uint_as_float(static_cast<uint32_t>(src[r * 8 + c]) << 16));
-  double o[4][8];
+  // the block as V[r][c], element r*gc + c (flat arrays: the factor sizes are run-time values)
+  double v[32], o[32];
+  for (int e = 0; e < 32; ++e) v[e] = static_cast<double>(__uint_as_float(static_cast<uint32_t>(src[e]) << 16));
   if (p.left != nullptr) {
+    const int gr = p.gr, gc = p.gc;
     const double* L = p.left + static_cast<int64_t>(j) * p.left_stride;
     const double* R = p.right + static_cast<int64_t>(j) * p.right_stride;
-    double U[4][8];
-    for (int r = 0; r < 4; ++r)
-      for (int c = 0; c < 8; ++c) {
+    double U[32];
+    for (int r = 0; r < gr; ++r)
+      for (int c = 0; c < gc; ++c) {
         double acc = 0.0;
-        for (int cc = 0; cc < 8; ++cc) acc = fma(v[r][cc], R[cc * 8 + c], acc);
-        U[r][c] = acc;
+        for (int cc = 0; cc < gc; ++cc) acc = fma(v[r * gc + cc], R[cc * gc + c], acc);
+        U[r * gc + c] = acc;
       }
-    for (int r = 0; r < 4; ++r)
-      for (int c = 0; c < 8; ++c) {
+    for (int r = 0; r < gr; ++r)
+      for (int c = 0; c < gc; ++c) {
         double acc = 0.0;
-        for (int i = 0; i < 4; ++i) acc = fma(L[i * 4 + r], U[i][c], acc);
-        o[r][c] = acc;
+        for (int i = 0; i < gr; ++i) acc = fma(L[i * gr + r], U[i * gc + c], acc);
+        o[r * gc + c] = acc;
       }
   } else {
-    for (int r = 0; r < 4; ++r)
-      for (int c = 0; c < 8; ++c) o[r][c] = v[r][c];
+    for (int e = 0; e < 32; ++e) o[e] = v[e];
   }
-  double mn = o[0][0], mx = o[0][0];
-  for (int r = 0; r < 4; ++r)
-    for (int c = 0; c < 8; ++c) {
-      mn = fmin(mn, o[r][c]);
-      mx = fmax(mx, o[r][c]);
-    }
+  double mn = o[0], mx = o[0];
+  for (int e = 0; e < 32; ++e) {
+    mn = fmin(mn, o[e]);
+    mx = fmax(mx, o[e]);
+  }
   if (p.clip_lo != nullptr) {
     const double lo = static_cast<double>(p.clip_lo[item]) * mn;
     const double hi = static_cast<double>(p.clip_hi[item]) * mx;
-    for (int r = 0; r < 4; ++r)
-      for (int c = 0; c < 8; ++c) o[r][c] = fmin(fmax(o[r][c], lo), hi);
+    for (int e = 0; e < 32; ++e) o[e] = fmin(fmax(o[e], lo), hi);
   }
   double amax = 0.0;
-  for (int r = 0; r < 4; ++r)
-    for (int c = 0; c < 8; ++c) amax = fmax(amax, fabs(o[r][c]));
+  for (int e = 0; e < 32; ++e) amax = fmax(amax, fabs(o[e]));
   int e = -127;
   if (amax > 0.0) {
     int ex;
@@ -94,7 +90,7 @@ __global__ void __launch_bounds__(128) prepare_weight_kernel(const PrepWeightPar
   uint32_t cw[4];
   for (int r = 0; r < 4; ++r) {
     uint32_t w = 0;
-    for (int c = 0; c < 8; ++c) w |= e2m1_code_f64(scalbn(o[r][c], -e)) << (4 * c);
+    for (int c = 0; c < 8; ++c) w |= e2m1_code_f64(scalbn(o[r * 8 + c], -e)) << (4 * c);
     cw[r] = w;
   }
   *reinterpret_cast<uint4*>(p.codes + row * (p.n / 2) + static_cast<int64_t>(j) * 16) =

@@ -60,7 +60,7 @@ def test_host_validation_without_a_device(lib):
     assert lib.batq_transform_create(C.byref(h), 128, 4, 8, p, 0, p, 0, p, None) == 1
     assert lib.batq_transform_create(C.byref(h), 100, 4, 8, p, 0, p, 0, None, None) == 2
     assert lib.batq_transform_create(C.byref(h), 128, 4, 4, p, 0, p, 0, None, None) == 2
-    assert lib.batq_transform_create(C.byref(h), 128, 8, 4, p, 0, p, 0, None, None) == 4
+    assert lib.batq_transform_create(C.byref(h), 128, 3, 11, p, 0, p, 0, None, None) == 2
     assert lib.batq_transform_create(C.byref(h), 128, 4, 8, p, 5, p, 0, None, None) == 2
     # quantize: shape / alignment / null, checked before any launch
     assert lib.batq_quantize_act(None, 16, 4, 100, 100, 16, 16, 0, None) == 2

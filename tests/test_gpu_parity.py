@@ -33,7 +33,8 @@ def gkernel(request, batq):
 
 
 def _mk_transform(batq, t):
-    return batq.batq_transform_create(t.n, t.left, t.right, t.clip_lo, t.clip_hi)
+    return batq.batq_transform_create(t.n, t.left, t.right, t.clip_lo, t.clip_hi, gr=t.left.shape[1],
+                                      gc=t.right.shape[1])
 
 
 def _gpu_quantize(batq, tr, xb, layout=0, ld=None):
@@ -167,6 +168,53 @@ def test_quantizer_row_stride_and_determinism(batq, qmode):
     c = _gpu_quantize(batq, tr, xb)
     for u, v, w in zip(a, b, c):
         assert np.array_equal(u, v) and np.array_equal(u, w)
+
+
+# ---------------------------------------------------------------------------- other factorisations of the block
+FACTOR_SIZES = [(1, 32), (2, 16), (8, 4), (16, 2), (32, 1)]
+
+
+@pytest.mark.parametrize("gr,gc", FACTOR_SIZES)
+@pytest.mark.parametrize("geometry", ["baseline", "paper", "naive"])
+@pytest.mark.parametrize("S,N", [(3, 96), (130, 1024)])
+def test_quantizer_other_factor_sizes(batq, gr, gc, geometry, S, N):
+    """The paper's ablation of the factor sizes (g1 in {1, 2, 4, 8, 16, 32}); (1, 32) with private
+    right factors is the undecomposed 32 x 32 block matrix."""
+    xb = synth.make_activations(S, N, 250 + S)
+    t = synth.make_transform(N, 12, geometry, gr=gr, gc=gc)
+    tr = _mk_transform(batq, t)
+    vhat = torch.empty((S, N), dtype=torch.float32, device="cuda")
+    batq.batq_debug_transform_clip_f32(tr, batq.bits_to_cuda_bf16(xb), vhat)
+    for layout in (0, 1):
+        gc_, gs = _gpu_quantize(batq, tr, xb, layout=layout)
+        # bit-exact on the GPU's own transformed values ...
+        oc, os_ = O.mxfp4_quantize(vhat.cpu().numpy().astype(np.float64))
+        assert np.array_equal(gs, os_) and np.array_equal(gc_, oc)
+    # ... which are the fp64 transform within the fp32 bound
+    V = O.transform_clip(xb, t.left, t.right, t.clip_lo, t.clip_hi)
+    X = np.abs(O.bf16_bits_to_f64(xb)).reshape(S, N // 32, 32)
+    P = np.abs(O.block_matrices(t.left, t.right, N // 32))
+    bound = FP32_REL * np.einsum("sje,jef->sjf", X, P).reshape(S, N)
+    assert np.all(np.abs(vhat.cpu().numpy().astype(np.float64) - V) <= bound + 1e-300)
+
+
+@pytest.mark.parametrize("gr,gc", FACTOR_SIZES)
+@pytest.mark.parametrize("S", [2, 40, 300])
+def test_linear_other_factor_sizes(batq, gr, gc, S):
+    M, N = 264, 1024
+    xb = synth.make_activations(S, N, 260 + S)
+    wb = synth.make_weight(M, N, 261)
+    t = synth.make_transform(N, 13, "paper", gr=gr, gc=gc)
+    tr = _mk_transform(batq, t)
+    w = batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(wb))
+    ws = batq.aligned_workspace(batq.batq_linear_workspace_bytes(w, S))
+    y = torch.empty((S, M), dtype=torch.float32, device="cuda")
+    batq.batq_linear_w4a4(tr, w, batq.bits_to_cuda_bf16(xb), y, ws)
+    assert batq.batq_last_device_status() == 0
+    got = y.cpu().numpy().astype(np.float64)
+    Y, Sabs, _, _ = O.linear_w4a4(xb, wb, t.left, t.right, t.clip_lo, t.clip_hi)
+    assert np.mean(np.abs(got - Y) > 1e-3 * Sabs + 1e-30) <= 1e-3
+    assert np.linalg.norm(got - Y) <= 1e-4 * np.linalg.norm(Sabs)
 
 
 # ---------------------------------------------------------------------------- weights
