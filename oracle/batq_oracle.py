@@ -175,6 +175,63 @@ def mxfp4_quantize(V: np.ndarray):
     return codes, (e + 127).astype(np.uint8)
 
 
+# ----------------------------------------------------------------------------
+# MXFP8 quantizer (E4M3 elements, Sec. 2: "we adopt E4M3 for MXFP8"), used for
+# 8-bit activations (W4A8) and the 8-bit KV cache
+# ----------------------------------------------------------------------------
+E4M3_EMAX = 8  # 448 = 1.75 * 2**8: exponent of the largest E4M3 magnitude
+
+
+def e4m3_decode(code: np.ndarray) -> np.ndarray:
+    """8-bit code -> real value: 1 sign, 4 exponent (bias 7), 3 mantissa bits;
+    E = 0 holds the subnormals M/8 * 2**-6; E = 15, M = 7 is NaN (no infinities)."""
+    code = np.asarray(code, dtype=np.uint8).astype(np.int64)
+    sgn, E, M = code >> 7, (code >> 3) & 15, code & 7
+    mag = np.where(E == 0, M / 8.0 * 2.0 ** -6, (1.0 + M / 8.0) * np.exp2((E - 7).astype(np.float64)))
+    mag = np.where((E == 15) & (M == 7), np.nan, mag)
+    return np.where(sgn == 1, -mag, mag)
+
+
+def e4m3_round_code(u: np.ndarray) -> np.ndarray:
+    """Round-to-nearest-even of u onto the E4M3 grid, saturating at +-448.  Written as the
+    definition: the nearest of the 127 finite magnitudes; on a tie the one with the even code."""
+    u = np.asarray(u, dtype=np.float64)
+    grid = e4m3_decode(np.arange(127, dtype=np.uint8))   # magnitudes of codes 0..126, increasing
+    mag = np.minimum(np.abs(u), grid[-1])
+    hi = np.clip(np.searchsorted(grid, mag, side="left"), 0, 126)   # first grid point >= mag
+    lo = np.maximum(hi - 1, 0)
+    d_hi, d_lo = grid[hi] - mag, mag - grid[lo]
+    pick_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))
+    code = np.where(pick_hi, hi, lo).astype(np.uint8)
+    return (code | (np.signbit(u).astype(np.uint8) << 7)).astype(np.uint8)
+
+
+def mxfp8_quantize(V: np.ndarray):
+    """Q(V) with E4M3 elements: per 32-block scale byte (e + 127, e = floor(log2 amax) - 8) and
+    one 8-bit code per element.  Returns (codes uint8 [S, N], scale_bytes uint8 [S, k])."""
+    S, N = V.shape
+    k = N // GROUP
+    Vb = V.reshape(S, k, GROUP)
+    amax = np.abs(Vb).max(axis=2)
+    mant, ex = np.frexp(amax)
+    e = np.where(amax == 0.0, -127, ex.astype(np.int64) - 1 - E4M3_EMAX)
+    e = np.clip(e, -127, 127).astype(np.int64)
+    u = Vb / np.exp2(e.astype(np.float64))[:, :, None]
+    return e4m3_round_code(u).reshape(S, N), (e + 127).astype(np.uint8)
+
+
+def quantize_act_mxfp8(x_bits, L, R, c_lo=None, c_hi=None):
+    """Stages 1+2 with 8-bit elements (transform -> clip -> MXFP8)."""
+    return mxfp8_quantize(transform_clip(x_bits, L, R, c_lo, c_hi))
+
+
+def dequantize_mxfp8(codes: np.ndarray, scale_bytes: np.ndarray) -> np.ndarray:
+    S, N = codes.shape
+    k = N // GROUP
+    scale = np.exp2(scale_bytes.astype(np.float64) - 127.0)
+    return (e4m3_decode(codes).reshape(S, k, GROUP) * scale[:, :, None]).reshape(S, N)
+
+
 def pack_codes(codes: np.ndarray) -> np.ndarray:
     """Two codes per byte: element 2i in bits 0-3, element 2i+1 in bits 4-7."""
     c = np.asarray(codes, dtype=np.uint8)

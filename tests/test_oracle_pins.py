@@ -311,3 +311,61 @@ def test_quantized_linear_is_close_to_fp():
     ref = O.bf16_bits_to_f64(xb) @ O.bf16_bits_to_f64(wb).T
     rel = np.linalg.norm(Y - ref) / np.linalg.norm(ref)
     assert rel < 0.35
+
+
+# ---------------------------------------------------------------- E4M3 / MXFP8
+def test_e4m3_decode_against_the_format_definition():
+    """1 sign / 4 exponent (bias 7) / 3 mantissa; the values the OCP format fixes."""
+    d = O.e4m3_decode(np.arange(256, dtype=np.uint8))
+    assert d[0] == 0.0 and d[1] == 2.0 ** -9 and d[7] == 7 * 2.0 ** -9      # subnormals
+    assert d[8] == 2.0 ** -6 and d[0x38] == 1.0 and d[0x40] == 2.0          # normals
+    assert d[0x7E] == 448.0 and np.isnan(d[0x7F]) and np.isnan(d[0xFF])     # largest finite, NaN
+    assert np.array_equal(d[128:255], -d[0:127])
+    assert np.all(np.diff(d[:127]) > 0)                                      # codes ordered like values
+
+
+def test_e4m3_rounding_against_torch_float8():
+    """An independent implementation of the same format: torch's float8_e4m3fn cast
+    (round-to-nearest-even) inside the finite range."""
+    import torch
+    rng = np.random.default_rng(4)
+    u = np.concatenate([rng.uniform(-448, 448, 20000), rng.standard_normal(20000) * 0.01,
+                        rng.standard_normal(5000) * 2.0 ** -8, np.array([0.0, -0.0, 448.0, -448.0, 2.0 ** -10])])
+    u = u.astype(np.float32).astype(np.float64)       # torch casts from fp32
+    want = torch.from_numpy(u.astype(np.float32)).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    got = O.e4m3_round_code(u)
+    assert np.array_equal(got & 0x7F, want & 0x7F)
+    nz = (got & 0x7F) != 0
+    assert np.array_equal(got[nz], want[nz])          # signs (torch may drop the sign of a zero result)
+
+
+def test_e4m3_rounding_properties():
+    codes = np.arange(127, dtype=np.uint8)
+    vals = O.e4m3_decode(codes)
+    assert np.array_equal(O.e4m3_round_code(vals), codes)                    # grid points are fixed points
+    mids = (vals[:-1] + vals[1:]) / 2                                         # exact ties
+    tie = O.e4m3_round_code(mids)
+    assert np.all(tie % 2 == 0) and np.all((tie == codes[:-1]) | (tie == codes[1:]))
+    assert O.e4m3_round_code(np.array([1e9]))[0] == 0x7E and O.e4m3_round_code(np.array([-500.0]))[0] == 0xFE
+    assert O.e4m3_round_code(np.array([-0.0]))[0] == 0x80
+    rng = np.random.default_rng(5)
+    u = np.sort(rng.uniform(-500, 500, 5000))
+    assert np.all(np.diff(O.e4m3_decode(O.e4m3_round_code(u))) >= 0)          # monotone
+
+
+def test_mxfp8_scale_rule_and_error_bound():
+    rng = np.random.default_rng(6)
+    V = rng.standard_normal((40, 128)) * np.exp2(rng.integers(-30, 30, (40, 1)))
+    codes, sb = O.mxfp8_quantize(V)
+    amax = np.abs(V).reshape(40, 4, 32).max(axis=2)
+    r = amax / np.exp2(sb.astype(float) - 127)
+    assert np.all((r >= 256) & (r < 512))            # amax / 2^e in [2^8, 2^9): e = floor(log2 amax) - 8
+    D = O.dequantize_mxfp8(codes, sb)
+    scale = np.repeat(np.exp2(sb.astype(float) - 127), 32, axis=1)
+    u = np.abs(V) / scale
+    ok = u <= 448
+    assert np.all(np.abs(D - V)[ok] <= np.maximum(2.0 ** -4 * np.abs(V)[ok], 2.0 ** -10 * scale[ok]))  # half an ulp
+    assert np.all(np.abs(D)[~ok] == 448 * scale[~ok])                          # (448, 512) saturates
+    z = np.zeros((1, 32)); z[0, 3] = -0.0
+    c, s_ = O.mxfp8_quantize(z)
+    assert s_[0, 0] == 0 and c[0, 3] == 0x80 and c[0, 0] == 0
