@@ -498,7 +498,10 @@ def run_ours(args):
         # written flush buffer would be drained to HBM during the timed launch)
         flush = torch.zeros(256 << 18, dtype=torch.int32, device="cuda")
         torch.cuda.synchronize()
-        variants = [("gpk", True), ("identity", False)]   # T_j = G (x) P_j with clip, and plain MXFP4 (T = I)
+        # T_j = G (x) P_j with clip to MXFP4, plain MXFP4 (T = I), and the transform with 8-bit (E4M3) elements
+        variants = [("gpk", True), ("identity", False), ("gpk_mxfp8", True)]
+        for L in cases:
+            L["codes8"] = torch.empty((L["S"], L["n"]), dtype=torch.uint8, device="cuda")
         marks = [[[(ev(), ev()) for _ in variants] for _ in cases] for _ in range(steps)]
 
         def step(k):
@@ -507,12 +510,15 @@ def run_ours(args):
                     flush.sum()
                     if k is not None:
                         marks[k][i][v][0].record()
-                    B.batq_quantize_act(L["tr"] if xf else None, L["x"], L["codes"], L["sf"], B.SF_MMA)
+                    if v == 2:
+                        B.batq_quantize_act_mxfp8(L["tr"], L["x"], L["codes8"], L["sf"], B.SF_MMA)
+                    else:
+                        B.batq_quantize_act(L["tr"] if xf else None, L["x"], L["codes"], L["sf"], B.SF_MMA)
                     if k is not None:
                         marks[k][i][v][1].record()
 
         ms, clocks = timed_region(h, step, steps, args.warmup)
-        t_ms = np.array([[[m[i][v][0].elapsed_time(m[i][v][1]) for v in range(2)] for i in range(len(cases))]
+        t_ms = np.array([[[m[i][v][0].elapsed_time(m[i][v][1]) for v in range(3)] for i in range(len(cases))]
                          for m in marks]).mean(axis=0)
         bytes_case = np.array([L["S"] * L["n"] * QUANT_BYTES_PER_ELEM for L in cases])
         gbs = bytes_case.sum() / (t_ms[:, 0].sum() * 1e-3) / 1e9
@@ -547,10 +553,13 @@ def run_ours(args):
             "kernels": [{"tokens": L["S"], "hidden": L["n"], "gpk_us": float(t_ms[i, 0] * 1e3),
                          "gpk_gbs": float(bytes_case[i] / (t_ms[i, 0] * 1e-3) / 1e9),
                          "identity_us": float(t_ms[i, 1] * 1e3),
-                         "identity_gbs": float(bytes_case[i] / (t_ms[i, 1] * 1e-3) / 1e9)} for i, L in enumerate(cases)],
+                         "identity_gbs": float(bytes_case[i] / (t_ms[i, 1] * 1e-3) / 1e9),
+                         "mxfp8_us": float(t_ms[i, 2] * 1e3),   # 2 + 1 + 1/32 bytes per element
+                         "mxfp8_gbs": float(L["S"] * L["n"] * 3.03125 / (t_ms[i, 2] * 1e-3) / 1e9)}
+                        for i, L in enumerate(cases)],
             "e2e": {"value": 24.0 * elems * h.world / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
                     "h2d_bytes_per_step": int(elems * 2), "d2h_bytes_per_step": int(elems // 2), "steps": 1},
-            "gpu_launches": 2 * len(cases) * steps,
+            "gpu_launches": 3 * len(cases) * steps,
         })
 
     status = B.batq_last_device_status()

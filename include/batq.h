@@ -98,6 +98,19 @@ batq_status batq_quantize_act(const batq_transform* t, const void* x_bf16, int64
                               int64_t ld, void* codes, void* scales, int32_t scale_layout,
                               void* stream);
 
+/* The same stages with 8-bit elements: MXFP8 with E4M3 codes (Sec. 2: "we adopt E4M3 for MXFP8"),
+ * the activation format of the paper's W4A8 configurations and of the 8-bit KV cache (the key and
+ * value transforms P_k, P_v of Sec. 3.2 are applied head by head: pass the cache as
+ * [tokens * heads x head_dim] with a transform of n = head_dim).  Shared scale
+ * e = floor(log2 amax) - 8, elements round to nearest even and saturate at +-448.
+ *   t        transform (required; an identity transform gives plain MXFP8 of X).
+ *   codes    dev, s * n bytes row-major, one E4M3 code per element.
+ *   scales   as batq_quantize_act.
+ * Errors as batq_quantize_act, plus NULL for t == NULL. */
+batq_status batq_quantize_act_mxfp8(const batq_transform* t, const void* x_bf16, int64_t s, int64_t n,
+                                    int64_t ld, void* codes, void* scales, int32_t scale_layout,
+                                    void* stream);
+
 /* Test hook: the exact fp32 values the quantiser rounds (after transform and
  * clip, before scaling), out dev fp32 [s x n] row-major. */
 batq_status batq_debug_transform_clip_f32(const batq_transform* t, const void* x_bf16, int64_t s,

@@ -30,6 +30,7 @@ SIGNATURES = {
     "batq_transform_destroy": (C.c_int, [_P]),
     "batq_sf_bytes": (_SZ, [_I64, _I64, _I32]),
     "batq_quantize_act": (C.c_int, [_P, _P, _I64, _I64, _I64, _P, _P, _I32, _P]),
+    "batq_quantize_act_mxfp8": (C.c_int, [_P, _P, _I64, _I64, _I64, _P, _P, _I32, _P]),
     "batq_debug_transform_clip_f32": (C.c_int, [_P, _P, _I64, _I64, _I64, _P, _P]),
     "batq_weight_bytes": (_SZ, [_I64, _I64]),
     "batq_prepare_weight": (C.c_int, [_P, _P, _I64, _I64, _I64, _P, _P, _P, C.POINTER(_P), _P]),
@@ -145,6 +146,16 @@ def batq_quantize_act(t, x, codes, scales, scale_layout=SF_ROWMAJOR, ld=None, s=
     st = load().batq_quantize_act(t.handle if t else None, _ptr(x), s, n, ld, _ptr(codes), _ptr(scales),
                                   scale_layout, _stream())
     _check(st, "batq_quantize_act")
+
+
+def batq_quantize_act_mxfp8(t, x, codes, scales, scale_layout=SF_ROWMAJOR, ld=None, s=None, n=None):
+    """As batq_quantize_act with E4M3 codes: codes is a uint8 CUDA buffer of s * n bytes."""
+    s = x.shape[0] if s is None else s
+    n = x.shape[1] if n is None else n
+    ld = x.stride(0) if ld is None else ld
+    st = load().batq_quantize_act_mxfp8(t.handle if t else None, _ptr(x), s, n, ld, _ptr(codes), _ptr(scales),
+                                        scale_layout, _stream())
+    _check(st, "batq_quantize_act_mxfp8")
 
 
 def batq_debug_transform_clip_f32(t, x, out):

@@ -106,6 +106,8 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(quantize_act_tc_kernel<false, false>, kQtSmemBytes);
     e = e ? e : set_smem(quantize_act_tc_kernel<true, true>, kQtSmemBytes);
     e = e ? e : set_smem(quantize_act_tc_kernel<false, true>, kQtSmemBytes);
+    e = e ? e : set_smem(quantize_act_tc_kernel<true, false, true>, kQtSmemBytes);
+    e = e ? e : set_smem(quantize_act_tc_kernel<false, false, true>, kQtSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<256, false>, GemmCfg<256>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<256, true>, GemmCfg<256>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<192, false>, GemmCfg<192>::kSmemBytes);
@@ -256,7 +258,8 @@ int g_force_quantizer = 0;  // tuning hook: 0 = automatic, 1 = ALU (Kronecker fo
 
 // Tensor-core version: 128-token x 4-block units.
 batq_status launch_quantize_tc(const batq_transform* t, const void* x, int64_t s, int64_t n, int64_t ld, void* codes,
-                               void* scales, int32_t layout, float* debug_out, cudaStream_t stream, int sm_count) {
+                               void* scales, int32_t layout, float* debug_out, cudaStream_t stream, int sm_count,
+                               bool fp8 = false) {
   QuantTcParams p{};
   p.s = s;
   p.n = static_cast<int32_t>(n);
@@ -276,8 +279,10 @@ batq_status launch_quantize_tc(const batq_transform* t, const void* x, int64_t s
   batq_status st = make_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x, n, s, ld * 2, 64, kQtRows,
                                 CU_TENSOR_MAP_SWIZZLE_128B);
   if (st == BATQ_OK && debug_out == nullptr)
-    st = make_tmap_2d(&tmap_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, n / 2, s, n / 2, 64, kQtRows,
-                      CU_TENSOR_MAP_SWIZZLE_64B);
+    st = fp8 ? make_tmap_2d(&tmap_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, n, s, n, 128, kQtRows,
+                            CU_TENSOR_MAP_SWIZZLE_128B)
+             : make_tmap_2d(&tmap_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, n / 2, s, n / 2, 64, kQtRows,
+                            CU_TENSOR_MAP_SWIZZLE_64B);
   if (st != BATQ_OK) return st;
   if (debug_out == nullptr && layout == BATQ_SF_MMA && p.sf_katoms > p.n_strips) {
     // an odd number of 4-block atoms: keep the padding atom finite
@@ -286,7 +291,10 @@ batq_status launch_quantize_tc(const batq_transform* t, const void* x, int64_t s
   const int grid = static_cast<int>(std::min<int64_t>(sm_count, p.n_units));
   const bool cl = t->has_clip, dbg = debug_out != nullptr;
 #define BATQ_QT(CL, DB) quantize_act_tc_kernel<CL, DB><<<grid, kQtThreads, kQtSmemBytes, stream>>>(tmap_x, tmap_codes, p)
-  if (cl && !dbg) BATQ_QT(true, false);
+  if (fp8 && !dbg) {
+    if (cl) quantize_act_tc_kernel<true, false, true><<<grid, kQtThreads, kQtSmemBytes, stream>>>(tmap_x, tmap_codes, p);
+    else quantize_act_tc_kernel<false, false, true><<<grid, kQtThreads, kQtSmemBytes, stream>>>(tmap_x, tmap_codes, p);
+  } else if (cl && !dbg) BATQ_QT(true, false);
   else if (!cl && !dbg) BATQ_QT(false, false);
   else if (cl && dbg) BATQ_QT(true, true);
   else BATQ_QT(false, true);
@@ -790,6 +798,25 @@ batq_status batq_quantize_act(const batq_transform* t, const void* x_bf16, int64
   if (codes == nullptr || scales == nullptr) return BATQ_ERR_NULL;
   if (!aligned(codes, 16) || (scale_layout == BATQ_SF_MMA && !aligned(scales, 16))) return BATQ_ERR_ALIGN;
   return launch_quantize(t, x_bf16, s, n, ld, codes, scales, scale_layout, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+batq_status batq_quantize_act_mxfp8(const batq_transform* t, const void* x_bf16, int64_t s, int64_t n, int64_t ld,
+                                    void* codes, void* scales, int32_t scale_layout, void* stream) {
+  batq_status st = check_x(x_bf16, s, n, ld);
+  if (st != BATQ_OK) return st;
+  if (t == nullptr) return BATQ_ERR_NULL;
+  if (t->n != n) return BATQ_ERR_SHAPE;
+  if (scale_layout != BATQ_SF_ROWMAJOR && scale_layout != BATQ_SF_MMA) return BATQ_ERR_UNSUPPORTED;
+  if (s == 0) return BATQ_OK;
+  if (codes == nullptr || scales == nullptr) return BATQ_ERR_NULL;
+  if (!aligned(codes, 16) || (scale_layout == BATQ_SF_MMA && !aligned(scales, 16))) return BATQ_ERR_ALIGN;
+  int dev;
+  const DeviceInfo* info;
+  st = device_setup(&dev, &info);
+  if (st != BATQ_OK) return st;
+  if (t->device != dev) return BATQ_ERR_CUDA;
+  return launch_quantize_tc(t, x_bf16, s, n, ld, codes, scales, scale_layout, nullptr,
+                            static_cast<cudaStream_t>(stream), info->sm_count, true);
 }
 
 batq_status batq_debug_transform_clip_f32(const batq_transform* t, const void* x_bf16, int64_t s, int64_t n,

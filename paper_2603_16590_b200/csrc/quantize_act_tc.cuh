@@ -32,8 +32,9 @@ constexpr int kQtImageBytes = 3 * kQtTermBytes;            // per block
 constexpr int kQtStripImageBytes = kQtGroups * kQtImageBytes;  // 24 KiB
 constexpr int kQtQuantWarps = 16;
 constexpr int kQtThreads = (2 + kQtQuantWarps) * 32;
-constexpr int kQtCodeTileBytes = kQtRows * kQtGroups * 16;  // codes of one unit: 128 rows x 64 bytes
-constexpr int kQtStagingBytes = 2 * kQtCodeTileBytes + 2 * 512;  // two code tiles, two scale atoms
+constexpr int kQtCodeTileBytes = kQtRows * kQtGroups * 16;  // 4-bit codes of one unit: 128 rows x 64 bytes
+constexpr int kQtCodeTileBytes8 = 2 * kQtCodeTileBytes;     // 8-bit codes: 128 rows x 128 bytes
+constexpr int kQtStagingBytes = 2 * kQtCodeTileBytes8 + 2 * 512;  // two code tiles (sized for 8-bit), two scale atoms
 constexpr int kQtSmemBytes = kQtStages * kQtStageBytes + 2 * kQtStripImageBytes + kQtStagingBytes + 1024;
 constexpr int kQtTmemCols = 256;              // 2 buffers x 4 blocks x 32 columns
 
@@ -90,7 +91,21 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   return d;
 }
 
-template <bool CLIP, bool DEBUG_OUT>
+// Four floats -> four E4M3 bytes (round to nearest even, saturating at +-448), first value in byte 0.
+__device__ __forceinline__ uint32_t e4m3x4_pack(float a, float b, float c, float d) {
+  uint32_t w;
+  asm("{\n\t.reg .b16 lo, hi;\n\t"
+      "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n\t"
+      "cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;\n\t"
+      "mov.b32 %0, {lo, hi};\n\t}"
+      : "=r"(w)
+      : "f"(a), "f"(b), "f"(c), "f"(d));
+  return w;
+}
+
+// FP8 = false: MXFP4 (E2M1 codes, two per byte).  FP8 = true: MXFP8 (E4M3 codes, Sec. 2), one byte per
+// element, shared scale e = floor(log2 amax) - 8.
+template <bool CLIP, bool DEBUG_OUT, bool FP8 = false>
 __global__ void __launch_bounds__(kQtThreads, 1)
 quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_codes,
                        const QuantTcParams p) {
@@ -309,20 +324,13 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         }
         continue;
       }
+      // shared scale: byte = max(biased_exponent(amax) - emax, 0), emax = 2 (E2M1) or 8 (E4M3)
       const int ef = static_cast<int>(__float_as_uint(amax) >> 23);
-      const int sbyte = max(ef - 2, 0);
+      const int sbyte = max(ef - (FP8 ? 8 : 2), 0);
       const float inv = __uint_as_float(static_cast<uint32_t>(254 - sbyte) << 23);
-      uint32_t cw[4];
-#pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        float uu[8];
-#pragma unroll
-        for (int c = 0; c < 8; ++c) uu[c] = o[8 * r + c] * inv;
-        cw[r] = e2m1x8_pack(uu);
-      }
-      // Codes and scale bytes of the whole unit meet in shared memory (128 rows x 64 bytes of codes,
-      // one 512-byte scale atom) and leave as one TMA store and one bulk copy: full 32-byte sectors
-      // instead of 16-byte and 1-byte pieces.
+      // Codes and scale bytes of the whole unit meet in shared memory (128 rows x 64 or 128 bytes of
+      // codes, one 512-byte scale atom) and leave as one TMA store and one bulk copy: full 32-byte
+      // sectors instead of 16-byte and 1-byte pieces.
       const int sb = it & 1;
       if (qw == 0 && lane == 0) {
         bulk_wait_group_read<1>();  // the stores of two units ago have read buffer sb
@@ -331,21 +339,45 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
       qt_named_barrier_sync(1, kQtQuantWarps * 32);
       if (!go_slot) break;
       const int trow = quad * 32 + lane;
-      *reinterpret_cast<uint4*>(staging + sb * kQtCodeTileBytes + trow * 64 + ((g ^ ((trow >> 1) & 3)) << 4)) =
-          make_uint4(cw[0], cw[1], cw[2], cw[3]);
+      if (FP8) {
+        uint8_t* tile = staging + sb * kQtCodeTileBytes8 + trow * 128;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          uint32_t cw[4];
+#pragma unroll
+          for (int r = 0; r < 4; ++r)
+            cw[r] = e4m3x4_pack(o[16 * h + 4 * r] * inv, o[16 * h + 4 * r + 1] * inv, o[16 * h + 4 * r + 2] * inv,
+                                o[16 * h + 4 * r + 3] * inv);
+          // 128-byte swizzle: 16-byte chunk index XOR (row & 7)
+          *reinterpret_cast<uint4*>(tile + (((2 * g + h) ^ (trow & 7)) << 4)) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+        }
+      } else {
+        uint32_t cw[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          float uu[8];
+#pragma unroll
+          for (int c = 0; c < 8; ++c) uu[c] = o[8 * r + c] * inv;
+          cw[r] = e2m1x8_pack(uu);
+        }
+        // 64-byte swizzle: 16-byte chunk index XOR ((row / 2) & 3)
+        *reinterpret_cast<uint4*>(staging + sb * kQtCodeTileBytes8 + trow * 64 + ((g ^ ((trow >> 1) & 3)) << 4)) =
+            make_uint4(cw[0], cw[1], cw[2], cw[3]);
+      }
       const uint8_t sbv = static_cast<uint8_t>(j < p.k ? sbyte : 0);
       if (p.sf_layout == 0) {
         if (row < p.s && j < p.k) p.scales[row * p.k + j] = sbv;
       } else {
-        staging[2 * kQtCodeTileBytes + sb * 512 + lane * 16 + quad * 4 + g] = sbv;
+        staging[2 * kQtCodeTileBytes8 + sb * 512 + lane * 16 + quad * 4 + g] = sbv;
       }
       fence_proxy_async_smem();
       qt_named_barrier_sync(1, kQtQuantWarps * 32);
       if (qw == 0 && lane == 0) {
         const int yrow = static_cast<int>(row_tile) * kQtRows;
-        tma_store_2d(&tmap_codes, static_cast<int>(strip) * (kQtGroups * 16), yrow, smem_u32(staging + sb * kQtCodeTileBytes));
+        tma_store_2d(&tmap_codes, static_cast<int>(strip) * (kQtGroups * (FP8 ? 32 : 16)), yrow,
+                     smem_u32(staging + sb * kQtCodeTileBytes8));
         if (p.sf_layout != 0)
-          bulk_s2g(p.scales + (row_tile * p.sf_katoms + strip) * 512, smem_u32(staging + 2 * kQtCodeTileBytes + sb * 512), 512);
+          bulk_s2g(p.scales + (row_tile * p.sf_katoms + strip) * 512, smem_u32(staging + 2 * kQtCodeTileBytes8 + sb * 512), 512);
         bulk_commit_group();
       }
     }

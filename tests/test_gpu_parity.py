@@ -217,6 +217,64 @@ def test_linear_other_factor_sizes(batq, gr, gc, S):
     assert np.linalg.norm(got - Y) <= 1e-4 * np.linalg.norm(Sabs)
 
 
+# ---------------------------------------------------------------------------- MXFP8 activations / KV cache
+@pytest.mark.parametrize("S,N", [(1, 32), (3, 96), (130, 1024), (257, 3584), (300, 4096 + 32)])
+@pytest.mark.parametrize("geometry", ["baseline", "paper"])
+def test_mxfp8_quantizer_vs_oracle(batq, S, N, geometry):
+    xb = synth.make_activations(S, N, 270 + S)
+    t = synth.make_transform(N, 14, geometry)
+    tr = _mk_transform(batq, t)
+    x = batq.bits_to_cuda_bf16(xb)
+    vhat = torch.empty((S, N), dtype=torch.float32, device="cuda")
+    batq.batq_debug_transform_clip_f32(tr, x, vhat)
+    V32 = vhat.cpu().numpy().astype(np.float64)
+    for layout in (0, 1):
+        codes = torch.full((S * N + 64,), 0xEE, dtype=torch.uint8, device="cuda")
+        nsf = batq.batq_sf_bytes(S, N, layout)
+        scales = torch.full((nsf + 64,), 0xEE, dtype=torch.uint8, device="cuda")
+        batq.batq_quantize_act_mxfp8(tr, x, codes, scales, layout)
+        assert batq.batq_last_device_status() == 0
+        c, sc = codes.cpu().numpy(), scales.cpu().numpy()
+        assert (c[S * N:] == 0xEE).all() and (sc[nsf:] == 0xEE).all(), "wrote past the output buffers"
+        gc_ = c[:S * N].reshape(S, N)
+        gs = sc[:nsf].reshape(S, N // 32) if layout == 0 else sf_mma_to_rowmajor(sc[:nsf], S, N // 32)
+        # bit-exact on the GPU's own transformed values
+        oc, os_ = O.mxfp8_quantize(V32)
+        assert np.array_equal(gs, os_) and np.array_equal(gc_, oc)
+    # and close to the fp64 path: neighbouring codes at most, rarely
+    oc64, os64 = O.quantize_act_mxfp8(xb, t.left, t.right, t.clip_lo, t.clip_hi)
+    same = np.repeat(gs == os64, 32, axis=1)
+    assert (gs != os64).mean() <= 1e-4
+    d = np.abs((gc_ & 0x7F).astype(int) - (oc64 & 0x7F).astype(int))
+    assert np.all(d[same] <= 1) and (d[same] != 0).mean() <= 1e-3
+
+
+def test_kv_cache_head_by_head(batq):
+    """Key/value transforms act head by head (Sec. 3.2): the cache [tokens, heads, head_dim] is the
+    matrix [tokens * heads, head_dim] with one transform of n = head_dim; KV4 and KV8."""
+    tokens, heads, hd = 70, 8, 128
+    xb = synth.make_activations(tokens * heads, hd, 31)
+    t = synth.make_transform(hd, 15, "paper")
+    tr = _mk_transform(batq, t)
+    x = batq.bits_to_cuda_bf16(xb)                       # contiguous [tokens, heads, head_dim]
+    vhat = torch.empty((tokens * heads, hd), dtype=torch.float32, device="cuda")
+    batq.batq_debug_transform_clip_f32(tr, x, vhat)
+    V32 = vhat.cpu().numpy().astype(np.float64)
+    c4, s4 = _gpu_quantize(batq, tr, xb)
+    o4, os4 = O.mxfp4_quantize(V32)
+    assert np.array_equal(c4, o4) and np.array_equal(s4, os4)
+    codes = torch.empty((tokens * heads, hd), dtype=torch.uint8, device="cuda")
+    scales = torch.empty((tokens * heads, hd // 32), dtype=torch.uint8, device="cuda")
+    batq.batq_quantize_act_mxfp8(tr, x, codes, scales, 0)
+    o8, os8 = O.mxfp8_quantize(V32)
+    assert np.array_equal(codes.cpu().numpy(), o8) and np.array_equal(scales.cpu().numpy(), os8)
+    # per head it is the oracle applied to that head's rows alone
+    h = 3
+    rows = np.arange(tokens) * heads + h
+    oh, osh = O.quantize_act_mxfp8(xb[rows], t.left, t.right, t.clip_lo, t.clip_hi)
+    assert (np.abs((codes.cpu().numpy()[rows] & 0x7F).astype(int) - (oh & 0x7F).astype(int)) <= 1).all()
+
+
 # ---------------------------------------------------------------------------- weights
 def _weight_mismatch_ok(gc, gs, oc, os_, Wt):
     sdiff = gs != os_
