@@ -34,7 +34,8 @@ constexpr int kQtQuantWarps = 16;
 constexpr int kQtThreads = (2 + kQtQuantWarps) * 32;
 constexpr int kQtCodeTileBytes = kQtRows * kQtGroups * 16;  // 4-bit codes of one unit: 128 rows x 64 bytes
 constexpr int kQtCodeTileBytes8 = 2 * kQtCodeTileBytes;     // 8-bit codes: 128 rows x 128 bytes
-constexpr int kQtStagingBytes = 2 * kQtCodeTileBytes8 + 2 * 512;  // two code tiles (sized for 8-bit), two scale atoms
+constexpr int kQtOutBufs = 3;   // staging buffers: with three, one barrier per unit orders their reuse
+constexpr int kQtStagingBytes = kQtOutBufs * (kQtCodeTileBytes8 + 512);  // code tiles (sized for 8-bit), scale atoms
 constexpr int kQtSmemBytes = kQtStages * kQtStageBytes + 2 * kQtStripImageBytes + kQtStagingBytes + 1024;
 constexpr int kQtTmemCols = 256;              // 2 buffers x 4 blocks x 32 columns
 
@@ -113,7 +114,7 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
   __shared__ __align__(8) uint64_t bars[2 * kQtStages + 8];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
-  __shared__ int go_slot;
+  __shared__ int go_slot[2];  // by unit parity: a slot is rewritten only after every warp has read it
   uint64_t* const x_full = bars;                     // [kQtStages]
   uint64_t* const x_empty = bars + kQtStages;        // [kQtStages]
   uint64_t* const p_full = bars + 2 * kQtStages;     // [2]
@@ -272,8 +273,8 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
       const int buf = it & 1;
       bool ok = mbar_wait(smem_u32(&d_full[buf]), (it >> 1) & 1u, &abort_flag);
       ok = __all_sync(0xFFFFFFFFu, ok);
-      // A warp whose wait gave up may not leave on its own: the sixteen quantiser warps meet at
-      // named barriers below, so they leave together (see `go_slot`).  The debug build has no barriers.
+      // A warp whose wait gave up may not leave on its own: the sixteen quantiser warps meet at a
+      // named barrier below, so they leave together (see `go_slot`).  The debug build has no barrier.
       if (DEBUG_OUT && !ok) break;
       tc_fence_after_sync();
       const int64_t row = row_tile * kQtRows + quad * 32 + lane;
@@ -331,13 +332,9 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
       // Codes and scale bytes of the whole unit meet in shared memory (128 rows x 64 or 128 bytes of
       // codes, one 512-byte scale atom) and leave as one TMA store and one bulk copy: full 32-byte
       // sectors instead of 16-byte and 1-byte pieces.
-      const int sb = it & 1;
-      if (qw == 0 && lane == 0) {
-        bulk_wait_group_read<1>();  // the stores of two units ago have read buffer sb
-        go_slot = *static_cast<volatile int*>(&abort_flag) == 0;  // one thread decides for all, published by the barrier
-      }
-      qt_named_barrier_sync(1, kQtQuantWarps * 32);
-      if (!go_slot) break;
+      // Buffer sb was last used by unit it - 3; its stores had been read out of shared memory before
+      // the issuing thread reached the barrier of unit it - 1 (see below), which every warp has passed.
+      const int sb = it % kQtOutBufs;
       const int trow = quad * 32 + lane;
       if (FP8) {
         uint8_t* tile = staging + sb * kQtCodeTileBytes8 + trow * 128;
@@ -368,17 +365,21 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
       if (p.sf_layout == 0) {
         if (row < p.s && j < p.k) p.scales[row * p.k + j] = sbv;
       } else {
-        staging[2 * kQtCodeTileBytes8 + sb * 512 + lane * 16 + quad * 4 + g] = sbv;
+        staging[kQtOutBufs * kQtCodeTileBytes8 + sb * 512 + lane * 16 + quad * 4 + g] = sbv;
       }
       fence_proxy_async_smem();
+      if (qw == 0 && lane == 0) go_slot[it & 1] = *static_cast<volatile int*>(&abort_flag) == 0;  // one thread decides for all
       qt_named_barrier_sync(1, kQtQuantWarps * 32);
+      if (!go_slot[it & 1]) break;
       if (qw == 0 && lane == 0) {
         const int yrow = static_cast<int>(row_tile) * kQtRows;
         tma_store_2d(&tmap_codes, static_cast<int>(strip) * (kQtGroups * (FP8 ? 32 : 16)), yrow,
                      smem_u32(staging + sb * kQtCodeTileBytes8));
         if (p.sf_layout != 0)
-          bulk_s2g(p.scales + (row_tile * p.sf_katoms + strip) * 512, smem_u32(staging + 2 * kQtCodeTileBytes8 + sb * 512), 512);
+          bulk_s2g(p.scales + (row_tile * p.sf_katoms + strip) * 512,
+                   smem_u32(staging + kQtOutBufs * kQtCodeTileBytes8 + sb * 512), 512);
         bulk_commit_group();
+        bulk_wait_group_read<1>();  // all but this unit's stores have read their buffers
       }
     }
     if (qw == 0 && lane == 0) bulk_wait_group<0>();
