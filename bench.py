@@ -168,17 +168,20 @@ def oracle_threads():
 
 def time_oracle(workload, seed, steps, warmup, budget_s):
     """Times the oracle as it stands on a sample sized so that warmup + steps take about
-    `budget_s` seconds: a small probe fixes the cost per (row x feature), then rows and
-    features are scaled up together."""
-    probe, pflops, _ = oracle_sample(workload, seed, 64, 512)
-    t0 = time.perf_counter()
-    probe()
-    per_flop = (time.perf_counter() - t0) / pflops
+    `budget_s` seconds: starting from a small sample, rows and features are doubled together
+    while one step of the doubled sample (about four times the work) still fits its share."""
     per_step = budget_s / max(steps + warmup, 1)
-    scale = max(1.0, per_step / (per_flop * pflops)) ** 0.5
-    rows, feats = int(64 * scale), int(512 * scale)
-    step, flops, desc = oracle_sample(workload, seed, rows, feats)
-    for _ in range(warmup):
+    rows, feats = 64, 512
+    while True:
+        step, flops, desc = oracle_sample(workload, seed, rows, feats)
+        t0 = time.perf_counter()
+        step()
+        once = time.perf_counter() - t0
+        _, tokens, projs, _, _ = WORKLOADS[workload]
+        if once * 4.0 > per_step or (rows >= tokens[-1] and feats >= max(projs[0][2], 1)):
+            break
+        rows, feats = rows * 2, feats * 2
+    for _ in range(max(warmup - 1, 0)):   # the sizing call above was the first warm-up
         step()
     t0 = time.perf_counter()
     for _ in range(steps):
