@@ -293,6 +293,7 @@ def run_ours(args):
     B.batq_debug_force_quantizer(args.quantizer)
     B.batq_debug_force_gemm_kernel(args.gemm_kernel)
     B.batq_debug_force_small_s_splits(args.splits)
+    B.batq_debug_force_small_s_path(args.small_path)
     peaks = load_peaks()
     kind, tokens, projs, _, _ = WORKLOADS[args.workload]
     # prefill: long enough (> 1 s) for the power cap to settle, so that the sustained peak is the fair denominator
@@ -587,6 +588,7 @@ def main():
     ap.add_argument("--quantizer", type=int, default=0, help="0 auto, 1 ALU kernel, 2 tensor-core kernel (tuning)")
     ap.add_argument("--gemm-kernel", type=int, default=0, help="0 auto, 1 one CTA per tile, 2 CTA pairs (tuning)")
     ap.add_argument("--tile-width", type=int, default=0, help="force the GEMM tile width (tuning); 0 = automatic")
+    ap.add_argument("--small-path", type=int, default=0, help="0 auto, 1 two kernels, 2 fused kernel (tuning)")
     ap.add_argument("--splits", type=int, default=0, help="force the small-s GEMM's K splits (tuning); 0 = automatic")
     args = ap.parse_args()
     if args.impl == "reference":

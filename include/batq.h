@@ -171,9 +171,11 @@ void batq_debug_force_tile_width(int32_t bn);
  * 256-token tile for s > 128, one CTA per 128-token tile otherwise), 1 = always one CTA per tile,
  * 2 = always CTA pairs (tile widths 192 and 256 only). */
 void batq_debug_force_gemm_kernel(int32_t which);
-/* Test / tuning hook: which activation quantiser later calls use.  0 = automatic (tensor-core
- * dense-block kernel for s >= 64 tokens, ALU Kronecker-form kernel below that and for the
- * identity transform), 1 = always the ALU kernel, 2 = always the tensor-core kernel. */
+/* Test / tuning hook: which activation quantiser later calls use.  0 = automatic (up to 64 tokens
+ * the one-thread-per-block kernel, above that the tensor-core dense-block kernel; the identity
+ * transform above 64 tokens and nothing else takes the streaming ALU kernel), 1 = the streaming ALU
+ * kernel (Kronecker form), 2 = the tensor-core kernel, 3 = the one-thread-per-block kernel.
+ * Factor sizes other than 4 x 8 always take the tensor-core kernel. */
 void batq_debug_force_quantizer(int32_t which);
 /* Test / tuning hook: number of K splits of the small-s GEMM (clamped to the number of
  * 256-element K steps and to 32); 0 restores the automatic choice.  Scratch sizes follow it. */

@@ -325,6 +325,32 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
     }
     return launch_quantize_tc(t, x, s, n, ld, codes, scales, layout, debug_out, stream, info->sm_count);
   }
+  // A handful of tokens: the ring of the streaming kernel below is all latency there; one thread
+  // per (token, block) with everything loaded up front is quicker.
+  if (g_force_quantizer == 3 || (g_force_quantizer == 0 && s <= kSmallSMax)) {
+    QuantSmallParams q{};
+    q.x = static_cast<const uint16_t*>(x);
+    q.ld = ld;
+    q.s = static_cast<int32_t>(s);
+    q.n = static_cast<int32_t>(n);
+    q.k = static_cast<int32_t>(n / 32);
+    if (t != nullptr) {
+      q.left = t->d_left; q.right = t->d_right;
+      q.left_stride = t->left_stride; q.right_stride = t->right_stride;
+      q.clip_lo = t->d_clip_lo; q.clip_hi = t->d_clip_hi;
+    }
+    q.codes = static_cast<uint8_t*>(codes);
+    q.scales = static_cast<uint8_t*>(scales);
+    q.sf_layout = layout;
+    q.sf_katoms = katoms_of(q.k);
+    q.debug_out = debug_out;
+    q.zero_words = zero_words;
+    q.n_zero_words = n_zero_words;
+    const unsigned blocks = static_cast<unsigned>((s * q.k + 127) / 128);
+    if (debug_out != nullptr) quantize_act_small_kernel<true><<<blocks, 128, 0, stream>>>(q);
+    else quantize_act_small_kernel<false><<<blocks, 128, 0, stream>>>(q);
+    return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
+  }
   QuantActParams p{};
   p.x = static_cast<const uint16_t*>(x);
   p.ld = ld;

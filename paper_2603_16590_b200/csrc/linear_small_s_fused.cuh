@@ -78,8 +78,8 @@ __device__ __forceinline__ float ld_shared_cluster_f32(uint32_t cluster_addr) {
 
 // One (token, block): 32 bf16 values -> transformed, clipped, quantised: 16 code bytes + scale byte.
 // Same arithmetic as quantize_act_kernel (fp32 fused multiply-adds over the Kronecker form).
-__device__ __forceinline__ void fused_quant_item(const uint16_t* xp, const float* L, const float* R, bool clip,
-                                                 float c_lo, float c_hi, uint32_t (&cw)[4], uint32_t& sbyte) {
+__device__ __forceinline__ void item_transform_clip(const uint16_t* xp, const float* L, const float* R, bool clip,
+                                                    float c_lo, float c_hi, float (&o)[4][8], float& amax) {
   // All loads of the item first (x: 4 x 16 bytes, R: 16 x 16 bytes, L: 4 x 16 bytes), so that their
   // latencies overlap: at this size the kernel is a chain of latencies.
   uint4 q[4];
@@ -108,7 +108,6 @@ __device__ __forceinline__ void fused_quant_item(const uint16_t* xp, const float
       v[i][2 * h + 1] = __uint_as_float(w[h] & 0xFFFF0000u);
     }
   }
-  float o[4][8];
   if (L != nullptr) {
     float U[4][8];
 #pragma unroll
@@ -143,7 +142,6 @@ __device__ __forceinline__ void fused_quant_item(const uint16_t* xp, const float
       mn = fminf(mn, o[r][c]);
       mx = fmaxf(mx, o[r][c]);
     }
-  float amax;
   if (clip) {
     const float lo = c_lo * mn, hi = c_hi * mx;
 #pragma unroll
@@ -154,6 +152,10 @@ __device__ __forceinline__ void fused_quant_item(const uint16_t* xp, const float
   } else {
     amax = fmaxf(fabsf(mn), fabsf(mx));
   }
+}
+
+// The transformed and clipped block -> 16 code bytes + scale byte (MXFP4, Sec. 2).
+__device__ __forceinline__ void item_encode(const float (&o)[4][8], float amax, uint32_t (&cw)[4], uint32_t& sbyte) {
   // shared scale: byte = max(biased_exponent(amax) - 2, 0) = clamp(floor(log2 amax) - 2) + 127
   const int ef = static_cast<int>(__float_as_uint(amax) >> 23);
   const int sb = max(ef - 2, 0);
@@ -166,6 +168,77 @@ __device__ __forceinline__ void fused_quant_item(const uint16_t* xp, const float
     cw[r] = e2m1x8_pack(uu);
   }
   sbyte = static_cast<uint32_t>(sb);
+}
+
+__device__ __forceinline__ void fused_quant_item(const uint16_t* xp, const float* L, const float* R, bool clip,
+                                                 float c_lo, float c_hi, uint32_t (&cw)[4], uint32_t& sbyte) {
+  float o[4][8];
+  float amax;
+  item_transform_clip(xp, L, R, clip, c_lo, c_hi, o, amax);
+  item_encode(o, amax, cw, sbyte);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Stages 1+2 alone for a handful of tokens: one (token, block) per thread, everything loaded
+// up front, no shared-memory ring -- a launch of a few microseconds in front of the small-s GEMM,
+// whose weight stream it releases at once (programmatic dependent launch).  Also clears the
+// GEMM's split-K tickets.
+struct QuantSmallParams {
+  const uint16_t* x;     // bf16 bits [s x n], row stride ld
+  int64_t ld;
+  int32_t s;
+  int32_t n;
+  int32_t k;             // n / 32
+  const float* left;     // [.][16], left_stride floats apart (0 = shared); NULL = identity transform
+  const float* right;    // [.][64]
+  int32_t left_stride;
+  int32_t right_stride;
+  const float* clip_lo;  // [k] or NULL
+  const float* clip_hi;
+  uint8_t* codes;        // [s x n/2]
+  uint8_t* scales;
+  int32_t sf_layout;     // BATQ_SF_ROWMAJOR / BATQ_SF_MMA
+  int32_t sf_katoms;
+  float* debug_out;      // [s x n] fp32 (DEBUG_OUT builds)
+  uint32_t* zero_words;  // optional: n_zero_words 32-bit words set to zero
+  int32_t n_zero_words;
+};
+
+template <bool DEBUG_OUT>
+__global__ void __launch_bounds__(128) quantize_act_small_kernel(const QuantSmallParams p) {
+  grid_launch_dependents();
+  if (blockIdx.x == 0)
+    for (int i = threadIdx.x; i < p.n_zero_words; i += 128) p.zero_words[i] = 0u;
+  const int64_t item = static_cast<int64_t>(blockIdx.x) * 128 + threadIdx.x;
+  if (item >= static_cast<int64_t>(p.s) * p.k) return;
+  const int64_t row = item / p.k;
+  const int j = static_cast<int>(item - row * p.k);
+  const bool clip = p.clip_lo != nullptr;
+  const float* L = p.left ? p.left + static_cast<int64_t>(j) * p.left_stride : nullptr;
+  const float* R = p.left ? p.right + static_cast<int64_t>(j) * p.right_stride : nullptr;
+  float o[4][8];
+  float amax;
+  item_transform_clip(p.x + row * p.ld + static_cast<int64_t>(j) * 32, L, R, clip, clip ? __ldg(p.clip_lo + j) : 1.0f,
+                      clip ? __ldg(p.clip_hi + j) : 1.0f, o, amax);
+  if (DEBUG_OUT) {
+    float4* dst = reinterpret_cast<float4*>(p.debug_out + row * p.n + static_cast<int64_t>(j) * 32);
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      dst[2 * r] = make_float4(o[r][0], o[r][1], o[r][2], o[r][3]);
+      dst[2 * r + 1] = make_float4(o[r][4], o[r][5], o[r][6], o[r][7]);
+    }
+    return;
+  }
+  uint32_t cw[4], sbyte;
+  item_encode(o, amax, cw, sbyte);
+  *reinterpret_cast<uint4*>(p.codes + row * (p.n / 2) + static_cast<int64_t>(j) * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+  if (p.sf_layout == 0) {
+    p.scales[row * p.k + j] = static_cast<uint8_t>(sbyte);
+  } else {
+    p.scales[sf_mma_offset(row, j, p.sf_katoms)] = static_cast<uint8_t>(sbyte);
+    if (j == p.k - 1)  // keep the padded blocks of this row finite
+      for (int jj = p.k; jj < p.sf_katoms * 4; ++jj) p.scales[sf_mma_offset(row, jj, p.sf_katoms)] = 0;
+  }
 }
 
 template <bool OUT_BF16>

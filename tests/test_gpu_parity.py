@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 FP32_REL = 32 * 2.0 ** -24
 
 
-@pytest.fixture(params=[1, 2], ids=["alu", "tensorcore"])
+@pytest.fixture(params=[1, 2, 3], ids=["alu", "tensorcore", "perblock"])
 def qmode(request, batq):
     """Runs a test once per activation-quantiser implementation."""
     batq.batq_debug_force_quantizer(request.param)
@@ -125,7 +125,7 @@ def test_identity_transform_is_bit_exact_plain_mxfp4(batq, S, N):
     assert np.array_equal(gs, os_) and np.array_equal(gc, oc)
     # identity *factors* through either transform kernel give the same bits
     t = synth.make_transform(N, 1, identity=True, clip=False)
-    for mode in (1, 2):
+    for mode in (1, 2, 3):
         batq.batq_debug_force_quantizer(mode)
         try:
             gc2, gs2 = _gpu_quantize(batq, _mk_transform(batq, t), xb)
