@@ -290,16 +290,27 @@ batq_status launch_quantize_tc(const batq_transform* t, const void* x, int64_t s
   }
   const int grid = static_cast<int>(std::min<int64_t>(sm_count, p.n_units));
   const bool cl = t->has_clip, dbg = debug_out != nullptr;
-#define BATQ_QT(CL, DB) quantize_act_tc_kernel<CL, DB><<<grid, kQtThreads, kQtSmemBytes, stream>>>(tmap_x, tmap_codes, p)
-  if (fp8 && !dbg) {
-    if (cl) quantize_act_tc_kernel<true, false, true><<<grid, kQtThreads, kQtSmemBytes, stream>>>(tmap_x, tmap_codes, p);
-    else quantize_act_tc_kernel<false, false, true><<<grid, kQtThreads, kQtSmemBytes, stream>>>(tmap_x, tmap_codes, p);
-  } else if (cl && !dbg) BATQ_QT(true, false);
-  else if (!cl && !dbg) BATQ_QT(false, false);
-  else if (cl && dbg) BATQ_QT(true, true);
-  else BATQ_QT(false, true);
+  // Launched as a programmatic dependent: if the kernel before it on the stream releases its
+  // dependents early (the GEMMs of this library do), the quantiser's CTAs take over the SMs that
+  // kernel has left and wait there; otherwise this is an ordinary launch.
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(grid));
+  cfg.blockDim = dim3(kQtThreads);
+  cfg.dynamicSmemBytes = kQtSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e;
+#define BATQ_QT(CL, DB, F8) cudaLaunchKernelEx(&cfg, quantize_act_tc_kernel<CL, DB, F8>, tmap_x, tmap_codes, p)
+  if (fp8 && !dbg) e = cl ? BATQ_QT(true, false, true) : BATQ_QT(false, false, true);
+  else if (!dbg) e = cl ? BATQ_QT(true, false, false) : BATQ_QT(false, false, false);
+  else e = cl ? BATQ_QT(true, true, false) : BATQ_QT(false, true, false);
 #undef BATQ_QT
-  return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
+  if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+  return BATQ_OK;
 }
 
 batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, int64_t n, int64_t ld, void* codes,

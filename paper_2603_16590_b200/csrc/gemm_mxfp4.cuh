@@ -90,6 +90,9 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
+  // A kernel launched as a programmatic dependent of this one may be scheduled on every SM this
+  // grid has left; it must still wait for this grid before it touches memory.
+  grid_launch_dependents();
   const int tid = threadIdx.x;
   const int warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0);  // warp-uniform for the compiler
   const int lane = tid & 31;

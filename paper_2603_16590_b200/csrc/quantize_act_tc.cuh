@@ -171,6 +171,7 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
     int n_img = 0;  // block-matrix images loaded so far
     bool ok = true;
     int issued = 0;
+    bool waited = false;
     for (int64_t u = u0; u < u1 && ok; ++u) {
       const int64_t strip = u / p.n_row_tiles;
       const int row0 = static_cast<int>(u - strip * p.n_row_tiles) * kQtRows;
@@ -187,6 +188,13 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                    static_cast<uint32_t>(ng) * kQtImageBytes, smem_u32(&p_full[pb]));
         }
         ++n_img;
+      }
+      if (!waited) {
+        // The block-matrix image above is the transform's own constant data; X may come from the
+        // kernel before this one, which this kernel may have been launched as a programmatic
+        // dependent of: wait for it here (nothing is written before data has flowed through).
+        grid_dependency_wait();
+        waited = true;
       }
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&x_empty[stage]), phase ^ 1u, &abort_flag));
       if (!ok) break;
