@@ -180,9 +180,14 @@ void batq_debug_force_quantizer(int32_t which);
 /* Test / tuning hook: number of K splits of the small-s GEMM (clamped to the number of
  * 256-element K steps and to 32); 0 restores the automatic choice.  Scratch sizes follow it. */
 void batq_debug_force_small_s_splits(int32_t splits);
+/* Test / tuning hook: how the small-s GEMM adds the partial tiles of its K splits.  0 = automatic
+ * (through a thread-block cluster's shared memory for up to 4 tokens, up to 8 splits and a grid
+ * below 90 % of the SM slots, where that measured faster; else through scratch and tickets),
+ * 1 = always scratch and tickets, 2 = the cluster whenever there are at most 8 splits. */
+void batq_debug_force_small_s_reduce(int32_t which);
 /* Test / tuning hook: how batq_linear_w4a4 runs a handful of tokens.  0 = automatic (one fused
  * kernel that quantises the activations inside the GEMM where that is the faster one -- tokens x
- * K-steps per CTA <= 8 and a grid of one wave --, else the quantiser kernel followed by the small-s
+ * K-steps per CTA <= 4 and a grid of one wave --, else the quantiser kernel followed by the small-s
  * GEMM), 1 = always the two kernels, 2 = the fused kernel up to 16 tokens.  The fused kernel needs
  * n <= 16384; other shapes take the two kernels. */
 void batq_debug_force_small_s_path(int32_t which);

@@ -41,6 +41,7 @@ SIGNATURES = {
     "batq_gemm_mxfp4_small_s": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _I64, _P, _SZ, _P]),
     "batq_debug_force_small_s_splits": (None, [_I32]),
     "batq_debug_force_small_s_path": (None, [_I32]),
+    "batq_debug_force_small_s_reduce": (None, [_I32]),
     "batq_debug_force_tile_width": (None, [_I32]),
     "batq_debug_force_gemm_kernel": (None, [_I32]),
     "batq_debug_force_quantizer": (None, [_I32]),
@@ -222,6 +223,10 @@ def batq_gemm_mxfp4_small_s(x_codes, x_scales_mma, w: Weight, s, y, scratch, ldy
 
 def batq_debug_force_small_s_splits(splits: int):
     load().batq_debug_force_small_s_splits(splits)
+
+
+def batq_debug_force_small_s_reduce(which: int):
+    load().batq_debug_force_small_s_reduce(which)
 
 
 def batq_debug_force_small_s_path(which: int):

@@ -555,6 +555,7 @@ batq_status launch_gemm(const void* x_codes, const void* x_sf, const batq_weight
 
 // ---- small-s (decode) GEMM: split choice, scratch layout, launch -------------------------------
 int g_force_splits = 0;  // tuning hook: 0 = automatic
+int g_small_reduce = 0;  // tuning hook: 0 = automatic, 1 = always tickets, 2 = cluster whenever splits <= 8
 constexpr int kMaxSplits = 32;
 
 inline int small_ntok(int64_t s) { return s <= 16 ? 16 : (s <= 32 ? 32 : 64); }
@@ -601,11 +602,22 @@ cudaError_t launch_small_kernel(dim3 grid, cudaStream_t stream, bool dependent, 
   cfg.blockDim = dim3(kSmallThreads);
   cfg.dynamicSmemBytes = SmallCfg<NTOK>::kSmemBytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute attr[2];
+  int na = 0;
+  if (p.cluster_reduce) {  // the K splits of a row tile as one cluster
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = 1;
+    attr[na].val.clusterDim.y = grid.y;
+    attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  if (dependent) {
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
   cfg.attrs = attr;
-  cfg.numAttrs = dependent ? 1 : 0;
+  cfg.numAttrs = na;
   return cudaLaunchKernelEx(&cfg, gemm_small_s_kernel<NTOK, BF>, tw, tx, p);
 }
 
@@ -634,6 +646,13 @@ batq_status launch_gemm_small(const void* x_codes, const void* x_sf, const batq_
   p.ldy = ldy;
   p.partial = reinterpret_cast<float*>(scratch);
   p.tickets = reinterpret_cast<uint32_t*>(scratch + sc.partial_bytes);
+  // Cluster reduction where it measured faster than tickets: few tokens (the leader reads
+  // tokens x splits remote values per thread) and a grid that leaves the gang scheduler of
+  // clusters some room (<= 90 % of the two-per-SM slots); 2 = forced on whenever splits <= 8.
+  const int64_t slots = 2 * static_cast<int64_t>(info->sm_count);
+  const bool fits = sc.splits > 1 && sc.splits <= 8;
+  p.cluster_reduce = (fits && (g_small_reduce == 2 ||
+                               (g_small_reduce == 0 && s <= 4 && sc.tiles * sc.splits * 10 <= slots * 9))) ? 1 : 0;
   const dim3 grid(static_cast<unsigned>(sc.tiles), static_cast<unsigned>(sc.splits));
   const bool bf = y_dtype == BATQ_BF16;
   cudaError_t e;
@@ -670,8 +689,8 @@ int pick_fused_splits(int64_t m, int64_t n, int sm_count) {
 }
 
 // Automatic choice: every CTA of a K split requantises its slice of the activations, which is only
-// hidden behind the weight stream while that is a few items per thread (tokens x K-steps <= 8) and
-// the grid fits the SMs in one wave; measured, the fused kernel then saves 10-20 % of a call.
+// hidden behind the weight stream while that is a few items per thread (tokens x K-steps <= 4) and
+// the grid fits the SMs in one wave; measured, the fused kernel then saves about 5 % of a call.
 bool use_fused_small(const batq_transform* t, const batq_weight* w, int64_t s) {
   if (g_force_small_path == 1 || s > kFusedTok) return false;
   if (t != nullptr && (t->gr != 4 || t->gc != 8)) return false;  // its in-kernel quantiser is the 4 x 8 form
@@ -681,7 +700,7 @@ bool use_fused_small(const batq_transform* t, const batq_weight* w, int64_t s) {
   const int64_t k_steps = (w->n + 255) / 256;
   const int64_t per = (k_steps + sp - 1) / sp;
   const int64_t slots = 2 * static_cast<int64_t>(w->sm_count > 0 ? w->sm_count : 148);
-  return s * per <= 8 && ((w->m + 127) / 128) * sp <= slots;
+  return s * per <= 4 && ((w->m + 127) / 128) * sp <= slots;
 }
 
 batq_status launch_linear_fused(const batq_transform* t, const batq_weight* w, const void* x, int64_t s, int64_t ld,
@@ -1074,6 +1093,7 @@ void batq_debug_force_quantizer(int32_t which) { g_force_quantizer = which; }
 void batq_debug_force_gemm_kernel(int32_t which) { g_force_gemm_kernel = which; }
 void batq_debug_force_small_s_splits(int32_t splits) { g_force_splits = splits; }
 void batq_debug_force_small_s_path(int32_t which) { g_force_small_path = which; }
+void batq_debug_force_small_s_reduce(int32_t which) { g_small_reduce = which; }
 
 size_t batq_static_workspace_capacity(void) { return BATQ_STATIC_WORKSPACE_BYTES - 1024; }
 

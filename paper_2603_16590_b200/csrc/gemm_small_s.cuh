@@ -9,8 +9,9 @@
 // columns), so no tensor-core row is spent on padding tokens.  The grid is
 // (row tiles) x (K splits): enough CTAs, two per SM, to keep the whole memory system
 // busy however few output features the layer has.  With more than one split every CTA
-// writes its partial tile to scratch and takes a ticket; the CTA that draws the last
-// ticket of a row tile adds the partials in split order (deterministic) and writes Y.
+// keeps its partial tile for a reduction in split order (deterministic): up to 8 splits form a
+// thread-block cluster whose leader reads the others' tiles from distributed shared memory;
+// beyond that the tiles go to scratch and the CTA that draws the last ticket of a row tile adds them.
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and tensor-memory owner,
 // warps 2..5 = epilogue.  The weight stream does not depend on the activation
@@ -53,8 +54,10 @@ struct SmallParams {
   int32_t splits;        // gridDim.y
   void* y;               // [s x m] fp32 or bf16, row stride ldy
   int64_t ldy;
-  float* partial;        // [row tile][split][NTOK][128] fp32 (splits > 1)
-  uint32_t* tickets;     // [row tiles], zero on entry, zero again on exit (splits > 1)
+  float* partial;        // [row tile][split][NTOK][128] fp32 (splits > 1, ticket mode)
+  uint32_t* tickets;     // [row tiles], zero on entry, zero again on exit (splits > 1, ticket mode)
+  int32_t cluster_reduce;  // 1: the splits of a row tile are one thread-block cluster (grid.y == cluster.y <= 8)
+                           // and add their partial tiles through distributed shared memory instead
 };
 
 // 32 lanes x 16 consecutive 32-bit columns -> 16 registers per thread.
@@ -115,6 +118,9 @@ gemm_small_s_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
   const int kt0 = static_cast<int>(static_cast<int64_t>(p.k_steps) * sp / p.splits);
   const int kt1 = static_cast<int>(static_cast<int64_t>(p.k_steps) * (sp + 1) / p.splits);
   const int n_steps = kt1 - kt0;                  // >= 1: the host keeps splits <= k_steps
+  const bool by_cluster = p.cluster_reduce != 0 && p.splits > 1;
+  bool epi_ok = false;
+  uint32_t v[NTOK];
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
@@ -225,14 +231,20 @@ gemm_small_s_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     if (ok) {
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
-      uint32_t v[NTOK];
 #pragma unroll
       for (int c = 0; c < NTOK; c += 16) tmem_ld_32x32b_x16(taddr + c, v + c);
       tmem_ld_wait();
       tc_fence_before_sync();
+      epi_ok = true;
 
-      bool write_out = true;
-      if (p.splits > 1) {
+      bool write_out = !by_cluster;
+      if (by_cluster) {
+        // every MMA has completed: the operand ring is free and takes this CTA's partial tile
+        float* part = reinterpret_cast<float*>(smem);
+#pragma unroll
+        for (int t = 0; t < NTOK; ++t)
+          if (t < p.s) part[t * 128 + row] = __uint_as_float(v[t]);
+      } else if (p.splits > 1) {
         float* mine = p.partial + (static_cast<int64_t>(rt) * p.splits + sp) * (NTOK * 128) + row;
 #pragma unroll
         for (int t = 0; t < NTOK; ++t)
@@ -301,6 +313,41 @@ gemm_small_s_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     }
   }
 
+  if (by_cluster) {
+    // Every thread of every CTA of the cluster takes both barriers, whatever happened above.
+    __syncthreads();
+    cluster_sync_all();
+    if (warp >= 2 && sp == 0 && epi_ok) {
+      const int row = (warp & 3) * 32 + lane;
+      const int64_t mrow = static_cast<int64_t>(rt) * 128 + row;
+      const uint32_t mine = smem_u32(smem) + row * 4;
+#pragma unroll
+      for (int t0 = 0; t0 < NTOK; t0 += 4) {
+        if (t0 < p.s) {
+          float part[7][4];
+#pragma unroll
+          for (int q = 1; q < 8; ++q)
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+              part[q - 1][t] = (q < p.splits && t0 + t < p.s)
+                                   ? ld_shared_cluster_f32(map_to_cta(mine + (t0 + t) * 512, q)) : 0.0f;
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            float acc = __uint_as_float(v[t0 + t]);  // split 0's own part, then splits 1.. in order
+#pragma unroll
+            for (int q = 1; q < 8; ++q) acc += part[q - 1][t];
+            if (t0 + t < p.s && mrow < p.m) {
+              if (OUT_BF16)
+                reinterpret_cast<__nv_bfloat16*>(p.y)[(t0 + t) * p.ldy + mrow] = __float2bfloat16_rn(acc);
+              else
+                reinterpret_cast<float*>(p.y)[(t0 + t) * p.ldy + mrow] = acc;
+            }
+          }
+        }
+      }
+    }
+    cluster_sync_all();  // the leader has read everybody's shared memory
+  }
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) {

@@ -70,12 +70,6 @@ struct FusedParams {
   int64_t ldy;
 };
 
-__device__ __forceinline__ float ld_shared_cluster_f32(uint32_t cluster_addr) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
-  return v;
-}
-
 // One (token, block): 32 bf16 values -> transformed, clipped, quantised: 16 code bytes + scale byte.
 // Same arithmetic as quantize_act_kernel (fp32 fused multiply-adds over the Kronecker form).
 __device__ __forceinline__ void item_transform_clip(const uint16_t* xp, const float* L, const float* R, bool clip,

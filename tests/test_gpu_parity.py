@@ -454,8 +454,13 @@ SMALL_SHAPES = [(1, 8, 32), (1, 1024, 1024), (4, 300, 544), (16, 4096, 4096), (1
 
 @pytest.mark.parametrize("S,M,N", SMALL_SHAPES)
 @pytest.mark.parametrize("splits", [0, 1, 3])
-def test_gemm_small_s_vs_oracle_same_codes(batq, S, M, N, splits):
-    got, Y, Sabs = _small_case(batq, S, M, N, 800 + S, splits=splits)
+@pytest.mark.parametrize("reduce", [2, 1], ids=["cluster", "tickets"])
+def test_gemm_small_s_vs_oracle_same_codes(batq, S, M, N, splits, reduce):
+    batq.batq_debug_force_small_s_reduce(reduce)
+    try:
+        got, Y, Sabs = _small_case(batq, S, M, N, 800 + S, splits=splits)
+    finally:
+        batq.batq_debug_force_small_s_reduce(0)
     assert np.all(np.isfinite(got))
     assert np.all(np.abs(got - Y) <= 1e-3 * Sabs + 1e-30)
     assert np.max(np.abs(got - Y) / (Sabs + 1e-30)) < 1e-5
