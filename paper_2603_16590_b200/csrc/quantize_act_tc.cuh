@@ -13,7 +13,10 @@
 // Work unit: 128 tokens x 4 blocks (one 512-byte scale atom).  Warp 0 = TMA
 // producer (X tiles, block-matrix images), warp 1 = MMA issuer and tensor-memory
 // owner, warps 2..17 = quantiser warps (4 lane quadrants x 4 blocks), one
-// (token, block) per thread and unit.
+// (token, block) per thread and unit; warp 18 = store warp: once the sixteen pieces of a unit
+// have arrived in the staging buffer it issues the unit's TMA store and scale-atom copy.  The
+// quantiser warps meet nowhere else, so they drift apart by up to a unit and their load, ALU
+// and store phases overlap.
 #pragma once
 #include <cuda.h>
 
@@ -31,10 +34,10 @@ constexpr int kQtTermBytes = 2048;            // one bf16 term of one 32 x 32 bl
 constexpr int kQtImageBytes = 3 * kQtTermBytes;            // per block
 constexpr int kQtStripImageBytes = kQtGroups * kQtImageBytes;  // 24 KiB
 constexpr int kQtQuantWarps = 16;
-constexpr int kQtThreads = (2 + kQtQuantWarps) * 32;
+constexpr int kQtThreads = (3 + kQtQuantWarps) * 32;  // + TMA producer, MMA issuer, store warp
 constexpr int kQtCodeTileBytes = kQtRows * kQtGroups * 16;  // 4-bit codes of one unit: 128 rows x 64 bytes
 constexpr int kQtCodeTileBytes8 = 2 * kQtCodeTileBytes;     // 8-bit codes: 128 rows x 128 bytes
-constexpr int kQtOutBufs = 3;   // staging buffers: with three, one barrier per unit orders their reuse
+constexpr int kQtOutBufs = 3;   // staging buffers between the quantiser warps and the store warp
 constexpr int kQtStagingBytes = kQtOutBufs * (kQtCodeTileBytes8 + 512);  // code tiles (sized for 8-bit), scale atoms
 constexpr int kQtSmemBytes = kQtStages * kQtStageBytes + 2 * kQtStripImageBytes + kQtStagingBytes + 1024;
 constexpr int kQtTmemCols = 256;              // 2 buffers x 4 blocks x 32 columns
@@ -77,10 +80,6 @@ __device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src_smem, uint32_t 
                : "memory");
 }
 
-__device__ __forceinline__ void qt_named_barrier_sync(int id, int threads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
-
 __device__ __forceinline__ float fmin3(float a, float b, float c) {
   float d;
   asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -111,16 +110,17 @@ __global__ void __launch_bounds__(kQtThreads, 1)
 quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_codes,
                        const QuantTcParams p) {
   extern __shared__ uint8_t qt_smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * kQtStages + 8];
+  __shared__ __align__(8) uint64_t bars[2 * kQtStages + 8 + 2 * kQtOutBufs];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
-  __shared__ int go_slot[2];  // by unit parity: a slot is rewritten only after every warp has read it
   uint64_t* const x_full = bars;                     // [kQtStages]
   uint64_t* const x_empty = bars + kQtStages;        // [kQtStages]
   uint64_t* const p_full = bars + 2 * kQtStages;     // [2]
   uint64_t* const p_empty = p_full + 2;              // [2]
   uint64_t* const d_full = p_full + 4;               // [2]
   uint64_t* const d_empty = p_full + 6;              // [2]
+  uint64_t* const t_full = p_full + 8;               // [kQtOutBufs] staging tile complete (16 warps)
+  uint64_t* const t_empty = t_full + kQtOutBufs;     // [kQtOutBufs] staging tile read out by its stores
 
   const int tid = threadIdx.x;
   const int warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0);
@@ -144,6 +144,10 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
       mbar_init(smem_u32(&p_empty[i]), 1);
       mbar_init(smem_u32(&d_full[i]), 1);
       mbar_init(smem_u32(&d_empty[i]), kQtQuantWarps);
+    }
+    for (int i = 0; i < kQtOutBufs; ++i) {
+      mbar_init(smem_u32(&t_full[i]), kQtQuantWarps);
+      mbar_init(smem_u32(&t_empty[i]), 1);
     }
     abort_flag = 0;
     mbar_fence_init();
@@ -269,6 +273,28 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
       if (++stage == kQtStages) { stage = 0; phase ^= 1u; }
     }
     __syncwarp();
+  } else if (warp == 2 + kQtQuantWarps) {
+    // ---------------------------------------------------------------- store warp
+    if (!DEBUG_OUT && lane == 0) {
+      int it = 0;
+      for (int64_t u = u0; u < u1; ++u, ++it) {
+        const int64_t strip = u / p.n_row_tiles;
+        const int64_t row_tile = u - strip * p.n_row_tiles;
+        const int sb = it % kQtOutBufs;
+        if (!mbar_wait(smem_u32(&t_full[sb]), static_cast<uint32_t>(it / kQtOutBufs) & 1u, &abort_flag)) break;
+        tma_store_2d(&tmap_codes, static_cast<int>(strip) * (kQtGroups * (FP8 ? 32 : 16)),
+                     static_cast<int>(row_tile) * kQtRows, smem_u32(staging + sb * kQtCodeTileBytes8));
+        if (p.sf_layout != 0)
+          bulk_s2g(p.scales + (row_tile * p.sf_katoms + strip) * 512,
+                   smem_u32(staging + kQtOutBufs * kQtCodeTileBytes8 + sb * 512), 512);
+        bulk_commit_group();
+        if (it > 0) {  // the stores of the unit before this one have read their buffer: hand it back
+          bulk_wait_group_read<1>();
+          mbar_arrive(smem_u32(&t_empty[(it - 1) % kQtOutBufs]));
+        }
+      }
+      bulk_wait_group<0>();  // all stores complete before the CTA exits
+    }
   } else {
     // ---------------------------------------------------------------- quantiser warps
     const int qw = warp - 2;            // 0..15
@@ -281,9 +307,7 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
       const int buf = it & 1;
       bool ok = mbar_wait(smem_u32(&d_full[buf]), (it >> 1) & 1u, &abort_flag);
       ok = __all_sync(0xFFFFFFFFu, ok);
-      // A warp whose wait gave up may not leave on its own: the sixteen quantiser warps meet at a
-      // named barrier below, so they leave together (see `go_slot`).  The debug build has no barrier.
-      if (DEBUG_OUT && !ok) break;
+      if (!ok) break;
       tc_fence_after_sync();
       const int64_t row = row_tile * kQtRows + quad * 32 + lane;
       const int j = static_cast<int>(strip) * kQtGroups + g;
@@ -340,9 +364,14 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
       // Codes and scale bytes of the whole unit meet in shared memory (128 rows x 64 or 128 bytes of
       // codes, one 512-byte scale atom) and leave as one TMA store and one bulk copy: full 32-byte
       // sectors instead of 16-byte and 1-byte pieces.
-      // Buffer sb was last used by unit it - 3; its stores had been read out of shared memory before
-      // the issuing thread reached the barrier of unit it - 1 (see below), which every warp has passed.
+      // Staging buffer sb was last used by unit it - 3; the store warp hands it back once that
+      // unit's stores have read it.
       const int sb = it % kQtOutBufs;
+      if (it >= kQtOutBufs) {
+        ok = mbar_wait(smem_u32(&t_empty[sb]), static_cast<uint32_t>(it / kQtOutBufs - 1) & 1u, &abort_flag);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+      }
       const int trow = quad * 32 + lane;
       if (FP8) {
         uint8_t* tile = staging + sb * kQtCodeTileBytes8 + trow * 128;
@@ -375,22 +404,10 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
       } else {
         staging[kQtOutBufs * kQtCodeTileBytes8 + sb * 512 + lane * 16 + quad * 4 + g] = sbv;
       }
-      fence_proxy_async_smem();
-      if (qw == 0 && lane == 0) go_slot[it & 1] = *static_cast<volatile int*>(&abort_flag) == 0;  // one thread decides for all
-      qt_named_barrier_sync(1, kQtQuantWarps * 32);
-      if (!go_slot[it & 1]) break;
-      if (qw == 0 && lane == 0) {
-        const int yrow = static_cast<int>(row_tile) * kQtRows;
-        tma_store_2d(&tmap_codes, static_cast<int>(strip) * (kQtGroups * (FP8 ? 32 : 16)), yrow,
-                     smem_u32(staging + sb * kQtCodeTileBytes8));
-        if (p.sf_layout != 0)
-          bulk_s2g(p.scales + (row_tile * p.sf_katoms + strip) * 512,
-                   smem_u32(staging + kQtOutBufs * kQtCodeTileBytes8 + sb * 512), 512);
-        bulk_commit_group();
-        bulk_wait_group_read<1>();  // all but this unit's stores have read their buffers
-      }
+      fence_proxy_async_smem();   // the staging writes become visible to the TMA store
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&t_full[sb]));
     }
-    if (qw == 0 && lane == 0) bulk_wait_group<0>();
   }
 
   tc_fence_before_sync();
