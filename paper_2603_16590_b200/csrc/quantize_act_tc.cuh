@@ -13,10 +13,11 @@
 // Work unit: 128 tokens x 4 blocks (one 512-byte scale atom).  Warp 0 = TMA
 // producer (X tiles, block-matrix images), warp 1 = MMA issuer and tensor-memory
 // owner, warps 2..17 = quantiser warps (4 lane quadrants x 4 blocks), one
-// (token, block) per thread and unit; warp 18 = store warp: once the sixteen pieces of a unit
-// have arrived in the staging buffer it issues the unit's TMA store and scale-atom copy.  The
-// quantiser warps meet nowhere else, so they drift apart by up to a unit and their load, ALU
-// and store phases overlap.
+// (token, block) per thread; warp 18 = store warp: once the pieces of a unit have arrived in
+// the staging buffer it issues the unit's TMA store and scale-atom copy.  The quantiser warps
+// form two groups of eight (4 lane quadrants x 2, two blocks per thread) that take alternate
+// units: the MMA issuer finishes their units half a period apart, so one group's tensor-memory
+// loads and stores fall into the other group's ALU phase.
 #pragma once
 #include <cuda.h>
 
@@ -37,10 +38,11 @@ constexpr int kQtQuantWarps = 16;
 constexpr int kQtThreads = (3 + kQtQuantWarps) * 32;  // + TMA producer, MMA issuer, store warp
 constexpr int kQtCodeTileBytes = kQtRows * kQtGroups * 16;  // 4-bit codes of one unit: 128 rows x 64 bytes
 constexpr int kQtCodeTileBytes8 = 2 * kQtCodeTileBytes;     // 8-bit codes: 128 rows x 128 bytes
-constexpr int kQtOutBufs = 3;   // staging buffers between the quantiser warps and the store warp
+constexpr int kQtOutBufs = 4;   // staging buffers between the quantiser warps and the store warp
+constexpr int kQtDBufs = 4;     // accumulator buffers in tensor memory: two per group of quantiser warps
 constexpr int kQtStagingBytes = kQtOutBufs * (kQtCodeTileBytes8 + 512);  // code tiles (sized for 8-bit), scale atoms
 constexpr int kQtSmemBytes = kQtStages * kQtStageBytes + 2 * kQtStripImageBytes + kQtStagingBytes + 1024;
-constexpr int kQtTmemCols = 256;              // 2 buffers x 4 blocks x 32 columns
+constexpr int kQtTmemCols = kQtDBufs * kQtGroups * 32;  // 4 buffers x 4 blocks x 32 columns = all 512
 
 struct QuantTcParams {
   int64_t s;
@@ -110,16 +112,16 @@ __global__ void __launch_bounds__(kQtThreads, 1)
 quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_codes,
                        const QuantTcParams p) {
   extern __shared__ uint8_t qt_smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * kQtStages + 8 + 2 * kQtOutBufs];
+  __shared__ __align__(8) uint64_t bars[2 * kQtStages + 4 + 2 * kQtDBufs + 2 * kQtOutBufs];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   uint64_t* const x_full = bars;                     // [kQtStages]
   uint64_t* const x_empty = bars + kQtStages;        // [kQtStages]
   uint64_t* const p_full = bars + 2 * kQtStages;     // [2]
   uint64_t* const p_empty = p_full + 2;              // [2]
-  uint64_t* const d_full = p_full + 4;               // [2]
-  uint64_t* const d_empty = p_full + 6;              // [2]
-  uint64_t* const t_full = p_full + 8;               // [kQtOutBufs] staging tile complete (16 warps)
+  uint64_t* const d_full = p_full + 4;               // [kQtDBufs]
+  uint64_t* const d_empty = d_full + kQtDBufs;       // [kQtDBufs]
+  uint64_t* const t_full = d_empty + kQtDBufs;       // [kQtOutBufs] staging tile complete (the 8 warps of a group)
   uint64_t* const t_empty = t_full + kQtOutBufs;     // [kQtOutBufs] staging tile read out by its stores
 
   const int tid = threadIdx.x;
@@ -142,11 +144,13 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&p_full[i]), 1);
       mbar_init(smem_u32(&p_empty[i]), 1);
+    }
+    for (int i = 0; i < kQtDBufs; ++i) {
       mbar_init(smem_u32(&d_full[i]), 1);
-      mbar_init(smem_u32(&d_empty[i]), kQtQuantWarps);
+      mbar_init(smem_u32(&d_empty[i]), kQtQuantWarps / 2);
     }
     for (int i = 0; i < kQtOutBufs; ++i) {
-      mbar_init(smem_u32(&t_full[i]), kQtQuantWarps);
+      mbar_init(smem_u32(&t_full[i]), kQtQuantWarps / 2);
       mbar_init(smem_u32(&t_empty[i]), 1);
     }
     abort_flag = 0;
@@ -242,8 +246,8 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         ++n_img;
       }
       const int pb = (n_img - 1) & 1;
-      const int buf = it & 1;
-      ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&d_empty[buf]), ((it >> 1) & 1u) ^ 1u, &abort_flag));
+      const int buf = it & (kQtDBufs - 1);
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&d_empty[buf]), ((it >> 2) & 1u) ^ 1u, &abort_flag));
       if (!ok) break;
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&x_full[stage]), phase, &abort_flag));
       if (!ok) break;
@@ -299,25 +303,39 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
     // ---------------------------------------------------------------- quantiser warps
     const int qw = warp - 2;            // 0..15
     const int quad = warp & 3;          // tensor-memory lanes [32 quad, 32 quad + 32)
-    const int g = qw >> 2;              // block of the unit this warp quantises
-    int it = 0;
-    for (int64_t u = u0; u < u1; ++u, ++it) {
+    const int grp = qw >> 3;            // takes the units of this CTA with it % 2 == grp
+    const int half = (qw & 7) >> 2;     // blocks 2 half and 2 half + 1 of the unit
+    for (int it = grp; u0 + it < u1; it += 2) {
+      const int64_t u = u0 + it;
       const int64_t strip = u / p.n_row_tiles;
       const int64_t row_tile = u - strip * p.n_row_tiles;
-      const int buf = it & 1;
-      bool ok = mbar_wait(smem_u32(&d_full[buf]), (it >> 1) & 1u, &abort_flag);
+      const int buf = it & (kQtDBufs - 1);
+      bool ok = mbar_wait(smem_u32(&d_full[buf]), (it >> 2) & 1u, &abort_flag);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after_sync();
+      // Staging buffer sb was last used by unit it - kQtOutBufs; the store warp hands it back once
+      // that unit's stores have read it.
+      const int sb = it % kQtOutBufs;
+      if (!DEBUG_OUT && it >= kQtOutBufs) {
+        ok = mbar_wait(smem_u32(&t_empty[sb]), static_cast<uint32_t>(it / kQtOutBufs - 1) & 1u, &abort_flag);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+      }
       const int64_t row = row_tile * kQtRows + quad * 32 + lane;
+#pragma unroll 1
+     for (int e = 0; e < 2; ++e) {
+      const int g = 2 * half + e;
       const int j = static_cast<int>(strip) * kQtGroups + g;
       const uint32_t taddr = tmem_base + buf * (kQtGroups * 32) + g * 32 + (static_cast<uint32_t>(quad * 32) << 16);
       uint32_t v[32];
       tmem_ld_32x32b_x32(taddr, v);
       tmem_ld_wait();
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&d_empty[buf]));  // the accumulator row is in registers now
+      if (e == 1) {
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&d_empty[buf]));  // both accumulator rows have been read
+      }
 
       float o[32];
 #pragma unroll
@@ -364,14 +382,6 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
       // Codes and scale bytes of the whole unit meet in shared memory (128 rows x 64 or 128 bytes of
       // codes, one 512-byte scale atom) and leave as one TMA store and one bulk copy: full 32-byte
       // sectors instead of 16-byte and 1-byte pieces.
-      // Staging buffer sb was last used by unit it - 3; the store warp hands it back once that
-      // unit's stores have read it.
-      const int sb = it % kQtOutBufs;
-      if (it >= kQtOutBufs) {
-        ok = mbar_wait(smem_u32(&t_empty[sb]), static_cast<uint32_t>(it / kQtOutBufs - 1) & 1u, &abort_flag);
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (!ok) break;
-      }
       const int trow = quad * 32 + lane;
       if (FP8) {
         uint8_t* tile = staging + sb * kQtCodeTileBytes8 + trow * 128;
@@ -404,9 +414,12 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
       } else {
         staging[kQtOutBufs * kQtCodeTileBytes8 + sb * 512 + lane * 16 + quad * 4 + g] = sbv;
       }
-      fence_proxy_async_smem();   // the staging writes become visible to the TMA store
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&t_full[sb]));
+     }  // the two blocks of this thread
+      if (!DEBUG_OUT) {
+        fence_proxy_async_smem();   // the staging writes become visible to the TMA store
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&t_full[sb]));
+      }
     }
   }
 
