@@ -357,10 +357,21 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
     q.debug_out = debug_out;
     q.zero_words = zero_words;
     q.n_zero_words = n_zero_words;
-    const unsigned blocks = static_cast<unsigned>((s * q.k + 127) / 128);
-    if (debug_out != nullptr) quantize_act_small_kernel<true><<<blocks, 128, 0, stream>>>(q);
-    else quantize_act_small_kernel<false><<<blocks, 128, 0, stream>>>(q);
-    return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
+    // Launched as a programmatic dependent of whatever precedes it on the stream (in a decode loop
+    // the GEMM of the layer before): it is scheduled early and waits inside the kernel.
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(static_cast<unsigned>((s * q.k + 127) / 128));
+    cfg.blockDim = dim3(128);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = debug_out != nullptr ? cudaLaunchKernelEx(&cfg, quantize_act_small_kernel<true>, q)
+                                               : cudaLaunchKernelEx(&cfg, quantize_act_small_kernel<false>, q);
+    if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+    return BATQ_OK;
   }
   QuantActParams p{};
   p.x = static_cast<const uint16_t*>(x);
@@ -733,13 +744,17 @@ batq_status launch_linear_fused(const batq_transform* t, const batq_weight* w, c
   cfg.blockDim = dim3(kFusedThreads);
   cfg.dynamicSmemBytes = FusedCfg::kSmemBytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 1;
   attr[0].val.clusterDim.y = static_cast<unsigned>(p.splits);
   attr[0].val.clusterDim.z = 1;
+  // A programmatic dependent of whatever precedes it on the stream: its weight stream starts
+  // while that still runs; x is read, and y written, after the wait inside the kernel.
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   const cudaError_t e = y_dtype == BATQ_BF16 ? cudaLaunchKernelEx(&cfg, linear_small_s_fused_kernel<true>, w->tmap_b128, p)
                                              : cudaLaunchKernelEx(&cfg, linear_small_s_fused_kernel<false>, w->tmap_b128, p);
   if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }

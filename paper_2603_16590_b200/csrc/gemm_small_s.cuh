@@ -88,6 +88,9 @@ gemm_small_s_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
   __shared__ uint32_t ticket_slot;
   __shared__ int abort_flag;
 
+  // The next grid on the stream (the quantiser of the next layer) may be scheduled at once; it
+  // writes nothing before its own grid_dependency_wait().
+  grid_launch_dependents();
   const int tid = threadIdx.x;
   const int warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0);
   const int lane = tid & 31;

@@ -74,11 +74,10 @@ struct FusedParams {
 // Same arithmetic as quantize_act_kernel (fp32 fused multiply-adds over the Kronecker form).
 __device__ __forceinline__ void item_transform_clip(const uint16_t* xp, const float* L, const float* R, bool clip,
                                                     float c_lo, float c_hi, float (&o)[4][8], float& amax) {
-  // All loads of the item first (x: 4 x 16 bytes, R: 16 x 16 bytes, L: 4 x 16 bytes), so that their
-  // latencies overlap: at this size the kernel is a chain of latencies.
-  uint4 q[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) q[i] = __ldg(reinterpret_cast<const uint4*>(xp) + i);
+  // All loads of the item first (R: 16 x 16 bytes, L: 4 x 16 bytes, x: 4 x 16 bytes), so that their
+  // latencies overlap: at this size the kernel is a chain of latencies.  The factors are constants
+  // of the layer and are requested before the wait for the previous grid; x, which that grid may
+  // have produced, after it.
   float Rr[64], Lr[16];
   if (L != nullptr) {
 #pragma unroll
@@ -92,6 +91,10 @@ __device__ __forceinline__ void item_transform_clip(const uint16_t* xp, const fl
       Lr[4 * i] = t.x; Lr[4 * i + 1] = t.y; Lr[4 * i + 2] = t.z; Lr[4 * i + 3] = t.w;
     }
   }
+  grid_dependency_wait();
+  uint4 q[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) q[i] = ld_global_ordered_v4(reinterpret_cast<const uint4*>(xp) + i);
   float v[4][8];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -201,10 +204,15 @@ struct QuantSmallParams {
 template <bool DEBUG_OUT>
 __global__ void __launch_bounds__(128) quantize_act_small_kernel(const QuantSmallParams p) {
   grid_launch_dependents();
-  if (blockIdx.x == 0)
-    for (int i = threadIdx.x; i < p.n_zero_words; i += 128) p.zero_words[i] = 0u;
   const int64_t item = static_cast<int64_t>(blockIdx.x) * 128 + threadIdx.x;
-  if (item >= static_cast<int64_t>(p.s) * p.k) return;
+  if (item >= static_cast<int64_t>(p.s) * p.k || blockIdx.x == 0) {
+    // Nothing is written before the grid in front of this one has finished: it may still read
+    // the codes, scales and tickets of its own call.
+    grid_dependency_wait();
+    if (blockIdx.x == 0)
+      for (int i = threadIdx.x; i < p.n_zero_words; i += 128) p.zero_words[i] = 0u;
+    if (item >= static_cast<int64_t>(p.s) * p.k) return;
+  }
   const int64_t row = item / p.k;
   const int j = static_cast<int>(item - row * p.k);
   const bool clip = p.clip_lo != nullptr;
@@ -247,6 +255,9 @@ linear_small_s_fused_kernel(const __grid_constant__ CUtensorMap tmap_w, const Fu
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
+  // The next grid on the stream may be scheduled at once: a kernel of this library touches nothing
+  // the grid before it reads or writes until its own grid_dependency_wait().
+  grid_launch_dependents();
   const int tid = threadIdx.x;
   const int warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0);
   const int lane = tid & 31;
@@ -383,6 +394,7 @@ linear_small_s_fused_kernel(const __grid_constant__ CUtensorMap tmap_w, const Fu
           make_uint4(cw[0], cw[1], cw[2], cw[3]);
       x_sf[step * Cfg::kSfBytes + (c >> 2) * 512 + t * 16 + (c & 3)] = static_cast<uint8_t>(sbyte);
     }
+    grid_dependency_wait();  // threads without an item: these warps write y below
     fence_proxy_async_smem();
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(&x_ready_bar));

@@ -26,6 +26,13 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 // dependent grid start being scheduled before this one has finished.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+// A 16-byte load that stays where it is written: data the previous grid produced is read with
+// this after grid_dependency_wait() (a read-only-cache load may be scheduled ahead of the wait).
+__device__ __forceinline__ uint4 ld_global_ordered_v4(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p) : "memory");
+  return r;
+}
 
 // ------------------------------------------------------------------ mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
