@@ -270,13 +270,19 @@ gemm_small_s_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 float acc[16];
 #pragma unroll
                 for (int t = 0; t < 16; ++t) acc[t] = 0.0f;
-                for (int q = 0; q < p.splits; ++q) {
-                  float part[16];
+                constexpr int QB = NTOK == 16 ? 4 : 2;  // splits per batch: 64 / 32 loads in flight
+                for (int q0 = 0; q0 < p.splits; q0 += QB) {
+                  float part[QB][16];
 #pragma unroll
-                  for (int t = 0; t < 16; ++t)
-                    part[t] = c + t < p.s ? __ldcg(all + q * (NTOK * 128) + (c + t) * 128) : 0.0f;
+                  for (int qq = 0; qq < QB; ++qq)
 #pragma unroll
-                  for (int t = 0; t < 16; ++t) acc[t] += part[t];
+                    for (int t = 0; t < 16; ++t)
+                      part[qq][t] = (q0 + qq < p.splits && c + t < p.s)
+                                        ? __ldcg(all + (q0 + qq) * (NTOK * 128) + (c + t) * 128) : 0.0f;
+#pragma unroll
+                  for (int qq = 0; qq < QB; ++qq)
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) acc[t] += part[qq][t];
                 }
 #pragma unroll
                 for (int t = 0; t < 16; ++t) v[c + t] = __float_as_uint(acc[t]);
