@@ -360,7 +360,7 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
     // Launched as a programmatic dependent of whatever precedes it on the stream (in a decode loop
     // the GEMM of the layer before): it is scheduled early and waits inside the kernel.
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(static_cast<unsigned>((s * q.k + 127) / 128));
+    cfg.gridDim = dim3(static_cast<unsigned>((s * q.k + 31) / 32));  // four lanes per (token, block)
     cfg.blockDim = dim3(128);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];

@@ -16,7 +16,7 @@
 // scratch in global memory, no atomics).
 //
 // Warp roles: warp 0 = TMA producer (weights), warp 1 = MMA issuer and tensor-memory owner,
-// warps 2..5 = activation quantisers, then epilogue.
+// warps 2..5 = activation quantisers (four lanes per (token, block)), then epilogue.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -70,116 +70,110 @@ struct FusedParams {
   int64_t ldy;
 };
 
-// One (token, block): 32 bf16 values -> transformed, clipped, quantised: 16 code bytes + scale byte.
-// Same arithmetic as quantize_act_kernel (fp32 fused multiply-adds over the Kronecker form).
-__device__ __forceinline__ void item_transform_clip(const uint16_t* xp, const float* L, const float* R, bool clip,
-                                                    float c_lo, float c_hi, float (&o)[4][8], float& amax) {
-  // All loads of the item first (R: 16 x 16 bytes, L: 4 x 16 bytes, x: 4 x 16 bytes), so that their
-  // latencies overlap: at this size the kernel is a chain of latencies.  The factors are constants
-  // of the layer and are requested before the wait for the previous grid; x, which that grid may
-  // have produced, after it.
-  float Rr[64], Lr[16];
-  if (L != nullptr) {
+// One (token, block) is worked on by FOUR lanes of a warp: lane r of the group holds row r of the
+// block's 4 x 8 matrix V and produces row r of V~ = L^T V R (Algorithm 1), i.e. 8 of the 32 outputs
+// and one 32-bit word of codes.  Same arithmetic, in the same order, as quantize_act_kernel (fp32
+// fused multiply-adds over the Kronecker form).  At this size a kernel is a chain of latencies: a
+// short instruction stream per lane (the code is executed once, from a cold instruction cache)
+// counts for more than the number of lanes.
+//
+// The constants of the layer; requested before the wait for the previous grid.
+struct QuadFactors {
+  float R[64];  // right factor, [cc][c]
+  float Lc[4];  // column r of the left factor: L[4 i + r], i = 0..3
+  float c_lo, c_hi;
+};
+
+// Lanes without an item (valid = false) get zeros and read nothing.
+__device__ __forceinline__ void quad_load_factors(bool valid, const float* L, const float* R, const float* clip_lo,
+                                                  const float* clip_hi, int j, int r, QuadFactors& f) {
+  const bool xf = valid && L != nullptr;
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const float4 t = __ldg(reinterpret_cast<const float4*>(R) + i);
-      Rr[4 * i] = t.x; Rr[4 * i + 1] = t.y; Rr[4 * i + 2] = t.z; Rr[4 * i + 3] = t.w;
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float4 t = __ldg(reinterpret_cast<const float4*>(L) + i);
-      Lr[4 * i] = t.x; Lr[4 * i + 1] = t.y; Lr[4 * i + 2] = t.z; Lr[4 * i + 3] = t.w;
-    }
+  for (int i = 0; i < 16; ++i) {
+    const float4 t = xf ? __ldg(reinterpret_cast<const float4*>(R) + i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    f.R[4 * i] = t.x; f.R[4 * i + 1] = t.y; f.R[4 * i + 2] = t.z; f.R[4 * i + 3] = t.w;
   }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) f.Lc[i] = xf ? __ldg(L + 4 * i + r) : 0.0f;
+  f.c_lo = (valid && clip_lo != nullptr) ? __ldg(clip_lo + j) : 1.0f;
+  f.c_hi = (valid && clip_hi != nullptr) ? __ldg(clip_hi + j) : 1.0f;
+}
+
+// Row r of the block (8 bf16 at xrow) -> this lane's 8 transformed, clipped values and the block's
+// amax (the same in the four lanes).  Every lane of the warp calls this (shuffles inside); lanes
+// without an item pass valid = false and get zeros.  x is read after the wait for the previous grid.
+__device__ __forceinline__ void quad_transform_clip(const uint16_t* xrow, bool valid, bool xform, bool clip,
+                                                    const QuadFactors& f, int lane, float (&o)[8], float& amax) {
   grid_dependency_wait();
-  uint4 q[4];
+  uint4 q = make_uint4(0u, 0u, 0u, 0u);
+  if (valid) q = ld_global_ordered_v4(xrow);
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+  float v[8];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) q[i] = ld_global_ordered_v4(reinterpret_cast<const uint4*>(xp) + i);
-  float v[4][8];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const uint32_t w[4] = {q[i].x, q[i].y, q[i].z, q[i].w};
-#pragma unroll
-    for (int h = 0; h < 4; ++h) {
-      v[i][2 * h] = __uint_as_float(w[h] << 16);
-      v[i][2 * h + 1] = __uint_as_float(w[h] & 0xFFFF0000u);
-    }
+  for (int h = 0; h < 4; ++h) {
+    v[2 * h] = __uint_as_float(w[h] << 16);
+    v[2 * h + 1] = __uint_as_float(w[h] & 0xFFFF0000u);
   }
-  if (L != nullptr) {
-    float U[4][8];
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        float acc = v[i][0] * Rr[c];
-#pragma unroll
-        for (int cc = 1; cc < 8; ++cc) acc = fmaf(v[i][cc], Rr[cc * 8 + c], acc);
-        U[i][c] = acc;
-      }
-#pragma unroll
-    for (int r = 0; r < 4; ++r)
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        float acc = Lr[r] * U[0][c];
-#pragma unroll
-        for (int i = 1; i < 4; ++i) acc = fmaf(Lr[4 * i + r], U[i][c], acc);
-        o[r][c] = acc;
-      }
-  } else {
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int c = 0; c < 8; ++c) o[i][c] = v[i][c];
-  }
-  float mn = o[0][0], mx = o[0][0];
-#pragma unroll
-  for (int r = 0; r < 4; ++r)
+  if (xform) {
+    float U[8];  // row r of V R
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
-      mn = fminf(mn, o[r][c]);
-      mx = fmaxf(mx, o[r][c]);
+      float acc = v[0] * f.R[c];
+#pragma unroll
+      for (int cc = 1; cc < 8; ++cc) acc = fmaf(v[cc], f.R[cc * 8 + c], acc);
+      U[c] = acc;
     }
+    const int base = lane & ~3;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {  // row r of L^T (V R): the rows of V R come from the other lanes
+      float acc = f.Lc[0] * __shfl_sync(0xFFFFFFFFu, U[c], base);
+#pragma unroll
+      for (int i = 1; i < 4; ++i) acc = fmaf(f.Lc[i], __shfl_sync(0xFFFFFFFFu, U[c], base + i), acc);
+      o[c] = acc;
+    }
+  } else {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) o[c] = v[c];
+  }
+  float mn = o[0], mx = o[0];
+#pragma unroll
+  for (int c = 1; c < 8; ++c) {
+    mn = fminf(mn, o[c]);
+    mx = fmaxf(mx, o[c]);
+  }
+#pragma unroll
+  for (int d = 1; d < 4; d <<= 1) {
+    mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, d));
+    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, d));
+  }
   if (clip) {
-    const float lo = c_lo * mn, hi = c_hi * mx;
+    const float lo = f.c_lo * mn, hi = f.c_hi * mx;
 #pragma unroll
-    for (int r = 0; r < 4; ++r)
-#pragma unroll
-      for (int c = 0; c < 8; ++c) o[r][c] = fminf(fmaxf(o[r][c], lo), hi);
+    for (int c = 0; c < 8; ++c) o[c] = fminf(fmaxf(o[c], lo), hi);
     amax = fmaxf(fabsf(fminf(fmaxf(mn, lo), hi)), fabsf(fminf(fmaxf(mx, lo), hi)));
   } else {
     amax = fmaxf(fabsf(mn), fabsf(mx));
   }
 }
 
-// The transformed and clipped block -> 16 code bytes + scale byte (MXFP4, Sec. 2).
-__device__ __forceinline__ void item_encode(const float (&o)[4][8], float amax, uint32_t (&cw)[4], uint32_t& sbyte) {
+// This lane's 8 values -> one word of codes; the block's scale byte (MXFP4, Sec. 2).
+__device__ __forceinline__ void quad_encode(const float (&o)[8], float amax, uint32_t& cw, uint32_t& sbyte) {
   // shared scale: byte = max(biased_exponent(amax) - 2, 0) = clamp(floor(log2 amax) - 2) + 127
   const int ef = static_cast<int>(__float_as_uint(amax) >> 23);
   const int sb = max(ef - 2, 0);
   const float inv = __uint_as_float(static_cast<uint32_t>(254 - sb) << 23);
+  float uu[8];
 #pragma unroll
-  for (int r = 0; r < 4; ++r) {
-    float uu[8];
-#pragma unroll
-    for (int c = 0; c < 8; ++c) uu[c] = o[r][c] * inv;
-    cw[r] = e2m1x8_pack(uu);
-  }
+  for (int c = 0; c < 8; ++c) uu[c] = o[c] * inv;
+  cw = e2m1x8_pack(uu);
   sbyte = static_cast<uint32_t>(sb);
 }
 
-__device__ __forceinline__ void fused_quant_item(const uint16_t* xp, const float* L, const float* R, bool clip,
-                                                 float c_lo, float c_hi, uint32_t (&cw)[4], uint32_t& sbyte) {
-  float o[4][8];
-  float amax;
-  item_transform_clip(xp, L, R, clip, c_lo, c_hi, o, amax);
-  item_encode(o, amax, cw, sbyte);
-}
-
 // ---------------------------------------------------------------------------------------------
-// Stages 1+2 alone for a handful of tokens: one (token, block) per thread, everything loaded
-// up front, no shared-memory ring -- a launch of a few microseconds in front of the small-s GEMM,
-// whose weight stream it releases at once (programmatic dependent launch).  Also clears the
-// GEMM's split-K tickets.
+// Stages 1+2 alone for a handful of tokens: four lanes per (token, block), the factors requested
+// before the wait for the previous grid and x right after it, no shared-memory ring -- a launch of
+// a few microseconds in front of the small-s GEMM, whose weight stream it releases at once
+// (programmatic dependent launch).  Also clears the GEMM's split-K tickets.
 struct QuantSmallParams {
   const uint16_t* x;     // bf16 bits [s x n], row stride ld
   int64_t ld;
@@ -204,36 +198,35 @@ struct QuantSmallParams {
 template <bool DEBUG_OUT>
 __global__ void __launch_bounds__(128) quantize_act_small_kernel(const QuantSmallParams p) {
   grid_launch_dependents();
-  const int64_t item = static_cast<int64_t>(blockIdx.x) * 128 + threadIdx.x;
-  if (item >= static_cast<int64_t>(p.s) * p.k || blockIdx.x == 0) {
-    // Nothing is written before the grid in front of this one has finished: it may still read
-    // the codes, scales and tickets of its own call.
-    grid_dependency_wait();
-    if (blockIdx.x == 0)
-      for (int i = threadIdx.x; i < p.n_zero_words; i += 128) p.zero_words[i] = 0u;
-    if (item >= static_cast<int64_t>(p.s) * p.k) return;
-  }
-  const int64_t row = item / p.k;
-  const int j = static_cast<int>(item - row * p.k);
-  const bool clip = p.clip_lo != nullptr;
-  const float* L = p.left ? p.left + static_cast<int64_t>(j) * p.left_stride : nullptr;
-  const float* R = p.left ? p.right + static_cast<int64_t>(j) * p.right_stride : nullptr;
-  float o[4][8];
+  const int lane = threadIdx.x & 31;
+  const int64_t gt = static_cast<int64_t>(blockIdx.x) * 128 + threadIdx.x;
+  const int r = static_cast<int>(gt & 3);
+  const int64_t item = gt >> 2;
+  const bool valid = item < static_cast<int64_t>(p.s) * p.k;
+  const int64_t row = valid ? item / p.k : 0;
+  const int j = valid ? static_cast<int>(item - row * p.k) : 0;
+  const bool xform = p.left != nullptr, clip = p.clip_lo != nullptr;
+  QuadFactors f;
+  quad_load_factors(valid, xform ? p.left + static_cast<int64_t>(j) * p.left_stride : nullptr,
+                    xform ? p.right + static_cast<int64_t>(j) * p.right_stride : nullptr, p.clip_lo, p.clip_hi, j, r, f);
+  float o[8];
   float amax;
-  item_transform_clip(p.x + row * p.ld + static_cast<int64_t>(j) * 32, L, R, clip, clip ? __ldg(p.clip_lo + j) : 1.0f,
-                      clip ? __ldg(p.clip_hi + j) : 1.0f, o, amax);
+  quad_transform_clip(p.x + row * p.ld + static_cast<int64_t>(j) * 32 + r * 8, valid, xform, clip, f, lane, o, amax);
+  // Past the wait inside quad_transform_clip: the grid in front of this one has finished and no
+  // longer reads the codes, scales and tickets of its own call.
+  if (blockIdx.x == 0)
+    for (int i = threadIdx.x; i < p.n_zero_words; i += 128) p.zero_words[i] = 0u;
+  if (!valid) return;
   if (DEBUG_OUT) {
-    float4* dst = reinterpret_cast<float4*>(p.debug_out + row * p.n + static_cast<int64_t>(j) * 32);
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      dst[2 * r] = make_float4(o[r][0], o[r][1], o[r][2], o[r][3]);
-      dst[2 * r + 1] = make_float4(o[r][4], o[r][5], o[r][6], o[r][7]);
-    }
+    float4* dst = reinterpret_cast<float4*>(p.debug_out + row * p.n + static_cast<int64_t>(j) * 32 + r * 8);
+    dst[0] = make_float4(o[0], o[1], o[2], o[3]);
+    dst[1] = make_float4(o[4], o[5], o[6], o[7]);
     return;
   }
-  uint32_t cw[4], sbyte;
-  item_encode(o, amax, cw, sbyte);
-  *reinterpret_cast<uint4*>(p.codes + row * (p.n / 2) + static_cast<int64_t>(j) * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+  uint32_t cw, sbyte;
+  quad_encode(o, amax, cw, sbyte);
+  *reinterpret_cast<uint32_t*>(p.codes + row * (p.n / 2) + static_cast<int64_t>(j) * 16 + r * 4) = cw;
+  if (r != 0) return;
   if (p.sf_layout == 0) {
     p.scales[row * p.k + j] = static_cast<uint8_t>(sbyte);
   } else {
@@ -374,25 +367,31 @@ linear_small_s_fused_kernel(const __grid_constant__ CUtensorMap tmap_w, const Fu
     __syncwarp();
   } else {
     // ---------------------------------------------------------------- activation quantisers, then epilogue
-    const int qt = tid - 64;                 // 0..127
+    const int qt = tid - 64;                 // 0..127: four lanes per (token, block), 32 items per pass
+    const int r = qt & 3;
     const int nb = n_steps * 8;              // blocks of this CTA's K slice
-    const bool clip = p.clip_lo != nullptr;
-    for (int item = qt; item < p.s * nb; item += 128) {
-      const int t = item / nb;
-      const int jj = item - t * nb;
+    const int total = p.s * nb;
+    const bool xform = p.left != nullptr, clip = p.clip_lo != nullptr;
+    for (int it0 = 0; it0 < total; it0 += 32) {  // the same trip count in every lane (shuffles inside)
+      const int item = it0 + (qt >> 2);
+      const bool valid = item < total;
+      const int t = valid ? item / nb : 0;
+      const int jj = valid ? item - t * nb : 0;
       const int j = kt0 * 8 + jj;
-      uint32_t cw[4] = {0u, 0u, 0u, 0u};
-      uint32_t sbyte = 0u;                   // blocks past the last channel: zero codes, finite scale
-      if (j < p.k) {
-        const float* L = p.left ? p.left + static_cast<int64_t>(j) * p.left_stride : nullptr;
-        const float* R = p.left ? p.right + static_cast<int64_t>(j) * p.right_stride : nullptr;
-        fused_quant_item(p.x + t * p.ld + static_cast<int64_t>(j) * 32, L, R, clip, clip ? __ldg(p.clip_lo + j) : 1.0f,
-                         clip ? __ldg(p.clip_hi + j) : 1.0f, cw, sbyte);
+      const bool real = valid && j < p.k;    // blocks past the last channel: zero codes, finite scale
+      QuadFactors f;
+      quad_load_factors(real, xform ? p.left + static_cast<int64_t>(j) * p.left_stride : nullptr,
+                        xform ? p.right + static_cast<int64_t>(j) * p.right_stride : nullptr, p.clip_lo, p.clip_hi, j, r, f);
+      float o[8];
+      float amax;
+      quad_transform_clip(p.x + t * p.ld + static_cast<int64_t>(j) * 32 + r * 8, real, xform, clip, f, lane, o, amax);
+      uint32_t cw = 0u, sbyte = 0u;
+      if (real) quad_encode(o, amax, cw, sbyte);
+      if (valid) {
+        const int step = jj >> 3, c = jj & 7;
+        *reinterpret_cast<uint32_t*>(x_codes + step * Cfg::kXStepBytes + t * 128 + ((c ^ (t & 7)) << 4) + r * 4) = cw;
+        if (r == 0) x_sf[step * Cfg::kSfBytes + (c >> 2) * 512 + t * 16 + (c & 3)] = static_cast<uint8_t>(sbyte);
       }
-      const int step = jj >> 3, c = jj & 7;
-      *reinterpret_cast<uint4*>(x_codes + step * Cfg::kXStepBytes + t * 128 + ((c ^ (t & 7)) << 4)) =
-          make_uint4(cw[0], cw[1], cw[2], cw[3]);
-      x_sf[step * Cfg::kSfBytes + (c >> 2) * 512 + t * 16 + (c & 3)] = static_cast<uint8_t>(sbyte);
     }
     grid_dependency_wait();  // threads without an item: these warps write y below
     fence_proxy_async_smem();
