@@ -294,6 +294,7 @@ def run_ours(args):
     B.batq_debug_force_gemm_kernel(args.gemm_kernel)
     B.batq_debug_force_small_s_splits(args.splits)
     B.batq_debug_force_small_s_path(args.small_path)
+    B.batq_debug_force_small_s_reduce(args.small_reduce)
     peaks = load_peaks()
     kind, tokens, projs, _, _ = WORKLOADS[args.workload]
     # prefill: long enough (> 1 s) for the power cap to settle, so that the sustained peak is the fair denominator
@@ -400,10 +401,12 @@ def run_ours(args):
         })
 
     elif kind == "decode":
-        # Per call: quantiser + small-s GEMM (one batq_linear_w4a4).  A decode loop is launch-bound
-        # from Python, so each case is captured once as a CUDA graph of `copies` calls, one per copy of
-        # the prepared weight: the copies cycle through more than 3 x L2 between reuses, so no call
-        # finds its weights in L2.  A step replays the graph of every case; events bracket each replay.
+        # Per call: quantiser + small-s GEMM, or the fused kernel (one batq_linear_w4a4).  A decode loop
+        # is launch-bound from Python, so for every token count the projections of `copies` layers, in
+        # model order (qkv, o, gate/up, down; layer after layer, each layer with its own copy of the
+        # prepared weights), are captured once as ONE CUDA graph.  The copies cycle through more than
+        # 3 x L2 between reuses, so no call finds its weights in L2.  A step replays the graph of every
+        # token count; events bracket each replay.
         copies = 4
         base = make_layer_inputs(args.workload, max(tokens), seed)
         cases = []
@@ -418,37 +421,64 @@ def run_ours(args):
                      "y": torch.empty((S, L["m"]), dtype=torch.bfloat16, device="cuda"),
                      "ws": B.aligned_workspace(B.batq_linear_workspace_bytes(L["ws_list"][0], S)),
                      "x_host": torch.from_numpy(L["x_bits"][:S].copy().view(np.int16)).pin_memory(),
-                     "y_host": torch.empty((S, L["m"]), dtype=torch.bfloat16).pin_memory()}
+                     "y_host": torch.empty((S, L["m"]), dtype=torch.bfloat16).pin_memory(),
+                     "launches": B.batq_linear_kernel_launches(L["tr"], L["ws_list"][0], S)}
                 cases.append(c)
         order = [c for S in tokens for c in cases if c["S"] == S]   # all projections at S=1, then S=4, ...
+
+        def call(c, layer):
+            B.batq_linear_w4a4(c["L"]["tr"], c["L"]["ws_list"][layer], c["x"], c["y"], c["ws"])
+
         side = torch.cuda.Stream()
+        layer_graphs = {}
         with torch.cuda.stream(side):
             for c in order:
-                for w in c["L"]["ws_list"]:   # first calls outside capture: per-device set-up
-                    B.batq_linear_w4a4(c["L"]["tr"], w, c["x"], c["y"], c["ws"])
+                for layer in range(copies):   # first calls outside capture: per-device set-up
+                    call(c, layer)
             torch.cuda.synchronize()
-            for c in order:
+            for S in tokens:
+                layer_graphs[S] = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(layer_graphs[S], stream=side):
+                    for layer in range(copies):
+                        for c in order:
+                            if c["S"] == S:
+                                call(c, layer)
+            for c in order:                   # per-projection detail: each case alone, `copies` calls
                 c["graph"] = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(c["graph"], stream=side):
-                    for w in c["L"]["ws_list"]:
-                        B.batq_linear_w4a4(c["L"]["tr"], w, c["x"], c["y"], c["ws"])
+                    for layer in range(copies):
+                        call(c, layer)
         torch.cuda.synchronize()
         flops_step = copies * sum(2.0 * c["S"] * c["L"]["n"] * c["L"]["m"] for c in order)
-        marks = [[(ev(), ev()) for _ in order] for _ in range(steps)]
+        marks = [[(ev(), ev()) for _ in tokens] for _ in range(steps)]
 
         def step(k):
-            for i, c in enumerate(order):
+            for i, S in enumerate(tokens):
                 if k is not None:
                     marks[k][i][0].record()
-                c["graph"].replay()
+                layer_graphs[S].replay()
                 if k is not None:
                     marks[k][i][1].record()
 
         ms, clocks = timed_region(h, step, steps, args.warmup)
-        c_ms = np.array([[m[i][0].elapsed_time(m[i][1]) for i in range(len(order))] for m in marks]) / copies
+        l_ms = np.array([[m[i][0].elapsed_time(m[i][1]) for i in range(len(tokens))] for m in marks]) / copies
+        layer_bytes = sum(L["n"] * L["m"] * WEIGHT_BYTES_PER_ELEM for L in base)
+        gbs = layer_bytes * len(tokens) / (l_ms.mean(axis=0).sum() * 1e-3) / 1e9
+
+        # Per-projection detail, outside the timed region: every case in a graph of its own.
+        d_steps = max(3, min(steps, 50))
+        d_marks = [[(ev(), ev()) for _ in order] for _ in range(d_steps)]
+        for k in range(-3, d_steps):
+            for i, c in enumerate(order):
+                if k >= 0:
+                    d_marks[k][i][0].record()
+                c["graph"].replay()
+                if k >= 0:
+                    d_marks[k][i][1].record()
+        torch.cuda.synchronize()
+        c_ms = np.array([[m[i][0].elapsed_time(m[i][1]) for i in range(len(order))] for m in d_marks]) / copies
         c_med = np.median(c_ms, axis=0)
         w_bytes = [c["L"]["n"] * c["L"]["m"] * WEIGHT_BYTES_PER_ELEM for c in order]
-        gbs = sum(w_bytes) / (c_ms.mean(axis=0).sum() * 1e-3) / 1e9
 
         def step_host():
             for c in order:
@@ -470,20 +500,27 @@ def run_ours(args):
             "value": h.whole_job_rate(flops_step, steps, ms) / 1e12, "ms_per_step": ms / steps,
             "config": {"workload": args.workload, "tokens": tokens, "projections": [list(p) for p in projs],
                        "transform": "shared 4x4 (x) private 8x8 per 32-group, clip U[0.8,1]", "output": "bf16",
-                       "launch": "one CUDA graph of %d calls per (tokens, projection) case" % copies,
+                       "launch": "per token count one CUDA graph of %d layers x %d projections in model order" % (
+                           copies, len(base)),
                        "l2": "%d copies of each prepared weight used in turn: %.0f MB cycle through L2 between reuses" % (
                            copies, copies * sum(L["n"] * L["m"] * WEIGHT_BYTES_PER_ELEM for L in base) / 1e6)},
             "roofline": {"bound": "hbm", "kernel": "gemm_small_s_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
-                         "peak_source": "%s copy bandwidth; achieved = weight bytes / whole-call time (quantiser + GEMM)" %
-                                        peaks["source"]},
+                         "peak_source": "%s copy bandwidth; achieved = weight bytes / time of the layer graphs "
+                                        "(quantisers + GEMMs)" % peaks["source"]},
+            "layers": [{"tokens": S, "layer_us": float(l_ms[:, i].mean() * 1e3),
+                        "layer_us_median": float(np.median(l_ms[:, i]) * 1e3),
+                        "weight_gbs": layer_bytes / (l_ms[:, i].mean() * 1e-3) / 1e9} for i, S in enumerate(tokens)],
             "kernels": [{"name": c["L"]["name"], "tokens": c["S"], "n": c["L"]["n"], "m": c["L"]["m"],
+                         "launches_per_call": c["launches"],
                          "call_us": float(c_ms[:, i].mean() * 1e3), "call_us_median": float(c_med[i] * 1e3),
                          "weight_gbs": w_bytes[i] / (c_ms[:, i].mean() * 1e-3) / 1e9} for i, c in enumerate(order)],
+            "kernels_note": "per projection, outside the timed region: each case alone in a graph of %d calls "
+                            "(includes that short graph's launch and ramp)" % copies,
             "e2e": {"value": flops_step / copies * e2e_steps * h.world / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                     "note": "one eager host-buffer call per case and step (no graph)"},
-            "gpu_launches": 2 * copies * len(order) * steps,
+            "gpu_launches": copies * sum(c["launches"] for c in order) * steps,
         })
 
     else:  # quantiser sweep
@@ -589,6 +626,7 @@ def main():
     ap.add_argument("--gemm-kernel", type=int, default=0, help="0 auto, 1 one CTA per tile, 2 CTA pairs (tuning)")
     ap.add_argument("--tile-width", type=int, default=0, help="force the GEMM tile width (tuning); 0 = automatic")
     ap.add_argument("--small-path", type=int, default=0, help="0 auto, 1 two kernels, 2 fused kernel (tuning)")
+    ap.add_argument("--small-reduce", type=int, default=0, help="0 auto, 1 tickets, 2 cluster (split-K reduction, tuning)")
     ap.add_argument("--splits", type=int, default=0, help="force the small-s GEMM's K splits (tuning); 0 = automatic")
     args = ap.parse_args()
     if args.impl == "reference":

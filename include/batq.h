@@ -201,6 +201,9 @@ void batq_debug_force_small_s_path(int32_t which);
  *              aligned; overwritten by every call (calls sharing a workspace
  *              must be ordered on one stream). */
 size_t batq_linear_workspace_bytes(const batq_weight* w, int64_t s);
+/* How many kernels one batq_linear_w4a4(t, w, ., s, ...) call launches with the current dispatch
+ * (1 = the fused kernel, 2 = quantiser + GEMM); 0 for a NULL weight or s <= 0.  Host only. */
+int32_t batq_linear_kernel_launches(const batq_transform* t, const batq_weight* w, int64_t s);
 batq_status batq_linear_w4a4(const batq_transform* t, const batq_weight* w, const void* x_bf16,
                              int64_t s, int64_t ld, void* y, int32_t y_dtype, int64_t ldy,
                              void* workspace, size_t workspace_bytes, void* stream);

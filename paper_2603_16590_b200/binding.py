@@ -46,6 +46,7 @@ SIGNATURES = {
     "batq_debug_force_gemm_kernel": (None, [_I32]),
     "batq_debug_force_quantizer": (None, [_I32]),
     "batq_linear_workspace_bytes": (_SZ, [_P, _I64]),
+    "batq_linear_kernel_launches": (C.c_int32, [_P, _P, _I64]),
     "batq_linear_w4a4": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P, _SZ, _P]),
     "batq_linear_w4a4_host": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _P, _P, _P, _SZ, _P]),
     "batq_static_workspace_capacity": (_SZ, []),
@@ -247,6 +248,10 @@ def batq_debug_force_quantizer(which: int):
 
 def batq_linear_workspace_bytes(w: Weight, s) -> int:
     return load().batq_linear_workspace_bytes(w.handle, s)
+
+
+def batq_linear_kernel_launches(t, w: Weight, s) -> int:
+    return load().batq_linear_kernel_launches(t.handle if t is not None else None, w.handle, s)
 
 
 def aligned_workspace(nbytes, device="cuda"):

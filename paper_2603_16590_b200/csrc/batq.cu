@@ -571,8 +571,20 @@ constexpr int kMaxSplits = 32;
 
 inline int small_ntok(int64_t s) { return s <= 16 ? 16 : (s <= 32 ? 32 : 64); }
 
+
+// The K splits of a row tile can meet as one thread-block cluster (reduction through distributed
+// shared memory) when there are at most 8 of them and the grid leaves the gang scheduler of
+// clusters some room: at most 90 % of the two-per-SM slots (measured: a fuller grid of clusters
+// no longer fits one wave).
+bool cluster_reduce_ok(int64_t tiles, int sp, int64_t slots) {
+  if (sp < 2 || sp > 8 || g_small_reduce == 1) return false;
+  return g_small_reduce == 2 || tiles * sp * 10 <= slots * 9;
+}
+
 // Number of K splits: the grid is (row tiles) x (splits) CTAs, two resident per SM.  Modelled
-// time = waves x (K-steps per CTA + fixed cost) + a reduction term that grows with the splits.
+// time = waves x (K-steps per CTA + fixed cost) + a reduction term that grows with the splits,
+// plus the round trip through scratch and tickets where the cluster reduction does not apply
+// (all in units of one K-step of streaming, about 0.5 us).
 int pick_splits(int64_t m, int64_t n, int sm_count) {
   const int k_steps = static_cast<int>((n + 255) / 256);
   if (g_force_splits > 0) return std::min(std::min(g_force_splits, k_steps), kMaxSplits);
@@ -582,7 +594,8 @@ int pick_splits(int64_t m, int64_t n, int sm_count) {
   double best_cost = 1e30;
   for (int sp = 1; sp <= std::min(k_steps, kMaxSplits); ++sp) {
     const int64_t waves = (tiles * sp + slots - 1) / slots;
-    const double cost = static_cast<double>(waves) * ((k_steps + sp - 1) / sp + 3.0) + 0.15 * sp;
+    double cost = static_cast<double>(waves) * ((k_steps + sp - 1) / sp + 3.0) + 0.15 * sp;
+    if (sp > 1 && !cluster_reduce_ok(tiles, sp, slots)) cost += 2.0;
     if (cost < best_cost - 1e-9) { best_cost = cost; best = sp; }
   }
   return best;
@@ -657,13 +670,7 @@ batq_status launch_gemm_small(const void* x_codes, const void* x_sf, const batq_
   p.ldy = ldy;
   p.partial = reinterpret_cast<float*>(scratch);
   p.tickets = reinterpret_cast<uint32_t*>(scratch + sc.partial_bytes);
-  // Cluster reduction where it measured faster than tickets: few tokens (the leader reads
-  // tokens x splits remote values per thread) and a grid that leaves the gang scheduler of
-  // clusters some room (<= 90 % of the two-per-SM slots); 2 = forced on whenever splits <= 8.
-  const int64_t slots = 2 * static_cast<int64_t>(info->sm_count);
-  const bool fits = sc.splits > 1 && sc.splits <= 8;
-  p.cluster_reduce = (fits && (g_small_reduce == 2 ||
-                               (g_small_reduce == 0 && s <= 4 && sc.tiles * sc.splits * 10 <= slots * 9))) ? 1 : 0;
+  p.cluster_reduce = cluster_reduce_ok(sc.tiles, sc.splits, 2 * static_cast<int64_t>(info->sm_count)) ? 1 : 0;
   const dim3 grid(static_cast<unsigned>(sc.tiles), static_cast<unsigned>(sc.splits));
   const bool bf = y_dtype == BATQ_BF16;
   cudaError_t e;
@@ -1047,6 +1054,11 @@ size_t batq_linear_workspace_bytes(const batq_weight* w, int64_t s) {
   if (w == nullptr || s < 0) return 0;
   const size_t q = round_up(static_cast<size_t>(s * (w->n / 2)), 1024) + round_up(batq_sf_bytes(s, w->n, BATQ_SF_MMA), 1024);
   return q + (s > 0 && s <= kSmallSMax ? small_scratch(w, s).total() : 0);
+}
+
+int32_t batq_linear_kernel_launches(const batq_transform* t, const batq_weight* w, int64_t s) {
+  if (w == nullptr || s <= 0) return 0;
+  return use_fused_small(t, w, s) ? 1 : 2;
 }
 
 batq_status batq_linear_w4a4(const batq_transform* t, const batq_weight* w, const void* x_bf16, int64_t s, int64_t ld,

@@ -9,9 +9,10 @@
 // columns), so no tensor-core row is spent on padding tokens.  The grid is
 // (row tiles) x (K splits): enough CTAs, two per SM, to keep the whole memory system
 // busy however few output features the layer has.  With more than one split every CTA
-// keeps its partial tile for a reduction in split order (deterministic): up to 8 splits form a
-// thread-block cluster whose leader reads the others' tiles from distributed shared memory;
-// beyond that the tiles go to scratch and the CTA that draws the last ticket of a row tile adds them.
+// keeps its partial tile for a reduction in split order (deterministic): up to 8 splits can form a
+// thread-block cluster that reduce-scatters the tiles through distributed shared memory (CTA q
+// adds and writes tokens q, q + splits, ...); otherwise the tiles go to scratch and the CTA that
+// draws the last ticket of a row tile adds them.
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and tensor-memory owner,
 // warps 2..5 = epilogue.  The weight stream does not depend on the activation
@@ -326,36 +327,30 @@ gemm_small_s_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     // Every thread of every CTA of the cluster takes both barriers, whatever happened above.
     __syncthreads();
     cluster_sync_all();
-    if (warp >= 2 && sp == 0 && epi_ok) {
+    if (warp >= 2 && epi_ok) {
+      // Reduce-scatter: CTA sp adds, in split order (deterministic), the partial sums of tokens
+      // sp, sp + splits, ... -- its own from local, the others' from distributed shared memory --
+      // and writes those tokens of y.
       const int row = (warp & 3) * 32 + lane;
       const int64_t mrow = static_cast<int64_t>(rt) * 128 + row;
       const uint32_t mine = smem_u32(smem) + row * 4;
+      for (int t = sp; t < p.s; t += p.splits) {
+        float part[8];
 #pragma unroll
-      for (int t0 = 0; t0 < NTOK; t0 += 4) {
-        if (t0 < p.s) {
-          float part[7][4];
+        for (int q = 0; q < 8; ++q)
+          part[q] = q < p.splits ? ld_shared_cluster_f32(map_to_cta(mine + t * 512, q)) : 0.0f;
+        float acc = part[0];
 #pragma unroll
-          for (int q = 1; q < 8; ++q)
-#pragma unroll
-            for (int t = 0; t < 4; ++t)
-              part[q - 1][t] = (q < p.splits && t0 + t < p.s)
-                                   ? ld_shared_cluster_f32(map_to_cta(mine + (t0 + t) * 512, q)) : 0.0f;
-#pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            float acc = __uint_as_float(v[t0 + t]);  // split 0's own part, then splits 1.. in order
-#pragma unroll
-            for (int q = 1; q < 8; ++q) acc += part[q - 1][t];
-            if (t0 + t < p.s && mrow < p.m) {
-              if (OUT_BF16)
-                reinterpret_cast<__nv_bfloat16*>(p.y)[(t0 + t) * p.ldy + mrow] = __float2bfloat16_rn(acc);
-              else
-                reinterpret_cast<float*>(p.y)[(t0 + t) * p.ldy + mrow] = acc;
-            }
-          }
+        for (int q = 1; q < 8; ++q) acc += part[q];
+        if (mrow < p.m) {
+          if (OUT_BF16)
+            reinterpret_cast<__nv_bfloat16*>(p.y)[t * p.ldy + mrow] = __float2bfloat16_rn(acc);
+          else
+            reinterpret_cast<float*>(p.y)[t * p.ldy + mrow] = acc;
         }
       }
     }
-    cluster_sync_all();  // the leader has read everybody's shared memory
+    cluster_sync_all();  // nobody leaves while its shared memory may still be read
   }
   tc_fence_before_sync();
   __syncthreads();

@@ -11,9 +11,9 @@
 // producer streams the weight slice, the four warps that will later run the epilogue quantise
 // the matching slice of the s activation rows straight into shared memory, in the operand
 // layout the MMA reads (the activations are tiny: every CTA of a K split redoes the same few
-// blocks).  The K splits of a row tile form a thread-block cluster; their partial tiles meet in
-// the leader's view of distributed shared memory and are added in rank order (deterministic; no
-// scratch in global memory, no atomics).
+// blocks).  The K splits of a row tile form a thread-block cluster; their partial tiles are
+// reduce-scattered through distributed shared memory (CTA q adds, in rank order, and writes tokens
+// q, q + splits, ...: deterministic; no scratch in global memory, no atomics).
 //
 // Warp roles: warp 0 = TMA producer (weights), warp 1 = MMA issuer and tensor-memory owner,
 // warps 2..5 = activation quantisers (four lanes per (token, block)), then epilogue.
@@ -424,33 +424,30 @@ linear_small_s_fused_kernel(const __grid_constant__ CUtensorMap tmap_w, const Fu
   tc_fence_before_sync();
   __syncthreads();
   cluster_sync_all();
-  if (warp >= 2 && sp == 0 && epi_ok) {
-    const int quad = warp & 3;
-    const int row = quad * 32 + lane;
+  if (warp >= 2 && epi_ok) {
+    const int row = (warp & 3) * 32 + lane;
     const int64_t mrow = static_cast<int64_t>(rt) * 128 + row;
     if (p.splits > 1) {
+      // Reduce-scatter: CTA sp adds, in rank order (deterministic), the partial sums of tokens sp,
+      // sp + splits, ... -- its own from local, the others' from distributed shared memory -- and
+      // writes those tokens of y.
       const uint32_t mine = smem_u32(x_codes) + row * 4;
+      for (int t = sp; t < p.s; t += p.splits) {
+        float part[kFusedMaxSplits];
 #pragma unroll
-      for (int t0 = 0; t0 < kFusedTok; t0 += 4) {
-        if (t0 < p.s) {
-          float part[kFusedMaxSplits - 1][4];
+        for (int q = 0; q < kFusedMaxSplits; ++q)
+          part[q] = q < p.splits ? ld_shared_cluster_f32(map_to_cta(mine + t * 512, q)) : 0.0f;
+        float acc = part[0];
 #pragma unroll
-          for (int q = 1; q < kFusedMaxSplits; ++q)
-#pragma unroll
-            for (int t = 0; t < 4; ++t)
-              part[q - 1][t] = (q < p.splits && t0 + t < p.s)
-                                   ? ld_shared_cluster_f32(map_to_cta(mine + (t0 + t) * 512, q)) : 0.0f;
-#pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            float acc = __uint_as_float(v[t0 + t]);  // rank 0's own part, then ranks 1.. in order
-#pragma unroll
-            for (int q = 1; q < kFusedMaxSplits; ++q) acc += part[q - 1][t];
-            v[t0 + t] = __float_as_uint(acc);
-          }
+        for (int q = 1; q < kFusedMaxSplits; ++q) acc += part[q];
+        if (mrow < p.m) {
+          if (OUT_BF16)
+            reinterpret_cast<__nv_bfloat16*>(p.y)[t * p.ldy + mrow] = __float2bfloat16_rn(acc);
+          else
+            reinterpret_cast<float*>(p.y)[t * p.ldy + mrow] = acc;
         }
       }
-    }
-    if (mrow < p.m) {
+    } else if (mrow < p.m) {
 #pragma unroll
       for (int t = 0; t < kFusedTok; ++t) {
         if (t < p.s) {
@@ -462,7 +459,7 @@ linear_small_s_fused_kernel(const __grid_constant__ CUtensorMap tmap_w, const Fu
       }
     }
   }
-  cluster_sync_all();  // the leader has read everybody's shared memory
+  cluster_sync_all();  // nobody leaves while its shared memory may still be read
   if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, Cfg::kTmemCols);

@@ -77,4 +77,5 @@ def test_host_validation_without_a_device(lib):
     assert lib.batq_prepare_weight(None, 16, 4, 128, 128, None, None, None, C.byref(h), None) == 1
     assert lib.batq_prepare_weight(None, 16, 4, 128, 128, None, None, 512, C.byref(h), None) == 3
     assert lib.batq_linear_workspace_bytes(None, 4) == 0
+    assert lib.batq_linear_kernel_launches(None, None, 4) == 0
     assert lib.batq_weight_destroy(None) == 0 and lib.batq_transform_destroy(None) == 0
