@@ -574,18 +574,20 @@ inline int small_ntok(int64_t s) { return s <= 16 ? 16 : (s <= 32 ? 32 : 64); }
 
 // The K splits of a row tile can meet as one thread-block cluster (reduction through distributed
 // shared memory) when there are at most 8 of them and the grid leaves the gang scheduler of
-// clusters some room: at most 90 % of the two-per-SM slots (measured: a fuller grid of clusters
-// no longer fits one wave).
-bool cluster_reduce_ok(int64_t tiles, int sp, int64_t slots) {
+// clusters some room: at most 90 % of the two-per-SM slots, 80 % above 4 tokens, where the CTAs
+// of the quantiser in front (tokens x blocks / 32 of them, resident while they wait) take room
+// too.  Measured: a fuller grid leaves a few clusters for a second wave, which costs a layer of
+// the decode benchmark about 5 us.
+bool cluster_reduce_ok(int64_t tiles, int sp, int64_t slots, int64_t s) {
   if (sp < 2 || sp > 8 || g_small_reduce == 1) return false;
-  return g_small_reduce == 2 || tiles * sp * 10 <= slots * 9;
+  return g_small_reduce == 2 || tiles * sp * 10 <= slots * (s > 4 ? 8 : 9);
 }
 
 // Number of K splits: the grid is (row tiles) x (splits) CTAs, two resident per SM.  Modelled
 // time = waves x (K-steps per CTA + fixed cost) + a reduction term that grows with the splits,
 // plus the round trip through scratch and tickets where the cluster reduction does not apply
 // (all in units of one K-step of streaming, about 0.5 us).
-int pick_splits(int64_t m, int64_t n, int sm_count) {
+int pick_splits(int64_t m, int64_t n, int64_t s, int sm_count) {
   const int k_steps = static_cast<int>((n + 255) / 256);
   if (g_force_splits > 0) return std::min(std::min(g_force_splits, k_steps), kMaxSplits);
   const int64_t tiles = (m + 127) / 128;
@@ -595,7 +597,7 @@ int pick_splits(int64_t m, int64_t n, int sm_count) {
   for (int sp = 1; sp <= std::min(k_steps, kMaxSplits); ++sp) {
     const int64_t waves = (tiles * sp + slots - 1) / slots;
     double cost = static_cast<double>(waves) * ((k_steps + sp - 1) / sp + 3.0) + 0.15 * sp;
-    if (sp > 1 && !cluster_reduce_ok(tiles, sp, slots)) cost += 2.0;
+    if (sp > 1 && !cluster_reduce_ok(tiles, sp, slots, s)) cost += 2.0;
     if (cost < best_cost - 1e-9) { best_cost = cost; best = sp; }
   }
   return best;
@@ -611,7 +613,7 @@ struct SmallScratch {
 SmallScratch small_scratch(const batq_weight* w, int64_t s) {
   SmallScratch sc{};
   sc.ntok = small_ntok(s);
-  sc.splits = pick_splits(w->m, w->n, w->sm_count);
+  sc.splits = pick_splits(w->m, w->n, s, w->sm_count);
   sc.tiles = (w->m + 127) / 128;
   sc.partial_bytes = sc.splits > 1 ? round_up(static_cast<size_t>(sc.tiles) * sc.splits * sc.ntok * 128 * 4, 1024) : 0;
   sc.ticket_bytes = round_up(static_cast<size_t>(sc.tiles) * 4, 1024);
@@ -670,7 +672,7 @@ batq_status launch_gemm_small(const void* x_codes, const void* x_sf, const batq_
   p.ldy = ldy;
   p.partial = reinterpret_cast<float*>(scratch);
   p.tickets = reinterpret_cast<uint32_t*>(scratch + sc.partial_bytes);
-  p.cluster_reduce = cluster_reduce_ok(sc.tiles, sc.splits, 2 * static_cast<int64_t>(info->sm_count)) ? 1 : 0;
+  p.cluster_reduce = cluster_reduce_ok(sc.tiles, sc.splits, 2 * static_cast<int64_t>(info->sm_count), s) ? 1 : 0;
   const dim3 grid(static_cast<unsigned>(sc.tiles), static_cast<unsigned>(sc.splits));
   const bool bf = y_dtype == BATQ_BF16;
   cudaError_t e;
