@@ -165,8 +165,17 @@ batq_status batq_gemm_mxfp4_small_s(const void* x_codes, const void* x_scales_mm
                                     size_t scratch_bytes, void* stream);
 
 /* Test / tuning hook: forces the GEMM's output-tile width to 128, 192 or 256 columns for all
- * later calls in this process; any other value restores the automatic choice. */
+ * later calls in this process (the CTA-pair kernel also takes 64, and 448 for columns of 256 and
+ * 192 alternating); any other value restores the automatic choice. */
 void batq_debug_force_tile_width(int32_t bn);
+
+/* Host only, no GPU needed: the work distribution of the CTA-pair GEMM for an s x m output
+ * over n input channels on a device with sm_count SMs.  pair < 0: returns the number of CTA pairs
+ * launched.  Otherwise returns the number of tiles pair `pair` works through, in order, and
+ * writes the first max_tiles of them to tiles (host, 3 ints each: index of the 256-token row
+ * block, first output feature, width in features).  -1 for arguments out of range. */
+int32_t batq_debug_pair_schedule(int64_t s, int64_t m, int64_t n, int32_t sm_count, int32_t pair,
+                                 int32_t* tiles, int32_t max_tiles);
 /* Test / tuning hook: which prefill GEMM kernel later calls use.  0 = automatic (CTA pairs sharing a
  * 256-token tile for s > 128, one CTA per 128-token tile otherwise), 1 = always one CTA per tile,
  * 2 = always CTA pairs (tile widths 192 and 256 only). */

@@ -6,6 +6,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <climits>
 #include <cmath>
 #include <cstring>
 #include <mutex>
@@ -45,10 +46,10 @@ struct batq_weight {
   int32_t sm_count;  // of the device the weight lives on (sizes the small-s split-K scratch)
   uint8_t* codes;   // [m x n/2]
   uint8_t* scales;  // BATQ_SF_MMA
-  CUtensorMap tmap_b256;  // boxes of 256 / 192 / 128 / 96 weight rows x 128 bytes
+  CUtensorMap tmap_b256;  // boxes of 256 / 192 / 128 weight rows x 128 bytes
   CUtensorMap tmap_b192;
   CUtensorMap tmap_b128;
-  CUtensorMap tmap_b96;
+  CUtensorMap tmap_b32;   // boxes of 32 weight rows: the CTA-pair kernel composes its half tiles from them
   CUtensorMap tmap_sf;    // scale atoms: [row tiles x KA] rows of 512 bytes, boxes of two atoms
 };
 
@@ -114,10 +115,8 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(gemm_mxfp4_kernel<192, true>, GemmCfg<192>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<128, false>, GemmCfg<128>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<128, true>, GemmCfg<128>::kSmemBytes);
-    e = e ? e : set_smem(gemm_mxfp4_pair_kernel<192, false>, PairCfg<192>::kSmemBytes);
-    e = e ? e : set_smem(gemm_mxfp4_pair_kernel<192, true>, PairCfg<192>::kSmemBytes);
-    e = e ? e : set_smem(gemm_mxfp4_pair_kernel<256, false>, PairCfg<256>::kSmemBytes);
-    e = e ? e : set_smem(gemm_mxfp4_pair_kernel<256, true>, PairCfg<256>::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_pair_kernel<false>, PairCfg::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_pair_kernel<true>, PairCfg::kSmemBytes);
     e = e ? e : set_smem(linear_small_s_fused_kernel<false>, FusedCfg::kSmemBytes);
     e = e ? e : set_smem(linear_small_s_fused_kernel<true>, FusedCfg::kSmemBytes);
     e = e ? e : set_smem(gemm_small_s_kernel<16, false>, SmallCfg<16>::kSmemBytes);
@@ -447,28 +446,72 @@ int pick_bn(int64_t s, int64_t m, int64_t n, int sm_count) {
 
 int g_force_gemm_kernel = 0;  // tuning hook: 0 = automatic, 1 = one CTA per tile, 2 = CTA pairs
 
-// CTA-pair kernel: tile width by the same wave model, over sm_count / 2 pairs.
-int pick_bn_pair(int64_t s, int64_t m, int64_t n, int sm_count) {
-  if (g_force_bn == 192 || g_force_bn == 256) return g_force_bn;
-  const int64_t mp = (s + 255) / 256;
-  const double k_steps = static_cast<double>((n + 255) / 256);
-  const int pairs = std::max(1, sm_count / 2);
-  auto cost = [&](int bn, double exposed_epilogue) {
-    const int64_t tiles = mp * ((m + bn - 1) / bn);
-    const int64_t waves = (tiles + pairs - 1) / pairs;
-    return static_cast<double>(waves) * (k_steps + exposed_epilogue) * bn / 256.0;
+// CTA-pair kernel: every pair takes an equal, contiguous share of the 256-token x 64-feature units
+// and walks it in tiles of up to cap0 / cap1 units (accumulator slots 0 / 1; 4 and 3 unless a
+// tile width is forced).
+// The schedule of the CTA-pair kernel for an s x m output with k_steps K-steps: column widths and
+// number of pairs.  Every candidate (columns of 128, 192 or 256 features, or 256 and 192
+// alternating) is walked exactly as the kernel walks it, and the pair that finishes last decides.
+// Model, in units of one K-step of a 192-wide tile (about 0.36 us): a K-step of a W-wide tile
+// moves 32 KiB of activations and W / 8 KiB of weights through L2, which is what its time follows;
+// a tile adds a small fixed cost, and the whole epilogue (about 3 us) when it has to wait for the
+// accumulator slot of the tile just before it.
+bool pair_schedule(int64_t s, int64_t m, int64_t k_steps, int sm_count, PairParams* p, int* pairs) {
+  const int64_t m_pairs = (s + 255) / 256;
+  const int max_pairs = std::max(1, sm_count / 2);
+  p->s = static_cast<int32_t>(s);
+  p->m = static_cast<int32_t>(m);
+  p->m_pairs = static_cast<int32_t>(m_pairs);
+  auto n_cols_of = [&](int w) -> int64_t {
+    if (w != 0) return (m + w - 1) / w;
+    const int64_t full = m / 448, rem = m % 448;
+    return 2 * full + (rem == 0 ? 0 : (rem <= 256 ? 1 : 2));
   };
-  return cost(192, 0.3) <= cost(256, 2.0) ? 192 : 256;
+  int best_w = -1;
+  double best_cost = 1e30;
+  const int cand[5] = {0, 256, 192, 128, 64};
+  for (int ci = 0; ci < 5; ++ci) {
+    const int w = cand[ci];
+    const bool forced = g_force_bn == 64 || g_force_bn == 128 || g_force_bn == 192 || g_force_bn == 256 || g_force_bn == 448;
+    if (forced ? (g_force_bn == 448 ? w != 0 : w != g_force_bn) : w == 64) continue;  // 64: only when forced
+    const int64_t n_cols = n_cols_of(w);
+    if (m_pairs * n_cols > INT32_MAX) return false;
+    p->tile_w = w;
+    p->n_cols = static_cast<int32_t>(n_cols);
+    const int np = static_cast<int>(std::min<int64_t>(max_pairs, m_pairs * n_cols));
+    double worst = 0.0;
+    for (int pr = 0; pr < np; ++pr) {
+      PairWalk walk(*p, pr, np);
+      PairSlots slots;
+      PairTile t;
+      int last = -1;
+      double cost = 0.0;
+      while (walk.next(t)) {
+        int slot;
+        uint32_t phase;
+        slots.take(t.bn, slot, phase);
+        cost += static_cast<double>(k_steps) * (32.0 + t.bn / 8.0) / 56.0 + (slot == last ? 8.0 : 1.0);
+        last = slot;
+      }
+      worst = std::max(worst, cost);
+    }
+    if (worst < best_cost - 1e-9) { best_cost = worst; best_w = w; }
+  }
+  if (best_w < 0) return false;
+  p->tile_w = best_w;
+  p->n_cols = static_cast<int32_t>(n_cols_of(best_w));
+  *pairs = static_cast<int>(std::min<int64_t>(max_pairs, m_pairs * p->n_cols));
+  return true;
 }
 
-template <int BN, bool BF>
+template <bool BF>
 cudaError_t launch_pair_kernel(int grid, cudaStream_t stream, bool dependent, const CUtensorMap& ta, const CUtensorMap& tb,
                                const CUtensorMap& tsfa, const CUtensorMap& tsfb, const CUtensorMap& ty,
                                const PairParams& p) {
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(static_cast<unsigned>(grid));
   cfg.blockDim = dim3(kPairThreads);
-  cfg.dynamicSmemBytes = PairCfg<BN>::kSmemBytes;
+  cfg.dynamicSmemBytes = PairCfg::kSmemBytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -479,7 +522,7 @@ cudaError_t launch_pair_kernel(int grid, cudaStream_t stream, bool dependent, co
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = dependent ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, gemm_mxfp4_pair_kernel<BN, BF>, ta, tb, tsfa, tsfb, ty, p);
+  return cudaLaunchKernelEx(&cfg, gemm_mxfp4_pair_kernel<BF>, ta, tb, tsfa, tsfb, ty, p);
 }
 
 batq_status launch_gemm_pair(const void* x_codes, const void* x_sf, const batq_weight* w, int64_t s, void* y,
@@ -489,23 +532,17 @@ batq_status launch_gemm_pair(const void* x_codes, const void* x_sf, const batq_w
   CUtensorMap tmap_sfa;
   batq_status st = make_sf_tmap(&tmap_sfa, x_sf, (s + 127) / 128, w->katoms);
   if (st != BATQ_OK) return st;
-  const int bn = pick_bn_pair(s, w->m, w->n, sm_count);
   PairParams p{};
-  p.s = static_cast<int32_t>(s);
-  p.m = static_cast<int32_t>(w->m);
+  int pairs = 0;
+  if (!pair_schedule(s, w->m, (w->n + 255) / 256, sm_count, &p, &pairs)) return BATQ_ERR_SHAPE;
   p.katoms = w->katoms;
   p.k_steps = static_cast<int32_t>((w->n + 255) / 256);
-  p.m_pairs = static_cast<int32_t>((s + 255) / 256);
-  p.n_tiles = static_cast<int32_t>((w->m + bn - 1) / bn);
   p.m16 = static_cast<int32_t>(m16);
   p.y = y;
   p.ldy = ldy;
-  const int grid = 2 * std::min(sm_count / 2, p.m_pairs * p.n_tiles);
-  cudaError_t e;
-  if (bn == 256) e = bf ? launch_pair_kernel<256, true>(grid, stream, dependent, tmap_a, w->tmap_b128, tmap_sfa, w->tmap_sf, tmap_y, p)
-                        : launch_pair_kernel<256, false>(grid, stream, dependent, tmap_a, w->tmap_b128, tmap_sfa, w->tmap_sf, tmap_y, p);
-  else e = bf ? launch_pair_kernel<192, true>(grid, stream, dependent, tmap_a, w->tmap_b96, tmap_sfa, w->tmap_sf, tmap_y, p)
-              : launch_pair_kernel<192, false>(grid, stream, dependent, tmap_a, w->tmap_b96, tmap_sfa, w->tmap_sf, tmap_y, p);
+  const int grid = 2 * pairs;
+  const cudaError_t e = bf ? launch_pair_kernel<true>(grid, stream, dependent, tmap_a, w->tmap_b32, tmap_sfa, w->tmap_sf, tmap_y, p)
+                           : launch_pair_kernel<false>(grid, stream, dependent, tmap_a, w->tmap_b32, tmap_sfa, w->tmap_sf, tmap_y, p);
   if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
   return BATQ_OK;
 }
@@ -991,7 +1028,7 @@ batq_status batq_prepare_weight(const batq_transform* t, const void* w_bf16, int
   st = make_codes_tmap(&w->tmap_b256, w->codes, m, n / 2, 256);
   if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b192, w->codes, m, n / 2, 192);
   if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b128, w->codes, m, n / 2, 128);
-  if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b96, w->codes, m, n / 2, 96);
+  if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b32, w->codes, m, n / 2, 32);
   if (st == BATQ_OK) st = make_sf_tmap(&w->tmap_sf, w->scales, (m + 127) / 128, w->katoms);
   if (st != BATQ_OK) { delete w; return st; }
   *out = w;
@@ -1118,6 +1155,28 @@ batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w,
 }
 
 void batq_debug_force_tile_width(int32_t bn) { g_force_bn = bn; }
+
+int32_t batq_debug_pair_schedule(int64_t s, int64_t m, int64_t n, int32_t sm_count, int32_t pair, int32_t* tiles,
+                                 int32_t max_tiles) {
+  if (s <= 0 || m <= 0 || n <= 0 || sm_count < 2) return -1;
+  PairParams p{};
+  int pairs = 0;
+  if (!pair_schedule(s, m, (n + 255) / 256, sm_count, &p, &pairs)) return -1;
+  if (pair < 0) return pairs;
+  if (pair >= pairs) return 0;
+  PairWalk w(p, pair, pairs);
+  PairTile t;
+  int32_t cnt = 0;
+  while (w.next(t)) {
+    if (tiles != nullptr && cnt < max_tiles) {
+      tiles[3 * cnt] = t.mp;
+      tiles[3 * cnt + 1] = t.n0;
+      tiles[3 * cnt + 2] = t.bn;
+    }
+    ++cnt;
+  }
+  return cnt;
+}
 void batq_debug_force_quantizer(int32_t which) { g_force_quantizer = which; }
 void batq_debug_force_gemm_kernel(int32_t which) { g_force_gemm_kernel = which; }
 void batq_debug_force_small_s_splits(int32_t splits) { g_force_splits = splits; }

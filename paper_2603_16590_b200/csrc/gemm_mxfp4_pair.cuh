@@ -5,14 +5,33 @@
 // the low-bit matrix multiplication Q(XP) Q(P^-1 W^T) of the paper's Sec. 3.
 //
 // Same pipeline as gemm_mxfp4.cuh, but two CTAs on the two SMs of a pair (a cluster of 2) share
-// one 256 x BN output tile: each CTA owns 128 token rows (its A tile, its accumulator rows in
-// its own tensor memory) and stages only half of the BN weight rows; one thread of the leader
+// one 256-token output tile: each CTA owns 128 token rows (its A tile, its accumulator rows in
+// its own tensor memory) and stages only half of the tile's weight rows; one thread of the leader
 // CTA issues tcgen05.mma.cta_group::2, which reads A and the two halves of B from both shared
-// memories.  Per CTA and K-step that is 16 KiB + BN/2 * 128 B instead of 16 KiB + BN * 128 B:
-// less traffic from L2, less shared-memory read bandwidth per MMA, and room for a deeper ring.
+// memories.
 //
-//   leader (cluster rank 0): rows [m0, m0+128),      weight rows [n0, n0+BN/2)
-//   peer   (cluster rank 1): rows [m0+128, m0+256),  weight rows [n0+BN/2, n0+BN)
+//   leader (cluster rank 0): rows [m0, m0+128),      weight rows [n0, n0+bn/2)
+//   peer   (cluster rank 1): rows [m0+128, m0+256),  weight rows [n0+bn/2, n0+bn)
+//
+// Work distribution.  Tiles are numbered column of tiles after column (all 256-token row blocks
+// of one range of output features are consecutive) and pair p of P takes tiles p, p + P, ...: at
+// any time the pairs work on a few neighbouring columns and all row blocks, in step along K, so
+// every weight tile is requested by many pairs at once and every activation tile by the others
+// -- measured, that sharing in L2 is worth a quarter of the throughput against a distribution in
+// which each pair walks its own stretch of a row.  The columns are all tile_w wide (64, 128, 192
+// or 256), or alternately 256 and 192 wide ("mixed", 224 on average); the host picks by a wave
+// model.  The last column is as narrow as the layer's edge allows.  Every column starts at a
+// multiple of 64 features: the MMA takes the weight scales from an even column of tensor memory
+// only (one column = 32 weight rows; an odd one raises a misaligned-address fault).
+//
+// Accumulators live in two slots of tensor memory, columns [0, 256) and [256, 448).  A tile wider
+// than 192 needs slot 0; a narrower one takes the slot the tile before it did not use, so that
+// its MMAs run under that tile's epilogue.  (Two 256-wide tiles in a row share slot 0: the second
+// waits for the first one's epilogue.)
+//
+// The scale factors of a K-step go through two alternating 24-column slots of tensor memory
+// behind the accumulators: tcgen05.cp and tcgen05.mma of one thread execute in issue order, so the
+// copy for step k+2 cannot overtake the MMAs of step k that still read the slot.
 //
 // Barriers.  full[stage] lives in the leader and counts the bytes of both CTAs' loads (the
 // peer's TMA loads name the leader's barrier); empty[stage] and acc_full[] exist in both CTAs
@@ -28,47 +47,87 @@
 namespace batq {
 
 constexpr int kPairThreads = 192;
+constexpr int kPairUnitCols = 64;   // output features per scheduling unit
 
-template <int BN>
 struct PairCfg {
   static constexpr int kABytes = kBM * kBKBytes;          // 16 KiB: this CTA's 128 token rows
-  static constexpr int kBBytes = (BN / 2) * kBKBytes;     // this CTA's half of the weight rows
+  static constexpr int kBBytes = 128 * kBKBytes;          // room for this CTA's half of the widest tile
   static constexpr int kSfaBytes = 1024;                  // 128 rows x 8 blocks
-  static constexpr int kSfbAtoms = 2;                     // 128-row scale tiles a BN-wide tile can touch
+  static constexpr int kSfbAtoms = 3;                     // 128-row scale tiles a tile can touch (256 columns from row 64)
   static constexpr int kSfbBytes = kSfbAtoms * 1024;
   static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
   static constexpr int kStages = 5;
-  static constexpr int kAccStages = (BN == 256) ? 1 : 2;
-  static constexpr int kAccCols = BN * kAccStages;
-  static constexpr int kSfColsPerStage = 8 + 2 * 4 * kSfbAtoms;
+  static constexpr int kSlot1Col = 256;                   // accumulator slot 0: [0, 256), slot 1: [256, 448)
+  static constexpr int kSlot1Width = 192;
+  static constexpr int kAccCols = 448;
+  static constexpr int kSfCols = 8 + 2 * 4 * kSfbAtoms;   // scale columns of one K-step
+  static constexpr int kSfSlots = 2;
   static constexpr int kTmemCols = 512;
-  static constexpr int kStagingBufs = (BN == 256) ? 1 : 2;
+  static constexpr int kStagingBufs = 2;
   static constexpr int kStagingBytes = 4 * kStagingBufs * 4096;
   static constexpr int kSmemBytes = kStages * kStageBytes + kStagingBytes + 1024;
-  static_assert(BN == 192 || BN == 256, "tile width");
-  static_assert(kAccCols + kStages * kSfColsPerStage <= kTmemCols, "tensor memory budget");
+  static_assert(kAccCols + kSfSlots * kSfCols <= kTmemCols, "tensor memory budget");
   static_assert(kSmemBytes <= 232448, "shared memory budget");
   static_assert(kStageBytes % 1024 == 0, "stage alignment");
 };
 
 struct PairParams {
-  int32_t s;            // rows of X (tokens)
-  int32_t m;            // rows of W (output features)
-  int32_t katoms;       // KA = 2*ceil(k/8): 512-byte scale atoms per 128-row tile
-  int32_t k_steps;      // ceil(n / 256)
-  int32_t m_pairs;      // ceil(s / 256)
-  int32_t n_tiles;      // ceil(m / BN)
-  int32_t m16;          // as in GemmParams: columns covered by the TMA store
+  int32_t s;              // rows of X (tokens)
+  int32_t m;              // rows of W (output features)
+  int32_t katoms;         // KA = 2*ceil(k/8): 512-byte scale atoms per 128-row tile
+  int32_t k_steps;        // ceil(n / 256)
+  int32_t m_pairs;        // ceil(s / 256)
+  int32_t tile_w;         // column width: 64, 128, 192 or 256; 0 = mixed (256, 192, 256, 192, ...)
+  int32_t n_cols;         // columns of tiles
+  int32_t m16;            // as in GemmParams: columns covered by the TMA store
   void* y;
   int64_t ldy;
 };
 
-template <int BN, bool OUT_BF16>
+// The tiles of one pair, in order.  Every warp role walks the same sequence.
+struct PairTile {
+  int mp;    // 256-token row block
+  int n0;    // first output feature (a multiple of 64)
+  int bn;    // width: the column's, less (a multiple of 64) in the last column
+};
+struct PairWalk {
+  int tile, total, step, m_pairs, tile_w, m;
+  __host__ __device__ __forceinline__ PairWalk(const PairParams& p, int pair, int n_pairs)
+      : tile(pair), total(p.m_pairs * p.n_cols), step(n_pairs), m_pairs(p.m_pairs), tile_w(p.tile_w), m(p.m) {}
+  __host__ __device__ __forceinline__ bool next(PairTile& t) {
+    if (tile >= total) return false;
+    const int nt = tile / m_pairs;
+    t.mp = tile - nt * m_pairs;
+    int w = tile_w;
+    if (tile_w == 0) {  // mixed: columns 2c and 2c + 1 share 448 features, 256 + 192
+      t.n0 = (nt >> 1) * 448 + (nt & 1) * 256;
+      w = (nt & 1) ? 192 : 256;
+    } else {
+      t.n0 = nt * tile_w;
+    }
+    const int rem = m - t.n0;
+    t.bn = rem >= w ? w : ((rem + 63) / 64) * 64;
+    tile += step;
+    return true;
+  }
+};
+// Which accumulator slot a tile takes, and the parity of that slot's barriers for it.
+struct PairSlots {
+  int prev, use0, use1;
+  __host__ __device__ __forceinline__ PairSlots() : prev(1), use0(0), use1(0) {}
+  __host__ __device__ __forceinline__ void take(int bn, int& slot, uint32_t& phase) {
+    slot = bn > PairCfg::kSlot1Width ? 0 : (prev == 0 ? 1 : 0);
+    phase = static_cast<uint32_t>(slot == 0 ? use0++ : use1++) & 1u;
+    prev = slot;
+  }
+};
+
+template <bool OUT_BF16>
 __global__ void __launch_bounds__(kPairThreads, 1)
-gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b32,
                        const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfb,
                        const __grid_constant__ CUtensorMap tmap_y, const PairParams p) {
-  using Cfg = PairCfg<BN>;
+  using Cfg = PairCfg;
   extern __shared__ uint8_t pair_smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[Cfg::kStages];   // used in the leader only
   __shared__ __align__(8) uint64_t empty_bar[Cfg::kStages];  // one set per CTA
@@ -103,7 +162,7 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmap_a);
-    tma_prefetch_desc(&tmap_b);
+    tma_prefetch_desc(&tmap_b32);
     tma_prefetch_desc(&tmap_sfa);
     tma_prefetch_desc(&tmap_sfb);
     tma_prefetch_desc(&tmap_y);
@@ -118,58 +177,76 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
   tc_fence_after_sync();
   const uint32_t tmem_base = tmem_base_slot;
 
-  const int total_tiles = p.m_pairs * p.n_tiles;
+  const PairWalk walk0(p, pair, n_pairs);
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer (both CTAs)
     bool ok = true;
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t full0_leader = map_to_cta(smem_u32(&full_bar[0]), 0);
-    const int my_tiles = pair < total_tiles ? (total_tiles - pair + n_pairs - 1) / n_pairs : 0;
-    const int my_steps = my_tiles * p.k_steps;
-    // Step g of this pair = K-step g % k_steps of its tile number g / k_steps.  `what`: 1 = the
-    // weight side (B tile half, weight scales; the leader also arms the barrier), 2 = the
-    // activation side (A tile, activation scales), 3 = both.
-    auto issue = [&](int g, int stage, int what) {
-      const int tile = pair + (g / p.k_steps) * n_pairs;
-      const int kt = g % p.k_steps;
-      const int mp = tile % p.m_pairs;
-      const int nt = tile / p.m_pairs;
-      const int m0 = mp * 256 + static_cast<int>(rank) * kBM;
-      const int n0 = nt * BN;
+    int my_steps = 0;
+    {
+      PairWalk w = walk0;
+      PairTile t;
+      while (w.next(t)) my_steps += p.k_steps;
+    }
+    // K-step kt of tile t into ring stage `stage`.  `what`: 1 = the weight side (this CTA's half of
+    // the B tile in boxes of 32 rows, weight scales; the leader also arms the barrier with the
+    // bytes of both CTAs), 2 = the activation side (A tile, activation scales), 3 = both.
+    auto issue = [&](const PairTile& t, int kt, int stage, int what) {
+      const int m0 = t.mp * 256 + static_cast<int>(rank) * kBM;
+      const int half = t.bn >> 1;
       const uint32_t st = smem_base + stage * Cfg::kStageBytes;
       const uint32_t bar = full0_leader + 8u * stage;
       if (what & 1) {
-        if (rank == 0) mbar_arrive_expect_tx(smem_u32(&full_bar[stage]), 2u * Cfg::kStageBytes);
-        tma_load_2d_pair(st + Cfg::kABytes, &tmap_b, kt * kBKBytes, n0 + static_cast<int>(rank) * (BN / 2), bar);
+        if (rank == 0)
+          mbar_arrive_expect_tx(smem_u32(&full_bar[stage]),
+                                2u * static_cast<uint32_t>(Cfg::kABytes + half * kBKBytes + Cfg::kSfaBytes + Cfg::kSfbBytes));
+        const int b0 = t.n0 + static_cast<int>(rank) * half;
+        for (int r = 0; r < half; r += 32)
+          tma_load_2d_pair(st + Cfg::kABytes + r * kBKBytes, &tmap_b32, kt * kBKBytes, b0 + r, bar);
 #pragma unroll
         for (int rt = 0; rt < Cfg::kSfbAtoms; ++rt)
           tma_load_2d_pair(st + Cfg::kABytes + Cfg::kBBytes + Cfg::kSfaBytes + rt * 1024, &tmap_sfb, 0,
-                           ((n0 >> 7) + rt) * p.katoms + 2 * kt, bar);
+                           ((t.n0 >> 7) + rt) * p.katoms + 2 * kt, bar);
       }
       if (what & 2) {
         tma_load_2d_pair(st, &tmap_a, kt * kBKBytes, m0, bar);
         tma_load_2d_pair(st + Cfg::kABytes + Cfg::kBBytes, &tmap_sfa, 0, (m0 >> 7) * p.katoms + 2 * kt, bar);
       }
     };
+    // The first `prefill` steps of the pair, side `what`, into stages 0, 1, ...
+    const int prefill = min(my_steps, Cfg::kStages);
+    auto issue_prefill = [&](int what) {
+      PairWalk w = walk0;
+      PairTile t;
+      int g = 0;
+      while (g < prefill && w.next(t))
+        for (int kt = 0; kt < p.k_steps && g < prefill; ++kt, ++g) issue(t, kt, g, what);
+    };
     // The weights do not depend on the kernel that quantises the activations: fill the ring's
     // weight side first, then wait for that kernel (programmatic dependent launch; an ordinary
     // launch does not wait here), then add the activation side.
-    const int prefill = min(my_steps, Cfg::kStages);
-    if (elect_one())
-      for (int g = 0; g < prefill; ++g) issue(g, g, 1);
+    if (elect_one()) issue_prefill(1);
     __syncwarp();
     grid_dependency_wait();
-    if (elect_one())
-      for (int g = 0; g < prefill; ++g) issue(g, g, 2);
+    if (elect_one()) issue_prefill(2);
     __syncwarp();
     int stage = prefill % Cfg::kStages;
     uint32_t phase = (prefill == Cfg::kStages) ? 1u : 0u;
-    for (int g = prefill; g < my_steps; ++g) {
-      ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag));
-      if (!ok) break;
-      if (elect_one()) issue(g, stage, 3);
-      if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+    {
+      PairWalk w = walk0;
+      PairTile t;
+      int g = 0;
+      while (ok && w.next(t)) {
+        for (int kt = 0; kt < p.k_steps; ++kt, ++g) {
+          if (g < prefill) continue;
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag));
+          if (!ok) break;
+          if (elect_one()) issue(t, kt, stage, 3);
+          if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
     }
     if (!ok && lane == 0) {
       // Given up: the loads of both CTAs are counted on the leader's barriers, so neither CTA can
@@ -180,8 +257,6 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer (leader CTA only)
     if (rank == 0) {
-      constexpr uint32_t idesc0 = mxf4_idesc(256, BN);
-      constexpr uint32_t idesc1 = idesc0 | (2u << 29) | (2u << 4);
       const uint32_t smem_base = smem_u32(smem);
       const uint64_t ab_desc0 = make_smem_desc(smem_base, 16, 1024, 2);
       const uint64_t sf_desc0 = make_smem_desc(smem_base + Cfg::kABytes + Cfg::kBBytes, 0, 128, 0);
@@ -191,18 +266,23 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
 
       int stage = 0;
       uint32_t phase = 0;
-      int it = 0;
+      uint32_t g = 0;  // K-steps issued so far: the scale slot alternates with it
       bool ok = true;
-      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++it) {
-        const int nt = tile / p.m_pairs;
-        const uint32_t sfb_sub = static_cast<uint32_t>((nt * BN) & 127) >> 5;
-        const int acc = it % Cfg::kAccStages;
-        const uint32_t acc_phase = (it / Cfg::kAccStages) & 1u;
+      PairWalk w = walk0;
+      PairTile t;
+      PairSlots slots;
+      while (ok && w.next(t)) {
+        const uint32_t idesc0 = mxf4_idesc(256, t.bn);
+        const uint32_t idesc1 = idesc0 | (2u << 29) | (2u << 4);
+        const uint32_t sfb_sub = static_cast<uint32_t>(t.n0 & 127) >> 5;
+        int acc;
+        uint32_t acc_phase;
+        slots.take(t.bn, acc, acc_phase);
         ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&acc_empty_bar[acc]), acc_phase ^ 1u, &abort_flag));
         if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int kt = 0; kt < p.k_steps; ++kt) {
+        const uint32_t d_tmem = tmem_base + acc * Cfg::kSlot1Col;
+        for (int kt = 0; kt < p.k_steps; ++kt, ++g) {
           ok = __all_sync(0xFFFFFFFFu, mbar_wait(full0 + 8u * stage, phase, &abort_flag));
           if (!ok) break;
           tc_fence_after_sync();
@@ -210,7 +290,7 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
           const uint64_t adesc = ab_desc0 + soff;
           const uint64_t bdesc = adesc + (Cfg::kABytes >> 4);
           const uint64_t sfd = sf_desc0 + soff;
-          const uint32_t sfa_col = sf_tmem0 + stage * Cfg::kSfColsPerStage;
+          const uint32_t sfa_col = sf_tmem0 + (g & 1u) * Cfg::kSfCols;
           const uint32_t sfb_col = sfa_col + 8 + sfb_sub;
           if (elect_one()) {
             tc_cp_32x128b_warpx4_pair(sfa_col, sfd);
@@ -250,20 +330,21 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     constexpr int kChunkCols = OUT_BF16 ? 64 : 32;
     const uint32_t acc_empty0_leader = map_to_cta(smem_u32(&acc_empty_bar[0]), 0);
     int buf = 0;
-    int it = 0;
-    for (int tile = pair; tile < total_tiles; tile += n_pairs, ++it) {
-      const int mp = tile % p.m_pairs;
-      const int nt = tile / p.m_pairs;
-      const int acc = it % Cfg::kAccStages;
-      const uint32_t acc_phase = (it / Cfg::kAccStages) & 1u;
+    PairWalk wk = walk0;
+    PairTile t;
+    PairSlots slots;
+    while (wk.next(t)) {
+      int acc;
+      uint32_t acc_phase;
+      slots.take(t.bn, acc, acc_phase);
       bool ok = mbar_wait(smem_u32(&acc_full_bar[acc]), acc_phase, &abort_flag);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after_sync();
-      const int row0 = mp * 256 + static_cast<int>(rank) * kBM + quad * 32;
-      const uint32_t taddr = tmem_base + acc * BN + (static_cast<uint32_t>(quad * 32) << 16);
+      const int row0 = t.mp * 256 + static_cast<int>(rank) * kBM + quad * 32;
+      const uint32_t taddr = tmem_base + acc * Cfg::kSlot1Col + (static_cast<uint32_t>(quad * 32) << 16);
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += kChunkCols) {
+      for (int c0 = 0; c0 < t.bn; c0 += kChunkCols) {
         uint32_t w[32];
         if (OUT_BF16) {
           uint32_t r0[32], r1[32];
@@ -281,7 +362,7 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
           tmem_ld_32x32b_x32(taddr + c0, w);
           tmem_ld_wait();
         }
-        const int col0 = nt * BN + c0;
+        const int col0 = t.n0 + c0;
         if (p.m16 < p.m && col0 < p.m && col0 + kChunkCols > p.m16 && row0 + lane < p.s) {
           if (OUT_BF16) {
             __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(p.y) + static_cast<int64_t>(row0 + lane) * p.ldy + col0;

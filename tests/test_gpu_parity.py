@@ -365,11 +365,9 @@ def test_gemm_vs_oracle_same_codes(batq, gkernel, S, M, N):
     assert np.max(np.abs(got - Y) / (Sabs + 1e-30)) < 1e-5
 
 
-@pytest.mark.parametrize("bn", [128, 192, 256])
-@pytest.mark.parametrize("S,M,N", [(300, 520, 3584), (129, 257, 2048 + 32), (260, 1000, 512)])
+@pytest.mark.parametrize("bn", [64, 128, 192, 256, 448])
+@pytest.mark.parametrize("S,M,N", [(300, 520, 3584), (129, 257, 2048 + 32), (260, 1000, 512), (600, 2300, 768)])
 def test_gemm_every_tile_width(batq, gkernel, bn, S, M, N):
-    if gkernel == 2 and bn == 128:
-        pytest.skip("CTA pairs have tile widths 192 and 256")
     batq.batq_debug_force_tile_width(bn)
     try:
         got, Y, Sabs = _gemm_case(batq, S, M, N, 700 + S)
@@ -381,7 +379,7 @@ def test_gemm_every_tile_width(batq, gkernel, bn, S, M, N):
     assert np.array_equal(got16.astype(np.float32), want16)
 
 
-@pytest.mark.parametrize("bn", [128, 192, 256])
+@pytest.mark.parametrize("bn", [64, 128, 192, 256, 448])
 def test_gemm_scale_layout_localising_case_every_tile_width(batq, gkernel, bn):
     batq.batq_debug_force_tile_width(bn)
     try:

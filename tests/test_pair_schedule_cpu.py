@@ -1,0 +1,80 @@
+"""Host logic of the CTA-pair GEMM: its work distribution, checked without a GPU.
+
+Tiles are numbered column of tiles after column and pair p of P takes tiles p, p + P, ...  The
+columns are all equally wide or alternately 256 and 192 wide.  The tiles of all pairs together
+must cover the s x m output exactly once, every column must start at a multiple of 64 features
+(the MMA cannot take weight scales from an odd 32-row group), only the last column may be narrower
+than its nominal width, and no pair may have more than one tile more than another."""
+import numpy as np
+import pytest
+
+from paper_2603_16590_b200 import binding as B
+
+SHAPES = [(2048, 4096, 4096), (2048, 6144, 4096), (2048, 28672, 4096), (2048, 4096, 14336), (2048, 4096 + 8, 512),
+          (300, 520, 3584), (129, 257, 2080), (260, 1000, 512), (8192, 3584, 3584), (8192, 18944, 3584),
+          (8192, 4608, 3584), (257, 192, 256), (1000, 1100, 768), (4096, 64, 1024), (256, 100000, 256)]
+
+
+def _check(sched, s, m):
+    rows = -(-s // 256)
+    cover = np.zeros((rows, -(-m // 64)), dtype=np.int32)
+    cols = {}
+    for p, tiles in enumerate(sched):
+        for i, (mp, n0, bn) in enumerate(tiles):
+            assert n0 % 64 == 0 and bn % 64 == 0 and 64 <= bn <= 256 and 0 <= mp < rows
+            cols.setdefault(n0, set()).add(bn)
+            cover[mp, n0 // 64:(n0 + bn) // 64] += 1
+    assert np.all(cover == 1)
+    starts = sorted(cols)
+    assert all(len(v) == 1 for v in cols.values())
+    widths = [next(iter(cols[c])) for c in starts]
+    # column-major round robin: tile number = column index * rows + row block
+    index = {c: k for k, c in enumerate(starts)}
+    for p, tiles in enumerate(sched):
+        for i, (mp, n0, bn) in enumerate(tiles):
+            assert index[n0] * rows + mp == p + i * len(sched)
+    body = widths[:-1]
+    uniform = len(set(body)) <= 1
+    mixed = all(w == (256 if k % 2 == 0 else 192) for k, w in enumerate(body))
+    assert uniform or mixed
+    nominal = (256 if (len(widths) - 1) % 2 == 0 else 192) if (mixed and not uniform) else (body[0] if body else widths[-1])
+    assert widths[-1] <= nominal and starts[-1] + widths[-1] >= m > starts[-1] + widths[-1] - 64
+    counts = [len(t) for t in sched]
+    assert max(counts) - min(counts) <= 1
+    return widths
+
+
+@pytest.mark.parametrize("s,m,n", SHAPES)
+@pytest.mark.parametrize("sm_count", [148, 132, 2])
+def test_tiles_cover_the_output_once(s, m, n, sm_count):
+    sched = B.batq_debug_pair_schedule(s, m, n, sm_count)
+    assert 1 <= len(sched) <= max(1, sm_count // 2)
+    _check(sched, s, m)
+
+
+@pytest.mark.parametrize("bn", [64, 128, 192, 256, 448])
+def test_forced_widths(bn):
+    for s, m, n in SHAPES[:8]:
+        B.batq_debug_force_tile_width(bn)
+        try:
+            sched = B.batq_debug_pair_schedule(s, m, n)
+        finally:
+            B.batq_debug_force_tile_width(0)
+        widths = _check(sched, s, m)
+        if len(widths) > 2:
+            assert set(widths[:-1]) == ({256, 192} if bn == 448 else {bn})
+
+
+def test_bad_arguments():
+    lib = B.load()
+    assert lib.batq_debug_pair_schedule(0, 128, 128, 148, -1, None, 0) == -1
+    assert lib.batq_debug_pair_schedule(128, 128, 128, 1, -1, None, 0) == -1
+    assert lib.batq_debug_pair_schedule(256, 128, 128, 148, 999, None, 0) == 0
+
+
+def test_width_follows_the_wave_model():
+    """Llama-8B prefill shapes at 2048 tokens on 74 pairs."""
+    w = lambda s, m, n: sorted({t[2] for tiles in B.batq_debug_pair_schedule(s, m, n) for t in tiles})
+    assert w(2048, 28672, 4096) == [192, 256]      # mixed: 1024 tiles = 13.8 waves instead of 16.2 of 192
+    assert w(2048, 4096, 14336) == [256]           # 2 tiles per pair however cut; the widest move least through L2
+    assert w(2048, 6144, 4096) == [192]
