@@ -555,6 +555,44 @@ def test_linear_fused_small_s_vs_oracle(batq, S, M, N, geometry, splits):
     assert np.linalg.norm(outs[1] - outs[2]) <= 1e-4 * np.linalg.norm(Sabs)
 
 
+@pytest.mark.parametrize("S", [1, 4, 16, 48, 300])
+def test_linear_calls_back_to_back_share_a_workspace(batq, S):
+    """Layers called one after the other on one stream, with one workspace, inside a replayed CUDA
+    graph: every kernel is a programmatic dependent of the one before it (the next layer's
+    quantiser or fused kernel is scheduled while the previous GEMM still runs), so a kernel that
+    touched the workspace, x or y before its wait would show up here.  Each output must be bit for
+    bit what the same call gives when it runs alone."""
+    shapes = [(1024, 1536), (1024, 1024), (1024, 2304), (2048, 1024), (1024, 264)]   # (n, m)
+    layers = []
+    for i, (n, m) in enumerate(shapes):
+        t = synth.make_transform(n, 40 + i, "baseline")
+        tr = _mk_transform(batq, t)
+        w = batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(synth.make_weight(m, n, 40 + i)))
+        x = batq.bits_to_cuda_bf16(synth.make_activations(S, n, 40 + i))
+        layers.append((tr, w, x, m))
+    ws = batq.aligned_workspace(max(batq.batq_linear_workspace_bytes(w, S) for _, w, _, _ in layers))
+    alone = []
+    for tr, w, x, m in layers:
+        y = torch.empty((S, m), dtype=torch.bfloat16, device="cuda")
+        batq.batq_linear_w4a4(tr, w, x, y, ws)
+        torch.cuda.synchronize()
+        alone.append(y)
+    outs = [torch.zeros((S, m), dtype=torch.bfloat16, device="cuda") for _, _, _, m in layers]
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(3):
+                for (tr, w, x, m), y in zip(layers, outs):
+                    batq.batq_linear_w4a4(tr, w, x, y, ws)
+        for _ in range(3):
+            g.replay()
+    torch.cuda.synchronize()
+    assert batq.batq_last_device_status() == 0
+    for a, b in zip(alone, outs):
+        assert torch.equal(a, b)
+
+
 def test_linear_host_entry_point_matches_device_entry_point(batq):
     S, M, N = 96, 256, 512
     xb = synth.make_activations(S, N, 5)
