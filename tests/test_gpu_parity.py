@@ -593,6 +593,22 @@ def test_linear_calls_back_to_back_share_a_workspace(batq, S):
         assert torch.equal(a, b)
 
 
+def test_linear_kernel_launches_reports_the_dispatch(batq):
+    """1 = the fused kernel (a token or so on a layer whose K slices are short), 2 = quantiser + GEMM."""
+    t = synth.make_transform(4096, 3, "baseline")
+    tr = _mk_transform(batq, t)
+    w = batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(synth.make_weight(4096, 4096, 3)))
+    assert batq.batq_linear_kernel_launches(tr, w, 1) == 1
+    assert batq.batq_linear_kernel_launches(tr, w, 16) == 2
+    assert batq.batq_linear_kernel_launches(tr, w, 2048) == 2
+    assert batq.batq_linear_kernel_launches(tr, w, 0) == 0
+    batq.batq_debug_force_small_s_path(1)
+    try:
+        assert batq.batq_linear_kernel_launches(tr, w, 1) == 2
+    finally:
+        batq.batq_debug_force_small_s_path(0)
+
+
 def test_linear_host_entry_point_matches_device_entry_point(batq):
     S, M, N = 96, 256, 512
     xb = synth.make_activations(S, N, 5)
