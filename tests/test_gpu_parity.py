@@ -170,6 +170,30 @@ def test_quantizer_row_stride_and_determinism(batq, qmode):
         assert np.array_equal(u, v) and np.array_equal(u, w)
 
 
+@pytest.mark.parametrize("S", [48, 1000])
+def test_quantizer_is_independent_of_the_row_order(batq, qmode, S):
+    """Mixed vision/text batch (first 75 % of the rows heavy-tailed Student-t, the rest Gaussian
+    with outlier channels): quantising the rows interleaved gives exactly the interleaved result of
+    quantising them in blocks, and a whole layer on the shuffled batch the shuffled output: no
+    statistic crosses a token row."""
+    N = 1792
+    xb = synth.make_activations(S, N, 77, outlier_channel_frac=0.005, vision_rows=(3 * S) // 4)
+    perm = np.random.default_rng(5).permutation(S)
+    t = synth.make_transform(N, 9, "baseline")
+    tr = _mk_transform(batq, t)
+    c0, s0 = _gpu_quantize(batq, tr, xb)
+    c1, s1 = _gpu_quantize(batq, tr, np.ascontiguousarray(xb[perm]))
+    assert np.array_equal(c0[perm], c1) and np.array_equal(s0[perm], s1)
+    w = batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(synth.make_weight(264, N, 77)))
+    ws = batq.aligned_workspace(batq.batq_linear_workspace_bytes(w, S))
+    y0 = torch.empty((S, 264), dtype=torch.float32, device="cuda")
+    y1 = torch.empty((S, 264), dtype=torch.float32, device="cuda")
+    batq.batq_linear_w4a4(tr, w, batq.bits_to_cuda_bf16(xb), y0, ws)
+    batq.batq_linear_w4a4(tr, w, batq.bits_to_cuda_bf16(np.ascontiguousarray(xb[perm])), y1, ws)
+    assert batq.batq_last_device_status() == 0
+    assert torch.equal(y0[torch.from_numpy(perm).cuda()], y1)
+
+
 # ---------------------------------------------------------------------------- other factorisations of the block
 FACTOR_SIZES = [(1, 32), (2, 16), (8, 4), (16, 2), (32, 1)]
 
