@@ -150,7 +150,7 @@ batq_status batq_weight_export(const batq_weight* w, void* codes_rowmajor, void*
 batq_status batq_gemm_mxfp4(const void* x_codes, const void* x_scales_mma, const batq_weight* w,
                             int64_t s, void* y, int32_t y_dtype, int64_t ldy, void* stream);
 
-/* Stage 3 alone for a handful of tokens (decode), s <= 64: the same contraction as
+/* Stage 3 alone for a handful of tokens (decode), s <= 128: the same contraction as
  * batq_gemm_mxfp4, organised for the case where streaming the weights from HBM once is the
  * whole cost.  The weights are the 128-row tensor-core operand and the tokens the narrow one;
  * the grid is (128-row weight tiles) x (K splits), and the partial sums of the splits meet in
@@ -158,7 +158,7 @@ batq_status batq_gemm_mxfp4(const void* x_codes, const void* x_scales_mma, const
  *   scratch        dev, batq_gemm_small_s_scratch_bytes(w, s) bytes, 1024-byte aligned; contents
  *                  need not be initialised; calls sharing it must be ordered on one stream.
  *   y              dev [s x m], fp32 or bf16, row stride ldy.
- * Errors as batq_gemm_mxfp4, plus SHAPE for s > 64 and WORKSPACE for a short scratch. */
+ * Errors as batq_gemm_mxfp4, plus SHAPE for s > 128 and WORKSPACE for a short scratch. */
 size_t batq_gemm_small_s_scratch_bytes(const batq_weight* w, int64_t s);
 batq_status batq_gemm_mxfp4_small_s(const void* x_codes, const void* x_scales_mma, const batq_weight* w,
                                     int64_t s, void* y, int32_t y_dtype, int64_t ldy, void* scratch,
@@ -180,10 +180,10 @@ int32_t batq_debug_pair_schedule(int64_t s, int64_t m, int64_t n, int32_t sm_cou
  * 256-token tile for s > 128, one CTA per 128-token tile otherwise), 1 = always one CTA per tile,
  * 2 = always CTA pairs (tile widths 192 and 256 only). */
 void batq_debug_force_gemm_kernel(int32_t which);
-/* Test / tuning hook: which activation quantiser later calls use.  0 = automatic (up to 64 tokens
- * the one-thread-per-block kernel, above that the tensor-core dense-block kernel; the identity
- * transform above 64 tokens and nothing else takes the streaming ALU kernel), 1 = the streaming ALU
- * kernel (Kronecker form), 2 = the tensor-core kernel, 3 = the one-thread-per-block kernel.
+/* Test / tuning hook: which activation quantiser later calls use.  0 = automatic (up to 128 tokens
+ * the per-block ALU kernel, above that the tensor-core dense-block kernel; the identity
+ * transform above 128 tokens and nothing else takes the streaming ALU kernel), 1 = the streaming ALU
+ * kernel (Kronecker form), 2 = the tensor-core kernel, 3 = the per-block ALU kernel.
  * Factor sizes other than 4 x 8 always take the tensor-core kernel. */
 void batq_debug_force_quantizer(int32_t which);
 /* Test / tuning hook: number of K splits of the small-s GEMM (clamped to the number of
@@ -201,11 +201,11 @@ void batq_debug_force_small_s_reduce(int32_t which);
  * n <= 16384; other shapes take the two kernels. */
 void batq_debug_force_small_s_path(int32_t which);
 
-/* The whole layer, stages 1+2+3: quantise X into the workspace, then the GEMM.  Up to 64
- * tokens take the small-s GEMM, launched so that its weight stream overlaps the quantiser; the
- * smallest cases take a single kernel that quantises the activations inside the GEMM (no
- * workspace traffic at all).  Above 64 tokens the GEMM is launched as a programmatic dependent of
- * the quantiser as well.
+/* The whole layer, stages 1+2+3: quantise X into the workspace, then the GEMM.  Up to 32
+ * tokens (up to 128 on layers of at least 40 M weights) take the small-s GEMM, launched so that
+ * its weight stream overlaps the quantiser; the smallest cases take a single kernel that
+ * quantises the activations inside the GEMM (no workspace traffic at all).  In every other case
+ * the GEMM is launched as a programmatic dependent of the quantiser as well.
  *   workspace  dev, at least batq_linear_workspace_bytes(w, s) bytes, 1024-byte
  *              aligned; overwritten by every call (calls sharing a workspace
  *              must be ordered on one stream). */

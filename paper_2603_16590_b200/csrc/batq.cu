@@ -125,6 +125,8 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(gemm_small_s_kernel<32, true>, SmallCfg<32>::kSmemBytes);
     e = e ? e : set_smem(gemm_small_s_kernel<64, false>, SmallCfg<64>::kSmemBytes);
     e = e ? e : set_smem(gemm_small_s_kernel<64, true>, SmallCfg<64>::kSmemBytes);
+    e = e ? e : set_smem(gemm_small_s_kernel<128, false>, SmallCfg<128>::kSmemBytes);
+    e = e ? e : set_smem(gemm_small_s_kernel<128, true>, SmallCfg<128>::kSmemBytes);
     if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
     if (g_encode_tiled == nullptr) {
       void* fn = nullptr;
@@ -252,7 +254,8 @@ batq_status check_x(const void* x, int64_t s, int64_t n, int64_t ld) {
   return BATQ_OK;
 }
 
-constexpr int64_t kSmallSMax = 64;  // token counts up to this take the swapped-operand split-K GEMM
+constexpr int64_t kSmallSMax = 128;       // the swapped-operand split-K GEMM takes up to this many tokens
+constexpr int64_t kSmallQuantAuto = 128;  // per-block ALU quantiser up to here, tensor cores above (12 us flat against 2-4 us)
 int g_force_quantizer = 0;  // tuning hook: 0 = automatic, 1 = ALU (Kronecker form), 2 = tensor cores (dense form)
 
 // Tensor-core version: 128-token x 4-block units.
@@ -325,8 +328,9 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
   // The ALU kernel is written for 4 x 8 factors; every other factorisation of 32 goes through the
   // tensor-core kernel, which only sees the dense block matrices.
   const bool only_tc = t != nullptr && (t->gr != 4 || t->gc != 8);
-  const bool use_tc = only_tc || (n_zero_words == 0 && t != nullptr &&
-                                  (g_force_quantizer == 2 || (g_force_quantizer == 0 && s > kSmallSMax)));
+  const bool small_path = n_zero_words > 0;  // in front of the small-s GEMM (its tickets to clear)
+  const bool use_tc = only_tc || (!small_path && t != nullptr &&
+                                  (g_force_quantizer == 2 || (g_force_quantizer == 0 && s > kSmallQuantAuto)));
   if (use_tc) {
     if (n_zero_words > 0 &&
         cudaMemsetAsync(zero_words, 0, static_cast<size_t>(n_zero_words) * 4, stream) != cudaSuccess) {
@@ -337,7 +341,7 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
   }
   // A handful of tokens: the ring of the streaming kernel below is all latency there; one thread
   // per (token, block) with everything loaded up front is quicker.
-  if (g_force_quantizer == 3 || (g_force_quantizer == 0 && s <= kSmallSMax)) {
+  if (g_force_quantizer == 3 || (g_force_quantizer == 0 && (s <= kSmallQuantAuto || (small_path && s <= kSmallSMax)))) {
     QuantSmallParams q{};
     q.x = static_cast<const uint16_t*>(x);
     q.ld = ld;
@@ -606,7 +610,7 @@ int g_force_splits = 0;  // tuning hook: 0 = automatic
 int g_small_reduce = 0;  // tuning hook: 0 = automatic, 1 = always tickets, 2 = cluster whenever splits <= 8
 constexpr int kMaxSplits = 32;
 
-inline int small_ntok(int64_t s) { return s <= 16 ? 16 : (s <= 32 ? 32 : 64); }
+inline int small_ntok(int64_t s) { return s <= 16 ? 16 : (s <= 32 ? 32 : (s <= 64 ? 64 : 128)); }
 
 
 // The K splits of a row tile can meet as one thread-block cluster (reduction through distributed
@@ -644,6 +648,7 @@ int pick_splits(int64_t m, int64_t n, int64_t s, int sm_count) {
 struct SmallScratch {
   size_t partial_bytes, ticket_bytes;
   int splits, ntok;
+  bool cluster;  // the splits of a row tile meet as a thread-block cluster (partials in shared memory)
   int64_t tiles;
   size_t total() const { return partial_bytes + ticket_bytes; }
 };
@@ -652,7 +657,9 @@ SmallScratch small_scratch(const batq_weight* w, int64_t s) {
   sc.ntok = small_ntok(s);
   sc.splits = pick_splits(w->m, w->n, s, w->sm_count);
   sc.tiles = (w->m + 127) / 128;
-  sc.partial_bytes = sc.splits > 1 ? round_up(static_cast<size_t>(sc.tiles) * sc.splits * sc.ntok * 128 * 4, 1024) : 0;
+  // the cluster reduction keeps its partial tiles in shared memory
+  sc.cluster = cluster_reduce_ok(sc.tiles, sc.splits, 2 * static_cast<int64_t>(w->sm_count > 0 ? w->sm_count : 148), s);
+  sc.partial_bytes = (sc.splits > 1 && !sc.cluster) ? round_up(static_cast<size_t>(sc.tiles) * sc.splits * sc.ntok * 128 * 4, 1024) : 0;
   sc.ticket_bytes = round_up(static_cast<size_t>(sc.tiles) * 4, 1024);
   return sc;
 }
@@ -709,7 +716,7 @@ batq_status launch_gemm_small(const void* x_codes, const void* x_sf, const batq_
   p.ldy = ldy;
   p.partial = reinterpret_cast<float*>(scratch);
   p.tickets = reinterpret_cast<uint32_t*>(scratch + sc.partial_bytes);
-  p.cluster_reduce = cluster_reduce_ok(sc.tiles, sc.splits, 2 * static_cast<int64_t>(info->sm_count), s) ? 1 : 0;
+  p.cluster_reduce = sc.cluster ? 1 : 0;
   const dim3 grid(static_cast<unsigned>(sc.tiles), static_cast<unsigned>(sc.splits));
   const bool bf = y_dtype == BATQ_BF16;
   cudaError_t e;
@@ -717,7 +724,8 @@ batq_status launch_gemm_small(const void* x_codes, const void* x_sf, const batq_
                            : launch_small_kernel<NT, false>(grid, stream, dependent, w->tmap_b128, tmap_x, p))
   if (sc.ntok == 16) e = BATQ_SMALL(16);
   else if (sc.ntok == 32) e = BATQ_SMALL(32);
-  else e = BATQ_SMALL(64);
+  else if (sc.ntok == 64) e = BATQ_SMALL(64);
+  else e = BATQ_SMALL(128);
 #undef BATQ_SMALL
   if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
   return BATQ_OK;
@@ -1089,10 +1097,21 @@ batq_status batq_gemm_mxfp4_small_s(const void* x_codes, const void* x_scales_mm
   return launch_gemm_small(x_codes, x_scales_mma, w, s, y, y_dtype, ldy, sp, sc, cs, false);
 }
 
+// The whole layer takes the small-s path (per-block quantiser + swapped-operand split-K GEMM) up
+// to 32 tokens, and up to 128 where the layer is large enough for the weight stream to dominate
+// (>= 40 M weights, e.g. 4096 x 14336).  The path's cost grows with the tokens (split-K reduction
+// of tokens x 128 partial sums per CTA), while the one-CTA-per-tile GEMM behind the same per-block
+// quantiser costs about the same from 33 to 128 tokens.  Measured, 4096 -> 6144 at 32 / 48 / 64 /
+// 96 / 128 tokens: 9.0 / 10.4 / 11.4 / 14.1 / 16.0 us on the small-s path, 9.7 / 8.8 / 9.6 / 10.1 us
+// from 48 tokens on the other; 4096 -> 28672 at 96 tokens: 17.9 against 19.5 us.
+static bool layer_takes_small_path(const batq_weight* w, int64_t s) {
+  return s <= 32 || (s <= kSmallSMax && w->m * w->n >= 40000000);
+}
+
 size_t batq_linear_workspace_bytes(const batq_weight* w, int64_t s) {
   if (w == nullptr || s < 0) return 0;
   const size_t q = round_up(static_cast<size_t>(s * (w->n / 2)), 1024) + round_up(batq_sf_bytes(s, w->n, BATQ_SF_MMA), 1024);
-  return q + (s > 0 && s <= kSmallSMax ? small_scratch(w, s).total() : 0);
+  return q + (s > 0 && layer_takes_small_path(w, s) ? small_scratch(w, s).total() : 0);
 }
 
 int32_t batq_linear_kernel_launches(const batq_transform* t, const batq_weight* w, int64_t s) {
@@ -1117,7 +1136,7 @@ batq_status batq_linear_w4a4(const batq_transform* t, const batq_weight* w, cons
   uint8_t* sf = codes + round_up(static_cast<size_t>(s * (w->n / 2)), 1024);
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   if (use_fused_small(t, w, s)) return launch_linear_fused(t, w, x_bf16, s, ld, y, y_dtype, ldy, cs);
-  if (s <= kSmallSMax) {
+  if (layer_takes_small_path(w, s)) {
     // A handful of tokens: the quantiser also clears the split-K tickets, and the GEMM is launched
     // as its programmatic dependent so that the weight stream starts while it still runs.
     uint8_t* scratch = sf + round_up(batq_sf_bytes(s, w->n, BATQ_SF_MMA), 1024);

@@ -1,11 +1,11 @@
-// MXFP4 x MXFP4 GEMM for a handful of tokens (decode: s <= 64), stage 3 of the path
+// MXFP4 x MXFP4 GEMM for a handful of tokens (decode: s <= 128), stage 3 of the path
 // where it is bound by streaming the weights from HBM once (0.53 bytes per weight).
 //
 //   Y[s, m] = sum_j 2^(ex[s,j] + ew[m,j]) * sum_{i<32} qx[s,j,i] * qw[m,j,i]
 //
 // the low-bit matrix multiplication Q(XP) Q(P^-1 W^T) of the paper's Sec. 3, with the
 // operands swapped for the tensor cores: a CTA owns 128 weight rows (the 128-row MMA
-// operand) and a slice of K; the tokens are the narrow MMA dimension (16, 32 or 64
+// operand) and a slice of K; the tokens are the narrow MMA dimension (16, 32, 64 or 128
 // columns), so no tensor-core row is spent on padding tokens.  The grid is
 // (row tiles) x (K splits): enough CTAs, two per SM, to keep the whole memory system
 // busy however few output features the layer has.  With more than one split every CTA
@@ -35,11 +35,12 @@ struct SmallCfg {
   static constexpr int kXBytes = NTOK * kBKBytes;    // activation codes
   static constexpr int kSfBytes = 1024;              // two 512-byte scale atoms (8 blocks), per operand
   static constexpr int kStageBytes = kWBytes + kXBytes + 2 * kSfBytes;
-  static constexpr int kStages = (NTOK == 64) ? 4 : 5;
+  static constexpr int kStages = (NTOK == 128) ? 3 : (NTOK == 64) ? 4 : 5;
   static constexpr int kSfColsPerStage = 16;         // W: 2 atoms x 4 columns, X: 2 atoms x 4 columns
-  static constexpr int kTmemCols = 128;
+  static constexpr int kTmemCols = (NTOK == 128) ? 256 : 128;
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024;
-  static_assert(NTOK == 16 || NTOK == 32 || NTOK == 64, "token tile");
+  static_assert(NTOK == 16 || NTOK == 32 || NTOK == 64 || NTOK == 128, "token tile");
+  static_assert(kStages * kStageBytes >= NTOK * 128 * 4, "the partial tile of the cluster reduction fits the ring");
   static_assert(NTOK + kStages * kSfColsPerStage <= kTmemCols, "tensor memory budget");
   static_assert(2 * (kSmemBytes + 2048) <= 232448, "two CTAs per SM");
   static_assert(kStageBytes % 1024 == 0, "stage alignment");
@@ -124,7 +125,6 @@ gemm_small_s_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
   const int n_steps = kt1 - kt0;                  // >= 1: the host keeps splits <= k_steps
   const bool by_cluster = p.cluster_reduce != 0 && p.splits > 1;
   bool epi_ok = false;
-  uint32_t v[NTOK];
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
@@ -224,6 +224,8 @@ gemm_small_s_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     __syncwarp();
   } else {
     // ---------------------------------------------------------------- epilogue warps
+    // The accumulator row of a thread (NTOK values) is handled 16 tokens at a time, so that the
+    // widest token tile needs no more registers than the narrowest.
     const int quad = warp & 3;  // tensor-memory lanes [32*quad, 32*quad + 32)
     const int row = quad * 32 + lane;              // weight row inside the tile
     const int64_t mrow = static_cast<int64_t>(rt) * 128 + row;
@@ -232,65 +234,86 @@ gemm_small_s_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     // agree on `ok` and take the barriers below together or not at all.
     named_barrier_sync(1, 128);
     const bool ok = *static_cast<volatile int*>(&abort_flag) == 0;
+    auto store16 = [&](int c, const float (&val)[16]) {
+      if (mrow < p.m) {
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+          if (c + t < p.s) {
+            if (OUT_BF16)
+              reinterpret_cast<__nv_bfloat16*>(p.y)[(c + t) * p.ldy + mrow] = __float2bfloat16_rn(val[t]);
+            else
+              reinterpret_cast<float*>(p.y)[(c + t) * p.ldy + mrow] = val[t];
+          }
+        }
+      }
+    };
     if (ok) {
       tc_fence_after_sync();
-      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
-#pragma unroll
-      for (int c = 0; c < NTOK; c += 16) tmem_ld_32x32b_x16(taddr + c, v + c);
-      tmem_ld_wait();
-      tc_fence_before_sync();
       epi_ok = true;
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+      float* part_smem = reinterpret_cast<float*>(smem);  // cluster mode: every MMA has completed, the ring is free
+      float* mine = p.partial + (static_cast<int64_t>(rt) * p.splits + sp) * (NTOK * 128) + row;
+#pragma unroll 1
+      for (int c = 0; c < NTOK; c += 16) {
+        if (c >= p.s) break;
+        uint32_t v[16];
+        tmem_ld_32x32b_x16(taddr + c, v);
+        tmem_ld_wait();
+        if (by_cluster) {
+#pragma unroll
+          for (int t = 0; t < 16; ++t)
+            if (c + t < p.s) part_smem[(c + t) * 128 + row] = __uint_as_float(v[t]);
+        } else if (p.splits > 1) {
+#pragma unroll
+          for (int t = 0; t < 16; ++t)
+            if (c + t < p.s) __stcg(mine + (c + t) * 128, __uint_as_float(v[t]));
+        } else {
+          float val[16];
+#pragma unroll
+          for (int t = 0; t < 16; ++t) val[t] = __uint_as_float(v[t]);
+          store16(c, val);
+        }
+      }
+      tc_fence_before_sync();
 
-      bool write_out = !by_cluster;
-      if (by_cluster) {
-        // every MMA has completed: the operand ring is free and takes this CTA's partial tile
-        float* part = reinterpret_cast<float*>(smem);
-#pragma unroll
-        for (int t = 0; t < NTOK; ++t)
-          if (t < p.s) part[t * 128 + row] = __uint_as_float(v[t]);
-      } else if (p.splits > 1) {
-        float* mine = p.partial + (static_cast<int64_t>(rt) * p.splits + sp) * (NTOK * 128) + row;
-#pragma unroll
-        for (int t = 0; t < NTOK; ++t)
-          if (t < p.s) __stcg(mine + t * 128, __uint_as_float(v[t]));
+      if (!by_cluster && p.splits > 1) {
         __threadfence();
         named_barrier_sync(1, 128);
         if (warp == 2 && lane == 0) ticket_slot = atomicAdd(p.tickets + rt, 1u);
         named_barrier_sync(1, 128);
-        write_out = ticket_slot == static_cast<uint32_t>(p.splits - 1);
-        if (write_out) {
+        if (ticket_slot == static_cast<uint32_t>(p.splits - 1)) {
           __threadfence();
           // Sum in split order (deterministic).  Loads are issued in independent batches -- over the
           // tokens when there are many, over the splits when there are few -- so that their latencies
           // overlap instead of adding up.
           const float* all = p.partial + static_cast<int64_t>(rt) * p.splits * (NTOK * 128) + row;
           if (p.s > 4) {
+#pragma unroll 1
+            for (int c = 0; c < NTOK; c += 16) {
+              if (c >= p.s) break;
+              float acc[16];
 #pragma unroll
-            for (int c = 0; c < NTOK; c += 16) {  // 16 tokens at a time keeps the registers in check
-              if (c < p.s) {
-                float acc[16];
+              for (int t = 0; t < 16; ++t) acc[t] = 0.0f;
+              constexpr int QB = 4;  // splits per batch: 64 loads in flight
+              for (int q0 = 0; q0 < p.splits; q0 += QB) {
+                float part[QB][16];
 #pragma unroll
-                for (int t = 0; t < 16; ++t) acc[t] = 0.0f;
-                constexpr int QB = NTOK == 16 ? 4 : 2;  // splits per batch: 64 / 32 loads in flight
-                for (int q0 = 0; q0 < p.splits; q0 += QB) {
-                  float part[QB][16];
+                for (int qq = 0; qq < QB; ++qq)
 #pragma unroll
-                  for (int qq = 0; qq < QB; ++qq)
+                  for (int t = 0; t < 16; ++t)
+                    part[qq][t] = (q0 + qq < p.splits && c + t < p.s)
+                                      ? __ldcg(all + (q0 + qq) * (NTOK * 128) + (c + t) * 128) : 0.0f;
 #pragma unroll
-                    for (int t = 0; t < 16; ++t)
-                      part[qq][t] = (q0 + qq < p.splits && c + t < p.s)
-                                        ? __ldcg(all + (q0 + qq) * (NTOK * 128) + (c + t) * 128) : 0.0f;
+                for (int qq = 0; qq < QB; ++qq)
 #pragma unroll
-                  for (int qq = 0; qq < QB; ++qq)
-#pragma unroll
-                    for (int t = 0; t < 16; ++t) acc[t] += part[qq][t];
-                }
-#pragma unroll
-                for (int t = 0; t < 16; ++t) v[c + t] = __float_as_uint(acc[t]);
+                  for (int t = 0; t < 16; ++t) acc[t] += part[qq][t];
               }
+              store16(c, acc);
             }
           } else {
-            float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            float acc[16];
+#pragma unroll
+            for (int t = 0; t < 16; ++t) acc[t] = 0.0f;
             for (int q0 = 0; q0 < p.splits; q0 += 8) {
               float part[8][4];
 #pragma unroll
@@ -303,21 +326,9 @@ gemm_small_s_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
 #pragma unroll
                 for (int t = 0; t < 4; ++t) acc[t] += part[qq][t];
             }
-#pragma unroll
-            for (int t = 0; t < 4; ++t) v[t] = __float_as_uint(acc[t]);
+            store16(0, acc);
           }
           if (warp == 2 && lane == 0) p.tickets[rt] = 0;  // ready for the next call
-        }
-      }
-      if (write_out && mrow < p.m) {
-#pragma unroll
-        for (int t = 0; t < NTOK; ++t) {
-          if (t < p.s) {
-            if (OUT_BF16)
-              reinterpret_cast<__nv_bfloat16*>(p.y)[t * p.ldy + mrow] = __float2bfloat16_rn(__uint_as_float(v[t]));
-            else
-              reinterpret_cast<float*>(p.y)[t * p.ldy + mrow] = __uint_as_float(v[t]);
-          }
         }
       }
     }

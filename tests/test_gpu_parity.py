@@ -471,7 +471,7 @@ def _small_case(batq, S, M, N, seed, out_dtype=torch.float32, splits=0):
 
 
 SMALL_SHAPES = [(1, 8, 32), (1, 1024, 1024), (4, 300, 544), (16, 4096, 4096), (17, 257, 2048 + 32), (32, 520, 3584),
-                (33, 128, 256), (64, 1000, 1024)]
+                (33, 128, 256), (64, 1000, 1024), (65, 264, 512), (100, 1032, 3584), (128, 4096, 2048)]
 
 
 @pytest.mark.parametrize("S,M,N", SMALL_SHAPES)
@@ -500,9 +500,9 @@ def test_gemm_small_s_many_splits_and_bf16(batq):
 def test_gemm_small_s_rejects_large_s_and_short_scratch(batq):
     w = batq.batq_prepare_weight(None, batq.bits_to_cuda_bf16(synth.make_weight(128, 256, 1)))
     z = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
-    y = torch.empty((65, 128), dtype=torch.float32, device="cuda")
+    y = torch.empty((129, 128), dtype=torch.float32, device="cuda")
     with pytest.raises(batq.BatqError) as e:
-        batq.batq_gemm_mxfp4_small_s(z, z, w, 65, y, batq.aligned_workspace(4096))
+        batq.batq_gemm_mxfp4_small_s(z, z, w, 129, y, batq.aligned_workspace(4096))
     assert e.value.status == 2
     with pytest.raises(batq.BatqError) as e:
         batq.batq_gemm_mxfp4_small_s(z, z, w, 8, y, batq.aligned_workspace(4096)[:512])
@@ -514,6 +514,9 @@ def test_gemm_small_s_rejects_large_s_and_short_scratch(batq):
                                             (50, 136, 544, "baseline"), (4, 1024, 1024, "baseline"),
                                             (1, 4096, 4096, "baseline"), (16, 6144, 4096, "paper"),
                                             (64, 520, 1024, "baseline"), (65, 520, 1024, "baseline"),
+                                            (100, 1032, 3584, "paper"), (128, 4096, 4096, "baseline"),
+                                            (100, 10240, 4096, "baseline"),   # 65..128 tokens on a large layer: small-s path
+                                            (129, 520, 1024, "baseline"),
                                             (520, 1032, 1024, "baseline")])
 def test_linear_w4a4_vs_oracle(batq, qmode, S, M, N, geometry):
     # automatic kernel choice: the small-s GEMM up to 64 tokens, one CTA per tile up to 128, CTA pairs above
@@ -579,7 +582,7 @@ def test_linear_fused_small_s_vs_oracle(batq, S, M, N, geometry, splits):
     assert np.linalg.norm(outs[1] - outs[2]) <= 1e-4 * np.linalg.norm(Sabs)
 
 
-@pytest.mark.parametrize("S", [1, 4, 16, 48, 300])
+@pytest.mark.parametrize("S", [1, 4, 16, 48, 100, 300])
 def test_linear_calls_back_to_back_share_a_workspace(batq, S):
     """Layers called one after the other on one stream, with one workspace, inside a replayed CUDA
     graph: every kernel is a programmatic dependent of the one before it (the next layer's
