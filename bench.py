@@ -382,7 +382,7 @@ def run_ours(args):
             "config": {"workload": args.workload, "tokens": S, "projections": [list(p) for p in projs],
                        "transform": "shared 4x4 (x) private 8x8 per 32-group, clip U[0.8,1]", "output": "bf16",
                        "l2": "inputs larger than L2: one step touches %.0f MB" % (touched / 1e6)},
-            "roofline": {"bound": "tensor", "kernel": "gemm_mxfp4_kernel", "achieved": gemm_achieved, "peak": fp4_peak,
+            "roofline": {"bound": "tensor", "kernel": "gemm_mxfp4_pair_kernel" if S > 128 else "gemm_mxfp4_kernel", "achieved": gemm_achieved, "peak": fp4_peak,
                          "events": "around every launch in every %dth step of the timed region (%d steps)" % (
                              EVENT_EVERY, len(sampled)),
                          "unit": "TFLOP/s", "frac": gemm_achieved / fp4_peak, "traffic": traffic,
