@@ -164,8 +164,8 @@ batq_status batq_gemm_mxfp4_small_s(const void* x_codes, const void* x_scales_mm
                                     int64_t s, void* y, int32_t y_dtype, int64_t ldy, void* scratch,
                                     size_t scratch_bytes, void* stream);
 
-/* Test / tuning hook: forces the GEMM's output-tile width to 128, 192 or 256 columns for all
- * later calls in this process (the CTA-pair kernel also takes 64, and 448 for columns of 256 and
+/* Test / tuning hook: forces the GEMM's output-tile width to 64, 128, 192 or 256 columns for all
+ * later calls in this process (the CTA-pair kernel also takes 448 for columns of 256 and
  * 192 alternating); any other value restores the automatic choice. */
 void batq_debug_force_tile_width(int32_t bn);
 

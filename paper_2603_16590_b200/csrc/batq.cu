@@ -49,6 +49,7 @@ struct batq_weight {
   CUtensorMap tmap_b256;  // boxes of 256 / 192 / 128 weight rows x 128 bytes
   CUtensorMap tmap_b192;
   CUtensorMap tmap_b128;
+  CUtensorMap tmap_b64;
   CUtensorMap tmap_b32;   // boxes of 32 weight rows: the CTA-pair kernel composes its half tiles from them
   CUtensorMap tmap_sf;    // scale atoms: [row tiles x KA] rows of 512 bytes, boxes of two atoms
 };
@@ -115,6 +116,8 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(gemm_mxfp4_kernel<192, true>, GemmCfg<192>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<128, false>, GemmCfg<128>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<128, true>, GemmCfg<128>::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_kernel<64, false>, GemmCfg<64>::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_kernel<64, true>, GemmCfg<64>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_pair_kernel<false>, PairCfg::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_pair_kernel<true>, PairCfg::kSmemBytes);
     e = e ? e : set_smem(linear_small_s_fused_kernel<false>, FusedCfg::kSmemBytes);
@@ -434,8 +437,11 @@ batq_status make_y_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_
 // loop proportional to the tile width.
 int g_force_bn = 0;  // test hook: 0 = automatic
 int pick_bn(int64_t s, int64_t m, int64_t n, int sm_count) {
-  if (g_force_bn == 128 || g_force_bn == 192 || g_force_bn == 256) return g_force_bn;
+  if (g_force_bn == 64 || g_force_bn == 128 || g_force_bn == 192 || g_force_bn == 256) return g_force_bn;
   const int64_t mt = (s + kBM - 1) / kBM;
+  // A few dozen tiles cannot pull the weights fast enough (a CTA streams what its ring keeps in
+  // flight): below half a wave of 128-wide tiles, twice as many 64-wide ones.
+  if (mt * ((m + 127) / 128) * 2 <= sm_count && m > 64) return 64;
   const double k_steps = static_cast<double>((n + 255) / 256);
   auto cost = [&](int bn, double exposed_epilogue) {
     const int64_t tiles = mt * ((m + bn - 1) / bn);
@@ -450,9 +456,6 @@ int pick_bn(int64_t s, int64_t m, int64_t n, int sm_count) {
 
 int g_force_gemm_kernel = 0;  // tuning hook: 0 = automatic, 1 = one CTA per tile, 2 = CTA pairs
 
-// CTA-pair kernel: every pair takes an equal, contiguous share of the 256-token x 64-feature units
-// and walks it in tiles of up to cap0 / cap1 units (accumulator slots 0 / 1; 4 and 3 unless a
-// tile width is forced).
 // The schedule of the CTA-pair kernel for an s x m output with k_steps K-steps: column widths and
 // number of pairs.  Every candidate (columns of 128, 192 or 256 features, or 256 and 192
 // alternating) is walked exactly as the kernel walks it, and the pair that finishes last decides.
@@ -599,7 +602,8 @@ batq_status launch_gemm(const void* x_codes, const void* x_sf, const batq_weight
   (cfg.dynamicSmemBytes = GemmCfg<BN>::kSmemBytes, cudaLaunchKernelEx(&cfg, gemm_mxfp4_kernel<BN, BF>, tmap_a, TB, tmap_y, p))
   if (bn == 256) e = bf ? BATQ_GEMM(256, true, w->tmap_b256) : BATQ_GEMM(256, false, w->tmap_b256);
   else if (bn == 192) e = bf ? BATQ_GEMM(192, true, w->tmap_b192) : BATQ_GEMM(192, false, w->tmap_b192);
-  else e = bf ? BATQ_GEMM(128, true, w->tmap_b128) : BATQ_GEMM(128, false, w->tmap_b128);
+  else if (bn == 128) e = bf ? BATQ_GEMM(128, true, w->tmap_b128) : BATQ_GEMM(128, false, w->tmap_b128);
+  else e = bf ? BATQ_GEMM(64, true, w->tmap_b64) : BATQ_GEMM(64, false, w->tmap_b64);
 #undef BATQ_GEMM
   if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
   return BATQ_OK;
@@ -1036,6 +1040,7 @@ batq_status batq_prepare_weight(const batq_transform* t, const void* w_bf16, int
   st = make_codes_tmap(&w->tmap_b256, w->codes, m, n / 2, 256);
   if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b192, w->codes, m, n / 2, 192);
   if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b128, w->codes, m, n / 2, 128);
+  if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b64, w->codes, m, n / 2, 64);
   if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b32, w->codes, m, n / 2, 32);
   if (st == BATQ_OK) st = make_sf_tmap(&w->tmap_sf, w->scales, (m + 127) / 128, w->katoms);
   if (st != BATQ_OK) { delete w; return st; }
