@@ -30,6 +30,10 @@ FP4_OVER_BF16 = 4.0       # nominal dense peak ratio 9 / 2.25 PFLOP/s
 QUANT_BYTES_PER_ELEM = 2.53125   # 2 (bf16 in) + 0.5 (codes) + 1/32 (scale byte)
 WEIGHT_BYTES_PER_ELEM = 0.53125  # 0.5 (codes) + 1/32 (scale byte)
 EVENT_EVERY = 8                  # prefill: every 8th timed step carries per-launch events
+MIN_BRACKETED = 50               # prefill: at least this many bracketed steps (extra ones follow the timed region)
+NOMINAL_FP4_TFLOPS = 9000.0      # vendor figure for dense FP4 at the maximum SM clock (context, not the denominator)
+# The CPU oracle is timed on this fixed sample of the workload's first projection (rows, output features)
+ORACLE_SAMPLE = {"prefill": (512, 4096), "decode": (16, 4096), "quant": (2048, 0)}
 
 # kind, tokens, projections (name, n in, m out), vision-row fraction, outlier-channel fraction
 WORKLOADS = {
@@ -68,6 +72,31 @@ def load_peaks():
         return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
                 "bf16_tflops_sustained": p["bf16_tflops_sustained"], "source": "measured"}
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def workload_config(workload):
+    """The `config` object of the JSON line: a function of the workload name alone, so that both
+    arms (--impl ours / reference) print the same object."""
+    kind, tokens, projs, vis_frac, och = WORKLOADS[workload]
+    cfg = {"workload": workload, "tokens": tokens[0] if kind == "prefill" else tokens,
+           "projections": [list(p) for p in projs],
+           "transform": "shared 4x4 (x) private 8x8 per 32-group, clip U[0.8,1]"}
+    if kind == "prefill":
+        S = tokens[0]
+        touched = sum(S * n * 2 + S * m * 2 + n * m * WEIGHT_BYTES_PER_ELEM for _, n, m in projs)
+        cfg.update({"output": "bf16", "l2": "inputs larger than L2: one step touches %.0f MB" % (touched / 1e6)})
+    elif kind == "decode":
+        copies = 4
+        cfg.update({"output": "bf16",
+                    "launch": "per token count one CUDA graph of %d layers x %d projections in model order" % (
+                        copies, len(projs)),
+                    "l2": "%d copies of each prepared weight used in turn: %.0f MB cycle through L2 between reuses" % (
+                        copies, copies * sum(n * m * WEIGHT_BYTES_PER_ELEM for _, n, m in projs) / 1e6)})
+    else:
+        cfg.update({"hidden": [p[1] for p in projs], "ablation": "T = I (plain MXFP4); 8-bit elements (MXFP8)",
+                    "l2": "a 256 MB buffer is read between launches (outside the per-launch events)",
+                    "value_note": "transform flops (24 per element) over quantiser time; the GB/s figures are the point"})
+    return cfg
 
 
 def make_layer_inputs(workload, S, seed):
@@ -166,41 +195,52 @@ def oracle_threads():
         return os.cpu_count() or 1
 
 
-def time_oracle(workload, seed, steps, warmup, budget_s):
-    """Times the oracle as it stands on a sample sized so that warmup + steps take about
-    `budget_s` seconds: starting from a small sample, rows and features are doubled together
-    while one step of the doubled sample (about four times the work) still fits its share."""
-    per_step = budget_s / max(steps + warmup, 1)
-    rows, feats = 64, 512
-    while True:
-        step, flops, desc = oracle_sample(workload, seed, rows, feats)
+def time_oracle(workload, seed, steps, warmup, threads=None):
+    """Times the oracle as it stands on the workload's fixed sample (ORACLE_SAMPLE); `threads`
+    limits the BLAS / OpenMP pools it runs on (None = as the libraries choose: all cores).
+    Returns (TFLOP/s, seconds per step, sample description, threads used)."""
+    kind = WORKLOADS[workload][0]
+    rows, feats = ORACLE_SAMPLE[kind]
+    step, flops, desc = oracle_sample(workload, seed, rows, feats)
+
+    def run():
+        for _ in range(warmup):
+            step()
         t0 = time.perf_counter()
-        step()
-        once = time.perf_counter() - t0
-        _, tokens, projs, _, _ = WORKLOADS[workload]
-        if once * 4.0 > per_step or (rows >= tokens[-1] and feats >= max(projs[0][2], 1)):
-            break
-        rows, feats = rows * 2, feats * 2
-    for _ in range(max(warmup - 1, 0)):   # the sizing call above was the first warm-up
-        step()
-    t0 = time.perf_counter()
-    for _ in range(steps):
-        step()
-    dt = (time.perf_counter() - t0) / max(steps, 1)
-    return flops / dt / 1e12, dt, desc
+        for _ in range(steps):
+            step()
+        return (time.perf_counter() - t0) / max(steps, 1)
+
+    if threads is None:
+        dt, used = run(), oracle_threads()
+    else:
+        from threadpoolctl import threadpool_limits
+        with threadpool_limits(limits=threads):
+            dt, used = run(), threads
+    return flops / dt / 1e12, dt, desc, used
+
+
+def cpu_baseline(workload, seed):
+    """The oracle on all host cores (3 steps) and on one core (1 step), same fixed sample."""
+    val, dt, desc, cores = time_oracle(workload, seed, 3, 1)
+    val1, dt1, _, _ = time_oracle(workload, seed, 1, 0, threads=1)
+    return {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc, "seconds_per_sample": dt,
+            "one_core": {"value": val1, "cores": 1, "seconds_per_sample": dt1}}
 
 
 def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    kind, tokens, projs, _, _ = WORKLOADS[args.workload]
+    if args.workload not in WORKLOADS:
+        print(json.dumps({"impl": "reference", "unavailable": "the MMA-only measurement has no CPU counterpart"}))
+        return
     steps = args.steps if args.steps is not None else 5
-    val, dt, desc = time_oracle(args.workload, synth.BASE_SEED, steps, args.warmup, 60.0)
+    val, dt, desc, cores = time_oracle(args.workload, synth.BASE_SEED, steps, args.warmup)
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "tokens": tokens, "projections": [list(p) for p in projs]},
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": desc},
+            "config": workload_config(args.workload),
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -283,19 +323,132 @@ def timed_region(h, step, steps, warmup):
     return h.max_over_ranks(e0.elapsed_time(e1)), clocks
 
 
+def measure_mma_peak(B, torch, iters):
+    """The block-scaled FP4 tensor-core rate with operands resident in shared memory (MMA-only loop,
+    every SM busy, nothing loaded or stored): CTA pairs on 256 x 256 tiles and single CTAs on
+    128 x 256 tiles, one timed launch each after a short warm-up launch."""
+    out = {}
+    for name, pair in (("pair_256x256", True), ("cta_128x256", False)):
+        B.batq_debug_mma_peak(pair, 256, max(64, iters // 50))
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        flops = B.batq_debug_mma_peak(pair, 256, iters)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        out[name] = {"tflops": flops / (ms * 1e-3) / 1e12, "ms": ms}
+    if B.batq_last_device_status() != 0:
+        raise SystemExit("device status after the MMA-only loop")
+    best = max(out, key=lambda k: out[k]["tflops"])
+    return {"tflops": out[best]["tflops"], "shape": best, "variants": out,
+            "how": "tcgen05.mma kind::mxf4.block_scale only, %d K-steps per CTA (pair), CUDA events" % iters}
+
+
+def measure_big_quantizer(B, torch, seed):
+    """The quantiser at the largest size of the sweep, 32768 x 8192 (537 MB in, 143 MB out: far larger
+    than L2), where it is meant to run at the HBM roofline.  The batch is a 4096-row draw repeated
+    eight times (the kernel's time does not depend on the values)."""
+    S, N, rep = 32768, 8192, 8
+    t = synth.make_transform(N, seed + 901, "baseline")
+    tr = B.batq_transform_create(N, t.left, t.right, t.clip_lo, t.clip_hi)
+    x = B.bits_to_cuda_bf16(synth.make_activations(S // rep, N, seed + 900)).repeat(rep, 1)
+    codes = torch.empty((S, N // 2), dtype=torch.uint8, device="cuda")
+    sf = torch.empty(B.batq_sf_bytes(S, N, B.SF_MMA), dtype=torch.uint8, device="cuda")
+    marks = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(10)]
+    for k in range(-3, len(marks)):
+        if k >= 0:
+            marks[k][0].record()
+        B.batq_quantize_act(tr, x, codes, sf, B.SF_MMA)
+        if k >= 0:
+            marks[k][1].record()
+    torch.cuda.synchronize()
+    us = float(np.median([a.elapsed_time(b) for a, b in marks]) * 1e3)
+    gbs = S * N * QUANT_BYTES_PER_ELEM / (us * 1e-6) / 1e9
+    peaks = load_peaks()
+    del x, codes, sf
+    return {"tokens": S, "hidden": N, "us": us, "achieved": gbs, "unit": "GB/s", "peak": peaks["hbm_gbs"],
+            "frac": gbs / peaks["hbm_gbs"], "events": "around each of 10 launches, median"}
+
+
+def sweep_parity_counts(B, torch, cases, rows_per_case=256):
+    """Part of the CPU-oracle leg of the quantiser sweep: for every case, the first and the last
+    `rows_per_case` token rows quantised by the library and by the oracle (fp64 transform), codes and
+    scale bytes compared.  Plain MXFP4 (T = I) must agree bit for bit; with the transform, the fp32
+    arithmetic may move an element next to a rounding boundary to the neighbouring code."""
+    from oracle import batq_oracle as O
+    out = []
+    for L in cases:
+        S, n, k = L["S"], L["n"], L["n"] // 32
+        rows = np.unique(np.concatenate([np.arange(min(rows_per_case, S)), np.arange(max(0, S - rows_per_case), S)]))
+        idx = torch.from_numpy(rows).cuda()
+        xb = L["x_bits"][rows]
+        t = L["t"]
+        rec = {"tokens": S, "hidden": n, "rows_checked": int(len(rows)), "elements_checked": int(len(rows)) * n}
+        for name, tr, want in (("gpk", L["tr"], O.quantize_act(xb, t.left, t.right, t.clip_lo, t.clip_hi)),
+                               ("identity", None, O.quantize_act(xb, None, None))):
+            scales = torch.empty((S, k), dtype=torch.uint8, device="cuda")
+            B.batq_quantize_act(tr, L["x"], L["codes"], scales, B.SF_ROWMAJOR)
+            gc = O.unpack_codes(L["codes"][idx].cpu().numpy())
+            gs = scales[idx].cpu().numpy()
+            rec[name + "_code_mismatch"] = int((gc != want[0]).sum())
+            rec[name + "_scale_mismatch"] = int((gs != want[1]).sum())
+        out.append(rec)
+    return out
+
+
+def run_peak(args, h, B, peaks):
+    """--workload peak_mxf4: the MMA-only rate as a burst (one launch of a few ms) and sustained
+    (launches back to back for about a second, under the power cap), with the clocks sampled."""
+    import torch
+    burst = measure_mma_peak(B, torch, 20000)
+    pair = burst["shape"].startswith("pair")
+    sampler = ClockSampler(h.local)
+    h.barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n = args.steps if args.steps is not None else 150
+    e0.record()
+    flops = 0.0
+    for _ in range(n):
+        flops += B.batq_debug_mma_peak(pair, 256, 20000)
+    e1.record()
+    h.barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    if B.batq_last_device_status() != 0:
+        raise SystemExit("device status after the MMA-only loop")
+    sustained = flops / (ms * 1e-3) / 1e12
+    if h.rank == 0:
+        print(json.dumps({
+            "metric": "mxf4_mma_only_tflops", "unit": UNIT, "value": sustained, "n_gpus": h.world, "steps": n,
+            "warmup": 1, "ms_per_step": ms / n, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "mxfp4", "data": "synthetic",
+            "config": {"workload": "peak_mxf4", "shape": burst["shape"], "k_steps_per_launch": 20000},
+            "burst": burst, "sustained": {"tflops": sustained, "ms": ms},
+            "context": {"cublas_bf16_x4_burst": peaks["bf16_tflops"] * FP4_OVER_BF16,
+                        "cublas_bf16_x4_sustained": peaks["bf16_tflops_sustained"] * FP4_OVER_BF16,
+                        "nominal": NOMINAL_FP4_TFLOPS, "source": peaks["source"]},
+            "gpu_launches": n + 4, "clocks": clocks}))
+    h.close()
+
+
 def run_ours(args):
     import torch
     from paper_2603_16590_b200 import binding as B
 
     h = Harness()
     B.load()
-    B.batq_debug_force_tile_width(args.tile_width)
-    B.batq_debug_force_quantizer(args.quantizer)
-    B.batq_debug_force_gemm_kernel(args.gemm_kernel)
-    B.batq_debug_force_small_s_splits(args.splits)
-    B.batq_debug_force_small_s_path(args.small_path)
-    B.batq_debug_force_small_s_reduce(args.small_reduce)
+    # tuning switches: touched only when a flag asks for something other than the automatic choice
+    for value, hook in ((args.tile_width, B.batq_debug_force_tile_width), (args.quantizer, B.batq_debug_force_quantizer),
+                        (args.gemm_kernel, B.batq_debug_force_gemm_kernel), (args.splits, B.batq_debug_force_small_s_splits),
+                        (args.small_path, B.batq_debug_force_small_s_path),
+                        (args.small_reduce, B.batq_debug_force_small_s_reduce)):
+        if value != 0:
+            hook(value)
     peaks = load_peaks()
+    if args.workload == "peak_mxf4":
+        return run_peak(args, h, B, peaks)
     kind, tokens, projs, _, _ = WORKLOADS[args.workload]
     # prefill: long enough (> 1 s) for the power cap to settle, so that the sustained peak is the fair denominator
     steps = args.steps if args.steps is not None else {"prefill": 5000, "decode": 300, "quant": 100}[kind]
@@ -346,8 +499,47 @@ def run_ours(args):
                 m[i][2].record()
 
         ms, clocks = timed_region(h, step, steps, args.warmup)
-        q_ms = np.array([[m[i][0].elapsed_time(m[i][1]) for i in range(len(layers))] for m in marks.values()]).mean(axis=0)
-        g_ms = np.array([[m[i][1].elapsed_time(m[i][2]) for i in range(len(layers))] for m in marks.values()]).mean(axis=0)
+        # A short run brackets only a few steps: add bracketed steps right after the timed region (same
+        # calls, same buffers, device still warm) until MIN_BRACKETED have been taken.
+        extra = max(0, MIN_BRACKETED - len(sampled))
+        for k in range(steps, steps + extra):
+            marks[k] = [(ev(), ev(), ev()) for _ in layers]
+            step(k)
+        torch.cuda.synchronize()
+        q_all = np.array([[m[i][0].elapsed_time(m[i][1]) for i in range(len(layers))] for m in marks.values()])
+        g_all = np.array([[m[i][1].elapsed_time(m[i][2]) for i in range(len(layers))] for m in marks.values()])
+        q_ms, g_ms = q_all.mean(axis=0), g_all.mean(axis=0)
+
+        # The same launches back to back (one CUDA graph of 8 steps' GEMMs, then one of 8 steps' quantisers):
+        # no event between launches, so each kernel's prologue hides behind the one before it as it does in
+        # the timed steps.  Reported next to the bracketed durations, not instead of them.
+        def graph_of(fn, reps=8):
+            side = torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    for _ in range(reps):
+                        fn()
+            return g, reps
+
+        def time_graph(g, reps, n=5):
+            g.replay()
+            torch.cuda.synchronize()
+            a, b = ev(), ev()
+            a.record()
+            for _ in range(n):
+                g.replay()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / (n * reps)
+
+        b2b = []
+        for L in layers:
+            gg, r = graph_of(lambda L=L: B.batq_gemm_mxfp4(L["codes"], L["sf"], L["w"], S, L["y"]))
+            gq, _ = graph_of(lambda L=L: B.batq_quantize_act(L["tr"], L["x"], L["codes"], L["sf"], B.SF_MMA))
+            b2b.append((time_graph(gq, r), time_graph(gg, r)))
+        mma_only = measure_mma_peak(B, torch, 20000) if S > 128 else None
+        big_quant = measure_big_quantizer(B, torch, seed) if (S > 128 and h.rank == 0) else None
 
         # end to end: host buffers in and out through the C-ABI host entry point
         def step_host():
@@ -376,25 +568,46 @@ def run_ours(args):
         traffic = None
         if GEMM_TRAFFIC["workload"] == args.workload and GEMM_TRAFFIC["source_sha256"] == kernel_source_hash():
             traffic = GEMM_TRAFFIC["mb_per_step"]
-        touched = h2d + d2h + sum(L["n"] * L["m"] * WEIGHT_BYTES_PER_ELEM for L in layers)
+        b2b_gemm = sum(gemm_flops) / (sum(t[1] for t in b2b) * 1e-3) / 1e12
+        b2b_quant = sum(q_bytes) / (sum(t[0] for t in b2b) * 1e-3) / 1e9
+        # context: the vendor's dense-FP4 figure scaled to the SM clock sampled during the timed region
+        mhz = (clocks or {}).get("sm_mhz") or 0.0
+        mhz_max = (clocks or {}).get("sm_max_mhz") or 0.0
+        nominal_at_clock = NOMINAL_FP4_TFLOPS * mhz / mhz_max if mhz and mhz_max else None
+        roof = {"bound": "tensor", "kernel": "gemm_mxfp4_pair_kernel" if S > 128 else "gemm_mxfp4_kernel",
+                "achieved": gemm_achieved, "peak": fp4_peak,
+                "events": "around every launch in every %dth step of the timed region (%d steps) and in %d more steps "
+                          "right after it" % (EVENT_EVERY, len(sampled), extra),
+                "unit": "TFLOP/s", "frac": gemm_achieved / fp4_peak, "traffic": traffic,
+                "traffic_unit": "MB per step (4 launches)" if traffic else None,
+                "peak_source": "%s cuBLAS bf16 %s x %.0f (nominal fp4:bf16 ratio): a proxy that inherits cuBLAS's own "
+                               "efficiency" % (peaks["source"], "sustained" if sustained else "burst", FP4_OVER_BF16),
+                "back_to_back": {"achieved": b2b_gemm, "frac": b2b_gemm / fp4_peak,
+                                 "how": "the same launches in a CUDA graph of 8 steps, no events between them"},
+                "nominal": {"peak": NOMINAL_FP4_TFLOPS, "frac": gemm_achieved / NOMINAL_FP4_TFLOPS,
+                            "peak_at_sampled_clock": nominal_at_clock,
+                            "frac_at_sampled_clock": gemm_achieved / nominal_at_clock if nominal_at_clock else None,
+                            "note": "vendor dense-FP4 figure; the 70 % target of the path is judged against this "
+                                    "one and is not met while frac here is below 0.70"}}
+        if mma_only is not None:
+            roof["mma_only"] = dict(mma_only, frac=gemm_achieved / mma_only["tflops"],
+                                    frac_back_to_back=b2b_gemm / mma_only["tflops"])
         line.update({
             "value": h.whole_job_rate(flops_step, steps, ms) / 1e12, "ms_per_step": ms / steps,
-            "config": {"workload": args.workload, "tokens": S, "projections": [list(p) for p in projs],
-                       "transform": "shared 4x4 (x) private 8x8 per 32-group, clip U[0.8,1]", "output": "bf16",
-                       "l2": "inputs larger than L2: one step touches %.0f MB" % (touched / 1e6)},
-            "roofline": {"bound": "tensor", "kernel": "gemm_mxfp4_pair_kernel" if S > 128 else "gemm_mxfp4_kernel", "achieved": gemm_achieved, "peak": fp4_peak,
-                         "events": "around every launch in every %dth step of the timed region (%d steps)" % (
-                             EVENT_EVERY, len(sampled)),
-                         "unit": "TFLOP/s", "frac": gemm_achieved / fp4_peak, "traffic": traffic,
-                         "traffic_unit": "MB per step (4 launches)" if traffic else None,
-                         "peak_source": "%s cuBLAS bf16 %s x %.0f (nominal fp4:bf16 ratio)" % (
-                             peaks["source"], "sustained" if sustained else "burst", FP4_OVER_BF16)},
+            "config": workload_config(args.workload),
+            "roofline": roof,
             "act_quant": {"bound": "hbm", "kernel": "quantize_act_tc_kernel", "achieved": quant_gbs,
                           "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": quant_gbs / peaks["hbm_gbs"],
-                          "peak_source": peaks["source"]},
+                          "peak_source": peaks["source"],
+                          "note": "between events: the kernel plus the launch gaps on both sides, at 17-59 MB per launch",
+                          "back_to_back": {"achieved": b2b_quant, "frac": b2b_quant / peaks["hbm_gbs"]},
+                          "largest_sweep_case": big_quant},
             "kernels": [{"name": L["name"], "n": L["n"], "m": L["m"], "quant_us": float(q_ms[i] * 1e3),
                          "quant_gbs": q_bytes[i] / (q_ms[i] * 1e-3) / 1e9, "gemm_us": float(g_ms[i] * 1e3),
-                         "gemm_tflops": gemm_flops[i] / (g_ms[i] * 1e-3) / 1e12} for i, L in enumerate(layers)],
+                         "gemm_tflops": gemm_flops[i] / (g_ms[i] * 1e-3) / 1e12,
+                         "quant_us_back_to_back": float(b2b[i][0] * 1e3), "gemm_us_back_to_back": float(b2b[i][1] * 1e3),
+                         "gemm_tflops_back_to_back": gemm_flops[i] / (b2b[i][1] * 1e-3) / 1e12}
+                        for i, L in enumerate(layers)],
             "e2e": {"value": flops_step * e2e_steps * h.world / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
             "gpu_launches": 2 * len(layers) * steps,
@@ -498,12 +711,7 @@ def run_ours(args):
         d2h = sum(c["S"] * c["L"]["m"] * 2 for c in order)
         line.update({
             "value": h.whole_job_rate(flops_step, steps, ms) / 1e12, "ms_per_step": ms / steps,
-            "config": {"workload": args.workload, "tokens": tokens, "projections": [list(p) for p in projs],
-                       "transform": "shared 4x4 (x) private 8x8 per 32-group, clip U[0.8,1]", "output": "bf16",
-                       "launch": "per token count one CUDA graph of %d layers x %d projections in model order" % (
-                           copies, len(base)),
-                       "l2": "%d copies of each prepared weight used in turn: %.0f MB cycle through L2 between reuses" % (
-                           copies, copies * sum(L["n"] * L["m"] * WEIGHT_BYTES_PER_ELEM for L in base) / 1e6)},
+            "config": workload_config(args.workload),
             "roofline": {"bound": "hbm", "kernel": "gemm_small_s_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
                          "peak_source": "%s copy bandwidth; achieved = weight bytes / time of the layer graphs "
@@ -583,10 +791,7 @@ def run_ours(args):
         line.update({
             "value": 24.0 * elems * steps * h.world / (t_ms[:, 0].sum() * steps * 1e-3) / 1e12,
             "ms_per_step": float(t_ms[:, 0].sum()),
-            "config": {"workload": args.workload, "tokens": tokens, "hidden": [p[1] for p in projs],
-                       "transform": "shared 4x4 (x) private 8x8 per 32-group, clip U[0.8,1]; ablation T = I",
-                       "l2": "a 256 MB buffer is read between launches (outside the per-launch events)",
-                       "value_note": "transform flops (24 per element) over quantiser time; the GB/s figures are the point"},
+            "config": workload_config(args.workload),
             "roofline": {"bound": "hbm", "kernel": "quantize_act_tc_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
                          "largest_case_gbs": float(bytes_case[big] / (t_ms[big, 0] * 1e-3) / 1e9),
@@ -607,9 +812,9 @@ def run_ours(args):
     if status != 0:
         raise SystemExit(f"device status {status} after the timed region")
     if h.rank == 0:
-        cpu_val, cpu_dt, cpu_desc = time_oracle(args.workload, synth.BASE_SEED, 3, 1, 20.0)
-        line["cpu_baseline"] = {"value": cpu_val, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
-                                "sample": cpu_desc, "seconds_per_sample": cpu_dt}
+        line["cpu_baseline"] = cpu_baseline(args.workload, synth.BASE_SEED)
+        if kind == "quant":
+            line["cpu_baseline"]["parity_check"] = sweep_parity_counts(B, torch, cases)
         line["clocks"] = clocks
         print(json.dumps(line))
     h.close()
@@ -621,7 +826,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None, help="timed steps (default: per workload, about 0.3-1 s of GPU time)")
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg1_llama8b_prefill", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="cfg1_llama8b_prefill", choices=sorted(WORKLOADS) + ["peak_mxf4"])
     ap.add_argument("--quantizer", type=int, default=0, help="0 auto, 1 ALU kernel, 2 tensor-core kernel (tuning)")
     ap.add_argument("--gemm-kernel", type=int, default=0, help="0 auto, 1 one CTA per tile, 2 CTA pairs (tuning)")
     ap.add_argument("--tile-width", type=int, default=0, help="force the GEMM tile width (tuning); 0 = automatic")

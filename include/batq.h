@@ -15,9 +15,12 @@
  * device, owned by the caller) or "host".  Calls validate on the host and
  * return a status; nothing throws or aborts.  Kernel launches are asynchronous
  * on the given stream (a cudaStream_t passed as void*; NULL = default stream).
- * The library allocates device memory only in batq_transform_create; every
- * other buffer is the caller's.  Device-side waits are bounded: a kernel that
+ * The library allocates device memory in batq_transform_create (held by the
+ * handle) and, temporarily, in batq_prepare_weight (offline: it allocates, frees
+ * and synchronises); every call on the online path (quantise, GEMM, layer) only
+ * uses the caller's buffers.  Device-side waits are bounded: a kernel that
  * gives up records BATQ_ERR_TIMEOUT, read back by batq_last_device_status.
+ * Test and tuning hooks live in batq_debug.h.
  */
 #ifndef BATQ_H_
 #define BATQ_H_
@@ -50,8 +53,8 @@ typedef struct batq_weight batq_weight;       /* one prepared (transformed, quan
 const char* batq_status_string(batq_status s);
 int batq_version(void);
 
-/* Theta = {A, {B_i}, {alpha_i}} of the paper's algorithm flow ("Store Theta for
- * online activation transformation"), as two Kronecker factors and clip ratios.
+/* Theta = {A, {B_i}, {alpha_i}}, the parameter set Algorithm 2 keeps for the online
+ * activation transform (its last step), as two Kronecker factors and clip ratios.
  *   n            channels, n % 32 == 0, k = n / 32 blocks.
  *   gr, gc       factor sizes, gr * gc == 32: (4, 8) is the paper's default (g2 = 4, g1 = 8);
  *                (1, 32), (2, 16), (8, 4), (16, 2), (32, 1) cover its ablation of the shared
@@ -98,7 +101,7 @@ batq_status batq_quantize_act(const batq_transform* t, const void* x_bf16, int64
                               int64_t ld, void* codes, void* scales, int32_t scale_layout,
                               void* stream);
 
-/* The same stages with 8-bit elements: MXFP8 with E4M3 codes (Sec. 2: "we adopt E4M3 for MXFP8"),
+/* The same stages with 8-bit elements: MXFP8 with E4M3 codes (the MXFP8 element type Sec. 2 settles on),
  * the activation format of the paper's W4A8 configurations and of the 8-bit KV cache (the key and
  * value transforms P_k, P_v of Sec. 3.2 are applied head by head: pass the cache as
  * [tokens * heads x head_dim] with a transform of n = head_dim).  Shared scale
@@ -111,13 +114,8 @@ batq_status batq_quantize_act_mxfp8(const batq_transform* t, const void* x_bf16,
                                     int64_t ld, void* codes, void* scales, int32_t scale_layout,
                                     void* stream);
 
-/* Test hook: the exact fp32 values the quantiser rounds (after transform and
- * clip, before scaling), out dev fp32 [s x n] row-major. */
-batq_status batq_debug_transform_clip_f32(const batq_transform* t, const void* x_bf16, int64_t s,
-                                          int64_t n, int64_t ld, float* out, void* stream);
-
-/* Offline weight fusion ("Offline Fusion for Deployment" in the paper's
- * algorithm flow): W~ = W P^-T per 32-block of each weight row, optional block
+/* Offline weight fusion (the deployment part of Algorithm 2):
+ * W~ = W P^-T per 32-block of each weight row, optional block
  * clip (Eq. 3-4 applied to weights), MXFP4 quantisation, written in the GEMM's
  * layout into a caller-provided buffer.  Computed in fp64 (inverse factors by
  * Gauss-Jordan on the host); not on the timed path.
@@ -163,43 +161,6 @@ size_t batq_gemm_small_s_scratch_bytes(const batq_weight* w, int64_t s);
 batq_status batq_gemm_mxfp4_small_s(const void* x_codes, const void* x_scales_mma, const batq_weight* w,
                                     int64_t s, void* y, int32_t y_dtype, int64_t ldy, void* scratch,
                                     size_t scratch_bytes, void* stream);
-
-/* Test / tuning hook: forces the GEMM's output-tile width to 64, 128, 192 or 256 columns for all
- * later calls in this process (the CTA-pair kernel also takes 448 for columns of 256 and
- * 192 alternating); any other value restores the automatic choice. */
-void batq_debug_force_tile_width(int32_t bn);
-
-/* Host only, no GPU needed: the work distribution of the CTA-pair GEMM for an s x m output
- * over n input channels on a device with sm_count SMs.  pair < 0: returns the number of CTA pairs
- * launched.  Otherwise returns the number of tiles pair `pair` works through, in order, and
- * writes the first max_tiles of them to tiles (host, 3 ints each: index of the 256-token row
- * block, first output feature, width in features).  -1 for arguments out of range. */
-int32_t batq_debug_pair_schedule(int64_t s, int64_t m, int64_t n, int32_t sm_count, int32_t pair,
-                                 int32_t* tiles, int32_t max_tiles);
-/* Test / tuning hook: which prefill GEMM kernel later calls use.  0 = automatic (CTA pairs sharing a
- * 256-token tile for s > 128, one CTA per 128-token tile otherwise), 1 = always one CTA per tile,
- * 2 = always CTA pairs (tile widths 192 and 256 only). */
-void batq_debug_force_gemm_kernel(int32_t which);
-/* Test / tuning hook: which activation quantiser later calls use.  0 = automatic (up to 128 tokens
- * the per-block ALU kernel, above that the tensor-core dense-block kernel; the identity
- * transform above 128 tokens and nothing else takes the streaming ALU kernel), 1 = the streaming ALU
- * kernel (Kronecker form), 2 = the tensor-core kernel, 3 = the per-block ALU kernel.
- * Factor sizes other than 4 x 8 always take the tensor-core kernel. */
-void batq_debug_force_quantizer(int32_t which);
-/* Test / tuning hook: number of K splits of the small-s GEMM (clamped to the number of
- * 256-element K steps and to 32); 0 restores the automatic choice.  Scratch sizes follow it. */
-void batq_debug_force_small_s_splits(int32_t splits);
-/* Test / tuning hook: how the small-s GEMM adds the partial tiles of its K splits.  0 = automatic
- * (through a thread-block cluster's shared memory for up to 4 tokens, up to 8 splits and a grid
- * below 90 % of the SM slots, where that measured faster; else through scratch and tickets),
- * 1 = always scratch and tickets, 2 = the cluster whenever there are at most 8 splits. */
-void batq_debug_force_small_s_reduce(int32_t which);
-/* Test / tuning hook: how batq_linear_w4a4 runs a handful of tokens.  0 = automatic (one fused
- * kernel that quantises the activations inside the GEMM where that is the faster one -- tokens x
- * K-steps per CTA <= 4 and a grid of one wave --, else the quantiser kernel followed by the small-s
- * GEMM), 1 = always the two kernels, 2 = the fused kernel up to 16 tokens.  The fused kernel needs
- * n <= 16384; other shapes take the two kernels. */
-void batq_debug_force_small_s_path(int32_t which);
 
 /* The whole layer, stages 1+2+3: quantise X into the workspace, then the GEMM.  Up to 32
  * tokens (up to 128 on layers of at least 40 M weights) take the small-s GEMM, launched so that

@@ -24,7 +24,7 @@ from __future__ import annotations
 
 import numpy as np
 
-GROUP = 32  # MX block size g (Sec. 2, "fixed block size of 32 elements")
+GROUP = 32  # MX block size g (Sec. 2: the MX formats share one scale per 32 elements)
 
 # The E2M1 magnitudes by code 0..7 (Sec. 2: 7 positive values + zero); bit 3
 # of a code is the sign.
@@ -176,7 +176,7 @@ def mxfp4_quantize(V: np.ndarray):
 
 
 # ----------------------------------------------------------------------------
-# MXFP8 quantizer (E4M3 elements, Sec. 2: "we adopt E4M3 for MXFP8"), used for
+# MXFP8 quantizer (E4M3 elements, the MXFP8 element type Sec. 2 settles on), used for
 # 8-bit activations (W4A8) and the 8-bit KV cache
 # ----------------------------------------------------------------------------
 E4M3_EMAX = 8  # 448 = 1.75 * 2**8: exponent of the largest E4M3 magnitude

@@ -1,4 +1,4 @@
-"""ctypes binding of the batq C-ABI (include/batq.h): argument marshalling only.
+"""ctypes binding of the batq C-ABI (include/batq.h, include/batq_debug.h): argument marshalling only.
 
 Every function has the name of the C entry point it calls.  Tensors are
 torch tensors used purely as device (or host) buffers; all arithmetic of the
@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "OK", 1: "ERR_NULL", 2: "ERR_SHAPE", 3: "ERR_ALIGN", 4: "ERR_
 _LIB = None
 _P, _I64, _I32, _SZ = C.c_void_p, C.c_int64, C.c_int32, C.c_size_t
 
-# name -> (restype, argtypes); must list every symbol include/batq.h declares
+# name -> (restype, argtypes); must list every symbol include/batq.h and include/batq_debug.h declare
 SIGNATURES = {
     "batq_status_string": (C.c_char_p, [C.c_int]),
     "batq_version": (C.c_int, []),
@@ -53,6 +53,8 @@ SIGNATURES = {
     "batq_static_workspace_capacity": (_SZ, []),
     "batq_linear_w4a4_noalloc": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P]),
     "batq_last_device_status": (C.c_int, [_P]),
+    "batq_debug_wait_timeout": (C.c_int, [_I64, _P]),
+    "batq_debug_mma_peak": (C.c_int, [_I32, _I32, _I32, C.POINTER(C.c_double), _P]),
 }
 
 
@@ -307,6 +309,18 @@ def batq_linear_w4a4_noalloc(t, w: Weight, x, y):
 
 def batq_last_device_status() -> int:
     return load().batq_last_device_status(_stream())
+
+
+def batq_debug_wait_timeout(limit_ns: int):
+    """Launches the one-warp kernel whose bounded wait runs out after limit_ns."""
+    _check(load().batq_debug_wait_timeout(limit_ns, _stream()), "batq_debug_wait_timeout")
+
+
+def batq_debug_mma_peak(pair: bool, bn: int, iters: int) -> float:
+    """Launches the MMA-only loop on the current stream; returns the flops of the launch."""
+    flops = C.c_double(0.0)
+    _check(load().batq_debug_mma_peak(1 if pair else 0, bn, iters, C.byref(flops), _stream()), "batq_debug_mma_peak")
+    return flops.value
 
 
 def bits_to_cuda_bf16(bits: np.ndarray) -> torch.Tensor:

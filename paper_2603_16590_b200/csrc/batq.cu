@@ -1,11 +1,12 @@
 // C-ABI of the batq library: host-side validation, handles and kernel launches.
 // The whole library is this one translation unit.
-#include "batq.h"
+#include "batq_debug.h"
 
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <climits>
 #include <cmath>
 #include <cstring>
@@ -17,6 +18,7 @@
 #include "gemm_mxfp4_pair.cuh"
 #include "gemm_small_s.cuh"
 #include "linear_small_s_fused.cuh"
+#include "mma_peak.cuh"
 #include "prepare_weight.cuh"
 #include "quantize_act.cuh"
 #include "quantize_act_tc.cuh"
@@ -118,6 +120,8 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(gemm_mxfp4_kernel<128, true>, GemmCfg<128>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<64, false>, GemmCfg<64>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<64, true>, GemmCfg<64>::kSmemBytes);
+    e = e ? e : set_smem(mma_peak_kernel<false>, kPeakSmemBytes);
+    e = e ? e : set_smem(mma_peak_kernel<true>, kPeakSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_pair_kernel<false>, PairCfg::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_pair_kernel<true>, PairCfg::kSmemBytes);
     e = e ? e : set_smem(linear_small_s_fused_kernel<false>, FusedCfg::kSmemBytes);
@@ -259,7 +263,7 @@ batq_status check_x(const void* x, int64_t s, int64_t n, int64_t ld) {
 
 constexpr int64_t kSmallSMax = 128;       // the swapped-operand split-K GEMM takes up to this many tokens
 constexpr int64_t kSmallQuantAuto = 128;  // per-block ALU quantiser up to here, tensor cores above (12 us flat against 2-4 us)
-int g_force_quantizer = 0;  // tuning hook: 0 = automatic, 1 = ALU (Kronecker form), 2 = tensor cores (dense form)
+std::atomic<int> g_force_quantizer{0};  // tuning hook: 0 = automatic, 1 = ALU (Kronecker form), 2 = tensor cores (dense form)
 
 // Tensor-core version: 128-token x 4-block units.
 batq_status launch_quantize_tc(const batq_transform* t, const void* x, int64_t s, int64_t n, int64_t ld, void* codes,
@@ -332,8 +336,9 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
   // tensor-core kernel, which only sees the dense block matrices.
   const bool only_tc = t != nullptr && (t->gr != 4 || t->gc != 8);
   const bool small_path = n_zero_words > 0;  // in front of the small-s GEMM (its tickets to clear)
+  const int force_q = g_force_quantizer.load(std::memory_order_relaxed);
   const bool use_tc = only_tc || (!small_path && t != nullptr &&
-                                  (g_force_quantizer == 2 || (g_force_quantizer == 0 && s > kSmallQuantAuto)));
+                                  (force_q == 2 || (force_q == 0 && s > kSmallQuantAuto)));
   if (use_tc) {
     if (n_zero_words > 0 &&
         cudaMemsetAsync(zero_words, 0, static_cast<size_t>(n_zero_words) * 4, stream) != cudaSuccess) {
@@ -344,7 +349,7 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
   }
   // A handful of tokens: the ring of the streaming kernel below is all latency there; one thread
   // per (token, block) with everything loaded up front is quicker.
-  if (g_force_quantizer == 3 || (g_force_quantizer == 0 && (s <= kSmallQuantAuto || (small_path && s <= kSmallSMax)))) {
+  if (force_q == 3 || (force_q == 0 && (s <= kSmallQuantAuto || (small_path && s <= kSmallSMax)))) {
     QuantSmallParams q{};
     q.x = static_cast<const uint16_t*>(x);
     q.ld = ld;
@@ -435,9 +440,10 @@ batq_status make_y_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_
 // overlaps the main loop of the next); 256 has the highest flop per byte staged but a single
 // accumulator.  Pick by modelled time: waves x (main loop + exposed epilogue), with the main
 // loop proportional to the tile width.
-int g_force_bn = 0;  // test hook: 0 = automatic
+std::atomic<int> g_force_bn{0};  // test hook: 0 = automatic
 int pick_bn(int64_t s, int64_t m, int64_t n, int sm_count) {
-  if (g_force_bn == 64 || g_force_bn == 128 || g_force_bn == 192 || g_force_bn == 256) return g_force_bn;
+  const int force_bn = g_force_bn.load(std::memory_order_relaxed);
+  if (force_bn == 64 || force_bn == 128 || force_bn == 192 || force_bn == 256) return force_bn;
   const int64_t mt = (s + kBM - 1) / kBM;
   // A few dozen tiles cannot pull the weights fast enough (a CTA streams what its ring keeps in
   // flight): below half a wave of 128-wide tiles, twice as many 64-wide ones.
@@ -454,7 +460,7 @@ int pick_bn(int64_t s, int64_t m, int64_t n, int sm_count) {
   return c256 <= c128 ? 256 : 128;
 }
 
-int g_force_gemm_kernel = 0;  // tuning hook: 0 = automatic, 1 = one CTA per tile, 2 = CTA pairs
+std::atomic<int> g_force_gemm_kernel{0};  // tuning hook: 0 = automatic, 1 = one CTA per tile, 2 = CTA pairs
 
 // The schedule of the CTA-pair kernel for an s x m output with k_steps K-steps: column widths and
 // number of pairs.  Every candidate (columns of 128, 192 or 256 features, or 256 and 192
@@ -476,11 +482,12 @@ bool pair_schedule(int64_t s, int64_t m, int64_t k_steps, int sm_count, PairPara
   };
   int best_w = -1;
   double best_cost = 1e30;
+  const int force_bn = g_force_bn.load(std::memory_order_relaxed);
   const int cand[5] = {0, 256, 192, 128, 64};
   for (int ci = 0; ci < 5; ++ci) {
     const int w = cand[ci];
-    const bool forced = g_force_bn == 64 || g_force_bn == 128 || g_force_bn == 192 || g_force_bn == 256 || g_force_bn == 448;
-    if (forced ? (g_force_bn == 448 ? w != 0 : w != g_force_bn) : w == 64) continue;  // 64: only when forced
+    const bool forced = force_bn == 64 || force_bn == 128 || force_bn == 192 || force_bn == 256 || force_bn == 448;
+    if (forced ? (force_bn == 448 ? w != 0 : w != force_bn) : w == 64) continue;  // 64: only when forced
     const int64_t n_cols = n_cols_of(w);
     if (m_pairs * n_cols > INT32_MAX) return false;
     p->tile_w = w;
@@ -571,7 +578,8 @@ batq_status launch_gemm(const void* x_codes, const void* x_sf, const batq_weight
   if (st == BATQ_OK && m16 > 0) st = make_y_tmap(&tmap_y, y, s, m16, ldy, bf);
   if (st != BATQ_OK) return st;
   // CTA pairs need at least two 128-token tiles to pay, and wide enough a layer for their tiles.
-  const bool use_pair = g_force_gemm_kernel == 2 || (g_force_gemm_kernel == 0 && s > 128 && w->m >= 192);
+  const int force_gemm = g_force_gemm_kernel.load(std::memory_order_relaxed);
+  const bool use_pair = force_gemm == 2 || (force_gemm == 0 && s > 128 && w->m >= 192);
   if (use_pair) return launch_gemm_pair(x_codes, x_sf, w, s, y, bf, ldy, stream, info->sm_count, tmap_a, tmap_y, m16, dependent);
   const int bn = pick_bn(s, w->m, w->n, info->sm_count);
   GemmParams p{};
@@ -610,8 +618,8 @@ batq_status launch_gemm(const void* x_codes, const void* x_sf, const batq_weight
 }
 
 // ---- small-s (decode) GEMM: split choice, scratch layout, launch -------------------------------
-int g_force_splits = 0;  // tuning hook: 0 = automatic
-int g_small_reduce = 0;  // tuning hook: 0 = automatic, 1 = always tickets, 2 = cluster whenever splits <= 8
+std::atomic<int> g_force_splits{0};  // tuning hook: 0 = automatic
+std::atomic<int> g_small_reduce{0};  // tuning hook: 0 = automatic, 1 = always tickets, 2 = cluster whenever splits <= 8
 constexpr int kMaxSplits = 32;
 
 inline int small_ntok(int64_t s) { return s <= 16 ? 16 : (s <= 32 ? 32 : (s <= 64 ? 64 : 128)); }
@@ -624,8 +632,9 @@ inline int small_ntok(int64_t s) { return s <= 16 ? 16 : (s <= 32 ? 32 : (s <= 6
 // too.  Measured: a fuller grid leaves a few clusters for a second wave, which costs a layer of
 // the decode benchmark about 5 us.
 bool cluster_reduce_ok(int64_t tiles, int sp, int64_t slots, int64_t s) {
-  if (sp < 2 || sp > 8 || g_small_reduce == 1) return false;
-  return g_small_reduce == 2 || tiles * sp * 10 <= slots * (s > 4 ? 8 : 9);
+  const int force_reduce = g_small_reduce.load(std::memory_order_relaxed);
+  if (sp < 2 || sp > 8 || force_reduce == 1) return false;
+  return force_reduce == 2 || tiles * sp * 10 <= slots * (s > 4 ? 8 : 9);
 }
 
 // Number of K splits: the grid is (row tiles) x (splits) CTAs, two resident per SM.  Modelled
@@ -634,7 +643,8 @@ bool cluster_reduce_ok(int64_t tiles, int sp, int64_t slots, int64_t s) {
 // (all in units of one K-step of streaming, about 0.5 us).
 int pick_splits(int64_t m, int64_t n, int64_t s, int sm_count) {
   const int k_steps = static_cast<int>((n + 255) / 256);
-  if (g_force_splits > 0) return std::min(std::min(g_force_splits, k_steps), kMaxSplits);
+  const int force_splits = g_force_splits.load(std::memory_order_relaxed);
+  if (force_splits > 0) return std::min(std::min(force_splits, k_steps), kMaxSplits);
   const int64_t tiles = (m + 127) / 128;
   const int64_t slots = 2 * static_cast<int64_t>(sm_count > 0 ? sm_count : 148);
   int best = 1;
@@ -736,7 +746,7 @@ batq_status launch_gemm_small(const void* x_codes, const void* x_sf, const batq_
 }
 
 // ---- fused small-s layer (quantiser inside the GEMM kernel) ------------------------------------
-int g_force_small_path = 0;  // tuning hook: 0 = automatic, 1 = two kernels, 2 = fused whenever it applies
+std::atomic<int> g_force_small_path{0};  // tuning hook: 0 = automatic, 1 = two kernels, 2 = fused whenever it applies
 // K splits of the fused kernel: a power of two (the cluster size), at most 8, with at most
 // kFusedMaxSteps K-steps per CTA; 0 if the shape does not fit.
 int pick_fused_splits(int64_t m, int64_t n, int sm_count) {
@@ -745,11 +755,12 @@ int pick_fused_splits(int64_t m, int64_t n, int sm_count) {
   const int64_t slots = 2 * static_cast<int64_t>(sm_count > 0 ? sm_count : 148);
   int best = 0;
   double best_cost = 1e30;
+  const int force_splits = g_force_splits.load(std::memory_order_relaxed);
   for (int sp = 1; sp <= kFusedMaxSplits; sp *= 2) {
     if (sp > k_steps) break;
     const int per = (k_steps + sp - 1) / sp;
     if (per > kFusedMaxSteps) continue;
-    if (g_force_splits > 0 && sp != g_force_splits) continue;
+    if (force_splits > 0 && sp != force_splits) continue;
     const int64_t waves = (tiles * sp + slots - 1) / slots;
     const double cost = static_cast<double>(waves) * (per + 3.0) + 0.15 * sp;
     if (cost < best_cost - 1e-9) { best_cost = cost; best = sp; }
@@ -761,11 +772,12 @@ int pick_fused_splits(int64_t m, int64_t n, int sm_count) {
 // hidden behind the weight stream while that is a few items per thread (tokens x K-steps <= 4) and
 // the grid fits the SMs in one wave; measured, the fused kernel then saves about 5 % of a call.
 bool use_fused_small(const batq_transform* t, const batq_weight* w, int64_t s) {
-  if (g_force_small_path == 1 || s > kFusedTok) return false;
+  const int force_path = g_force_small_path.load(std::memory_order_relaxed);
+  if (force_path == 1 || s > kFusedTok) return false;
   if (t != nullptr && (t->gr != 4 || t->gc != 8)) return false;  // its in-kernel quantiser is the 4 x 8 form
   const int sp = pick_fused_splits(w->m, w->n, w->sm_count);
   if (sp == 0) return false;
-  if (g_force_small_path == 2) return true;
+  if (force_path == 2) return true;
   const int64_t k_steps = (w->n + 255) / 256;
   const int64_t per = (k_steps + sp - 1) / sp;
   const int64_t slots = 2 * static_cast<int64_t>(w->sm_count > 0 ? w->sm_count : 148);
@@ -1178,7 +1190,7 @@ batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w,
   return BATQ_OK;
 }
 
-void batq_debug_force_tile_width(int32_t bn) { g_force_bn = bn; }
+void batq_debug_force_tile_width(int32_t bn) { g_force_bn.store(bn, std::memory_order_relaxed); }
 
 int32_t batq_debug_pair_schedule(int64_t s, int64_t m, int64_t n, int32_t sm_count, int32_t pair, int32_t* tiles,
                                  int32_t max_tiles) {
@@ -1201,11 +1213,46 @@ int32_t batq_debug_pair_schedule(int64_t s, int64_t m, int64_t n, int32_t sm_cou
   }
   return cnt;
 }
-void batq_debug_force_quantizer(int32_t which) { g_force_quantizer = which; }
-void batq_debug_force_gemm_kernel(int32_t which) { g_force_gemm_kernel = which; }
-void batq_debug_force_small_s_splits(int32_t splits) { g_force_splits = splits; }
-void batq_debug_force_small_s_path(int32_t which) { g_force_small_path = which; }
-void batq_debug_force_small_s_reduce(int32_t which) { g_small_reduce = which; }
+void batq_debug_force_quantizer(int32_t which) { g_force_quantizer.store(which, std::memory_order_relaxed); }
+void batq_debug_force_gemm_kernel(int32_t which) { g_force_gemm_kernel.store(which, std::memory_order_relaxed); }
+void batq_debug_force_small_s_splits(int32_t splits) { g_force_splits.store(splits, std::memory_order_relaxed); }
+void batq_debug_force_small_s_path(int32_t which) { g_force_small_path.store(which, std::memory_order_relaxed); }
+void batq_debug_force_small_s_reduce(int32_t which) { g_small_reduce.store(which, std::memory_order_relaxed); }
+
+batq_status batq_debug_wait_timeout(int64_t limit_ns, void* stream) {
+  batq_status st = device_setup(nullptr, nullptr);
+  if (st != BATQ_OK) return st;
+  const uint64_t lim = static_cast<uint64_t>(std::min<int64_t>(std::max<int64_t>(limit_ns, 1000), 10000000));
+  wait_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(lim);
+  return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
+}
+
+batq_status batq_debug_mma_peak(int32_t pair, int32_t bn, int32_t iters, double* flops_out, void* stream) {
+  if (bn != 64 && bn != 128 && bn != 192 && bn != 256) return BATQ_ERR_SHAPE;
+  if (iters <= 0 || iters > (1 << 24)) return BATQ_ERR_SHAPE;
+  const DeviceInfo* info;
+  batq_status st = device_setup(nullptr, &info);
+  if (st != BATQ_OK) return st;
+  PeakParams p{iters, bn};
+  const int ctas = pair ? (info->sm_count / 2) * 2 : info->sm_count;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(ctas));
+  cfg.blockDim = dim3(kPeakThreads);
+  cfg.dynamicSmemBytes = kPeakSmemBytes;
+  cfg.stream = static_cast<cudaStream_t>(stream);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pair ? 1 : 0;
+  const cudaError_t e = pair ? cudaLaunchKernelEx(&cfg, mma_peak_kernel<true>, p) : cudaLaunchKernelEx(&cfg, mma_peak_kernel<false>, p);
+  if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+  if (flops_out != nullptr)
+    *flops_out = 2.0 * (pair ? 256.0 : 128.0) * bn * 256.0 * iters * (pair ? ctas / 2 : ctas);
+  return BATQ_OK;
+}
 
 size_t batq_static_workspace_capacity(void) { return BATQ_STATIC_WORKSPACE_BYTES - 1024; }
 

@@ -1,0 +1,150 @@
+// Measurement kernels: (1) the block-scaled FP4 tensor-core rate with operands resident in shared
+// memory (the denominator of the GEMM's roofline fraction), (2) a wait that runs out on purpose,
+// to show that the library's bounded waits report and return.
+#pragma once
+#include <cuda.h>
+
+#include "gemm_mxfp4.cuh"
+#include "ptx.cuh"
+
+namespace batq {
+
+constexpr int kPeakThreads = 128;
+constexpr int kPeakBatch = 8;            // K-steps between two commits
+constexpr int kPeakSfbAtoms = 2;         // 256 weight rows
+constexpr int kPeakABytes = 128 * kBKBytes;
+constexpr int kPeakBBytes = 256 * kBKBytes;
+constexpr int kPeakSfBytes = 1024 + kPeakSfbAtoms * 1024;
+constexpr int kPeakSmemBytes = kPeakABytes + kPeakBBytes + kPeakSfBytes + 1024;
+constexpr int kPeakSfCols = 8 + 2 * 4 * kPeakSfbAtoms;
+
+struct PeakParams {
+  int32_t iters;   // K-steps (four MMAs of K = 64 each)
+  int32_t bn;      // tile width
+};
+
+// PAIR = false: every CTA issues tcgen05.mma.cta_group::1 on a 128 x bn tile.
+// PAIR = true:  clusters of two; the leader issues cta_group::2 on a 256 x bn tile whose A rows and
+//               B rows are split over the two CTAs' shared memories, as in the CTA-pair GEMM.
+template <bool PAIR>
+__global__ void __launch_bounds__(kPeakThreads, 1) mma_peak_kernel(const PeakParams p) {
+  extern __shared__ uint8_t peak_smem_raw[];
+  __shared__ __align__(8) uint64_t batch_bar[2];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+  const int tid = threadIdx.x;
+  const int warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0);
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(peak_smem_raw) + 1023) & ~uintptr_t(1023));
+
+  // Operands: every byte pattern is a pair of valid E2M1 codes; scale bytes 125..129 (2^-2..2^2).
+  uint32_t h = 0x9E3779B9u * (blockIdx.x * kPeakThreads + tid + 1u);
+  for (int i = tid; i < (kPeakABytes + kPeakBBytes) / 4; i += kPeakThreads) {
+    h = h * 1664525u + 1013904223u;
+    reinterpret_cast<uint32_t*>(smem)[i] = h ^ (h >> 15);
+  }
+  for (int i = tid; i < kPeakSfBytes; i += kPeakThreads) {
+    h = h * 1664525u + 1013904223u;
+    smem[kPeakABytes + kPeakBBytes + i] = static_cast<uint8_t>(125u + (h >> 24) % 5u);
+  }
+  if (tid == 0) {
+    mbar_init(smem_u32(&batch_bar[0]), 1);
+    mbar_init(smem_u32(&batch_bar[1]), 1);
+    abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    if (PAIR) { tmem_alloc_pair(smem_u32(&tmem_base_slot), 512); tmem_relinquish_pair(); }
+    else      { tmem_alloc(smem_u32(&tmem_base_slot), 512); tmem_relinquish(); }
+  }
+  fence_proxy_async_smem();   // the generic-proxy writes above are read by the tensor cores
+  tc_fence_before_sync();
+  __syncthreads();
+  if (PAIR) cluster_sync_all();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 1 && rank == 0) {
+    const uint32_t smem_base = smem_u32(smem);
+    const uint64_t adesc = make_smem_desc(smem_base, 16, 1024, 2);
+    const uint64_t bdesc = adesc + (kPeakABytes >> 4);
+    const uint64_t sfd = make_smem_desc(smem_base + kPeakABytes + kPeakBBytes, 0, 128, 0);
+    const uint32_t sfa_col = tmem_base + 256;
+    const uint32_t sfb_col = sfa_col + 8;
+    const uint32_t idesc0 = mxf4_idesc(PAIR ? 256 : 128, p.bn);
+    const uint32_t idesc1 = idesc0 | (2u << 29) | (2u << 4);
+    bool ok = true;
+    if (elect_one()) {
+      // scale factors once: shared -> tensor memory, the layout of the GEMM kernels
+      if (PAIR) {
+        tc_cp_32x128b_warpx4_pair(sfa_col, sfd);
+        tc_cp_32x128b_warpx4_pair(sfa_col + 4, sfd + 32);
+      } else {
+        tc_cp_32x128b_warpx4(sfa_col, sfd);
+        tc_cp_32x128b_warpx4(sfa_col + 4, sfd + 32);
+      }
+#pragma unroll
+      for (int rt = 0; rt < kPeakSfbAtoms; ++rt)
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          const uint32_t col = sfa_col + 8 + c * 4 * kPeakSfbAtoms + 4 * rt;
+          const uint64_t src = sfd + ((1024 + rt * 1024 + c * 512) >> 4);
+          if (PAIR) tc_cp_32x128b_warpx4_pair(col, src); else tc_cp_32x128b_warpx4(col, src);
+        }
+    }
+    __syncwarp();
+    const int n_batches = (p.iters + kPeakBatch - 1) / kPeakBatch;
+    for (int b = 0; b < n_batches && ok; ++b) {
+      // at most two batches in flight, like a ring of stages
+      if (b >= 2) {
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&batch_bar[b & 1]), ((b >> 1) - 1) & 1u, &abort_flag));
+        if (!ok) break;
+      }
+      if (elect_one()) {
+        const int k1 = min(p.iters, (b + 1) * kPeakBatch);
+        for (int kt = b * kPeakBatch; kt < k1; ++kt) {
+#pragma unroll
+          for (int kb = 0; kb < 4; ++kb) {
+            const uint32_t c = kb >> 1;
+            const uint32_t sfid = (kb & 1) * 2;
+            const uint32_t sa = (sfa_col + 4 * c) | (sfid << 30);
+            const uint32_t sb = (sfb_col + c * 4 * kPeakSfbAtoms) | (sfid << 30);
+            const uint32_t acc = (kt | kb) != 0 ? 1u : 0u;
+            if (PAIR) tc_mma_mxf4_pair(tmem_base, adesc + 2 * kb, bdesc + 2 * kb, (kb & 1) ? idesc1 : idesc0, sa, sb, acc);
+            else      tc_mma_mxf4(tmem_base, adesc + 2 * kb, bdesc + 2 * kb, (kb & 1) ? idesc1 : idesc0, sa, sb, acc);
+          }
+        }
+        if (PAIR) tc_commit_pair_local(smem_u32(&batch_bar[b & 1])); else tc_commit(smem_u32(&batch_bar[b & 1]));
+      }
+      __syncwarp();
+    }
+    // drain: the last two batches (fewer if there were fewer)
+    for (int b = max(0, n_batches - 2); b < n_batches; ++b)
+      if (!mbar_wait(smem_u32(&batch_bar[b & 1]), (b >> 1) & 1u, &abort_flag)) break;
+    __syncwarp();
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (PAIR) cluster_sync_all();   // the peer's shared memory is read until the leader has drained
+  if (warp == 1) {
+    tc_fence_after_sync();
+    if (PAIR) tmem_dealloc_pair(tmem_base, 512); else tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// One warp waits on a barrier nothing signals; the bounded wait gives up after limit_ns, records
+// the time-out for the host and the kernel returns normally.
+__global__ void wait_timeout_kernel(uint64_t limit_ns) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+  mbar_wait(smem_u32(&bar), 0, &abort_flag, limit_ns);
+}
+
+}  // namespace batq

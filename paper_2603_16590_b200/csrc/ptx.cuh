@@ -77,12 +77,13 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t pari
 
 // Bounded wait.  Returns false when the wait was given up: either another
 // thread of the CTA already raised *abort_flag (shared memory), or this wait
-// exceeded kWaitLimitNs, in which case it raises the flag and records the
+// exceeded limit_ns (kWaitLimitNs in every product kernel), in which case it raises the flag and records the
 // error for the host.  Callers leave their loops and fall through to the
 // kernel's common exit, so tensor memory is always released.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s: ~1000x the longest kernel here
 constexpr uint32_t kParkNs = 20000u;              // longest single park; the limits are checked between parks
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   uint64_t t0 = 0;
   for (;;) {
@@ -90,7 +91,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (*abort_flag) return false;
     const uint64_t now = global_timer_ns();
     if (t0 == 0) t0 = now;
-    if (now - t0 > kWaitLimitNs) {
+    if (now - t0 > limit_ns) {
       *abort_flag = 1;
       atomicExch(&g_device_error, 1);
       return false;

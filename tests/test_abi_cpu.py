@@ -20,9 +20,13 @@ def lib():
 
 
 def _declared_symbols():
-    src = open(os.path.join(ROOT, "include", "batq.h")).read()
-    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
-    return sorted(set(re.findall(r"\b(batq_[a-z0-9_]+)\s*\(", src)))
+    names = set()
+    for header in sorted(os.listdir(os.path.join(ROOT, "include"))):
+        assert header.endswith(".h")
+        src = open(os.path.join(ROOT, "include", header)).read()
+        src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+        names |= set(re.findall(r"\b(batq_[a-z0-9_]+)\s*\(", src))
+    return sorted(names)
 
 
 def test_every_declared_symbol_is_exported_and_bound(lib):
@@ -79,3 +83,11 @@ def test_host_validation_without_a_device(lib):
     assert lib.batq_linear_workspace_bytes(None, 4) == 0
     assert lib.batq_linear_kernel_launches(None, None, 4) == 0
     assert lib.batq_weight_destroy(None) == 0 and lib.batq_transform_destroy(None) == 0
+    assert lib.batq_debug_mma_peak(0, 100, 10, None, None) == 2
+    assert lib.batq_debug_mma_peak(0, 256, 0, None, None) == 2
+
+
+def test_debug_hooks_are_not_in_the_public_header():
+    src = open(os.path.join(ROOT, "include", "batq.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    assert "batq_debug_" not in src

@@ -293,6 +293,11 @@ def test_gemm_exact_integer_variant_and_unit_scales():
     Yi = O.gemm_mxfp4_exact_int(cx, sx, cw, sw)
     assert np.array_equal(Y, Yi)   # small exponents: fp64 sum is exact too
     assert np.all(np.abs(Y) <= Sabs)
+    # Sabs pinned from both sides: with every sign bit cleared no product is negative, so the exact
+    # contraction of the magnitudes *is* sum |a*b| (Python integers and fractions, no floating point)
+    Sabs_exact = O.gemm_mxfp4_exact_int(cx & 7, sx, cw & 7, sw)
+    assert np.array_equal(Sabs, Sabs_exact)
+    assert np.all(Sabs_exact >= np.abs(Yi)) and np.any(Sabs_exact > np.abs(Yi))
     # all scales 2^0: plain integer dot product of doubled values / 4
     one = np.full((S, N // 32), 127, np.uint8)
     Y1, _ = O.gemm_mxfp4(cx, one, cw, np.full((M, N // 32), 127, np.uint8))

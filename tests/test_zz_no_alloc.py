@@ -28,17 +28,17 @@ def test_noalloc_entry_point_matches_regular_one_twice_in_a_row(batq):
     # two calls in a row on different shapes: the second sees the first one's stale scratch
     cases = [(300, 520, 2048, 1, torch.float32), (77, 264, 544, 2, torch.bfloat16)]
     layers = [_layer(batq, *c) for c in cases]
+    outs = [torch.full_like(want, float("nan")) for (_, _, _, want) in layers]
+    # one call first: it resolves the array's address on this device (documented set-up step)
+    batq.batq_linear_w4a4_noalloc(*layers[0][:3], torch.empty_like(layers[0][3]))
     torch.cuda.synchronize()
-    before = torch.cuda.memory_allocated()
-    outs = []
-    for (tr, w, x, want) in layers:
-        got = torch.full_like(want, float("nan"))
-        outs.append(got)
-    mid = torch.cuda.memory_allocated()
+    # what the driver itself hands out (torch's own counter would not see a cudaMalloc inside the library)
+    free_before = torch.cuda.mem_get_info()[0]
+    torch_before = torch.cuda.memory_allocated()
     for (tr, w, x, want), got in zip(layers, outs):
         batq.batq_linear_w4a4_noalloc(tr, w, x, got)
     assert batq.batq_last_device_status() == 0
-    assert torch.cuda.memory_allocated() == mid and mid >= before
+    assert torch.cuda.mem_get_info()[0] == free_before and torch.cuda.memory_allocated() == torch_before
     for (tr, w, x, want), got in zip(layers, outs):
         # same kernels, same inputs: bit-identical, which is inside every tolerance used elsewhere
         assert torch.equal(got, want)
@@ -48,6 +48,35 @@ def test_noalloc_entry_point_matches_regular_one_twice_in_a_row(batq):
     batq.batq_linear_w4a4_noalloc(tr, w, x, again)
     torch.cuda.synchronize()
     assert torch.equal(again, want)
+
+
+def test_noalloc_small_token_paths_after_a_large_call(batq):
+    """The decode-sized paths keep more than codes in the scratch: split-K partial tiles and one
+    ticket word per row tile (which must read zero when the GEMM starts).  Run them through the
+    built-in array right after a large call has filled it with other bytes: 16 tokens with 12 K
+    splits (partials and tickets in the array), 4 tokens (cluster reduction) and 1 token (the fused
+    single-kernel path), each twice."""
+    big = _layer(batq, 1500, 264, 4096, 5, torch.bfloat16)
+    small = []
+    batq.batq_debug_force_small_s_splits(12)
+    try:
+        small.append(_layer(batq, 16, 520, 3584, 6, torch.float32))
+        got = [torch.full_like(small[0][3], float("nan")) for _ in range(2)]
+        batq.batq_linear_w4a4_noalloc(*big[:3], torch.empty_like(big[3]))
+        for g in got:
+            batq.batq_linear_w4a4_noalloc(*small[0][:3], g)
+        assert batq.batq_last_device_status() == 0
+        assert torch.equal(got[0], small[0][3]) and torch.equal(got[1], small[0][3])
+    finally:
+        batq.batq_debug_force_small_s_splits(0)
+    for S, M, N, seed in [(4, 1032, 2048, 7), (1, 4096, 4096, 8)]:
+        tr, w, x, want = _layer(batq, S, M, N, seed, torch.float32)
+        batq.batq_linear_w4a4_noalloc(*big[:3], torch.empty_like(big[3]))
+        got = [torch.full_like(want, float("nan")) for _ in range(2)]
+        for g in got:
+            batq.batq_linear_w4a4_noalloc(tr, w, x, g)
+        assert batq.batq_last_device_status() == 0
+        assert torch.equal(got[0], want) and torch.equal(got[1], want)
 
 
 def test_noalloc_rejects_sizes_beyond_the_array(batq):
