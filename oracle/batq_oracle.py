@@ -232,6 +232,46 @@ def dequantize_mxfp8(codes: np.ndarray, scale_bytes: np.ndarray) -> np.ndarray:
     return (e4m3_decode(codes).reshape(S, k, GROUP) * scale[:, :, None]).reshape(S, N)
 
 
+def gemm_mxfp8_mxfp4(codes_x8, scales_x, codes_w, scales_w):
+    """Stage 3 of the W4A8 configuration (MXFP8-E4M3 activations x MXFP4 weights, the W4A8
+    settings of Sec. 4): Y[s,m] = sum_e deq8_x[s,e] * deq4_w[m,e] in fp64 and
+    Sabs[s,m] = sum_e |deq8_x * deq4_w|.  Returns (Y, Sabs)."""
+    dx = dequantize_mxfp8(codes_x8, scales_x)
+    dw = dequantize(codes_w, scales_w)
+    return dx @ dw.T, np.abs(dx) @ np.abs(dw).T
+
+
+def gemm_mxfp8_mxfp4_exact(codes_x8, scales_x, codes_w, scales_w):
+    """The same contraction in exact rational arithmetic, for tiny shapes: every finite E4M3 value
+    is an integer multiple of 2**-9 and every E2M1 value of 2**-1, so a block contributes
+    2**(ex + ew - 10) times an integer dot product.  Returns fp64 after the exact evaluation."""
+    from fractions import Fraction
+    S, N = codes_x8.shape
+    M = codes_w.shape[0]
+    k = N // GROUP
+    ix = np.rint(512 * e4m3_decode(codes_x8)).astype(np.int64)
+    iw = np.rint(2 * e2m1_decode(codes_w)).astype(np.int64)
+    Y = np.zeros((S, M), dtype=np.float64)
+    for s in range(S):
+        for m in range(M):
+            acc = Fraction(0)
+            for j in range(k):
+                blk = int(np.dot(ix[s, j * GROUP:(j + 1) * GROUP], iw[m, j * GROUP:(j + 1) * GROUP]))
+                ex = int(scales_x[s, j]) - 127 + int(scales_w[m, j]) - 127
+                acc += Fraction(blk, 1024) * (Fraction(2) ** ex)
+            Y[s, m] = float(acc)
+    return Y
+
+
+def linear_w4a8(x_bits, w_bits, L, R, c_lo=None, c_hi=None):
+    """The W4A8 layer: Q8(XP) Q4(P^{-1} W^T), activations in MXFP8 (E4M3), weights in MXFP4.
+    Returns (Y, Sabs, (codes_x8, scales_x), (codes_w, scales_w))."""
+    qx = quantize_act_mxfp8(x_bits, L, R, c_lo, c_hi)
+    qw = prepare_weight(w_bits, L, R)
+    Y, Sabs = gemm_mxfp8_mxfp4(qx[0], qx[1], qw[0], qw[1])
+    return Y, Sabs, qx, qw
+
+
 def pack_codes(codes: np.ndarray) -> np.ndarray:
     """Two codes per byte: element 2i in bits 0-3, element 2i+1 in bits 4-7."""
     c = np.asarray(codes, dtype=np.uint8)

@@ -374,3 +374,40 @@ def test_mxfp8_scale_rule_and_error_bound():
     z = np.zeros((1, 32)); z[0, 3] = -0.0
     c, s_ = O.mxfp8_quantize(z)
     assert s_[0, 0] == 0 and c[0, 3] == 0x80 and c[0, 0] == 0
+
+
+def test_w4a8_gemm_exact_rational_variant_and_sabs():
+    """MXFP8 x MXFP4 contraction: fp64 equals the exact rational evaluation on tiny shapes, Sabs
+    equals the exact contraction of the magnitudes, and with unit scales the result is the integer
+    dot product of (512 * e4m3) and (2 * e2m1) over 1024."""
+    rng = np.random.default_rng(18)
+    S, M, N = 3, 4, 96
+    cx = rng.integers(0, 256, (S, N)).astype(np.uint8)
+    cx[(cx & 0x7F) == 0x7F] = 0x7E                      # no NaN codes
+    cw = rng.integers(0, 16, (M, N)).astype(np.uint8)
+    sx = rng.integers(120, 135, (S, N // 32)).astype(np.uint8)
+    sw = rng.integers(120, 135, (M, N // 32)).astype(np.uint8)
+    Y, Sabs = O.gemm_mxfp8_mxfp4(cx, sx, cw, sw)
+    assert np.array_equal(Y, O.gemm_mxfp8_mxfp4_exact(cx, sx, cw, sw))
+    assert np.array_equal(Sabs, O.gemm_mxfp8_mxfp4_exact(cx & 0x7F, sx, cw & 7, sw))
+    assert np.all(np.abs(Y) <= Sabs)
+    one_x, one_w = np.full((S, N // 32), 127, np.uint8), np.full((M, N // 32), 127, np.uint8)
+    Y1, _ = O.gemm_mxfp8_mxfp4(cx, one_x, cw, one_w)
+    ix = np.rint(512 * O.e4m3_decode(cx)).astype(np.int64)
+    iw = np.rint(2 * O.e2m1_decode(cw)).astype(np.int64)
+    assert np.array_equal(Y1, (ix @ iw.T) / 1024.0)
+
+
+def test_w4a8_layer_is_closer_to_fp_than_w4a4():
+    """The 8-bit activation format loses less than the 4-bit one (the paper's W4A8 rows sit above
+    its W4A4 rows): on the same layer the W4A8 oracle output is nearer the full-precision product."""
+    S, M, N = 32, 48, 256
+    xb = synth.make_activations(S, N, 33)
+    wb = synth.make_weight(M, N, 33)
+    t = synth.make_transform(N, 33, "baseline")
+    ref = O.bf16_bits_to_f64(xb) @ O.bf16_bits_to_f64(wb).T
+    y8 = O.linear_w4a8(xb, wb, t.left, t.right, t.clip_lo, t.clip_hi)[0]
+    y4 = O.linear_w4a4(xb, wb, t.left, t.right, t.clip_lo, t.clip_hi)[0]
+    assert np.linalg.norm(y8 - ref) < np.linalg.norm(y4 - ref)
+    # unquantised activations would leave only the weight error: W4A8 must sit between the two
+    assert np.linalg.norm(y8 - ref) / np.linalg.norm(ref) < 0.35
