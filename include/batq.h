@@ -148,6 +148,29 @@ batq_status batq_weight_export(const batq_weight* w, void* codes_rowmajor, void*
 batq_status batq_gemm_mxfp4(const void* x_codes, const void* x_scales_mma, const batq_weight* w,
                             int64_t s, void* y, int32_t y_dtype, int64_t ldy, void* stream);
 
+/* Stage 3 of the W4A8 configurations (Sec. 4: MXFP8 activations, MXFP4 weights; E4M3 is the MXFP8
+ * element type of Sec. 2):  Y[s, m] = sum_j 2^(ex[s,j] + ew[m,j]) * sum_{i<32} q8x[s,j,i] * qw[m,j,i]
+ * on the block-scaled tensor cores, fp32 accumulation.
+ *   x_codes8      dev [s x n] bytes, one E4M3 code per element, 16-byte aligned, as written by
+ *                 batq_quantize_act_mxfp8.
+ *   x_scales_mma  dev, BATQ_SF_MMA layout for [s x n].
+ *   w             a prepared weight with n % 128 == 0 (else UNSUPPORTED): the same 4-bit codes
+ *                 and scales as for batq_gemm_mxfp4, nothing is stored twice.
+ *   y             as batq_gemm_mxfp4.
+ * s == 0 is a no-op. */
+batq_status batq_gemm_mxfp8_mxfp4(const void* x_codes8, const void* x_scales_mma, const batq_weight* w,
+                                  int64_t s, void* y, int32_t y_dtype, int64_t ldy, void* stream);
+
+/* The whole W4A8 layer: transform + clip + MXFP8 quantisation of X into the workspace (Eq. 1-4,
+ * Sec. 2), then batq_gemm_mxfp8_mxfp4, launched as a programmatic dependent of the quantiser.
+ *   t          transform (required, as for batq_quantize_act_mxfp8).
+ *   workspace  dev, at least batq_linear_w4a8_workspace_bytes(w, s) bytes, 1024-byte aligned.
+ * Errors as batq_linear_w4a4, plus UNSUPPORTED for n % 128 != 0. */
+size_t batq_linear_w4a8_workspace_bytes(const batq_weight* w, int64_t s);
+batq_status batq_linear_w4a8(const batq_transform* t, const batq_weight* w, const void* x_bf16,
+                             int64_t s, int64_t ld, void* y, int32_t y_dtype, int64_t ldy,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
 /* Stage 3 alone for a handful of tokens (decode), s <= 128: the same contraction as
  * batq_gemm_mxfp4, organised for the case where streaming the weights from HBM once is the
  * whole cost.  The weights are the 128-row tensor-core operand and the tokens the narrow one;

@@ -37,6 +37,9 @@ SIGNATURES = {
     "batq_weight_destroy": (C.c_int, [_P]),
     "batq_weight_export": (C.c_int, [_P, _P, _P, _P]),
     "batq_gemm_mxfp4": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _I64, _P]),
+    "batq_gemm_mxfp8_mxfp4": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _I64, _P]),
+    "batq_linear_w4a8_workspace_bytes": (_SZ, [_P, _I64]),
+    "batq_linear_w4a8": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P, _SZ, _P]),
     "batq_gemm_small_s_scratch_bytes": (_SZ, [_P, _I64]),
     "batq_gemm_mxfp4_small_s": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _I64, _P, _SZ, _P]),
     "batq_debug_force_small_s_splits": (None, [_I32]),
@@ -212,6 +215,24 @@ def batq_gemm_mxfp4(x_codes, x_scales_mma, w: Weight, s, y, ldy=None):
     st = load().batq_gemm_mxfp4(_ptr(x_codes), _ptr(x_scales_mma), w.handle, s, _ptr(y), dt,
                                 y.stride(0) if ldy is None else ldy, _stream())
     _check(st, "batq_gemm_mxfp4")
+
+
+def batq_gemm_mxfp8_mxfp4(x_codes8, x_scales_mma, w: Weight, s, y, ldy=None):
+    dt = F32 if y.dtype == torch.float32 else BF16
+    st = load().batq_gemm_mxfp8_mxfp4(_ptr(x_codes8), _ptr(x_scales_mma), w.handle, s, _ptr(y), dt,
+                                      y.stride(0) if ldy is None else ldy, _stream())
+    _check(st, "batq_gemm_mxfp8_mxfp4")
+
+
+def batq_linear_w4a8_workspace_bytes(w: Weight, s) -> int:
+    return load().batq_linear_w4a8_workspace_bytes(w.handle, s)
+
+
+def batq_linear_w4a8(t, w: Weight, x, y, workspace):
+    dt = F32 if y.dtype == torch.float32 else BF16
+    st = load().batq_linear_w4a8(t.handle if t else None, w.handle, _ptr(x), x.shape[0], x.stride(0), _ptr(y), dt,
+                                 y.stride(0), _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "batq_linear_w4a8")
 
 
 def batq_gemm_small_s_scratch_bytes(w: Weight, s) -> int:

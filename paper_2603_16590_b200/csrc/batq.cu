@@ -17,6 +17,7 @@
 #include "gemm_mxfp4.cuh"
 #include "gemm_mxfp4_pair.cuh"
 #include "gemm_small_s.cuh"
+#include "gemm_w4a8.cuh"
 #include "linear_small_s_fused.cuh"
 #include "mma_peak.cuh"
 #include "prepare_weight.cuh"
@@ -54,6 +55,9 @@ struct batq_weight {
   CUtensorMap tmap_b64;
   CUtensorMap tmap_b32;   // boxes of 32 weight rows: the CTA-pair kernel composes its half tiles from them
   CUtensorMap tmap_sf;    // scale atoms: [row tiles x KA] rows of 512 bytes, boxes of two atoms
+  bool has_u4;            // n % 128 == 0: the maps below exist (W4A8 GEMM)
+  CUtensorMap tmap_u4_128;  // packed 4-bit codes widened to 8-bit containers by the TMA unit: boxes of
+  CUtensorMap tmap_u4_256;  // 128 elements x 128 / 256 weight rows
 };
 
 // Scratch for batq_linear_w4a4_noalloc: part of the library image, one copy per GPU.
@@ -120,6 +124,10 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(gemm_mxfp4_kernel<128, true>, GemmCfg<128>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<64, false>, GemmCfg<64>::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_kernel<64, true>, GemmCfg<64>::kSmemBytes);
+    e = e ? e : set_smem(gemm_w4a8_kernel<128, false>, W4A8Cfg<128>::kSmemBytes);
+    e = e ? e : set_smem(gemm_w4a8_kernel<128, true>, W4A8Cfg<128>::kSmemBytes);
+    e = e ? e : set_smem(gemm_w4a8_kernel<256, false>, W4A8Cfg<256>::kSmemBytes);
+    e = e ? e : set_smem(gemm_w4a8_kernel<256, true>, W4A8Cfg<256>::kSmemBytes);
     e = e ? e : set_smem(mma_peak_kernel<false>, kPeakSmemBytes);
     e = e ? e : set_smem(mma_peak_kernel<true>, kPeakSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_pair_kernel<false>, PairCfg::kSmemBytes);
@@ -159,6 +167,19 @@ batq_status make_codes_tmap(CUtensorMap* map, const void* base, int64_t rows, in
   const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBKBytes), static_cast<cuuint32_t>(box_rows)};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides,
+                                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? BATQ_OK : BATQ_ERR_CUDA;
+}
+
+// Tensor map over packed 4-bit codes [rows x n] (n elements per row, n % 128 == 0) whose loads widen
+// every 16 codes (8 bytes) into a 16-byte slot of shared memory: box = 128 elements x box_rows.
+batq_status make_u4_unpack_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t n, int box_rows) {
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(n), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(n / 2)};
+  const cuuint32_t box[2] = {128, static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 2, const_cast<void*>(base), dims, strides,
                                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? BATQ_OK : BATQ_ERR_CUDA;
@@ -831,6 +852,70 @@ batq_status launch_linear_fused(const batq_transform* t, const batq_weight* w, c
   return BATQ_OK;
 }
 
+// ---- W4A8: MXFP8 activations x MXFP4 weights --------------------------------------------------
+// Bytes one weight row of a K-step (128 four-bit codes, 64 bytes in global memory, 128 bytes of
+// 8-bit containers in shared memory) adds to the mbarrier's transaction count.
+constexpr int kU4RowTxBytes = 128;
+
+batq_status launch_gemm_w4a8(const void* x_codes8, const void* x_sf, const batq_weight* w, int64_t s, void* y,
+                             int32_t y_dtype, int64_t ldy, cudaStream_t stream, bool dependent) {
+  int dev;
+  const DeviceInfo* info;
+  batq_status st = device_setup(&dev, &info);
+  if (st != BATQ_OK) return st;
+  if (w->device != dev) return BATQ_ERR_CUDA;
+  if (!w->has_u4) return BATQ_ERR_UNSUPPORTED;
+  const bool bf = y_dtype == BATQ_BF16;
+  CUtensorMap tmap_a, tmap_y;
+  std::memset(&tmap_y, 0, sizeof(tmap_y));
+  st = make_tmap_2d(&tmap_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, x_codes8, w->n, s, w->n, 128, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+  const int64_t m16 = w->m / (bf ? 8 : 4) * (bf ? 8 : 4);
+  if (st == BATQ_OK && m16 > 0) st = make_y_tmap(&tmap_y, y, s, m16, ldy, bf);
+  if (st != BATQ_OK) return st;
+  // Tile width: 256 (one accumulator, highest flop per byte staged) unless 128-wide tiles (two
+  // accumulators, epilogue overlapped) fill the SMs in fewer waves' worth of time.
+  const int64_t mt = (s + kBM - 1) / kBM;
+  auto waves = [&](int bn) { return ((mt * ((w->m + bn - 1) / bn)) + info->sm_count - 1) / info->sm_count; };
+  const int force_bn = g_force_bn.load(std::memory_order_relaxed);
+  int bn = (w->m <= 128 || waves(128) * 128 * 1.08 < waves(256) * 256 * 1.1) ? 128 : 256;
+  if (force_bn == 128 || force_bn == 256) bn = force_bn;
+  W4A8Params p{};
+  p.sfa = static_cast<const uint8_t*>(x_sf);
+  p.sfb = w->scales;
+  p.s = static_cast<int32_t>(s);
+  p.m = static_cast<int32_t>(w->m);
+  p.katoms = w->katoms;
+  p.k_steps = static_cast<int32_t>(w->n / kW4A8KElems);
+  p.m_tiles = static_cast<int32_t>(mt);
+  p.n_tiles = static_cast<int32_t>((w->m + bn - 1) / bn);
+  p.sfb_row_tiles = static_cast<int32_t>((w->m + 127) / 128);
+  p.m16 = static_cast<int32_t>(m16);
+  p.b_row_tx = kU4RowTxBytes;
+  p.y = y;
+  p.ldy = ldy;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(std::min<int64_t>(info->sm_count, static_cast<int64_t>(p.m_tiles) * p.n_tiles)));
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = dependent ? 1 : 0;
+  cudaError_t e;
+  if (bn == 256) {
+    cfg.dynamicSmemBytes = W4A8Cfg<256>::kSmemBytes;
+    e = bf ? cudaLaunchKernelEx(&cfg, gemm_w4a8_kernel<256, true>, tmap_a, w->tmap_u4_256, tmap_y, p)
+           : cudaLaunchKernelEx(&cfg, gemm_w4a8_kernel<256, false>, tmap_a, w->tmap_u4_256, tmap_y, p);
+  } else {
+    cfg.dynamicSmemBytes = W4A8Cfg<128>::kSmemBytes;
+    e = bf ? cudaLaunchKernelEx(&cfg, gemm_w4a8_kernel<128, true>, tmap_a, w->tmap_u4_128, tmap_y, p)
+           : cudaLaunchKernelEx(&cfg, gemm_w4a8_kernel<128, false>, tmap_a, w->tmap_u4_128, tmap_y, p);
+  }
+  if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+  return BATQ_OK;
+}
+
 batq_status check_y(const void* y, int32_t y_dtype, int64_t ldy, int64_t m) {
   if (y_dtype != BATQ_F32 && y_dtype != BATQ_BF16) return BATQ_ERR_UNSUPPORTED;
   if (ldy < m) return BATQ_ERR_SHAPE;
@@ -1055,6 +1140,9 @@ batq_status batq_prepare_weight(const batq_transform* t, const void* w_bf16, int
   if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b64, w->codes, m, n / 2, 64);
   if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b32, w->codes, m, n / 2, 32);
   if (st == BATQ_OK) st = make_sf_tmap(&w->tmap_sf, w->scales, (m + 127) / 128, w->katoms);
+  w->has_u4 = n % 128 == 0;
+  if (st == BATQ_OK && w->has_u4) st = make_u4_unpack_tmap(&w->tmap_u4_128, w->codes, m, n, 128);
+  if (st == BATQ_OK && w->has_u4) st = make_u4_unpack_tmap(&w->tmap_u4_256, w->codes, m, n, 256);
   if (st != BATQ_OK) { delete w; return st; }
   *out = w;
   return BATQ_OK;
@@ -1089,6 +1177,51 @@ batq_status batq_gemm_mxfp4(const void* x_codes, const void* x_scales_mma, const
   batq_status st = check_y(y, y_dtype, ldy, w->m);
   if (st != BATQ_OK) return st;
   return launch_gemm(x_codes, x_scales_mma, w, s, y, y_dtype, ldy, static_cast<cudaStream_t>(stream));
+}
+
+batq_status batq_gemm_mxfp8_mxfp4(const void* x_codes8, const void* x_scales_mma, const batq_weight* w, int64_t s, void* y,
+                                  int32_t y_dtype, int64_t ldy, void* stream) {
+  if (w == nullptr) return BATQ_ERR_NULL;
+  if (s < 0 || s > (int64_t(1) << 30)) return BATQ_ERR_SHAPE;
+  if (!w->has_u4) return BATQ_ERR_UNSUPPORTED;
+  if (s == 0) return BATQ_OK;
+  if (x_codes8 == nullptr || x_scales_mma == nullptr || y == nullptr) return BATQ_ERR_NULL;
+  if (!aligned(x_codes8, 16) || !aligned(x_scales_mma, 16)) return BATQ_ERR_ALIGN;
+  batq_status st = check_y(y, y_dtype, ldy, w->m);
+  if (st != BATQ_OK) return st;
+  return launch_gemm_w4a8(x_codes8, x_scales_mma, w, s, y, y_dtype, ldy, static_cast<cudaStream_t>(stream), false);
+}
+
+size_t batq_linear_w4a8_workspace_bytes(const batq_weight* w, int64_t s) {
+  if (w == nullptr || s < 0) return 0;
+  return round_up(static_cast<size_t>(s * w->n), 1024) + round_up(batq_sf_bytes(s, w->n, BATQ_SF_MMA), 1024);
+}
+
+batq_status batq_linear_w4a8(const batq_transform* t, const batq_weight* w, const void* x_bf16, int64_t s, int64_t ld,
+                             void* y, int32_t y_dtype, int64_t ldy, void* workspace, size_t workspace_bytes,
+                             void* stream) {
+  if (w == nullptr || t == nullptr) return BATQ_ERR_NULL;
+  batq_status st = check_x(x_bf16, s, w->n, ld);
+  if (st != BATQ_OK) return st;
+  if (t->n != w->n) return BATQ_ERR_SHAPE;
+  if (!w->has_u4) return BATQ_ERR_UNSUPPORTED;
+  if (s == 0) return BATQ_OK;
+  if (y == nullptr || workspace == nullptr) return BATQ_ERR_NULL;
+  st = check_y(y, y_dtype, ldy, w->m);
+  if (st != BATQ_OK) return st;
+  if (!aligned(workspace, 1024)) return BATQ_ERR_ALIGN;
+  if (workspace_bytes < batq_linear_w4a8_workspace_bytes(w, s)) return BATQ_ERR_WORKSPACE;
+  int dev;
+  const DeviceInfo* info;
+  st = device_setup(&dev, &info);
+  if (st != BATQ_OK) return st;
+  if (t->device != dev || w->device != dev) return BATQ_ERR_CUDA;
+  uint8_t* codes = static_cast<uint8_t*>(workspace);
+  uint8_t* sf = codes + round_up(static_cast<size_t>(s * w->n), 1024);
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  st = launch_quantize_tc(t, x_bf16, s, w->n, ld, codes, sf, BATQ_SF_MMA, nullptr, cs, info->sm_count, true);
+  if (st != BATQ_OK) return st;
+  return launch_gemm_w4a8(codes, sf, w, s, y, y_dtype, ldy, cs, true);
 }
 
 size_t batq_gemm_small_s_scratch_bytes(const batq_weight* w, int64_t s) {
