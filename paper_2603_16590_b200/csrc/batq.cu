@@ -853,9 +853,10 @@ batq_status launch_linear_fused(const batq_transform* t, const batq_weight* w, c
 }
 
 // ---- W4A8: MXFP8 activations x MXFP4 weights --------------------------------------------------
-// Bytes one weight row of a K-step (128 four-bit codes, 64 bytes in global memory, 128 bytes of
-// 8-bit containers in shared memory) adds to the mbarrier's transaction count.
-constexpr int kU4RowTxBytes = 128;
+// Bytes one weight row of a K-step adds to the mbarrier's transaction count: 128 four-bit codes
+// are 64 bytes in global memory and land in 128 bytes of shared memory (8 data bytes at the start
+// of every 16-byte slot, the other 8 left untouched); the copy reports the 64 bytes it moved.
+constexpr int kU4RowTxBytes = 64;
 
 batq_status launch_gemm_w4a8(const void* x_codes8, const void* x_sf, const batq_weight* w, int64_t s, void* y,
                              int32_t y_dtype, int64_t ldy, cudaStream_t stream, bool dependent) {
