@@ -443,6 +443,7 @@ def run_ours(args):
     for value, hook in ((args.tile_width, B.batq_debug_force_tile_width), (args.quantizer, B.batq_debug_force_quantizer),
                         (args.gemm_kernel, B.batq_debug_force_gemm_kernel), (args.splits, B.batq_debug_force_small_s_splits),
                         (args.small_path, B.batq_debug_force_small_s_path),
+                        (args.prefill_path, B.batq_debug_force_prefill_path),
                         (args.small_reduce, B.batq_debug_force_small_s_reduce)):
         if value != 0:
             hook(value)
@@ -831,6 +832,7 @@ def main():
     ap.add_argument("--gemm-kernel", type=int, default=0, help="0 auto, 1 one CTA per tile, 2 CTA pairs (tuning)")
     ap.add_argument("--tile-width", type=int, default=0, help="force the GEMM tile width (tuning); 0 = automatic")
     ap.add_argument("--small-path", type=int, default=0, help="0 auto, 1 two kernels, 2 fused kernel (tuning)")
+    ap.add_argument("--prefill-path", type=int, default=0, help="0 auto, 1 quantiser + GEMM kernels, 2 one kernel (tuning)")
     ap.add_argument("--small-reduce", type=int, default=0, help="0 auto, 1 tickets, 2 cluster (split-K reduction, tuning)")
     ap.add_argument("--splits", type=int, default=0, help="force the small-s GEMM's K splits (tuning); 0 = automatic")
     args = ap.parse_args()

@@ -63,6 +63,11 @@ void batq_debug_force_small_s_reduce(int32_t which);
  * other shapes take the two kernels. */
 void batq_debug_force_small_s_path(int32_t which);
 
+/* How batq_linear_w4a4 runs prefill shapes (s > 128, m >= 192, a transform, k % 8 == 0).
+ * 0 = automatic, 1 = always two kernels (quantiser, then the CTA-pair GEMM as its programmatic
+ * dependent), 2 = one kernel (quantise phase and GEMM phase on the same grid) wherever it applies. */
+void batq_debug_force_prefill_path(int32_t which);
+
 /* Failure-detection check that harms nothing: launches one warp that waits, with the library's
  * bounded wait and a limit of limit_ns nanoseconds (clamped to [1000, 10000000]), on a barrier
  * that nothing ever signals.  The wait runs out, the kernel records it exactly as a product

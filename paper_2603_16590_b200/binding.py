@@ -46,6 +46,7 @@ SIGNATURES = {
     "batq_debug_force_small_s_path": (None, [_I32]),
     "batq_debug_force_small_s_reduce": (None, [_I32]),
     "batq_debug_force_tile_width": (None, [_I32]),
+    "batq_debug_force_prefill_path": (None, [_I32]),
     "batq_debug_force_gemm_kernel": (None, [_I32]),
     "batq_debug_force_quantizer": (None, [_I32]),
     "batq_linear_workspace_bytes": (_SZ, [_P, _I64]),
@@ -256,6 +257,10 @@ def batq_debug_force_small_s_reduce(which: int):
 
 def batq_debug_force_small_s_path(which: int):
     load().batq_debug_force_small_s_path(which)
+
+
+def batq_debug_force_prefill_path(which: int):
+    load().batq_debug_force_prefill_path(which)
 
 
 def batq_debug_force_tile_width(bn: int):

@@ -18,6 +18,7 @@
 #include "gemm_mxfp4_pair.cuh"
 #include "gemm_small_s.cuh"
 #include "gemm_w4a8.cuh"
+#include "linear_prefill_fused.cuh"
 #include "linear_small_s_fused.cuh"
 #include "mma_peak.cuh"
 #include "prepare_weight.cuh"
@@ -40,6 +41,7 @@ struct batq_transform {
   float* d_clip_lo;
   float* d_clip_hi;
   uint8_t* d_pimg;                    // [k][3][2048]: dense P_j^T as three bf16 terms, tensor-core operand layout
+  CUtensorMap tmap_pimg;              // the same bytes as [k][3 terms][2 halves of 16 rows][1024]: boxes of 4 blocks x 3 terms x one half
 };
 
 struct batq_weight {
@@ -132,6 +134,10 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(mma_peak_kernel<true>, kPeakSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_pair_kernel<false>, PairCfg::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_pair_kernel<true>, PairCfg::kSmemBytes);
+    e = e ? e : set_smem(linear_prefill_fused_kernel<false, false>, kPfSmemBytes);
+    e = e ? e : set_smem(linear_prefill_fused_kernel<false, true>, kPfSmemBytes);
+    e = e ? e : set_smem(linear_prefill_fused_kernel<true, false>, kPfSmemBytes);
+    e = e ? e : set_smem(linear_prefill_fused_kernel<true, true>, kPfSmemBytes);
     e = e ? e : set_smem(linear_small_s_fused_kernel<false>, FusedCfg::kSmemBytes);
     e = e ? e : set_smem(linear_small_s_fused_kernel<true>, FusedCfg::kSmemBytes);
     e = e ? e : set_smem(gemm_small_s_kernel<16, false>, SmallCfg<16>::kSmemBytes);
@@ -852,6 +858,88 @@ batq_status launch_linear_fused(const batq_transform* t, const batq_weight* w, c
   return BATQ_OK;
 }
 
+// ---- prefill layer in one kernel (quantise phase + GEMM phase on one grid of CTA pairs) --------
+std::atomic<int> g_force_prefill_path{0};  // tuning hook: 0 = automatic, 1 = two kernels, 2 = one kernel wherever it applies
+std::atomic<unsigned long long> g_call_tag{1};  // tags the readiness counters of one call; never reused within a process
+
+inline size_t prefill_ready_bytes(int64_t s) { return round_up(static_cast<size_t>(((s + 255) / 256) * 2 + 1) * 8, 1024); }
+
+// Applies to what the CTA-pair GEMM takes (s > 128, m >= 192) with a transform whose scale atoms
+// come in pairs (k % 8 == 0: no padding atom to keep finite).
+bool fused_prefill_applies(const batq_transform* t, const batq_weight* w, int64_t s) {
+  return t != nullptr && s > 128 && w->m >= 192 && w->k % 8 == 0 &&
+         g_force_gemm_kernel.load(std::memory_order_relaxed) != 1 && g_force_quantizer.load(std::memory_order_relaxed) == 0;
+}
+bool use_fused_prefill(const batq_transform* t, const batq_weight* w, int64_t s) {
+  const int f = g_force_prefill_path.load(std::memory_order_relaxed);
+  if (f == 1 || !fused_prefill_applies(t, w, s)) return false;
+  return f == 2;
+}
+
+batq_status launch_linear_prefill_fused(const batq_transform* t, const batq_weight* w, const void* x, int64_t s, int64_t ld,
+                                        void* y, int32_t y_dtype, int64_t ldy, uint8_t* codes, uint8_t* sf, uint8_t* ready,
+                                        cudaStream_t stream) {
+  int dev;
+  const DeviceInfo* info;
+  batq_status st = device_setup(&dev, &info);
+  if (st != BATQ_OK) return st;
+  if (w->device != dev || t->device != dev) return BATQ_ERR_CUDA;
+  const bool bf = y_dtype == BATQ_BF16;
+  const int64_t n = w->n;
+  CUtensorMap tmap_x, tmap_codes, tmap_a, tmap_sfa, tmap_y;
+  std::memset(&tmap_y, 0, sizeof(tmap_y));
+  st = make_tmap_2d(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x, n, s, ld * 2, 64, kQtRows, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (st == BATQ_OK)
+    st = make_tmap_2d(&tmap_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, n / 2, s, n / 2, 64, kQtRows, CU_TENSOR_MAP_SWIZZLE_64B);
+  if (st == BATQ_OK) st = make_codes_tmap(&tmap_a, codes, s, n / 2, kBM);
+  if (st == BATQ_OK) st = make_sf_tmap(&tmap_sfa, sf, (s + 127) / 128, w->katoms);
+  const int64_t m16 = w->m / (bf ? 8 : 4) * (bf ? 8 : 4);
+  if (st == BATQ_OK && m16 > 0) st = make_y_tmap(&tmap_y, y, s, m16, ldy, bf);
+  if (st != BATQ_OK) return st;
+  PrefillFusedParams q{};
+  int pairs = 0;
+  if (!pair_schedule(s, w->m, (n + 255) / 256, info->sm_count, &q.g, &pairs)) return BATQ_ERR_SHAPE;
+  q.g.katoms = w->katoms;
+  q.g.k_steps = static_cast<int32_t>((n + 255) / 256);
+  q.g.m16 = static_cast<int32_t>(m16);
+  q.g.y = y;
+  q.g.ldy = ldy;
+  q.n = static_cast<int32_t>(n);
+  q.k = w->k;
+  q.n_strips = w->k / kQtGroups;
+  q.n_row_tiles = static_cast<int32_t>((s + 127) / 128);
+  q.n_units = q.g.m_pairs * q.n_strips;
+  q.clip_lo = t->d_clip_lo;
+  q.clip_hi = t->d_clip_hi;
+  q.scales = sf;
+  q.ready = reinterpret_cast<unsigned long long*>(ready);
+  q.tag = g_call_tag.fetch_add(1, std::memory_order_relaxed) & ((1ull << 40) - 1ull);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs));
+  cfg.blockDim = dim3(kPfThreads);
+  cfg.dynamicSmemBytes = kPfSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  // A programmatic dependent of whatever precedes it on the stream: its CTAs take over the SMs that
+  // kernel has left and wait, inside the kernel, before they read x.
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  cudaError_t e;
+#define BATQ_PF(CL, BF) cudaLaunchKernelEx(&cfg, linear_prefill_fused_kernel<CL, BF>, tmap_x, t->tmap_pimg, tmap_codes, tmap_a, \
+                                           w->tmap_b32, tmap_sfa, w->tmap_sf, tmap_y, q)
+  if (t->has_clip) e = bf ? BATQ_PF(true, true) : BATQ_PF(true, false);
+  else e = bf ? BATQ_PF(false, true) : BATQ_PF(false, false);
+#undef BATQ_PF
+  if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+  return BATQ_OK;
+}
+
 // ---- W4A8: MXFP8 activations x MXFP4 weights --------------------------------------------------
 // Bytes one weight row of a K-step adds to the mbarrier's transaction count: 128 four-bit codes
 // are 64 bytes in global memory and land in 128 bytes of shared memory (8 data bytes at the start
@@ -991,6 +1079,19 @@ batq_status batq_transform_create(batq_transform** out, int32_t n, int32_t gr, i
     cudaGetLastError();
     batq_transform_destroy(t);
     return BATQ_ERR_CUDA;
+  }
+  {
+    // the block-matrix images seen as [k blocks][3 terms][2 halves][256 words]
+    const cuuint64_t dims[4] = {256, 2, 3, static_cast<cuuint64_t>(t->k)};
+    const cuuint64_t strides[3] = {1024, 2048, static_cast<cuuint64_t>(kQtImageBytes)};
+    const cuuint32_t box[4] = {256, 1, 3, static_cast<cuuint32_t>(kQtGroups)};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (g_encode_tiled(&t->tmap_pimg, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, t->d_pimg, dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+      batq_transform_destroy(t);
+      return BATQ_ERR_CUDA;
+    }
   }
   *out = t;
   return BATQ_OK;
@@ -1262,12 +1363,13 @@ static bool layer_takes_small_path(const batq_weight* w, int64_t s) {
 size_t batq_linear_workspace_bytes(const batq_weight* w, int64_t s) {
   if (w == nullptr || s < 0) return 0;
   const size_t q = round_up(static_cast<size_t>(s * (w->n / 2)), 1024) + round_up(batq_sf_bytes(s, w->n, BATQ_SF_MMA), 1024);
+  if (s > 128) return q + prefill_ready_bytes(s);   // readiness counters of the one-kernel prefill path
   return q + (s > 0 && layer_takes_small_path(w, s) ? small_scratch(w, s).total() : 0);
 }
 
 int32_t batq_linear_kernel_launches(const batq_transform* t, const batq_weight* w, int64_t s) {
   if (w == nullptr || s <= 0) return 0;
-  return use_fused_small(t, w, s) ? 1 : 2;
+  return (use_fused_small(t, w, s) || use_fused_prefill(t, w, s)) ? 1 : 2;
 }
 
 batq_status batq_linear_w4a4(const batq_transform* t, const batq_weight* w, const void* x_bf16, int64_t s, int64_t ld,
@@ -1297,6 +1399,9 @@ batq_status batq_linear_w4a4(const batq_transform* t, const batq_weight* w, cons
     if (st != BATQ_OK) return st;
     return launch_gemm_small(codes, sf, w, s, y, y_dtype, ldy, scratch, sc, cs, true);
   }
+  if (use_fused_prefill(t, w, s))
+    return launch_linear_prefill_fused(t, w, x_bf16, s, ld, y, y_dtype, ldy, codes, sf,
+                                       sf + round_up(batq_sf_bytes(s, w->n, BATQ_SF_MMA), 1024), cs);
   st = launch_quantize(t, x_bf16, s, w->n, ld, codes, sf, BATQ_SF_MMA, nullptr, cs);
   if (st != BATQ_OK) return st;
   return launch_gemm(codes, sf, w, s, y, y_dtype, ldy, cs, true);
@@ -1352,6 +1457,7 @@ void batq_debug_force_gemm_kernel(int32_t which) { g_force_gemm_kernel.store(whi
 void batq_debug_force_small_s_splits(int32_t splits) { g_force_splits.store(splits, std::memory_order_relaxed); }
 void batq_debug_force_small_s_path(int32_t which) { g_force_small_path.store(which, std::memory_order_relaxed); }
 void batq_debug_force_small_s_reduce(int32_t which) { g_small_reduce.store(which, std::memory_order_relaxed); }
+void batq_debug_force_prefill_path(int32_t which) { g_force_prefill_path.store(which, std::memory_order_relaxed); }
 
 batq_status batq_debug_wait_timeout(int64_t limit_ns, void* stream) {
   batq_status st = device_setup(nullptr, nullptr);
