@@ -862,7 +862,8 @@ batq_status launch_linear_fused(const batq_transform* t, const batq_weight* w, c
 std::atomic<int> g_force_prefill_path{0};  // tuning hook: 0 = automatic, 1 = two kernels, 2 = one kernel wherever it applies
 std::atomic<unsigned long long> g_call_tag{1};  // tags the readiness counters of one call; never reused within a process
 
-inline size_t prefill_ready_bytes(int64_t s) { return round_up(static_cast<size_t>(((s + 255) / 256) * 2 + 1) * 8, 1024); }
+// a run counter and one flag word per CTA of the grid (at most one CTA per SM)
+inline size_t prefill_flag_bytes(const batq_weight* w) { return round_up(static_cast<size_t>(std::max(w->sm_count, 148) + 1) * 8, 1024); }
 
 // Applies to what the CTA-pair GEMM takes (s > 128, m >= 192) with a transform whose scale atoms
 // come in pairs (k % 8 == 0: no padding atom to keep finite).
@@ -912,7 +913,7 @@ batq_status launch_linear_prefill_fused(const batq_transform* t, const batq_weig
   q.clip_lo = t->d_clip_lo;
   q.clip_hi = t->d_clip_hi;
   q.scales = sf;
-  q.ready = reinterpret_cast<unsigned long long*>(ready);
+  q.sync = reinterpret_cast<unsigned long long*>(ready);
   q.tag = g_call_tag.fetch_add(1, std::memory_order_relaxed) & ((1ull << 40) - 1ull);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs));
@@ -1363,7 +1364,7 @@ static bool layer_takes_small_path(const batq_weight* w, int64_t s) {
 size_t batq_linear_workspace_bytes(const batq_weight* w, int64_t s) {
   if (w == nullptr || s < 0) return 0;
   const size_t q = round_up(static_cast<size_t>(s * (w->n / 2)), 1024) + round_up(batq_sf_bytes(s, w->n, BATQ_SF_MMA), 1024);
-  if (s > 128) return q + prefill_ready_bytes(s);   // readiness counters of the one-kernel prefill path
+  if (s > 128) return q + prefill_flag_bytes(w);   // flag words of the one-kernel prefill path
   return q + (s > 0 && layer_takes_small_path(w, s) ? small_scratch(w, s).total() : 0);
 }
 

@@ -10,14 +10,21 @@
 // quantize_act_tc.cuh; each CTA stages the 16 output channels of P_j^T that its half of the B
 // operand holds), sixteen quantiser warps clip, scale and round their token rows out of tensor
 // memory, and a store warp writes the unit's codes (one TMA store) and scale atom (one bulk
-// copy) to the workspace.  When a CTA's stores of a unit have completed it bumps the counter of
-// that (256-token row block, half): counter words carry the call's tag in their upper bits, so
-// stale contents of the workspace never count.
+// copy) to the workspace.  When all stores of a CTA have completed it publishes that in its own
+// flag word in the workspace (no atomics: one release store per CTA).
 //
 // Phase 2 (GEMM).  Exactly the CTA-pair GEMM of gemm_mxfp4_pair.cuh (same schedule, same
 // barriers, same tensor-memory plan); instead of waiting for a preceding grid, the TMA producer
-// of a CTA waits -- bounded -- until the counter of the row block it is about to load says that
-// all of its channel strips have been quantised.  Weight tiles never wait.
+// of a CTA first waits -- bounded -- until every CTA's flag says that its share of X is in the
+// workspace.
+//
+// Flag words.  The workspace holds a run counter and one flag per CTA.  Every CTA reads the run
+// counter once the grid before it has completed (griddepcontrol.wait); counter + 1 is the number
+// of this run, and a CTA that has finished phase 1 stores that number, mixed with a tag unique to
+// the call (host counter), in its flag.  Flags of earlier runs -- of this launch or of any other
+// that shares the workspace, replays of a CUDA graph included -- hold smaller numbers and never
+// read as done, and neither does whatever an uninitialised workspace holds.  CTA 0 writes the new
+// run number back after it has seen every flag, i.e. after every CTA has read the old one.
 //
 // All tcgen05 instructions of the kernel use cta_group::2.  Every wait is bounded; a wait that
 // gives up raises the CTA's abort flag, records the time-out for the host and falls through to
@@ -43,7 +50,7 @@ constexpr int kPfSmemBytes = PairCfg::kSmemBytes;
 static_assert(kPfPhase1Bytes + 1024 <= kPfSmemBytes, "phase 1 fits the GEMM's shared memory");
 static_assert((kPfXStages * kQtStageBytes) % 1024 == 0 && kPfStripImageBytes % 1024 == 0 && kPfOutBufBytes % 512 == 0,
               "alignment of the phase-1 regions");
-constexpr int kPfTagShift = 24;               // counter word: (tag << 24) | units done
+constexpr int kPfTagShift = 24;               // flag word: run number ^ (tag << 24)
 
 struct PrefillFusedParams {
   PairParams g;            // the GEMM: shapes, schedule, y
@@ -55,7 +62,7 @@ struct PrefillFusedParams {
   const float* clip_lo;    // [k] or NULL
   const float* clip_hi;
   uint8_t* scales;         // activation scale atoms (BATQ_SF_MMA layout) in the workspace
-  unsigned long long* ready;   // [m_pairs][2] counter words in the workspace, then one word counting finished CTAs
+  unsigned long long* sync;    // in the workspace: [0] run counter, [1 + i] flag of CTA i
   unsigned long long tag;      // this call's tag (40 bits)
 };
 
@@ -84,35 +91,29 @@ __device__ __forceinline__ unsigned long long ld_acquire_gpu_u64(const unsigned 
   return v;
 }
 
-// One more unit of (row block, half) is in the workspace: tagged increment, release order.  A word
-// whose upper bits are not this call's tag (stale or never written) counts as zero.  Returns the
-// new count (0 if the update could not be made in 2^20 tries).
-__device__ __forceinline__ uint32_t ready_bump(unsigned long long* word, unsigned long long tag) {
-  __threadfence();
-  unsigned long long old = *reinterpret_cast<volatile unsigned long long*>(word);
-  for (int tries = 0; tries < (1 << 20); ++tries) {
-    const unsigned long long nw = ((old >> kPfTagShift) == tag) ? old + 1ull : ((tag << kPfTagShift) | 1ull);
-    const unsigned long long seen = atomicCAS(word, old, nw);
-    if (seen == old) return static_cast<uint32_t>(nw & ((1ull << kPfTagShift) - 1ull));
-    old = seen;
-  }
-  return 0u;
+__device__ __forceinline__ void st_release_gpu_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
-// Bounded wait until `word` says that `expect` units of this call are done.
-__device__ __forceinline__ bool ready_wait(const unsigned long long* word, unsigned long long tag, uint32_t expect,
-                                           volatile int* abort_flag) {
-  const unsigned long long want = (tag << kPfTagShift) | expect;
-  if (ld_acquire_gpu_u64(word) == want) return true;
-  const uint64_t t0 = global_timer_ns();
+// Bounded wait of a whole warp until all n flag words equal `want` (lane l polls words l, l + 32, ...).
+__device__ __forceinline__ bool flags_wait_all(const unsigned long long* flags, int n, unsigned long long want,
+                                               volatile int* abort_flag) {
+  const int lane = threadIdx.x & 31;
+  uint64_t t0 = 0;
   for (;;) {
-    if (ld_acquire_gpu_u64(word) == want) return true;
-    if (*abort_flag) return false;
-    if (global_timer_ns() - t0 > kWaitLimitNs) {
-      *abort_flag = 1;
-      atomicExch(&g_device_error, 1);
+    bool mine = true;
+    for (int i = lane; i < n; i += 32) mine = mine && (ld_acquire_gpu_u64(flags + i) == want);
+    if (__all_sync(0xFFFFFFFFu, mine)) return true;
+    if (__any_sync(0xFFFFFFFFu, *abort_flag != 0)) return false;
+    const uint64_t now = global_timer_ns();
+    if (t0 == 0) t0 = now;
+    if (__any_sync(0xFFFFFFFFu, now - t0 > kWaitLimitNs)) {
+      if (lane == 0) {
+        *abort_flag = 1;
+        atomicExch(&g_device_error, 1);
+      }
       return false;
     }
-    __nanosleep(64);
+    __nanosleep(200);
   }
 }
 
@@ -144,6 +145,8 @@ linear_prefill_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
   __shared__ __align__(8) uint64_t drain_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
+  __shared__ unsigned long long run_number;                  // this run's number
+  __shared__ unsigned long long flag_value;                  // what a finished CTA's flag holds in this run
 
   grid_launch_dependents();
   const int tid = threadIdx.x;
@@ -300,6 +303,11 @@ linear_prefill_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
   } else if (warp == 2 + kQtQuantWarps) {
     // ------------------------------------------------------------ store warp (both CTAs)
     if (lane == 0) {
+      // The grid before this one (possibly an earlier run of this very launch) has completed once
+      // this returns: only then is the run counter final.
+      grid_dependency_wait();
+      run_number = *reinterpret_cast<volatile unsigned long long*>(q.sync) + 1ull;
+      flag_value = run_number ^ (q.tag << kPfTagShift);
       int it = 0;
       bool ok = true;
       for (int u = u0; u < u1; ++u, ++it) {
@@ -313,23 +321,17 @@ linear_prefill_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
         if (row_tile < q.n_row_tiles)
           bulk_s2g(q.scales + (static_cast<int64_t>(row_tile) * p.katoms + strip) * 512, smem_u32(ob + kQtCodeTileBytes), 512);
         bulk_commit_group();
-        if (it > 0) {
-          // The unit before this one: its stores have completed (the buffer is free and the bytes
-          // are in global memory), so it may be counted.
-          bulk_wait_group<1>();
-          fence_proxy_async_all();
-          const int up = u - 1;
-          const int sp = up / p.m_pairs;
-          ready_bump(q.ready + (static_cast<int64_t>(up - sp * p.m_pairs) * 2 + rank), q.tag);
+        if (it > 0) {  // the stores of the unit before this one have read their buffer: hand it back
+          bulk_wait_group_read<1>();
           mbar_arrive(smem_u32(&t_empty[(it - 1) % kPfOutBufs]));
         }
       }
+      // All stores of this CTA are in global memory: publish it (also with no units at all).
       bulk_wait_group<0>();
-      if (ok && u1 > u0) {
+      if (ok) {
         fence_proxy_async_all();
-        const int up = u1 - 1;
-        const int sp = up / p.m_pairs;
-        ready_bump(q.ready + (static_cast<int64_t>(up - sp * p.m_pairs) * 2 + rank), q.tag);
+        __threadfence();
+        st_release_gpu_u64(q.sync + 1 + blockIdx.x, flag_value);
       }
     }
   } else {
@@ -442,7 +444,6 @@ linear_prefill_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     bool ok = true;
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t full0_leader = map_to_cta(smem_u32(&full_bar[0]), 0);
-    unsigned long long confirmed = 0ull;   // row blocks < 64 already seen complete
     auto issue = [&](const PairTile& t, int kt, int stage) {
       const int m0 = t.mp * 256 + static_cast<int>(rank) * kBM;
       const int half = t.bn >> 1;
@@ -465,17 +466,13 @@ linear_prefill_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     uint32_t phase = 0;
     PairWalk w = walk0;
     PairTile t;
+    // Every CTA's share of X quantised and in global memory?  (Every lane takes the acquire
+    // itself, so whichever lane is elected to issue the copies below has observed the flags.)
+    ok = flags_wait_all(q.sync + 1, static_cast<int>(gridDim.x), flag_value, &abort_flag);
+    fence_proxy_async_all();   // the TMA loads below read what other SMs wrote
+    // every CTA has read the run counter (it publishes its flag after that): CTA 0 moves it on
+    if (ok && blockIdx.x == 0 && lane == 0) *reinterpret_cast<volatile unsigned long long*>(q.sync) = run_number;
     while (ok && w.next(t)) {
-      // this CTA's 128 token rows of the row block: all strips quantised and in global memory?
-      if (t.mp >= 64 || !((confirmed >> t.mp) & 1ull)) {
-        // every lane takes the acquire itself (one broadcast load), so whichever lane is elected
-        // to issue the copies below has observed the counter
-        ok = __all_sync(0xFFFFFFFFu, ready_wait(q.ready + (static_cast<int64_t>(t.mp) * 2 + rank), q.tag,
-                                                 static_cast<uint32_t>(q.n_strips), &abort_flag));
-        if (!ok) break;
-        fence_proxy_async_all();   // the TMA loads below read what other SMs wrote
-        if (t.mp < 64) confirmed |= 1ull << t.mp;
-      }
       for (int kt = 0; kt < p.k_steps; ++kt) {
         ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag));
         if (!ok) break;
@@ -639,16 +636,6 @@ linear_prefill_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
   if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc_pair(tmem_base, Cfg::kTmemCols);
-  }
-  // The CTA that finishes last puts every counter word back to zero: nobody reads them any more
-  // (each CTA counts itself only after its last wait), and a replay of the same launch -- a CUDA
-  // graph carries the same tag -- starts from clean words.
-  if (tid == 0) {
-    unsigned long long* const done = q.ready + static_cast<int64_t>(p.m_pairs) * 2;
-    if (ready_bump(done, q.tag) == gridDim.x) {
-      for (int i = 0; i <= p.m_pairs * 2; ++i) q.ready[i] = 0ull;
-      __threadfence();
-    }
   }
 }
 
