@@ -328,19 +328,20 @@ def measure_mma_peak(B, torch, iters):
     every SM busy, nothing loaded or stored): CTA pairs on 256 x 256 tiles and single CTAs on
     128 x 256 tiles, one timed launch each after a short warm-up launch."""
     out = {}
-    for name, pair in (("pair_256x256", True), ("cta_128x256", False)):
-        B.batq_debug_mma_peak(pair, 256, max(64, iters // 50))
+    for name, pair, sfc in (("pair_256x256", True, False), ("cta_128x256", False, False),
+                            ("pair_256x256_with_scale_copies", True, True), ("cta_128x256_with_scale_copies", False, True)):
+        B.batq_debug_mma_peak(pair, 256, max(64, iters // 50), sfc)
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        flops = B.batq_debug_mma_peak(pair, 256, iters)
+        flops = B.batq_debug_mma_peak(pair, 256, iters, sfc)
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1)
         out[name] = {"tflops": flops / (ms * 1e-3) / 1e12, "ms": ms}
     if B.batq_last_device_status() != 0:
         raise SystemExit("device status after the MMA-only loop")
-    best = max(out, key=lambda k: out[k]["tflops"])
+    best = max((k for k in out if "scale_copies" not in k), key=lambda k: out[k]["tflops"])
     return {"tflops": out[best]["tflops"], "shape": best, "variants": out,
             "how": "tcgen05.mma kind::mxf4.block_scale only, %d K-steps per CTA (pair), CUDA events" % iters}
 
@@ -411,7 +412,7 @@ def run_peak(args, h, B, peaks):
     e0.record()
     flops = 0.0
     for _ in range(n):
-        flops += B.batq_debug_mma_peak(pair, 256, 20000)
+        flops += B.batq_debug_mma_peak(pair, 256, 20000, False)
     e1.record()
     h.barrier()
     clocks = sampler.stop()

@@ -22,8 +22,9 @@ batq_status batq_debug_transform_clip_f32(const batq_transform* t, const void* x
                                           int64_t n, int64_t ld, float* out, void* stream);
 
 /* Forces the GEMM's output-tile width to 64, 128, 192 or 256 columns for all later calls in this
- * process (the CTA-pair kernel also takes 448 for columns of 256 and 192 alternating); any other
- * value restores the automatic choice. */
+ * process (the CTA-pair kernel also takes 448 for columns of 256 and 192 alternating, and 1 for
+ * its automatic choice restricted to one width pattern for the whole layer); any other value
+ * restores the automatic choice. */
 void batq_debug_force_tile_width(int32_t bn);
 
 /* Host only, no GPU needed: the work distribution of the CTA-pair GEMM for an s x m output
@@ -79,11 +80,13 @@ batq_status batq_debug_wait_timeout(int64_t limit_ns, void* stream);
  * Every CTA (one per SM; pair != 0: every pair of CTAs, tcgen05 cta_group::2) issues `iters`
  * K-steps of four tcgen05.mma kind::mxf4.block_scale (K = 64 each, 128 or 256 rows x bn columns)
  * on operands that stay resident in shared memory (seeded pseudo-random codes, scale bytes near
- * 2^0), accumulating in tensor memory; nothing is loaded or stored in the loop.  The caller
+ * 2^0), accumulating in tensor memory; nothing is loaded or stored in the loop.  sf_copies != 0:
+ * the scale factors are copied from shared to tensor memory (tcgen05.cp) again before every
+ * K-step, as a GEMM whose scales change with K has to; 0: once, before the loop.  The caller
  * times the launch; *flops_out (host) receives the floating-point operations of the launch
  * (2 * rows * bn * 256 per K-step and CTA or pair).  bn in {64, 128, 192, 256}. */
-batq_status batq_debug_mma_peak(int32_t pair, int32_t bn, int32_t iters, double* flops_out,
-                                void* stream);
+batq_status batq_debug_mma_peak(int32_t pair, int32_t bn, int32_t iters, int32_t sf_copies,
+                                double* flops_out, void* stream);
 
 #ifdef __cplusplus
 }

@@ -58,7 +58,7 @@ SIGNATURES = {
     "batq_linear_w4a4_noalloc": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P]),
     "batq_last_device_status": (C.c_int, [_P]),
     "batq_debug_wait_timeout": (C.c_int, [_I64, _P]),
-    "batq_debug_mma_peak": (C.c_int, [_I32, _I32, _I32, C.POINTER(C.c_double), _P]),
+    "batq_debug_mma_peak": (C.c_int, [_I32, _I32, _I32, _I32, C.POINTER(C.c_double), _P]),
 }
 
 
@@ -342,10 +342,11 @@ def batq_debug_wait_timeout(limit_ns: int):
     _check(load().batq_debug_wait_timeout(limit_ns, _stream()), "batq_debug_wait_timeout")
 
 
-def batq_debug_mma_peak(pair: bool, bn: int, iters: int) -> float:
+def batq_debug_mma_peak(pair: bool, bn: int, iters: int, sf_copies: bool = False) -> float:
     """Launches the MMA-only loop on the current stream; returns the flops of the launch."""
     flops = C.c_double(0.0)
-    _check(load().batq_debug_mma_peak(1 if pair else 0, bn, iters, C.byref(flops), _stream()), "batq_debug_mma_peak")
+    _check(load().batq_debug_mma_peak(1 if pair else 0, bn, iters, 1 if sf_copies else 0, C.byref(flops), _stream()),
+           "batq_debug_mma_peak")
     return flops.value
 
 

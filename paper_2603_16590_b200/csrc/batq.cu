@@ -57,6 +57,10 @@ struct batq_weight {
   CUtensorMap tmap_b64;
   CUtensorMap tmap_b32;   // boxes of 32 weight rows: the CTA-pair kernel composes its half tiles from them
   CUtensorMap tmap_sf;    // scale atoms: [row tiles x KA] rows of 512 bytes, boxes of two atoms
+  // CTA-pair schedules already worked out for this weight, by token count (host only)
+  struct SchedEntry { int64_t s; int force_bn; int32_t n_cols, n_segs, pairs; batq::PairSeg seg[batq::kPairMaxSegs]; };
+  mutable std::mutex sched_mutex;
+  mutable std::vector<SchedEntry> sched_cache;
   bool has_u4;            // n % 128 == 0: the maps below exist (W4A8 GEMM)
   CUtensorMap tmap_u4_128;  // packed 4-bit codes widened to 8-bit containers by the TMA unit: boxes of
   CUtensorMap tmap_u4_256;  // 128 elements x 128 / 256 weight rows
@@ -489,59 +493,175 @@ int pick_bn(int64_t s, int64_t m, int64_t n, int sm_count) {
 
 std::atomic<int> g_force_gemm_kernel{0};  // tuning hook: 0 = automatic, 1 = one CTA per tile, 2 = CTA pairs
 
-// The schedule of the CTA-pair kernel for an s x m output with k_steps K-steps: column widths and
-// number of pairs.  Every candidate (columns of 128, 192 or 256 features, or 256 and 192
-// alternating) is walked exactly as the kernel walks it, and the pair that finishes last decides.
+// The schedule of the CTA-pair kernel for an s x m output with k_steps K-steps: the segments of
+// column widths and the number of pairs.  Candidates: columns all 128, 192 or 256 wide; 256 and
+// 192 alternating; and every split of the features into a columns of 256 and b of 192, arranged as
+// 256s-192s-256s or 192s-256s-192s with the outer group cut at several places.  Each candidate is
+// walked exactly as the kernel walks it, and the pair that finishes last decides.
 // Model, in units of one K-step of a 192-wide tile (about 0.36 us): a K-step of a W-wide tile
 // moves 32 KiB of activations and W / 8 KiB of weights through L2, which is what its time follows;
-// a tile adds a small fixed cost, and the whole epilogue (about 3 us) when it has to wait for the
-// accumulator slot of the tile just before it.
+// a tile adds a small fixed cost, and about 2 us when it has to wait for the accumulator slot of
+// the tile just before it (that tile's epilogue, less what the filled ring wins back afterwards;
+// fitted to measured layers); the epilogue of a pair's last tile (about 3 us at 256 columns) is
+// always exposed.
+struct PairSched {
+  int32_t n_cols, n_segs, pairs;
+  PairSeg seg[kPairMaxSegs];
+};
+
+inline int64_t seg_span(int wa, int wb, int64_t cols) { return (cols / 2) * (wa + wb) + (cols & 1) * wa; }
+
+// Appends columns to a candidate; false if it does not fit the segment table.
+bool sched_add(PairSched* c, int wa, int wb, int64_t cols) {
+  if (cols <= 0) return true;
+  if (c->n_segs > 0) {
+    PairSeg& l = c->seg[c->n_segs - 1];
+    if (l.wa == l.wb && wa == wb && l.wa == wa) { l.cols += static_cast<int32_t>(cols); c->n_cols += static_cast<int32_t>(cols); return true; }
+  }
+  if (c->n_segs == kPairMaxSegs) return false;
+  PairSeg& g = c->seg[c->n_segs];
+  g.col0 = c->n_cols;
+  g.n0 = c->n_segs == 0 ? 0 : static_cast<int32_t>(c->seg[c->n_segs - 1].n0 +
+                                                   seg_span(c->seg[c->n_segs - 1].wa, c->seg[c->n_segs - 1].wb, c->seg[c->n_segs - 1].cols));
+  g.cols = static_cast<int32_t>(cols);
+  g.wa = static_cast<int16_t>(wa);
+  g.wb = static_cast<int16_t>(wb);
+  ++c->n_segs;
+  c->n_cols += static_cast<int32_t>(cols);
+  return true;
+}
+
+double sched_cost(const PairSched& c, PairParams* p, int64_t k_steps, int max_pairs, int* pairs_out) {
+  p->n_cols = c.n_cols;
+  p->n_segs = c.n_segs;
+  for (int i = 0; i < kPairMaxSegs; ++i) p->seg[i] = c.seg[i];
+  const int np = static_cast<int>(std::min<int64_t>(max_pairs, static_cast<int64_t>(p->m_pairs) * c.n_cols));
+  *pairs_out = np;
+  double worst = 0.0;
+  for (int pr = 0; pr < np; ++pr) {
+    PairWalk walk(*p, pr, np);
+    PairSlots slots;
+    PairTile t;
+    int last = -1, last_bn = 0;
+    double cost = 0.0;
+    while (walk.next(t)) {
+      int slot;
+      uint32_t phase;
+      slots.take(t.bn, slot, phase);
+      cost += static_cast<double>(k_steps) * (32.0 + t.bn / 8.0) / 56.0 + (slot == last ? 5.0 : 1.0);
+      last = slot;
+      last_bn = t.bn;
+    }
+    cost += 8.0 * last_bn / 256.0;
+    worst = std::max(worst, cost);
+  }
+  return worst;
+}
+
 bool pair_schedule(int64_t s, int64_t m, int64_t k_steps, int sm_count, PairParams* p, int* pairs) {
   const int64_t m_pairs = (s + 255) / 256;
   const int max_pairs = std::max(1, sm_count / 2);
+  if (m_pairs * ((m + 63) / 64) > INT32_MAX) return false;
   p->s = static_cast<int32_t>(s);
   p->m = static_cast<int32_t>(m);
   p->m_pairs = static_cast<int32_t>(m_pairs);
-  auto n_cols_of = [&](int w) -> int64_t {
-    if (w != 0) return (m + w - 1) / w;
-    const int64_t full = m / 448, rem = m % 448;
-    return 2 * full + (rem == 0 ? 0 : (rem <= 256 ? 1 : 2));
-  };
-  int best_w = -1;
-  double best_cost = 1e30;
   const int force_bn = g_force_bn.load(std::memory_order_relaxed);
-  const int cand[5] = {0, 256, 192, 128, 64};
+  const bool forced = force_bn == 64 || force_bn == 128 || force_bn == 192 || force_bn == 256 || force_bn == 448;
+  PairSched best{};
+  double best_cost = 1e30;
+  auto consider = [&](const PairSched& c) {
+    // every column must start inside the layer and the columns must reach its edge
+    const PairSeg& l = c.seg[c.n_segs - 1];
+    const int64_t end = l.n0 + seg_span(l.wa, l.wb, l.cols);
+    const int64_t last_w = (l.cols & 1) ? l.wa : l.wb;
+    if (end < m || end - last_w >= m) return;
+    int np;
+    const double cost = sched_cost(c, p, k_steps, max_pairs, &np);
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = c; best.pairs = np; }
+  };
+  // columns all equally wide, or 256 and 192 alternating
+  const int uniform[5] = {0, 256, 192, 128, 64};
   for (int ci = 0; ci < 5; ++ci) {
-    const int w = cand[ci];
-    const bool forced = force_bn == 64 || force_bn == 128 || force_bn == 192 || force_bn == 256 || force_bn == 448;
+    const int w = uniform[ci];
     if (forced ? (force_bn == 448 ? w != 0 : w != force_bn) : w == 64) continue;  // 64: only when forced
-    const int64_t n_cols = n_cols_of(w);
-    if (m_pairs * n_cols > INT32_MAX) return false;
-    p->tile_w = w;
-    p->n_cols = static_cast<int32_t>(n_cols);
-    const int np = static_cast<int>(std::min<int64_t>(max_pairs, m_pairs * n_cols));
-    double worst = 0.0;
-    for (int pr = 0; pr < np; ++pr) {
-      PairWalk walk(*p, pr, np);
-      PairSlots slots;
-      PairTile t;
-      int last = -1;
-      double cost = 0.0;
-      while (walk.next(t)) {
-        int slot;
-        uint32_t phase;
-        slots.take(t.bn, slot, phase);
-        cost += static_cast<double>(k_steps) * (32.0 + t.bn / 8.0) / 56.0 + (slot == last ? 8.0 : 1.0);
-        last = slot;
-      }
-      worst = std::max(worst, cost);
+    PairSched c{};
+    if (w != 0) {
+      sched_add(&c, w, w, (m + w - 1) / w);
+    } else {
+      const int64_t full = m / 448, rem = m % 448;
+      sched_add(&c, 256, 192, 2 * full + (rem == 0 ? 0 : (rem <= 256 ? 1 : 2)));
     }
-    if (worst < best_cost - 1e-9) { best_cost = worst; best_w = w; }
+    consider(c);
   }
-  if (best_w < 0) return false;
-  p->tile_w = best_w;
-  p->n_cols = static_cast<int32_t>(n_cols_of(best_w));
-  *pairs = static_cast<int>(std::min<int64_t>(max_pairs, m_pairs * p->n_cols));
+  if (!forced && force_bn != 1) {   // 1: only the uniform and alternating candidates above
+    // a columns of 256 and b of 192 (the last one as narrow as the edge allows), in three groups;
+    // with many tiles per pair the balance matters less and fewer splits are tried
+    const int64_t a_max = (m + 255) / 256;
+    const int64_t a_step = std::max<int64_t>(1, a_max * m_pairs / (24 * max_pairs));
+    for (int64_t a = 1; a < a_max; a += a_step) {
+      const int64_t rest = m - 256 * a;
+      if (rest <= 0) break;
+      const int64_t b = (rest + 191) / 192;
+      const int64_t cuts[7] = {0, 1, 2, 3, 4, 5, 6};
+      for (int ci = 0; ci < 7; ++ci) {
+        const int64_t a1 = a * cuts[ci] / 6, b1 = b * cuts[ci] / 6;
+        {
+          PairSched c{};
+          if (sched_add(&c, 256, 256, a1) && sched_add(&c, 192, 192, b) && sched_add(&c, 256, 256, a - a1)) consider(c);
+        }
+        if (ci > 0 && ci < 6) {
+          PairSched c{};
+          if (sched_add(&c, 192, 192, b1) && sched_add(&c, 256, 256, a) && sched_add(&c, 192, 192, b - b1)) consider(c);
+        }
+      }
+    }
+    // 256 and 192 alternating for the first 2c columns, then all 192 or all 256 to the edge
+    const int64_t c_max = m / 448;
+    const int64_t c_step = std::max<int64_t>(1, c_max * m_pairs / (24 * max_pairs));
+    for (int64_t cp = 1; cp <= c_max; cp += c_step) {
+      const int64_t rest = m - 448 * cp;
+      if (rest <= 0) break;
+      for (int w = 192; w <= 256; w += 64) {
+        PairSched c{};
+        if (sched_add(&c, 256, 192, 2 * cp) && sched_add(&c, w, w, (rest + w - 1) / w)) consider(c);
+        PairSched d{};
+        if (sched_add(&d, w, w, rest / w) && rest % w == 0 && sched_add(&d, 256, 192, 2 * cp)) consider(d);
+      }
+    }
+  }
+  if (best_cost >= 1e30) return false;
+  p->n_cols = best.n_cols;
+  p->n_segs = best.n_segs;
+  for (int i = 0; i < kPairMaxSegs; ++i) p->seg[i] = best.seg[i];
+  *pairs = best.pairs;
+  return true;
+}
+
+// The same, remembered per prepared weight and token count (the search walks a few hundred
+// candidates; a layer is called with few distinct token counts).
+bool pair_schedule_cached(const batq_weight* w, int64_t s, int sm_count, PairParams* p, int* pairs) {
+  const int force_bn = g_force_bn.load(std::memory_order_relaxed);
+  {
+    std::lock_guard<std::mutex> lock(w->sched_mutex);
+    for (const auto& e : w->sched_cache)
+      if (e.s == s && e.force_bn == force_bn) {
+        p->s = static_cast<int32_t>(s);
+        p->m = static_cast<int32_t>(w->m);
+        p->m_pairs = static_cast<int32_t>((s + 255) / 256);
+        p->n_cols = e.n_cols;
+        p->n_segs = e.n_segs;
+        for (int i = 0; i < kPairMaxSegs; ++i) p->seg[i] = e.seg[i];
+        *pairs = e.pairs;
+        return true;
+      }
+  }
+  if (!pair_schedule(s, w->m, (w->n + 255) / 256, sm_count, p, pairs)) return false;
+  batq_weight::SchedEntry e{};
+  e.s = s; e.force_bn = force_bn; e.n_cols = p->n_cols; e.n_segs = p->n_segs; e.pairs = *pairs;
+  for (int i = 0; i < kPairMaxSegs; ++i) e.seg[i] = p->seg[i];
+  std::lock_guard<std::mutex> lock(w->sched_mutex);
+  if (w->sched_cache.size() >= 16) w->sched_cache.erase(w->sched_cache.begin());
+  w->sched_cache.push_back(e);
   return true;
 }
 
@@ -575,7 +695,7 @@ batq_status launch_gemm_pair(const void* x_codes, const void* x_sf, const batq_w
   if (st != BATQ_OK) return st;
   PairParams p{};
   int pairs = 0;
-  if (!pair_schedule(s, w->m, (w->n + 255) / 256, sm_count, &p, &pairs)) return BATQ_ERR_SHAPE;
+  if (!pair_schedule_cached(w, s, sm_count, &p, &pairs)) return BATQ_ERR_SHAPE;
   p.katoms = w->katoms;
   p.k_steps = static_cast<int32_t>((w->n + 255) / 256);
   p.m16 = static_cast<int32_t>(m16);
@@ -899,7 +1019,7 @@ batq_status launch_linear_prefill_fused(const batq_transform* t, const batq_weig
   if (st != BATQ_OK) return st;
   PrefillFusedParams q{};
   int pairs = 0;
-  if (!pair_schedule(s, w->m, (n + 255) / 256, info->sm_count, &q.g, &pairs)) return BATQ_ERR_SHAPE;
+  if (!pair_schedule_cached(w, s, info->sm_count, &q.g, &pairs)) return BATQ_ERR_SHAPE;
   q.g.katoms = w->katoms;
   q.g.k_steps = static_cast<int32_t>((n + 255) / 256);
   q.g.m16 = static_cast<int32_t>(m16);
@@ -1468,13 +1588,13 @@ batq_status batq_debug_wait_timeout(int64_t limit_ns, void* stream) {
   return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
 }
 
-batq_status batq_debug_mma_peak(int32_t pair, int32_t bn, int32_t iters, double* flops_out, void* stream) {
+batq_status batq_debug_mma_peak(int32_t pair, int32_t bn, int32_t iters, int32_t sf_copies, double* flops_out, void* stream) {
   if (bn != 64 && bn != 128 && bn != 192 && bn != 256) return BATQ_ERR_SHAPE;
   if (iters <= 0 || iters > (1 << 24)) return BATQ_ERR_SHAPE;
   const DeviceInfo* info;
   batq_status st = device_setup(nullptr, &info);
   if (st != BATQ_OK) return st;
-  PeakParams p{iters, bn};
+  PeakParams p{iters, bn, sf_copies ? 1 : 0};
   const int ctas = pair ? (info->sm_count / 2) * 2 : info->sm_count;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(static_cast<unsigned>(ctas));

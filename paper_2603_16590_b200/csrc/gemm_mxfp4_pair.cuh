@@ -18,11 +18,15 @@
 // any time the pairs work on a few neighbouring columns and all row blocks, in step along K, so
 // every weight tile is requested by many pairs at once and every activation tile by the others
 // -- measured, that sharing in L2 is worth a quarter of the throughput against a distribution in
-// which each pair walks its own stretch of a row.  The columns are all tile_w wide (64, 128, 192
-// or 256), or alternately 256 and 192 wide ("mixed", 224 on average); the host picks by a wave
-// model.  The last column is as narrow as the layer's edge allows.  Every column starts at a
-// multiple of 64 features: the MMA takes the weight scales from an even column of tensor memory
-// only (one column = 32 weight rows; an odd one raises a misaligned-address fault).
+// which each pair walks its own stretch of a row.  Column widths come in up to kPairMaxSegs
+// segments of consecutive columns; inside a segment the columns are all equally wide (64, 128,
+// 192 or 256) or alternately wa and wb wide (256 and 192: 224 on average).  The host picks the
+// segments by walking candidates through a cost model, so that the pairs' last tiles end together
+// (e.g. 6144 features at 2048 tokens: nine columns of 256, twelve of 192, six of 256 give every
+// pair at most three tiles and never two 256-wide ones in a row).  The last column is as narrow
+// as the layer's edge allows.  Every column starts at a multiple of 64 features: the MMA takes
+// the weight scales from an even column of tensor memory only (one column = 32 weight rows; an
+// odd one raises a misaligned-address fault).
 //
 // Accumulators live in two slots of tensor memory, columns [0, 256) and [256, 448).  A tile wider
 // than 192 needs slot 0; a narrower one takes the slot the tile before it did not use, so that
@@ -48,6 +52,7 @@ namespace batq {
 
 constexpr int kPairThreads = 192;
 constexpr int kPairUnitCols = 64;   // output features per scheduling unit
+constexpr int kPairMaxSegs = 4;     // segments of columns with one width pattern each
 
 struct PairCfg {
   static constexpr int kABytes = kBM * kBKBytes;          // 16 KiB: this CTA's 128 token rows
@@ -71,14 +76,21 @@ struct PairCfg {
   static_assert(kStageBytes % 1024 == 0, "stage alignment");
 };
 
+// Columns [col0, col0 + cols) of tiles: they start at feature n0 and are alternately wa and wb wide
+// (wa == wb: all equally wide).
+struct PairSeg {
+  int32_t col0, cols, n0;
+  int16_t wa, wb;
+};
 struct PairParams {
   int32_t s;              // rows of X (tokens)
   int32_t m;              // rows of W (output features)
   int32_t katoms;         // KA = 2*ceil(k/8): 512-byte scale atoms per 128-row tile
   int32_t k_steps;        // ceil(n / 256)
   int32_t m_pairs;        // ceil(s / 256)
-  int32_t tile_w;         // column width: 64, 128, 192 or 256; 0 = mixed (256, 192, 256, 192, ...)
   int32_t n_cols;         // columns of tiles
+  int32_t n_segs;         // segments in use
+  PairSeg seg[kPairMaxSegs];
   int32_t m16;            // as in GemmParams: columns covered by the TMA store
   void* y;
   int64_t ldy;
@@ -91,21 +103,21 @@ struct PairTile {
   int bn;    // width: the column's, less (a multiple of 64) in the last column
 };
 struct PairWalk {
-  int tile, total, step, m_pairs, tile_w, m;
-  __host__ __device__ __forceinline__ PairWalk(const PairParams& p, int pair, int n_pairs)
-      : tile(pair), total(p.m_pairs * p.n_cols), step(n_pairs), m_pairs(p.m_pairs), tile_w(p.tile_w), m(p.m) {}
+  const PairParams* p;
+  int tile, total, step;
+  __host__ __device__ __forceinline__ PairWalk(const PairParams& params, int pair, int n_pairs)
+      : p(&params), tile(pair), total(params.m_pairs * params.n_cols), step(n_pairs) {}
   __host__ __device__ __forceinline__ bool next(PairTile& t) {
     if (tile >= total) return false;
-    const int nt = tile / m_pairs;
-    t.mp = tile - nt * m_pairs;
-    int w = tile_w;
-    if (tile_w == 0) {  // mixed: columns 2c and 2c + 1 share 448 features, 256 + 192
-      t.n0 = (nt >> 1) * 448 + (nt & 1) * 256;
-      w = (nt & 1) ? 192 : 256;
-    } else {
-      t.n0 = nt * tile_w;
-    }
-    const int rem = m - t.n0;
+    const int nt = tile / p->m_pairs;
+    t.mp = tile - nt * p->m_pairs;
+    int sg = 0;
+    while (sg + 1 < p->n_segs && nt >= p->seg[sg + 1].col0) ++sg;
+    const PairSeg& g = p->seg[sg];
+    const int i = nt - g.col0;
+    t.n0 = g.n0 + (i >> 1) * (g.wa + g.wb) + (i & 1) * g.wa;
+    const int w = (i & 1) ? g.wb : g.wa;
+    const int rem = p->m - t.n0;
     t.bn = rem >= w ? w : ((rem + 63) / 64) * 64;
     tile += step;
     return true;
@@ -126,7 +138,7 @@ template <bool OUT_BF16>
 __global__ void __launch_bounds__(kPairThreads, 1)
 gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b32,
                        const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfb,
-                       const __grid_constant__ CUtensorMap tmap_y, const PairParams p) {
+                       const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ PairParams p) {
   using Cfg = PairCfg;
   extern __shared__ uint8_t pair_smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[Cfg::kStages];   // used in the leader only

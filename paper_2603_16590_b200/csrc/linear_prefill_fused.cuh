@@ -123,7 +123,7 @@ linear_prefill_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                             const __grid_constant__ CUtensorMap tmap_codes, const __grid_constant__ CUtensorMap tmap_a,
                             const __grid_constant__ CUtensorMap tmap_b32, const __grid_constant__ CUtensorMap tmap_sfa,
                             const __grid_constant__ CUtensorMap tmap_sfb, const __grid_constant__ CUtensorMap tmap_y,
-                            const PrefillFusedParams q) {
+                            const __grid_constant__ PrefillFusedParams q) {
   using Cfg = PairCfg;
   const PairParams& p = q.g;
   extern __shared__ uint8_t pf_smem_raw[];

@@ -19,8 +19,9 @@ constexpr int kPeakSmemBytes = kPeakABytes + kPeakBBytes + kPeakSfBytes + 1024;
 constexpr int kPeakSfCols = 8 + 2 * 4 * kPeakSfbAtoms;
 
 struct PeakParams {
-  int32_t iters;   // K-steps (four MMAs of K = 64 each)
-  int32_t bn;      // tile width
+  int32_t iters;      // K-steps (four MMAs of K = 64 each)
+  int32_t bn;         // tile width
+  int32_t sf_copies;  // 0: scale factors copied to tensor memory once; 1: again before every K-step, as a GEMM must
 };
 
 // PAIR = false: every CTA issues tcgen05.mma.cta_group::1 on a 128 x bn tile.
@@ -103,6 +104,23 @@ __global__ void __launch_bounds__(kPeakThreads, 1) mma_peak_kernel(const PeakPar
       if (elect_one()) {
         const int k1 = min(p.iters, (b + 1) * kPeakBatch);
         for (int kt = b * kPeakBatch; kt < k1; ++kt) {
+          if (p.sf_copies) {
+            if (PAIR) {
+              tc_cp_32x128b_warpx4_pair(sfa_col, sfd);
+              tc_cp_32x128b_warpx4_pair(sfa_col + 4, sfd + 32);
+            } else {
+              tc_cp_32x128b_warpx4(sfa_col, sfd);
+              tc_cp_32x128b_warpx4(sfa_col + 4, sfd + 32);
+            }
+#pragma unroll
+            for (int rt = 0; rt < kPeakSfbAtoms; ++rt)
+#pragma unroll
+              for (int c = 0; c < 2; ++c) {
+                const uint32_t col = sfa_col + 8 + c * 4 * kPeakSfbAtoms + 4 * rt;
+                const uint64_t src = sfd + ((1024 + rt * 1024 + c * 512) >> 4);
+                if (PAIR) tc_cp_32x128b_warpx4_pair(col, src); else tc_cp_32x128b_warpx4(col, src);
+              }
+          }
 #pragma unroll
           for (int kb = 0; kb < 4; ++kb) {
             const uint32_t c = kb >> 1;

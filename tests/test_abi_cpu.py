@@ -83,8 +83,8 @@ def test_host_validation_without_a_device(lib):
     assert lib.batq_linear_workspace_bytes(None, 4) == 0
     assert lib.batq_linear_kernel_launches(None, None, 4) == 0
     assert lib.batq_weight_destroy(None) == 0 and lib.batq_transform_destroy(None) == 0
-    assert lib.batq_debug_mma_peak(0, 100, 10, None, None) == 2
-    assert lib.batq_debug_mma_peak(0, 256, 0, None, None) == 2
+    assert lib.batq_debug_mma_peak(0, 100, 10, 0, None, None) == 2
+    assert lib.batq_debug_mma_peak(0, 256, 0, 0, None, None) == 2
 
 
 def test_debug_hooks_are_not_in_the_public_header():

@@ -1,10 +1,10 @@
 """Host logic of the CTA-pair GEMM: its work distribution, checked without a GPU.
 
 Tiles are numbered column of tiles after column and pair p of P takes tiles p, p + P, ...  The
-columns are all equally wide or alternately 256 and 192 wide.  The tiles of all pairs together
-must cover the s x m output exactly once, every column must start at a multiple of 64 features
-(the MMA cannot take weight scales from an odd 32-row group), only the last column may be narrower
-than its nominal width, and no pair may have more than one tile more than another."""
+columns come in a few segments, each all equally wide or alternately 256 and 192 wide.  The tiles
+of all pairs together must cover the s x m output exactly once, every column must start at a
+multiple of 64 features (the MMA cannot take weight scales from an odd 32-row group), only the
+last column may be ragged, and no pair may have more than one tile more than another."""
 import numpy as np
 import pytest
 
@@ -34,11 +34,11 @@ def _check(sched, s, m):
         for i, (mp, n0, bn) in enumerate(tiles):
             assert index[n0] * rows + mp == p + i * len(sched)
     body = widths[:-1]
-    uniform = len(set(body)) <= 1
-    mixed = all(w == (256 if k % 2 == 0 else 192) for k, w in enumerate(body))
-    assert uniform or mixed
-    nominal = (256 if (len(widths) - 1) % 2 == 0 else 192) if (mixed and not uniform) else (body[0] if body else widths[-1])
-    assert widths[-1] <= nominal and starts[-1] + widths[-1] >= m > starts[-1] + widths[-1] - 64
+    assert all(w in (64, 128, 192, 256) for w in body)
+    # a handful of segments: the width pattern changes rarely
+    changes = sum(1 for k in range(2, len(body)) if body[k] != body[k - 2])
+    assert changes <= 8
+    assert starts[-1] + widths[-1] >= m > starts[-1] + widths[-1] - 64
     counts = [len(t) for t in sched]
     assert max(counts) - min(counts) <= 1
     return widths
@@ -72,9 +72,25 @@ def test_bad_arguments():
     assert lib.batq_debug_pair_schedule(256, 128, 128, 148, 999, None, 0) == 0
 
 
-def test_width_follows_the_wave_model():
-    """Llama-8B prefill shapes at 2048 tokens on 74 pairs."""
-    w = lambda s, m, n: sorted({t[2] for tiles in B.batq_debug_pair_schedule(s, m, n) for t in tiles})
-    assert w(2048, 28672, 4096) == [192, 256]      # mixed: 1024 tiles = 13.8 waves instead of 16.2 of 192
-    assert w(2048, 4096, 14336) == [256]           # 2 tiles per pair however cut; the widest move least through L2
-    assert w(2048, 6144, 4096) == [192]
+def test_forced_single_pattern():
+    """Width 1 = the automatic choice among single-pattern schedules (all columns equally wide, or 256
+    and 192 alternating)."""
+    B.batq_debug_force_tile_width(1)
+    try:
+        for s, m, n in SHAPES[:8]:
+            widths = _check(B.batq_debug_pair_schedule(s, m, n), s, m)
+            body = widths[:-1]
+            assert len(set(body)) <= 1 or all(w == (256 if k % 2 == 0 else 192) for k, w in enumerate(body))
+    finally:
+        B.batq_debug_force_tile_width(0)
+
+
+def test_schedule_ends_the_pairs_together():
+    """Llama-8B prefill shapes at 2048 tokens on 74 pairs: 6144 features are cut so that no pair has
+    more than three tiles (four 192-wide ones otherwise) and none works on two 256-wide tiles in a
+    row (they would share one accumulator slot)."""
+    sched = B.batq_debug_pair_schedule(2048, 6144, 4096)
+    assert max(len(t) for t in sched) == 3
+    for tiles in sched:
+        assert all(not (a[2] == 256 and b[2] == 256) for a, b in zip(tiles, tiles[1:]))
+    assert sum(t[2] for tiles in sched for t in tiles) == 8 * 6144
