@@ -43,12 +43,17 @@ WORKLOADS = {
     "cfg3_qwen2vl7b_prefill": ("prefill", [8192], synth.QWEN2VL7B_PREFILL, 0.75, 0.005),
     "cfg4_quantizer_sweep": ("quant", [1024, 8192, 32768], [("h2048", 2048, 0), ("h4096", 4096, 0), ("h8192", 8192, 0)],
                              0.0, 0.01),
+    # the W4A8 settings (MXFP8 activations x MXFP4 weights) on the config-1 shapes
+    "cfg1_llama8b_prefill_w4a8": ("prefill", [2048], synth.LLAMA8B_PREFILL, 0.0, 0.01),
     # single-kernel cases for profiler captures (inputs larger than L2, a few hundred MB on the device)
     "profile_gemm_gate_up": ("prefill", [2048], [("gate_up", 4096, 28672)], 0.0, 0.01),
     "profile_gemm_down": ("prefill", [2048], [("down", 14336, 4096)], 0.0, 0.01),
     "profile_quant_32768x4096": ("quant", [32768], [("h4096", 4096, 0)], 0.0, 0.01),
     "profile_decode_gate_up": ("decode", [16], [("gate_up", 4096, 28672)] * 4, 0.0, 0.01),
 }
+
+A8_WORKLOADS = {"cfg1_llama8b_prefill_w4a8"}   # activations quantised to MXFP8 (E4M3), GEMM on kind::mxf8f6f4
+FP8_OVER_BF16 = 2.0       # nominal dense peak ratio 4.5 / 2.25 PFLOP/s
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, MB per step = the four GEMM launches of
 # cfg1_llama8b_prefill) from the ncu capture summarised under profiles/, valid for the kernel source
@@ -81,6 +86,8 @@ def workload_config(workload):
     cfg = {"workload": workload, "tokens": tokens[0] if kind == "prefill" else tokens,
            "projections": [list(p) for p in projs],
            "transform": "shared 4x4 (x) private 8x8 per 32-group, clip U[0.8,1]"}
+    if workload in A8_WORKLOADS:
+        cfg["activations"] = "MXFP8 (E4M3), weights MXFP4"
     if kind == "prefill":
         S = tokens[0]
         touched = sum(S * n * 2 + S * m * 2 + n * m * WEIGHT_BYTES_PER_ELEM for _, n, m in projs)
@@ -179,6 +186,9 @@ def oracle_sample(workload, seed, rows, feats):
     qw = O.prepare_weight(wb, t.left, t.right)
 
     def step():
+        if workload in A8_WORKLOADS:
+            qx = O.quantize_act_mxfp8(xb, t.left, t.right, t.clip_lo, t.clip_hi)
+            return O.gemm_mxfp8_mxfp4(qx[0], qx[1], qw[0], qw[1])[0]
         qx = O.quantize_act(xb, t.left, t.right, t.clip_lo, t.clip_hi)
         return O.gemm_mxfp4(qx[0], qx[1], qw[0], qw[1])[0]
 
@@ -466,17 +476,25 @@ def run_ours(args):
 
     if kind == "prefill":
         S = tokens[0]
+        a8 = args.workload in A8_WORKLOADS
+        # the three calls of the path, in the 4-bit or the 8-bit activation format
+        f_linear = B.batq_linear_w4a8 if a8 else B.batq_linear_w4a4
+        f_quant = B.batq_quantize_act_mxfp8 if a8 else B.batq_quantize_act
+        f_gemm = B.batq_gemm_mxfp8_mxfp4 if a8 else B.batq_gemm_mxfp4
+        f_ws = B.batq_linear_w4a8_workspace_bytes if a8 else B.batq_linear_workspace_bytes
+        if a8:
+            line["metric"], line["dtype"] = "w4a8_linear_tflops", "mxfp8 x mxfp4"
         layers = make_layer_inputs(args.workload, S, seed)
         for L in layers:
             L["tr"] = mk_transform(L)
             L["x"] = B.bits_to_cuda_bf16(L["x_bits"])
-            L["codes"] = torch.empty((S, L["n"] // 2), dtype=torch.uint8, device="cuda")
+            L["codes"] = torch.empty((S, L["n"] if a8 else L["n"] // 2), dtype=torch.uint8, device="cuda")
             L["sf"] = torch.empty(B.batq_sf_bytes(S, L["n"], B.SF_MMA), dtype=torch.uint8, device="cuda")
             wdev = B.bits_to_cuda_bf16(synth.make_weight(L["m"], L["n"], L["w_seed"]))
             L["w"] = B.batq_prepare_weight(L["tr"], wdev)
             del wdev
             L["y"] = torch.empty((S, L["m"]), dtype=torch.bfloat16, device="cuda")
-            L["ws"] = B.aligned_workspace(B.batq_linear_workspace_bytes(L["w"], S))
+            L["ws"] = B.aligned_workspace(f_ws(L["w"], S))
             L["x_host"] = torch.from_numpy(L["x_bits"].view(np.int16)).pin_memory()
             L["y_host"] = torch.empty((S, L["m"]), dtype=torch.bfloat16).pin_memory()
         torch.cuda.synchronize()
@@ -492,12 +510,12 @@ def run_ours(args):
             m = marks.get(k)
             for i, L in enumerate(layers):
                 if m is None:
-                    B.batq_linear_w4a4(L["tr"], L["w"], L["x"], L["y"], L["ws"])
+                    f_linear(L["tr"], L["w"], L["x"], L["y"], L["ws"])
                     continue
                 m[i][0].record()
-                B.batq_quantize_act(L["tr"], L["x"], L["codes"], L["sf"], B.SF_MMA)
+                f_quant(L["tr"], L["x"], L["codes"], L["sf"], B.SF_MMA)
                 m[i][1].record()
-                B.batq_gemm_mxfp4(L["codes"], L["sf"], L["w"], S, L["y"])
+                f_gemm(L["codes"], L["sf"], L["w"], S, L["y"])
                 m[i][2].record()
 
         ms, clocks = timed_region(h, step, steps, args.warmup)
@@ -537,16 +555,22 @@ def run_ours(args):
 
         b2b = []
         for L in layers:
-            gg, r = graph_of(lambda L=L: B.batq_gemm_mxfp4(L["codes"], L["sf"], L["w"], S, L["y"]))
-            gq, _ = graph_of(lambda L=L: B.batq_quantize_act(L["tr"], L["x"], L["codes"], L["sf"], B.SF_MMA))
+            gg, r = graph_of(lambda L=L: f_gemm(L["codes"], L["sf"], L["w"], S, L["y"]))
+            gq, _ = graph_of(lambda L=L: f_quant(L["tr"], L["x"], L["codes"], L["sf"], B.SF_MMA))
             b2b.append((time_graph(gq, r), time_graph(gg, r)))
-        mma_only = measure_mma_peak(B, torch, 20000) if S > 128 else None
-        big_quant = measure_big_quantizer(B, torch, seed) if (S > 128 and h.rank == 0) else None
+        mma_only = measure_mma_peak(B, torch, 20000) if (S > 128 and not a8) else None
+        big_quant = measure_big_quantizer(B, torch, seed) if (S > 128 and h.rank == 0 and not a8) else None
 
         # end to end: host buffers in and out through the C-ABI host entry point
         def step_host():
             for L in layers:
-                B.batq_linear_w4a4_host(L["tr"], L["w"], L["x_host"], L["y_host"], L["x"], L["y"], L["ws"])
+                if a8:   # no host entry point for the 8-bit format: the same copies around the device call
+                    L["x"].copy_(L["x_host"].view(torch.bfloat16), non_blocking=True)
+                    f_linear(L["tr"], L["w"], L["x"], L["y"], L["ws"])
+                    L["y_host"].copy_(L["y"], non_blocking=True)
+                    torch.cuda.synchronize()
+                else:
+                    B.batq_linear_w4a4_host(L["tr"], L["w"], L["x_host"], L["y_host"], L["x"], L["y"], L["ws"])
 
         e2e_steps = max(1, min(steps, 5))
         for _ in range(2):
@@ -562,11 +586,11 @@ def run_ours(args):
 
         gemm_flops = [2.0 * S * L["n"] * L["m"] for L in layers]
         gemm_achieved = sum(gemm_flops) / (g_ms.sum() * 1e-3) / 1e12
-        q_bytes = [S * L["n"] * QUANT_BYTES_PER_ELEM for L in layers]
+        q_bytes = [S * L["n"] * (3.03125 if a8 else QUANT_BYTES_PER_ELEM) for L in layers]
         quant_gbs = sum(q_bytes) / (q_ms.sum() * 1e-3) / 1e9
         sustained = ms >= 500.0   # a timed region this long runs under the power cap
         bf16_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
-        fp4_peak = bf16_peak * FP4_OVER_BF16
+        fp4_peak = bf16_peak * (FP8_OVER_BF16 if a8 else FP4_OVER_BF16)   # the 8-bit-container MMA runs at the FP8 rate
         traffic = None
         if GEMM_TRAFFIC["workload"] == args.workload and GEMM_TRAFFIC["source_sha256"] == kernel_source_hash():
             traffic = GEMM_TRAFFIC["mb_per_step"]
@@ -575,18 +599,20 @@ def run_ours(args):
         # context: the vendor's dense-FP4 figure scaled to the SM clock sampled during the timed region
         mhz = (clocks or {}).get("sm_mhz") or 0.0
         mhz_max = (clocks or {}).get("sm_max_mhz") or 0.0
-        nominal_at_clock = NOMINAL_FP4_TFLOPS * mhz / mhz_max if mhz and mhz_max else None
-        roof = {"bound": "tensor", "kernel": "gemm_mxfp4_pair_kernel" if S > 128 else "gemm_mxfp4_kernel",
+        nominal_at_clock = (NOMINAL_FP4_TFLOPS / 2 if a8 else NOMINAL_FP4_TFLOPS) * mhz / mhz_max if mhz and mhz_max else None
+        nominal_peak = NOMINAL_FP4_TFLOPS / 2 if a8 else NOMINAL_FP4_TFLOPS
+        roof = {"bound": "tensor", "kernel": "gemm_w4a8_kernel" if a8 else ("gemm_mxfp4_pair_kernel" if S > 128 else "gemm_mxfp4_kernel"),
                 "achieved": gemm_achieved, "peak": fp4_peak,
                 "events": "around every launch in every %dth step of the timed region (%d steps) and in %d more steps "
                           "right after it" % (EVENT_EVERY, len(sampled), extra),
                 "unit": "TFLOP/s", "frac": gemm_achieved / fp4_peak, "traffic": traffic,
                 "traffic_unit": "MB per step (4 launches)" if traffic else None,
-                "peak_source": "%s cuBLAS bf16 %s x %.0f (nominal fp4:bf16 ratio): a proxy that inherits cuBLAS's own "
-                               "efficiency" % (peaks["source"], "sustained" if sustained else "burst", FP4_OVER_BF16),
+                "peak_source": "%s cuBLAS bf16 %s x %.0f (nominal %s:bf16 ratio): a proxy that inherits cuBLAS's own "
+                               "efficiency" % (peaks["source"], "sustained" if sustained else "burst",
+                                               FP8_OVER_BF16 if a8 else FP4_OVER_BF16, "fp8" if a8 else "fp4"),
                 "back_to_back": {"achieved": b2b_gemm, "frac": b2b_gemm / fp4_peak,
                                  "how": "the same launches in a CUDA graph of 8 steps, no events between them"},
-                "nominal": {"peak": NOMINAL_FP4_TFLOPS, "frac": gemm_achieved / NOMINAL_FP4_TFLOPS,
+                "nominal": {"peak": nominal_peak, "frac": gemm_achieved / nominal_peak,
                             "peak_at_sampled_clock": nominal_at_clock,
                             "frac_at_sampled_clock": gemm_achieved / nominal_at_clock if nominal_at_clock else None,
                             "note": "vendor dense-FP4 figure; the 70 % target of the path is judged against this "

@@ -104,6 +104,32 @@ def transform_fast(X: np.ndarray, L: np.ndarray, R: np.ndarray) -> np.ndarray:
     return out.reshape(S, N)
 
 
+def round_to_bf16(v: np.ndarray) -> np.ndarray:
+    """Round real values (fp64) to the nearest bf16 value (8 significant bits, ties to even), as
+    fp64.  Written from the format: v = m * 2**e with m in [0.5, 1); keep 8 bits of m."""
+    v = np.asarray(v, dtype=np.float64)
+    m, e = np.frexp(v)
+    return np.ldexp(np.rint(m * 256.0) / 256.0, e)     # np.rint rounds halves to even
+
+
+def transform_fast_bf16(X: np.ndarray, L: np.ndarray, R: np.ndarray) -> np.ndarray:
+    """The two contractions of Algorithm 1 as the paper runs them (Sec. 3.2 keeps the
+    pre-quantization transforms in BF16): the result of each contraction is a bf16 tensor, i.e.
+    V R is rounded to bf16 before L^T is applied, and the output is rounded to bf16 again.  Each
+    contraction itself is exact here (a BF16 matmul accumulates wider than it stores)."""
+    L = np.asarray(L, dtype=np.float64)
+    R = np.asarray(R, dtype=np.float64)
+    S, N = X.shape
+    k = N // GROUP
+    gr, gc = L.shape[1], R.shape[1]
+    V = X.reshape(S, k, gr, gc)
+    out = np.empty_like(V)
+    for j in range(k):
+        U = round_to_bf16(V[:, j] @ _factor_for_block(R, j))
+        out[:, j] = round_to_bf16(np.einsum("ra,src->sac", _factor_for_block(L, j), U))
+    return out.reshape(S, N)
+
+
 # ----------------------------------------------------------------------------
 # Block-wise clipping: Eq. 3 / Eq. 4
 # ----------------------------------------------------------------------------
@@ -297,22 +323,25 @@ def dequantize(codes: np.ndarray, scale_bytes: np.ndarray) -> np.ndarray:
 # ----------------------------------------------------------------------------
 # The three stages
 # ----------------------------------------------------------------------------
-def transform_clip(x_bits, L, R, c_lo=None, c_hi=None) -> np.ndarray:
+def transform_clip(x_bits, L, R, c_lo=None, c_hi=None, round_intermediate_bf16=False) -> np.ndarray:
     """Stage 1 in fp64: x~ = x P (dense form), then the block clip.  L / R may
-    be None for the identity transform (plain MXFP4 of X)."""
+    be None for the identity transform (plain MXFP4 of X).  round_intermediate_bf16: the
+    transform as the paper's BF16 implementation computes it (transform_fast_bf16)."""
     X = bf16_bits_to_f64(x_bits)
     k = X.shape[1] // GROUP
-    if L is not None:
+    if L is not None and round_intermediate_bf16:
+        X = transform_fast_bf16(X, L, R)
+    elif L is not None:
         X = transform_dense(X, block_matrices(L, R, k))
     if c_lo is not None:
         X = block_clip(X, c_lo, c_hi)
     return X
 
 
-def quantize_act(x_bits, L, R, c_lo=None, c_hi=None):
+def quantize_act(x_bits, L, R, c_lo=None, c_hi=None, round_intermediate_bf16=False):
     """Stages 1+2 (transform -> clip -> Q, the order of the paper's algorithm
     flow).  Returns (codes [S, N] unpacked, scale_bytes [S, k])."""
-    return mxfp4_quantize(transform_clip(x_bits, L, R, c_lo, c_hi))
+    return mxfp4_quantize(transform_clip(x_bits, L, R, c_lo, c_hi, round_intermediate_bf16))
 
 
 def invert_blocks(P: np.ndarray) -> np.ndarray:

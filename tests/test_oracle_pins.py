@@ -411,3 +411,44 @@ def test_w4a8_layer_is_closer_to_fp_than_w4a4():
     assert np.linalg.norm(y8 - ref) < np.linalg.norm(y4 - ref)
     # unquantised activations would leave only the weight error: W4A8 must sit between the two
     assert np.linalg.norm(y8 - ref) / np.linalg.norm(ref) < 0.35
+
+
+def test_round_to_bf16_against_torch_and_the_format():
+    """An independent implementation of the same rounding: torch's float32 -> bfloat16 cast."""
+    import torch
+    rng = np.random.default_rng(21)
+    v = np.concatenate([rng.standard_normal(50000) * np.exp2(rng.integers(-40, 40, 50000)),
+                        np.array([0.0, -0.0, 1.0, 1.00390625, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -257.0, 255.5])])
+    v = v.astype(np.float32).astype(np.float64)
+    want = torch.from_numpy(v.astype(np.float32)).bfloat16().float().numpy().astype(np.float64)
+    got = O.round_to_bf16(v)
+    assert np.array_equal(got, want)
+    assert np.array_equal(O.round_to_bf16(got), got)                         # idempotent
+    assert O.round_to_bf16(np.array([1.0 + 2.0 ** -8]))[0] == 1.0            # tie -> even mantissa
+    assert O.round_to_bf16(np.array([1.0 + 3 * 2.0 ** -8]))[0] == 1.0 + 2.0 ** -6
+    bits = synth.f32_to_bf16_bits(v.astype(np.float32))                       # the input generator's own rounding agrees
+    assert np.array_equal(O.bf16_bits_to_f64(bits), got)
+
+
+def test_bf16_intermediate_transform_properties():
+    """With values that need no rounding (small integers, integer factors) the BF16 form equals the
+    exact transform; in general it differs from it by at most the two roundings (2^-8 relative each,
+    propagated through the second contraction)."""
+    rng = np.random.default_rng(22)
+    S, N = 5, 96
+    X = rng.integers(-3, 4, (S, N)).astype(np.float64)
+    L = rng.integers(-1, 2, (1, 4, 4)).astype(np.float64)
+    R = rng.integers(-1, 2, (3, 8, 8)).astype(np.float64)
+    assert np.array_equal(O.transform_fast_bf16(X, L, R), O.transform_fast(X, L, R))
+    t = synth.make_transform(N, 23, "baseline")
+    Xr = O.bf16_bits_to_f64(synth.make_activations(S, N, 23))
+    exact = O.transform_fast(Xr, t.left, t.right)
+    got = O.transform_fast_bf16(Xr, t.left, t.right)
+    assert np.array_equal(O.round_to_bf16(got), got)                          # the output is a bf16 tensor
+    Vb = np.abs(Xr).reshape(S, 3, 4, 8)
+    bound = np.zeros_like(Vb)
+    for j in range(3):
+        U = Vb[:, j] @ np.abs(t.right[j].astype(np.float64))
+        bound[:, j] = np.einsum("ra,src->sac", np.abs(t.left[0].astype(np.float64)), U)
+    assert np.all(np.abs(got - exact) <= 2.0 ** -7 * bound.reshape(S, N) + 1e-300)
+    assert np.any(got != exact)
