@@ -76,6 +76,17 @@ batq_status batq_transform_create(batq_transform** out, int32_t n, int32_t gr, i
                                   const float* clip_lo, const float* clip_hi);
 batq_status batq_transform_destroy(batq_transform* t);
 
+/* Emulation of a BF16 implementation of the transform (Sec. 3.2 keeps the pre-quantization
+ * transforms in BF16; Algorithm 1 is two contractions, each of which then stores a bf16 tensor).
+ * on != 0: later calls with this transform round V R to bf16 before L^T is applied and round the
+ * result to bf16 again, then clip and quantise as usual; on == 0 (the default): fp32 throughout,
+ * nothing is rounded before the quantiser.  Needs the factored form, so only (gr, gc) = (4, 8)
+ * (else UNSUPPORTED) and only MXFP4 (batq_quantize_act_mxfp8 and batq_linear_w4a8 return
+ * UNSUPPORTED while it is on); the activation quantiser then always runs on the ALUs.  The
+ * offline weight side is not affected (it is computed in fp64).  Not thread-safe against calls
+ * that use the transform at the same time. */
+batq_status batq_transform_set_bf16_intermediates(batq_transform* t, int32_t on);
+
 /* Size in bytes of a scale-byte buffer for a [rows x n] tensor.
  *   BATQ_SF_ROWMAJOR: rows * k bytes, byte (row, j) at row*k + j.
  *   BATQ_SF_MMA: the layout the block-scaled tensor-core instruction reads.

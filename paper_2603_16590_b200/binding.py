@@ -28,6 +28,7 @@ SIGNATURES = {
     "batq_version": (C.c_int, []),
     "batq_transform_create": (C.c_int, [C.POINTER(_P), _I32, _I32, _I32, _P, _I64, _P, _I64, _P, _P]),
     "batq_transform_destroy": (C.c_int, [_P]),
+    "batq_transform_set_bf16_intermediates": (C.c_int, [_P, _I32]),
     "batq_sf_bytes": (_SZ, [_I64, _I64, _I32]),
     "batq_quantize_act": (C.c_int, [_P, _P, _I64, _I64, _I64, _P, _P, _I32, _P]),
     "batq_quantize_act_mxfp8": (C.c_int, [_P, _P, _I64, _I64, _I64, _P, _P, _I32, _P]),
@@ -137,6 +138,10 @@ class Transform:
 
 def batq_transform_create(n, left, right, clip_lo=None, clip_hi=None, gr=4, gc=8) -> Transform:
     return Transform(n, left, right, clip_lo, clip_hi, gr, gc)
+
+
+def batq_transform_set_bf16_intermediates(t: Transform, on: bool):
+    _check(load().batq_transform_set_bf16_intermediates(t.handle, 1 if on else 0), "batq_transform_set_bf16_intermediates")
 
 
 def batq_sf_bytes(rows, n, layout) -> int:

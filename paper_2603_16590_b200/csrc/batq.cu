@@ -35,6 +35,7 @@ struct batq_transform {
   int32_t n, k, gr, gc;
   int32_t left_stride, right_stride;  // 0 = shared
   bool has_clip;
+  bool bf16_mid;                      // the transform's two contractions store bf16 (emulation of a BF16 implementation)
   std::vector<float> left, right;     // host copies (for the inverse)
   float* d_left;                      // device copies (for the kernels)
   float* d_right;
@@ -366,9 +367,10 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
   // The ALU kernel is written for 4 x 8 factors; every other factorisation of 32 goes through the
   // tensor-core kernel, which only sees the dense block matrices.
   const bool only_tc = t != nullptr && (t->gr != 4 || t->gc != 8);
+  const bool mid = t != nullptr && t->bf16_mid;   // needs the factored form: the ALU kernels (4 x 8 only, checked when it is set)
   const bool small_path = n_zero_words > 0;  // in front of the small-s GEMM (its tickets to clear)
   const int force_q = g_force_quantizer.load(std::memory_order_relaxed);
-  const bool use_tc = only_tc || (!small_path && t != nullptr &&
+  const bool use_tc = only_tc || (!mid && !small_path && t != nullptr &&
                                   (force_q == 2 || (force_q == 0 && s > kSmallQuantAuto)));
   if (use_tc) {
     if (n_zero_words > 0 &&
@@ -399,6 +401,7 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
     q.debug_out = debug_out;
     q.zero_words = zero_words;
     q.n_zero_words = n_zero_words;
+    q.bf16_mid = mid ? 1 : 0;
     // Launched as a programmatic dependent of whatever precedes it on the stream (in a decode loop
     // the GEMM of the layer before): it is scheduled early and waits inside the kernel.
     cudaLaunchConfig_t cfg{};
@@ -440,6 +443,7 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
   p.debug_out = debug_out;
   p.zero_words = zero_words;
   p.n_zero_words = n_zero_words;
+  p.bf16_mid = mid ? 1 : 0;
   const int grid = static_cast<int>(std::min<int64_t>(info->sm_count, p.n_units));
   const bool xf = t != nullptr, cl = t != nullptr && t->has_clip, dbg = debug_out != nullptr;
 #define BATQ_QA(XF, CL, DB) quantize_act_kernel<XF, CL, DB><<<grid, kQaThreads, kQaSmemBytes, stream>>>(p)
@@ -921,7 +925,7 @@ int pick_fused_splits(int64_t m, int64_t n, int sm_count) {
 bool use_fused_small(const batq_transform* t, const batq_weight* w, int64_t s) {
   const int force_path = g_force_small_path.load(std::memory_order_relaxed);
   if (force_path == 1 || s > kFusedTok) return false;
-  if (t != nullptr && (t->gr != 4 || t->gc != 8)) return false;  // its in-kernel quantiser is the 4 x 8 form
+  if (t != nullptr && (t->gr != 4 || t->gc != 8 || t->bf16_mid)) return false;  // its in-kernel quantiser is the plain 4 x 8 form
   const int sp = pick_fused_splits(w->m, w->n, w->sm_count);
   if (sp == 0) return false;
   if (force_path == 2) return true;
@@ -988,7 +992,7 @@ inline size_t prefill_flag_bytes(const batq_weight* w) { return round_up(static_
 // Applies to what the CTA-pair GEMM takes (s > 128, m >= 192) with a transform whose scale atoms
 // come in pairs (k % 8 == 0: no padding atom to keep finite).
 bool fused_prefill_applies(const batq_transform* t, const batq_weight* w, int64_t s) {
-  return t != nullptr && s > 128 && w->m >= 192 && w->k % 8 == 0 &&
+  return t != nullptr && !t->bf16_mid && s > 128 && w->m >= 192 && w->k % 8 == 0 &&
          g_force_gemm_kernel.load(std::memory_order_relaxed) != 1 && g_force_quantizer.load(std::memory_order_relaxed) == 0;
 }
 bool use_fused_prefill(const batq_transform* t, const batq_weight* w, int64_t s) {
@@ -1176,6 +1180,7 @@ batq_status batq_transform_create(batq_transform** out, int32_t n, int32_t gr, i
   t->left_stride = static_cast<int32_t>(left_stride);
   t->right_stride = static_cast<int32_t>(right_stride);
   t->has_clip = clip_lo != nullptr;
+  t->bf16_mid = false;
   const size_t nl = static_cast<size_t>(left_stride ? t->k : 1) * gr * gr;
   const size_t nr = static_cast<size_t>(right_stride ? t->k : 1) * gc * gc;
   t->left.assign(left, left + nl);
@@ -1218,6 +1223,13 @@ batq_status batq_transform_create(batq_transform** out, int32_t n, int32_t gr, i
   return BATQ_OK;
 }
 
+batq_status batq_transform_set_bf16_intermediates(batq_transform* t, int32_t on) {
+  if (t == nullptr) return BATQ_ERR_NULL;
+  if (on != 0 && (t->gr != 4 || t->gc != 8)) return BATQ_ERR_UNSUPPORTED;
+  t->bf16_mid = on != 0;
+  return BATQ_OK;
+}
+
 batq_status batq_transform_destroy(batq_transform* t) {
   if (t == nullptr) return BATQ_OK;
   cudaFree(t->d_left);
@@ -1255,6 +1267,7 @@ batq_status batq_quantize_act_mxfp8(const batq_transform* t, const void* x_bf16,
   if (st != BATQ_OK) return st;
   if (t == nullptr) return BATQ_ERR_NULL;
   if (t->n != n) return BATQ_ERR_SHAPE;
+  if (t->bf16_mid) return BATQ_ERR_UNSUPPORTED;   // the 8-bit quantiser has the dense form only
   if (scale_layout != BATQ_SF_ROWMAJOR && scale_layout != BATQ_SF_MMA) return BATQ_ERR_UNSUPPORTED;
   if (s == 0) return BATQ_OK;
   if (codes == nullptr || scales == nullptr) return BATQ_ERR_NULL;
@@ -1427,7 +1440,7 @@ batq_status batq_linear_w4a8(const batq_transform* t, const batq_weight* w, cons
   batq_status st = check_x(x_bf16, s, w->n, ld);
   if (st != BATQ_OK) return st;
   if (t->n != w->n) return BATQ_ERR_SHAPE;
-  if (!w->has_u4) return BATQ_ERR_UNSUPPORTED;
+  if (!w->has_u4 || t->bf16_mid) return BATQ_ERR_UNSUPPORTED;
   if (s == 0) return BATQ_OK;
   if (y == nullptr || workspace == nullptr) return BATQ_ERR_NULL;
   st = check_y(y, y_dtype, ldy, w->m);

@@ -103,7 +103,8 @@ __device__ __forceinline__ void quad_load_factors(bool valid, const float* L, co
 // amax (the same in the four lanes).  Every lane of the warp calls this (shuffles inside); lanes
 // without an item pass valid = false and get zeros.  x is read after the wait for the previous grid.
 __device__ __forceinline__ void quad_transform_clip(const uint16_t* xrow, bool valid, bool xform, bool clip,
-                                                    const QuadFactors& f, int lane, float (&o)[8], float& amax) {
+                                                    const QuadFactors& f, int lane, float (&o)[8], float& amax,
+                                                    bool bf16_mid = false) {
   grid_dependency_wait();
   uint4 q = make_uint4(0u, 0u, 0u, 0u);
   if (valid) q = ld_global_ordered_v4(xrow);
@@ -121,7 +122,7 @@ __device__ __forceinline__ void quad_transform_clip(const uint16_t* xrow, bool v
       float acc = v[0] * f.R[c];
 #pragma unroll
       for (int cc = 1; cc < 8; ++cc) acc = fmaf(v[cc], f.R[cc * 8 + c], acc);
-      U[c] = acc;
+      U[c] = bf16_mid ? round_bf16(acc) : acc;   // a BF16 implementation stores V R as bf16
     }
     const int base = lane & ~3;
 #pragma unroll
@@ -129,7 +130,7 @@ __device__ __forceinline__ void quad_transform_clip(const uint16_t* xrow, bool v
       float acc = f.Lc[0] * __shfl_sync(0xFFFFFFFFu, U[c], base);
 #pragma unroll
       for (int i = 1; i < 4; ++i) acc = fmaf(f.Lc[i], __shfl_sync(0xFFFFFFFFu, U[c], base + i), acc);
-      o[c] = acc;
+      o[c] = bf16_mid ? round_bf16(acc) : acc;
     }
   } else {
 #pragma unroll
@@ -193,6 +194,7 @@ struct QuantSmallParams {
   float* debug_out;      // [s x n] fp32 (DEBUG_OUT builds)
   uint32_t* zero_words;  // optional: n_zero_words 32-bit words set to zero
   int32_t n_zero_words;
+  int32_t bf16_mid;      // != 0: both contractions of the transform store their result as bf16
 };
 
 template <bool DEBUG_OUT>
@@ -211,7 +213,8 @@ __global__ void __launch_bounds__(128) quantize_act_small_kernel(const QuantSmal
                     xform ? p.right + static_cast<int64_t>(j) * p.right_stride : nullptr, p.clip_lo, p.clip_hi, j, r, f);
   float o[8];
   float amax;
-  quad_transform_clip(p.x + row * p.ld + static_cast<int64_t>(j) * 32 + r * 8, valid, xform, clip, f, lane, o, amax);
+  quad_transform_clip(p.x + row * p.ld + static_cast<int64_t>(j) * 32 + r * 8, valid, xform, clip, f, lane, o, amax,
+                      p.bf16_mid != 0);
   // Past the wait inside quad_transform_clip: the grid in front of this one has finished and no
   // longer reads the codes, scales and tickets of its own call.
   if (blockIdx.x == 0)

@@ -12,6 +12,8 @@
 // A producer warp streams tiles into a shared-memory ring with 1-D bulk copies
 // (one per row); eight consumer warps transform, clip and quantise them.
 #pragma once
+#include <cuda_bf16.h>
+
 #include "ptx.cuh"
 
 namespace batq {
@@ -46,7 +48,11 @@ struct QuantActParams {
   float* debug_out;      // [s x n] fp32 when the kernel is built with DEBUG_OUT
   uint32_t* zero_words;  // optional: n_zero_words 32-bit words set to zero (tickets of the kernel that follows)
   int32_t n_zero_words;
+  int32_t bf16_mid;      // != 0: V R and L^T (V R) are rounded to bf16, as a BF16 implementation of Algorithm 1 stores them
 };
+
+// fp32 -> nearest bf16 value (ties to even), as fp32.
+__device__ __forceinline__ float round_bf16(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 
 // Two floats -> one byte holding two E2M1 codes (hi in bits 4-7, lo in bits 0-3),
 // four such bytes -> one 32-bit word (byte 0 = first pair).
@@ -198,7 +204,7 @@ __global__ void __launch_bounds__(kQaThreads, 1) quantize_act_kernel(const Quant
             float acc = v[i][0] * R[c];
 #pragma unroll
             for (int cc = 1; cc < 8; ++cc) acc = fmaf(v[i][cc], R[cc * 8 + c], acc);
-            U[i][c] = acc;
+            U[i][c] = p.bf16_mid ? round_bf16(acc) : acc;
           }
 #pragma unroll
         for (int r = 0; r < 4; ++r)
@@ -207,7 +213,7 @@ __global__ void __launch_bounds__(kQaThreads, 1) quantize_act_kernel(const Quant
             float acc = Lr[r] * U[0][c];
 #pragma unroll
             for (int i = 1; i < 4; ++i) acc = fmaf(Lr[4 * i + r], U[i][c], acc);
-            o[r][c] = acc;
+            o[r][c] = p.bf16_mid ? round_bf16(acc) : acc;
           }
       } else {
 #pragma unroll
