@@ -826,6 +826,7 @@ def run_ours(args):
                          "peak_source": "%s copy bandwidth" % peaks["source"]},
             "kernels": [{"tokens": L["S"], "hidden": L["n"], "gpk_us": float(t_ms[i, 0] * 1e3),
                          "gpk_gbs": float(bytes_case[i] / (t_ms[i, 0] * 1e-3) / 1e9),
+                         "gpk_frac": float(bytes_case[i] / (t_ms[i, 0] * 1e-3) / 1e9 / peaks["hbm_gbs"]),
                          "identity_us": float(t_ms[i, 1] * 1e3),
                          "identity_gbs": float(bytes_case[i] / (t_ms[i, 1] * 1e-3) / 1e9),
                          "mxfp8_us": float(t_ms[i, 2] * 1e3),   # 2 + 1 + 1/32 bytes per element
