@@ -617,8 +617,8 @@ def run_ours(args):
                 "nominal": {"peak": nominal_peak, "frac": gemm_achieved / nominal_peak,
                             "peak_at_sampled_clock": nominal_at_clock,
                             "frac_at_sampled_clock": gemm_achieved / nominal_at_clock if nominal_at_clock else None,
-                            "note": "vendor dense-FP4 figure; the 70 % target of the path is judged against this "
-                                    "one and is not met while frac here is below 0.70"}}
+                            "note": "vendor dense-FP4 figure (context, not the denominator of `frac` above); 70 % of "
+                                    "the dense FP4 peak means frac >= 0.70 here"}}
         if mma_only is not None:
             roof["mma_only"] = dict(mma_only, frac=gemm_achieved / mma_only["tflops"],
                                     frac_back_to_back=b2b_gemm / mma_only["tflops"])

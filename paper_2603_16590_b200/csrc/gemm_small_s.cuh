@@ -12,7 +12,11 @@
 // keeps its partial tile for a reduction in split order (deterministic): up to 8 splits can form a
 // thread-block cluster that reduce-scatters the tiles through distributed shared memory (CTA q
 // adds and writes tokens q, q + splits, ...); otherwise the tiles go to scratch and the CTA that
-// draws the last ticket of a row tile adds them.
+// draws the last ticket of a row tile adds them.  Up to 16 tokens the cluster's CTAs PUSH: each
+// stores the partial sums of token t straight into a receive buffer of CTA t mod splits (remote
+// stores are posted, nothing waits for them), one cluster barrier, and every CTA adds what it
+// received from local shared memory -- one barrier and no remote load instead of two barriers
+// around a round of remote loads.
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and tensor-memory owner,
 // warps 2..5 = epilogue.  The weight stream does not depend on the activation
@@ -38,7 +42,11 @@ struct SmallCfg {
   static constexpr int kStages = (NTOK == 128) ? 3 : (NTOK == 64) ? 4 : 5;
   static constexpr int kSfColsPerStage = 16;         // W: 2 atoms x 4 columns, X: 2 atoms x 4 columns
   static constexpr int kTmemCols = (NTOK == 128) ? 256 : 128;
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024;
+  // Receive buffer of the push reduction (16-token tile only): [source split][ceil(s / splits)][128] fp32,
+  // at most (16 + 7 - 1) / 7 * 7 = 21 token slots of 512 bytes.  It is apart from the ring: a faster
+  // CTA of the cluster writes into it while this CTA's MMAs may still read the ring.
+  static constexpr int kRecvBytes = (NTOK == 16) ? 21 * 512 : 0;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kRecvBytes + 1024;
   static_assert(NTOK == 16 || NTOK == 32 || NTOK == 64 || NTOK == 128, "token tile");
   static_assert(kStages * kStageBytes >= NTOK * 128 * 4, "the partial tile of the cluster reduction fits the ring");
   static_assert(NTOK + kStages * kSfColsPerStage <= kTmemCols, "tensor memory budget");
@@ -259,7 +267,16 @@ gemm_small_s_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         uint32_t v[16];
         tmem_ld_32x32b_x16(taddr + c, v);
         tmem_ld_wait();
-        if (by_cluster) {
+        if (by_cluster && NTOK == 16) {
+          // push: token t goes to CTA t mod splits, slot [this split][t / splits]
+          const int per = (p.s + p.splits - 1) / p.splits;
+          const uint32_t recv0 = smem_u32(smem + Cfg::kStages * Cfg::kStageBytes) + static_cast<uint32_t>(sp * per * 512 + row * 4);
+#pragma unroll
+          for (int t = 0; t < 16; ++t)
+            if (t < p.s)
+              st_shared_cluster_f32(map_to_cta(recv0 + static_cast<uint32_t>((t / p.splits) * 512), static_cast<uint32_t>(t % p.splits)),
+                                    __uint_as_float(v[t]));
+        } else if (by_cluster) {
 #pragma unroll
           for (int t = 0; t < 16; ++t)
             if (c + t < p.s) part_smem[(c + t) * 128 + row] = __uint_as_float(v[t]);
@@ -338,7 +355,32 @@ gemm_small_s_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     // Every thread of every CTA of the cluster takes both barriers, whatever happened above.
     __syncthreads();
     cluster_sync_all();
-    if (warp >= 2 && epi_ok) {
+    if (NTOK == 16) {
+      // Push mode: everything this CTA owns has arrived in its receive buffer (the barrier above
+      // orders the other CTAs' remote stores before this point); add in split order (deterministic).
+      // No CTA touches another's shared memory any more, so no second barrier.
+      if (warp >= 2 && epi_ok) {
+        const int row = (warp & 3) * 32 + lane;
+        const int64_t mrow = static_cast<int64_t>(rt) * 128 + row;
+        const int per = (p.s + p.splits - 1) / p.splits;
+        const float* recv = reinterpret_cast<const float*>(smem + Cfg::kStages * Cfg::kStageBytes) + row;
+        for (int j = 0; sp + j * p.splits < p.s; ++j) {
+          const int t = sp + j * p.splits;
+          float part[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) part[q] = q < p.splits ? recv[(q * per + j) * 128] : 0.0f;
+          float acc = part[0];
+#pragma unroll
+          for (int q = 1; q < 8; ++q) acc += part[q];
+          if (mrow < p.m) {
+            if (OUT_BF16)
+              reinterpret_cast<__nv_bfloat16*>(p.y)[t * p.ldy + mrow] = __float2bfloat16_rn(acc);
+            else
+              reinterpret_cast<float*>(p.y)[t * p.ldy + mrow] = acc;
+          }
+        }
+      }
+    } else if (warp >= 2 && epi_ok) {
       // Reduce-scatter: CTA sp adds, in split order (deterministic), the partial sums of tokens
       // sp, sp + splits, ... -- its own from local, the others' from distributed shared memory --
       // and writes those tokens of y.
@@ -361,7 +403,7 @@ gemm_small_s_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         }
       }
     }
-    cluster_sync_all();  // nobody leaves while its shared memory may still be read
+    if (NTOK != 16) cluster_sync_all();  // pull mode: nobody leaves while its shared memory may still be read
   }
   tc_fence_before_sync();
   __syncthreads();

@@ -220,6 +220,9 @@ __device__ __forceinline__ float ld_shared_cluster_f32(uint32_t cluster_addr) { 
   asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
   return v;
 }
+__device__ __forceinline__ void st_shared_cluster_f32(uint32_t cluster_addr, float v) {  // any CTA's shared memory
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {  // arrive on a barrier of any CTA of the cluster
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
