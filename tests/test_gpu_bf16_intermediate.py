@@ -110,3 +110,16 @@ def test_bf16_intermediates_need_the_factored_4x8_form(batq):
     with pytest.raises(batq.BatqError) as e:
         batq.batq_quantize_act_mxfp8(tr, x, z, z, 0)
     assert e.value.status == 4
+
+
+def test_switching_the_emulation_off_restores_the_fp32_path(batq):
+    S, N = 50, 512
+    xb = synth.make_activations(S, N, 41)
+    t = synth.make_transform(N, 41, "paper")
+    ref = _quantize(batq, _mk(batq, t, on=False), xb)
+    tr = _mk(batq, t, on=True)
+    on = _quantize(batq, tr, xb)
+    batq.batq_transform_set_bf16_intermediates(tr, False)
+    off = _quantize(batq, tr, xb)
+    assert np.array_equal(off[0], ref[0]) and np.array_equal(off[1], ref[1]) and np.array_equal(off[2], ref[2])
+    assert not np.array_equal(on[2], ref[2])

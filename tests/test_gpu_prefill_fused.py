@@ -123,3 +123,32 @@ def test_one_kernel_prefill_in_a_replayed_graph(batq, fused):
     assert batq.batq_last_device_status() == 0
     for a, b in zip(alone, outs):
         assert torch.equal(a, b)
+
+
+def test_one_kernel_prefill_with_row_strides(batq, fused):
+    """x with a row stride larger than n and y with a row stride larger than m: same bits as the
+    dense call, nothing written between the rows."""
+    S, M, N = 300, 520, 1024
+    t, tr, w, xb, wb = _layer(batq, S, M, N, 77)
+    x = batq.bits_to_cuda_bf16(xb)
+    xp = torch.zeros((S, N + 72), dtype=torch.bfloat16, device="cuda")
+    xp[:, :N] = x
+    ws = batq.aligned_workspace(batq.batq_linear_workspace_bytes(w, S))
+    y = torch.empty((S, M), dtype=torch.bfloat16, device="cuda")
+    batq.batq_linear_w4a4(tr, w, x, y, ws)
+    yp = torch.full((S, M + 24), 7.0, dtype=torch.bfloat16, device="cuda")
+    batq.batq_linear_w4a4(tr, w, xp[:, :N], yp[:, :M], ws)
+    assert batq.batq_last_device_status() == 0
+    assert torch.equal(yp[:, :M], y) and (yp[:, M:] == 7.0).all()
+
+
+def test_empty_batches_are_no_ops(batq):
+    N, M = 256, 192
+    t = synth.make_transform(N, 5, "baseline")
+    tr = batq.batq_transform_create(N, t.left, t.right, t.clip_lo, t.clip_hi)
+    w = batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(synth.make_weight(M, N, 5)))
+    lib = batq.load()
+    x = torch.zeros((8, N), dtype=torch.bfloat16, device="cuda")
+    assert lib.batq_linear_w4a4(tr.handle, w.handle, x.data_ptr(), 0, N, None, 1, M, None, 0, None) == 0
+    assert lib.batq_linear_w4a8(tr.handle, w.handle, x.data_ptr(), 0, N, None, 1, M, None, 0, None) == 0
+    assert lib.batq_gemm_mxfp8_mxfp4(None, None, w.handle, 0, None, 1, M, None) == 0

@@ -163,3 +163,21 @@ def test_w4a8_rejects_channel_counts_the_tensor_map_cannot_take(batq):
     with pytest.raises(batq.BatqError) as e:
         batq.batq_gemm_mxfp8_mxfp4(z, z, w, S, y)
     assert e.value.status == 4
+
+
+def test_linear_w4a8_with_row_strides_and_bf16_output(batq):
+    S, M, N = 200, 264, 1024
+    xb = synth.make_activations(S, N, 61)
+    t = synth.make_transform(N, 61, "baseline")
+    tr = _mk(batq, t)
+    w = batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(synth.make_weight(M, N, 61)))
+    ws = batq.aligned_workspace(batq.batq_linear_w4a8_workspace_bytes(w, S))
+    x = batq.bits_to_cuda_bf16(xb)
+    y32 = torch.empty((S, M), dtype=torch.float32, device="cuda")
+    batq.batq_linear_w4a8(tr, w, x, y32, ws)
+    xp = torch.zeros((S, N + 40), dtype=torch.bfloat16, device="cuda")
+    xp[:, :N] = x
+    yp = torch.full((S, M + 16), 3.0, dtype=torch.bfloat16, device="cuda")
+    batq.batq_linear_w4a8(tr, w, xp[:, :N], yp[:, :M], ws)
+    assert batq.batq_last_device_status() == 0
+    assert torch.equal(yp[:, :M], y32.bfloat16()) and (yp[:, M:] == 3.0).all()
