@@ -43,8 +43,9 @@ void batq_debug_force_gemm_kernel(int32_t which);
 /* Which activation quantiser later calls use.  0 = automatic (up to 128 tokens the per-block ALU
  * kernel, above that the tensor-core dense-block kernel; the identity transform above 128 tokens
  * and nothing else takes the streaming ALU kernel), 1 = the streaming ALU kernel (Kronecker
- * form), 2 = the tensor-core kernel, 3 = the per-block ALU kernel.  Factor sizes other than
- * 4 x 8 always take the tensor-core kernel. */
+ * form), 2 = the tensor-core kernel, 3 = the per-block ALU kernel.  The streaming ALU kernel is
+ * built for 4 x 8 factors and the per-block ALU kernel for 4 x 8, 8 x 4 and 16 x 2; a transform
+ * of another size takes the tensor-core kernel where the forced one cannot run it. */
 void batq_debug_force_quantizer(int32_t which);
 
 /* Number of K splits of the small-s GEMM (clamped to the number of 256-element K steps and to

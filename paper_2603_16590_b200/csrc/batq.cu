@@ -143,8 +143,12 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(linear_prefill_fused_kernel<false, true>, kPfSmemBytes);
     e = e ? e : set_smem(linear_prefill_fused_kernel<true, false>, kPfSmemBytes);
     e = e ? e : set_smem(linear_prefill_fused_kernel<true, true>, kPfSmemBytes);
-    e = e ? e : set_smem(linear_small_s_fused_kernel<false>, FusedCfg::kSmemBytes);
-    e = e ? e : set_smem(linear_small_s_fused_kernel<true>, FusedCfg::kSmemBytes);
+    e = e ? e : set_smem(linear_small_s_fused_kernel<false, 8>, FusedCfg::kSmemBytes);
+    e = e ? e : set_smem(linear_small_s_fused_kernel<true, 8>, FusedCfg::kSmemBytes);
+    e = e ? e : set_smem(linear_small_s_fused_kernel<false, 4>, FusedCfg::kSmemBytes);
+    e = e ? e : set_smem(linear_small_s_fused_kernel<true, 4>, FusedCfg::kSmemBytes);
+    e = e ? e : set_smem(linear_small_s_fused_kernel<false, 2>, FusedCfg::kSmemBytes);
+    e = e ? e : set_smem(linear_small_s_fused_kernel<true, 2>, FusedCfg::kSmemBytes);
     e = e ? e : set_smem(gemm_small_s_kernel<16, false>, SmallCfg<16>::kSmemBytes);
     e = e ? e : set_smem(gemm_small_s_kernel<16, true>, SmallCfg<16>::kSmemBytes);
     e = e ? e : set_smem(gemm_small_s_kernel<32, false>, SmallCfg<32>::kSmemBytes);
@@ -354,6 +358,11 @@ batq_status launch_quantize_tc(const batq_transform* t, const void* x, int64_t s
   return BATQ_OK;
 }
 
+// Factor sizes the four-lanes-per-block ALU code (small quantiser, fused small-s layer) is built for.
+bool alu_small_geometry(const batq_transform* t) {
+  return t == nullptr || t->gc == 8 || t->gc == 4 || t->gc == 2;
+}
+
 batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, int64_t n, int64_t ld, void* codes,
                             void* scales, int32_t layout, float* debug_out, cudaStream_t stream,
                             uint32_t* zero_words = nullptr, int32_t n_zero_words = 0) {
@@ -364,14 +373,20 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
   if (t != nullptr && t->device != dev) return BATQ_ERR_CUDA;
   // The dense-block tensor-core kernel works on 128-token tiles; tiny batches (decode) and the
   // identity transform stay on the ALU kernel.
-  // The ALU kernel is written for 4 x 8 factors; every other factorisation of 32 goes through the
-  // tensor-core kernel, which only sees the dense block matrices.
-  const bool only_tc = t != nullptr && (t->gr != 4 || t->gc != 8);
+  // The per-block ALU kernel takes right factors of 8, 4 or 2 columns (4 x 8, 8 x 4, 16 x 2), the
+  // streaming ALU kernel 4 x 8 only; every other case goes through the tensor-core kernel, which
+  // only sees the dense block matrices.
+  const bool small_ok = alu_small_geometry(t);
+  const bool stream_ok = t == nullptr || (t->gr == 4 && t->gc == 8);
   const bool mid = t != nullptr && t->bf16_mid;   // needs the factored form: the ALU kernels (4 x 8 only, checked when it is set)
   const bool small_path = n_zero_words > 0;  // in front of the small-s GEMM (its tickets to clear)
   const int force_q = g_force_quantizer.load(std::memory_order_relaxed);
-  const bool use_tc = only_tc || (!mid && !small_path && t != nullptr &&
-                                  (force_q == 2 || (force_q == 0 && s > kSmallQuantAuto)));
+  // Narrower right factors cost the four lanes more work per block (8 x 4: 2.0 us at 16 tokens and
+  // 4.5 us at 128 for n = 4096; 16 x 2: 2.9 and 7.8 us; the tensor-core kernel 4.0-4.2 us throughout).
+  const int64_t small_limit = stream_ok ? kSmallQuantAuto : (t->gc == 4 ? 64 : 32);
+  const bool want_small = force_q == 3 || (force_q == 0 && (s <= small_limit || (stream_ok && small_path && s <= kSmallSMax)));
+  const bool use_tc = !small_ok || (!stream_ok && !want_small) ||
+                      (!mid && !small_path && t != nullptr && (force_q == 2 || (force_q == 0 && s > kSmallQuantAuto)));
   if (use_tc) {
     if (n_zero_words > 0 &&
         cudaMemsetAsync(zero_words, 0, static_cast<size_t>(n_zero_words) * 4, stream) != cudaSuccess) {
@@ -382,7 +397,7 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
   }
   // A handful of tokens: the ring of the streaming kernel below is all latency there; one thread
   // per (token, block) with everything loaded up front is quicker.
-  if (force_q == 3 || (force_q == 0 && (s <= kSmallQuantAuto || (small_path && s <= kSmallSMax)))) {
+  if (want_small) {
     QuantSmallParams q{};
     q.x = static_cast<const uint16_t*>(x);
     q.ld = ld;
@@ -413,8 +428,15 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t e = debug_out != nullptr ? cudaLaunchKernelEx(&cfg, quantize_act_small_kernel<true>, q)
-                                               : cudaLaunchKernelEx(&cfg, quantize_act_small_kernel<false>, q);
+    const int gc = t != nullptr ? t->gc : 8;
+    const bool dbg = debug_out != nullptr;
+    cudaError_t e;
+    if (gc == 8)      e = dbg ? cudaLaunchKernelEx(&cfg, quantize_act_small_kernel<true, 8>, q)
+                              : cudaLaunchKernelEx(&cfg, quantize_act_small_kernel<false, 8>, q);
+    else if (gc == 4) e = dbg ? cudaLaunchKernelEx(&cfg, quantize_act_small_kernel<true, 4>, q)
+                              : cudaLaunchKernelEx(&cfg, quantize_act_small_kernel<false, 4>, q);
+    else              e = dbg ? cudaLaunchKernelEx(&cfg, quantize_act_small_kernel<true, 2>, q)
+                              : cudaLaunchKernelEx(&cfg, quantize_act_small_kernel<false, 2>, q);
     if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
     return BATQ_OK;
   }
@@ -925,7 +947,7 @@ int pick_fused_splits(int64_t m, int64_t n, int sm_count) {
 bool use_fused_small(const batq_transform* t, const batq_weight* w, int64_t s) {
   const int force_path = g_force_small_path.load(std::memory_order_relaxed);
   if (force_path == 1 || s > kFusedTok) return false;
-  if (t != nullptr && (t->gr != 4 || t->gc != 8 || t->bf16_mid)) return false;  // its in-kernel quantiser is the plain 4 x 8 form
+  if (!alu_small_geometry(t) || (t != nullptr && t->bf16_mid)) return false;  // its in-kernel quantiser: right factors of 8, 4, 2 columns, fp32
   const int sp = pick_fused_splits(w->m, w->n, w->sm_count);
   if (sp == 0) return false;
   if (force_path == 2) return true;
@@ -976,8 +998,15 @@ batq_status launch_linear_fused(const batq_transform* t, const batq_weight* w, c
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  const cudaError_t e = y_dtype == BATQ_BF16 ? cudaLaunchKernelEx(&cfg, linear_small_s_fused_kernel<true>, w->tmap_b128, p)
-                                             : cudaLaunchKernelEx(&cfg, linear_small_s_fused_kernel<false>, w->tmap_b128, p);
+  const int gc = t != nullptr ? t->gc : 8;
+  const bool bf = y_dtype == BATQ_BF16;
+  cudaError_t e;
+  if (gc == 8)      e = bf ? cudaLaunchKernelEx(&cfg, linear_small_s_fused_kernel<true, 8>, w->tmap_b128, p)
+                           : cudaLaunchKernelEx(&cfg, linear_small_s_fused_kernel<false, 8>, w->tmap_b128, p);
+  else if (gc == 4) e = bf ? cudaLaunchKernelEx(&cfg, linear_small_s_fused_kernel<true, 4>, w->tmap_b128, p)
+                           : cudaLaunchKernelEx(&cfg, linear_small_s_fused_kernel<false, 4>, w->tmap_b128, p);
+  else              e = bf ? cudaLaunchKernelEx(&cfg, linear_small_s_fused_kernel<true, 2>, w->tmap_b128, p)
+                           : cudaLaunchKernelEx(&cfg, linear_small_s_fused_kernel<false, 2>, w->tmap_b128, p);
   if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
   return BATQ_OK;
 }

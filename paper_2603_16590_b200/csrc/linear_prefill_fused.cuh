@@ -408,7 +408,7 @@ linear_prefill_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
         for (int r = 0; r < 4; ++r) {
           float uu[8];
 #pragma unroll
-          for (int c = 0; c < 8; ++c) uu[c] = o[8 * r + c] * inv;
+          for (int c = 0; c < 8; c += 2) mul2(o[8 * r + c], o[8 * r + c + 1], inv, uu[c], uu[c + 1]);
           cw[r] = e2m1x8_pack(uu);
         }
         // 64-byte swizzle: 16-byte chunk index XOR ((row / 2) & 3)

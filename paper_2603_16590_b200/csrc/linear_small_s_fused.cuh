@@ -55,8 +55,8 @@ struct FusedParams {
   int32_t s;             // tokens (<= 16)
   int32_t n;
   int32_t k;             // n / 32
-  const float* left;     // [.][16], left_stride floats apart (0 = shared); NULL = identity transform
-  const float* right;    // [.][64]
+  const float* left;     // [.][gr x gr], left_stride floats apart (0 = shared); NULL = identity transform
+  const float* right;    // [.][gc x gc]
   int32_t left_stride;
   int32_t right_stride;
   const float* clip_lo;  // [k] or NULL
@@ -70,41 +70,52 @@ struct FusedParams {
   int64_t ldy;
 };
 
-// One (token, block) is worked on by FOUR lanes of a warp: lane r of the group holds row r of the
-// block's 4 x 8 matrix V and produces row r of V~ = L^T V R (Algorithm 1), i.e. 8 of the 32 outputs
-// and one 32-bit word of codes.  Same arithmetic, in the same order, as quantize_act_kernel (fp32
-// fused multiply-adds over the Kronecker form).  At this size a kernel is a chain of latencies: a
-// short instruction stream per lane (the code is executed once, from a cold instruction cache)
-// counts for more than the number of lanes.
+// One (token, block) is worked on by FOUR lanes of a warp.  The block is a gr x gc matrix V
+// (row-major, gr * gc = 32) and lane q of the group holds its elements 8 q .. 8 q + 7, i.e.
+// 8 / GC whole rows when gc = GC is 8, 4 or 2; it produces the same elements of V~ = L^T V R
+// (Algorithm 1) and one 32-bit word of codes.  Same arithmetic, in the same order, for every GC:
+// fp32 fused multiply-adds, V R first (ascending inner index), then L^T (ascending row index).
+// At this size a kernel is a chain of latencies: a short instruction stream per lane (the code is
+// executed once, from a cold instruction cache) counts for more than the number of lanes.
 //
 // The constants of the layer; requested before the wait for the previous grid.
+template <int GC>
 struct QuadFactors {
-  float R[64];  // right factor, [cc][c]
-  float Lc[4];  // column r of the left factor: L[4 i + r], i = 0..3
+  static constexpr int kGR = 32 / GC;   // rows of V = size of the left factor
+  static constexpr int kRows = 8 / GC;  // rows of V held by one lane
+  float R[GC * GC];        // right factor, [cc][c]
+  float Lc[kRows * kGR];   // [rr][i] = L[i][q * kRows + rr]: the columns of L this lane's rows need
   float c_lo, c_hi;
 };
 
-// Lanes without an item (valid = false) get zeros and read nothing.
+// Lanes without an item (valid = false) get zeros and read nothing.  q = lane within the group.
+template <int GC>
 __device__ __forceinline__ void quad_load_factors(bool valid, const float* L, const float* R, const float* clip_lo,
-                                                  const float* clip_hi, int j, int r, QuadFactors& f) {
+                                                  const float* clip_hi, int j, int q, QuadFactors<GC>& f) {
+  using F = QuadFactors<GC>;
   const bool xf = valid && L != nullptr;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
+  for (int i = 0; i < GC * GC / 4; ++i) {
     const float4 t = xf ? __ldg(reinterpret_cast<const float4*>(R) + i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
     f.R[4 * i] = t.x; f.R[4 * i + 1] = t.y; f.R[4 * i + 2] = t.z; f.R[4 * i + 3] = t.w;
   }
 #pragma unroll
-  for (int i = 0; i < 4; ++i) f.Lc[i] = xf ? __ldg(L + 4 * i + r) : 0.0f;
+  for (int rr = 0; rr < F::kRows; ++rr)
+#pragma unroll
+    for (int i = 0; i < F::kGR; ++i) f.Lc[rr * F::kGR + i] = xf ? __ldg(L + i * F::kGR + q * F::kRows + rr) : 0.0f;
   f.c_lo = (valid && clip_lo != nullptr) ? __ldg(clip_lo + j) : 1.0f;
   f.c_hi = (valid && clip_hi != nullptr) ? __ldg(clip_hi + j) : 1.0f;
 }
 
-// Row r of the block (8 bf16 at xrow) -> this lane's 8 transformed, clipped values and the block's
-// amax (the same in the four lanes).  Every lane of the warp calls this (shuffles inside); lanes
-// without an item pass valid = false and get zeros.  x is read after the wait for the previous grid.
+// Elements 8 q .. 8 q + 7 of the block (8 bf16 at xrow) -> this lane's 8 transformed, clipped
+// values and the block's amax (the same in the four lanes).  Every lane of the warp calls this
+// (shuffles inside); lanes without an item pass valid = false and get zeros.  x is read after the
+// wait for the previous grid.
+template <int GC>
 __device__ __forceinline__ void quad_transform_clip(const uint16_t* xrow, bool valid, bool xform, bool clip,
-                                                    const QuadFactors& f, int lane, float (&o)[8], float& amax,
+                                                    const QuadFactors<GC>& f, int lane, float (&o)[8], float& amax,
                                                     bool bf16_mid = false) {
+  using F = QuadFactors<GC>;
   grid_dependency_wait();
   uint4 q = make_uint4(0u, 0u, 0u, 0u);
   if (valid) q = ld_global_ordered_v4(xrow);
@@ -116,21 +127,30 @@ __device__ __forceinline__ void quad_transform_clip(const uint16_t* xrow, bool v
     v[2 * h + 1] = __uint_as_float(w[h] & 0xFFFF0000u);
   }
   if (xform) {
-    float U[8];  // row r of V R
+    float U[8];  // this lane's rows of V R
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      float acc = v[0] * f.R[c];
+    for (int rr = 0; rr < F::kRows; ++rr)
 #pragma unroll
-      for (int cc = 1; cc < 8; ++cc) acc = fmaf(v[cc], f.R[cc * 8 + c], acc);
-      U[c] = bf16_mid ? round_bf16(acc) : acc;   // a BF16 implementation stores V R as bf16
-    }
+      for (int c = 0; c < GC; ++c) {
+        float acc = v[rr * GC] * f.R[c];
+#pragma unroll
+        for (int cc = 1; cc < GC; ++cc) acc = fmaf(v[rr * GC + cc], f.R[cc * GC + c], acc);
+        U[rr * GC + c] = bf16_mid ? round_bf16(acc) : acc;   // a BF16 implementation stores V R as bf16
+      }
     const int base = lane & ~3;
+    // this lane's rows of L^T (V R): row i of V R sits in lane i / kRows of the group
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {  // row r of L^T (V R): the rows of V R come from the other lanes
-      float acc = f.Lc[0] * __shfl_sync(0xFFFFFFFFu, U[c], base);
+    for (int i = 0; i < F::kGR; ++i)
 #pragma unroll
-      for (int i = 1; i < 4; ++i) acc = fmaf(f.Lc[i], __shfl_sync(0xFFFFFFFFu, U[c], base + i), acc);
-      o[c] = bf16_mid ? round_bf16(acc) : acc;
+      for (int c = 0; c < GC; ++c) {
+        const float u = __shfl_sync(0xFFFFFFFFu, U[(i % F::kRows) * GC + c], base + i / F::kRows);
+#pragma unroll
+        for (int rr = 0; rr < F::kRows; ++rr)
+          o[rr * GC + c] = i == 0 ? f.Lc[rr * F::kGR] * u : fmaf(f.Lc[rr * F::kGR + i], u, o[rr * GC + c]);
+      }
+    if (bf16_mid) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) o[c] = round_bf16(o[c]);
     }
   } else {
 #pragma unroll
@@ -181,8 +201,8 @@ struct QuantSmallParams {
   int32_t s;
   int32_t n;
   int32_t k;             // n / 32
-  const float* left;     // [.][16], left_stride floats apart (0 = shared); NULL = identity transform
-  const float* right;    // [.][64]
+  const float* left;     // [.][gr x gr], left_stride floats apart (0 = shared); NULL = identity transform
+  const float* right;    // [.][gc x gc]
   int32_t left_stride;
   int32_t right_stride;
   const float* clip_lo;  // [k] or NULL
@@ -197,7 +217,7 @@ struct QuantSmallParams {
   int32_t bf16_mid;      // != 0: both contractions of the transform store their result as bf16
 };
 
-template <bool DEBUG_OUT>
+template <bool DEBUG_OUT, int GC>
 __global__ void __launch_bounds__(128) quantize_act_small_kernel(const QuantSmallParams p) {
   grid_launch_dependents();
   const int lane = threadIdx.x & 31;
@@ -208,12 +228,12 @@ __global__ void __launch_bounds__(128) quantize_act_small_kernel(const QuantSmal
   const int64_t row = valid ? item / p.k : 0;
   const int j = valid ? static_cast<int>(item - row * p.k) : 0;
   const bool xform = p.left != nullptr, clip = p.clip_lo != nullptr;
-  QuadFactors f;
-  quad_load_factors(valid, xform ? p.left + static_cast<int64_t>(j) * p.left_stride : nullptr,
-                    xform ? p.right + static_cast<int64_t>(j) * p.right_stride : nullptr, p.clip_lo, p.clip_hi, j, r, f);
+  QuadFactors<GC> f;
+  quad_load_factors<GC>(valid, xform ? p.left + static_cast<int64_t>(j) * p.left_stride : nullptr,
+                        xform ? p.right + static_cast<int64_t>(j) * p.right_stride : nullptr, p.clip_lo, p.clip_hi, j, r, f);
   float o[8];
   float amax;
-  quad_transform_clip(p.x + row * p.ld + static_cast<int64_t>(j) * 32 + r * 8, valid, xform, clip, f, lane, o, amax,
+  quad_transform_clip<GC>(p.x + row * p.ld + static_cast<int64_t>(j) * 32 + r * 8, valid, xform, clip, f, lane, o, amax,
                       p.bf16_mid != 0);
   // Past the wait inside quad_transform_clip: the grid in front of this one has finished and no
   // longer reads the codes, scales and tickets of its own call.
@@ -239,7 +259,7 @@ __global__ void __launch_bounds__(128) quantize_act_small_kernel(const QuantSmal
   }
 }
 
-template <bool OUT_BF16>
+template <bool OUT_BF16, int GC>
 __global__ void __launch_bounds__(kFusedThreads, 2)
 linear_small_s_fused_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams p) {
   using Cfg = FusedCfg;
@@ -382,12 +402,12 @@ linear_small_s_fused_kernel(const __grid_constant__ CUtensorMap tmap_w, const Fu
       const int jj = valid ? item - t * nb : 0;
       const int j = kt0 * 8 + jj;
       const bool real = valid && j < p.k;    // blocks past the last channel: zero codes, finite scale
-      QuadFactors f;
-      quad_load_factors(real, xform ? p.left + static_cast<int64_t>(j) * p.left_stride : nullptr,
-                        xform ? p.right + static_cast<int64_t>(j) * p.right_stride : nullptr, p.clip_lo, p.clip_hi, j, r, f);
+      QuadFactors<GC> f;
+      quad_load_factors<GC>(real, xform ? p.left + static_cast<int64_t>(j) * p.left_stride : nullptr,
+                            xform ? p.right + static_cast<int64_t>(j) * p.right_stride : nullptr, p.clip_lo, p.clip_hi, j, r, f);
       float o[8];
       float amax;
-      quad_transform_clip(p.x + t * p.ld + static_cast<int64_t>(j) * 32 + r * 8, real, xform, clip, f, lane, o, amax);
+      quad_transform_clip<GC>(p.x + t * p.ld + static_cast<int64_t>(j) * 32 + r * 8, real, xform, clip, f, lane, o, amax);
       uint32_t cw = 0u, sbyte = 0u;
       if (real) quad_encode(o, amax, cw, sbyte);
       if (valid) {

@@ -93,6 +93,18 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   return d;
 }
 
+// (a, b) * s with one packed instruction (the products are the same fp32 values as two scalar
+// multiplications give: s is a power of two here).
+__device__ __forceinline__ void mul2(float a, float b, float s, float& ra, float& rb) {
+  asm("{\n\t.reg .b64 v, w, r;\n\t"
+      "mov.b64 v, {%2, %3};\n\t"
+      "mov.b64 w, {%4, %4};\n\t"
+      "mul.rn.f32x2 r, v, w;\n\t"
+      "mov.b64 {%0, %1}, r;\n\t}"
+      : "=f"(ra), "=f"(rb)
+      : "f"(a), "f"(b), "f"(s));
+}
+
 // Four floats -> four E4M3 bytes (round to nearest even, saturating at +-448), first value in byte 0.
 __device__ __forceinline__ uint32_t e4m3x4_pack(float a, float b, float c, float d) {
   uint32_t w;
@@ -401,7 +413,7 @@ quantize_act_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         for (int r = 0; r < 4; ++r) {
           float uu[8];
 #pragma unroll
-          for (int c = 0; c < 8; ++c) uu[c] = o[8 * r + c] * inv;
+          for (int c = 0; c < 8; c += 2) mul2(o[8 * r + c], o[8 * r + c + 1], inv, uu[c], uu[c + 1]);
           cw[r] = e2m1x8_pack(uu);
         }
         // 64-byte swizzle: 16-byte chunk index XOR ((row / 2) & 3)

@@ -348,6 +348,72 @@ def test_linear_other_factor_sizes(batq, gr, gc, S):
     assert np.linalg.norm(got - Y) <= 1e-4 * np.linalg.norm(Sabs)
 
 
+@pytest.mark.parametrize("gr,gc", [(8, 4), (16, 2)])
+@pytest.mark.parametrize("geometry", ["paper", "naive"])
+@pytest.mark.parametrize("S,N", [(1, 4096), (16, 1056), (128, 544)])
+def test_small_quantizer_other_factor_sizes_vs_dense_form(batq, gr, gc, geometry, S, N):
+    """Right factors of 4 and 2 columns run through the four-lanes-per-block ALU quantiser at
+    decode sizes (Kronecker form, Algorithm 1) and through the tensor-core quantiser (dense block
+    matrices, Eq. 1-2) when forced: both within the fp32 bound of the fp64 transform, each
+    bit-exact on its own transformed values."""
+    xb = synth.make_activations(S, N, 270 + S)
+    t = synth.make_transform(N, 15, geometry, gr=gr, gc=gc)
+    tr = _mk_transform(batq, t)
+    V = O.transform_clip(xb, t.left, t.right, t.clip_lo, t.clip_hi)
+    X = np.abs(O.bf16_bits_to_f64(xb)).reshape(S, N // 32, 32)
+    P = np.abs(O.block_matrices(t.left, t.right, N // 32))
+    bound = FP32_REL * np.einsum("sje,jef->sjf", X, P).reshape(S, N)
+    vh = {}
+    try:
+        for mode in (3, 2):
+            batq.batq_debug_force_quantizer(mode)
+            vhat = torch.empty((S, N), dtype=torch.float32, device="cuda")
+            batq.batq_debug_transform_clip_f32(tr, batq.bits_to_cuda_bf16(xb), vhat)
+            vh[mode] = vhat.cpu().numpy().astype(np.float64)
+            assert np.all(np.abs(vh[mode] - V) <= bound + 1e-300)
+            for layout in (0, 1):
+                gc_, gs = _gpu_quantize(batq, tr, xb, layout=layout)
+                oc, os_ = O.mxfp4_quantize(vh[mode])
+                assert np.array_equal(gs, os_) and np.array_equal(gc_, oc)
+    finally:
+        batq.batq_debug_force_quantizer(0)
+    assert batq.batq_last_device_status() == 0
+    # two different summation orders of the same product: not the same bits everywhere
+    assert np.all(np.abs(vh[2] - vh[3]) <= 2 * bound + 1e-300)
+
+
+@pytest.mark.parametrize("gr,gc", [(8, 4), (16, 2)])
+@pytest.mark.parametrize("S,M,N", [(1, 1032, 4096), (4, 520, 2048), (16, 264, 1056)])
+def test_linear_fused_small_s_other_factor_sizes(batq, gr, gc, S, M, N):
+    """The single-kernel decode path with 8 x 4 and 16 x 2 factors: against the oracle, and equal
+    to the two-kernel path (the same four-lane arithmetic in both)."""
+    xb = synth.make_activations(S, N, 280 + S)
+    wb = synth.make_weight(M, N, 281)
+    t = synth.make_transform(N, 16, "paper", gr=gr, gc=gc)
+    tr = _mk_transform(batq, t)
+    w = batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(wb))
+    x = batq.bits_to_cuda_bf16(xb)
+    outs = {}
+    try:
+        for path in (1, 2):
+            batq.batq_debug_force_small_s_path(path)
+            assert batq.batq_linear_kernel_launches(tr, w, S) == (2 if path == 1 else 1)
+            ws = batq.aligned_workspace(batq.batq_linear_workspace_bytes(w, S))
+            y = torch.full((S + 1, M + 8), float("nan"), dtype=torch.float32, device="cuda")
+            batq.batq_linear_w4a4(tr, w, x, y[:S, :M], ws)
+            assert batq.batq_last_device_status() == 0
+            yh = y.cpu().numpy()
+            assert np.isnan(yh[S]).all() and np.isnan(yh[:S, M:]).all(), "wrote outside [S x M]"
+            outs[path] = yh[:S, :M].astype(np.float64)
+    finally:
+        batq.batq_debug_force_small_s_path(0)
+    Y, Sabs, _, _ = O.linear_w4a4(xb, wb, t.left, t.right, t.clip_lo, t.clip_hi)
+    for got in outs.values():
+        assert np.mean(np.abs(got - Y) > 1e-3 * Sabs + 1e-30) <= 1e-3
+        assert np.linalg.norm(got - Y) <= 1e-4 * np.linalg.norm(Sabs)
+    assert np.linalg.norm(outs[1] - outs[2]) <= 1e-4 * np.linalg.norm(Sabs)
+
+
 # ---------------------------------------------------------------------------- MXFP8 activations / KV cache
 @pytest.mark.parametrize("S,N", [(1, 32), (3, 96), (130, 1024), (257, 3584), (300, 4096 + 32)])
 @pytest.mark.parametrize("geometry", ["baseline", "paper"])
