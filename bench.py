@@ -356,6 +356,33 @@ def measure_mma_peak(B, torch, iters):
             "how": "tcgen05.mma kind::mxf4.block_scale only, %d K-steps per CTA (pair), CUDA events" % iters}
 
 
+def measure_mma_with_loads(B, torch, w, iters=8192):
+    """What a streaming GEMM can reach at most with 256 x 256 tiles per CTA pair: the MMA-only loop
+    with, beside it in every CTA, a TMA load stream of the GEMM's volume (32 KiB of a prepared
+    weight, L2-resident, per K-step) into a ring nobody reads.  No barrier couples the two, so the
+    result is what the tensor cores and the path from L2 to shared memory sustain together; a GEMM
+    adds its hand-shakes on top.  Also the two alone, and the MMAs with half the loads."""
+    def timed(it, lit):
+        B.batq_debug_mma_peak_with_loads(w, True, 256, min(it, 256), min(lit, 256))
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        flops, nbytes = B.batq_debug_mma_peak_with_loads(w, True, 256, it, lit)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        return {"tflops": flops / (ms * 1e-3) / 1e12, "load_gbs": nbytes / (ms * 1e-3) / 1e9, "ms": ms}
+    out = {"mma_and_loads": timed(iters, iters), "loads_only": timed(0, iters), "mma_only": timed(iters, 0),
+           "mma_and_three_quarters_of_the_loads": timed(iters, iters * 3 // 4),
+           "mma_and_half_the_loads": timed(iters, iters // 2)}
+    if B.batq_last_device_status() != 0:
+        raise SystemExit("device status after the MMA + loads loop")
+    return {"tflops": out["mma_and_loads"]["tflops"], "variants": out,
+            "how": "CTA pairs, tcgen05.mma kind::mxf4.block_scale on resident operands (scale copies every K-step) "
+                   "and an unsynchronised TMA stream of 32 KiB per K-step and CTA from an L2-resident weight, "
+                   "%d K-steps, CUDA events" % iters}
+
+
 def measure_big_quantizer(B, torch, seed):
     """The quantiser at the largest size of the sweep, 32768 x 8192 (537 MB in, 143 MB out: far larger
     than L2), where it is meant to run at the HBM roofline.  The batch is a 4096-row draw repeated
@@ -419,6 +446,8 @@ def run_peak(args, h, B, peaks):
     import torch
     burst = measure_mma_peak(B, torch, 20000)
     pair = burst["shape"].startswith("pair")
+    wq = B.batq_prepare_weight(None, B.bits_to_cuda_bf16(synth.make_weight(8192, 4096, synth.BASE_SEED + 77)))
+    with_loads = measure_mma_with_loads(B, torch, wq)
     sampler = ClockSampler(h.local)
     h.barrier()
     sampler.start()
@@ -441,11 +470,11 @@ def run_peak(args, h, B, peaks):
             "warmup": 1, "ms_per_step": ms / n, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "mxfp4", "data": "synthetic",
             "config": {"workload": "peak_mxf4", "shape": burst["shape"], "k_steps_per_launch": 20000},
-            "burst": burst, "sustained": {"tflops": sustained, "ms": ms},
+            "burst": burst, "sustained": {"tflops": sustained, "ms": ms}, "with_loads": with_loads,
             "context": {"cublas_bf16_x4_burst": peaks["bf16_tflops"] * FP4_OVER_BF16,
                         "cublas_bf16_x4_sustained": peaks["bf16_tflops_sustained"] * FP4_OVER_BF16,
                         "nominal": NOMINAL_FP4_TFLOPS, "source": peaks["source"]},
-            "gpu_launches": n + 4, "clocks": clocks}))
+            "gpu_launches": n + 4 + 10, "clocks": clocks}))
     h.close()
 
 
@@ -564,6 +593,8 @@ def run_ours(args):
             gq, _ = graph_of(lambda L=L: f_quant(L["tr"], L["x"], L["codes"], L["sf"], B.SF_MMA))
             b2b.append((time_graph(gq, r), time_graph(gg, r)))
         mma_only = measure_mma_peak(B, torch, 20000) if (S > 128 and not a8) else None
+        big_w = max(layers, key=lambda L: L["m"] * L["n"])["w"]
+        mma_loads = measure_mma_with_loads(B, torch, big_w) if (S > 128 and not a8) else None
         big_quant = measure_big_quantizer(B, torch, seed) if (S > 128 and h.rank == 0 and not a8) else None
 
         # end to end: host buffers in and out through the C-ABI host entry point
@@ -627,6 +658,9 @@ def run_ours(args):
         if mma_only is not None:
             roof["mma_only"] = dict(mma_only, frac=gemm_achieved / mma_only["tflops"],
                                     frac_back_to_back=b2b_gemm / mma_only["tflops"])
+        if mma_loads is not None:
+            roof["mma_with_loads"] = dict(mma_loads, frac=gemm_achieved / mma_loads["tflops"],
+                                          frac_back_to_back=b2b_gemm / mma_loads["tflops"])
         line.update({
             "value": h.whole_job_rate(flops_step, steps, ms) / 1e12, "ms_per_step": ms / steps,
             "config": workload_config(args.workload),

@@ -89,6 +89,23 @@ batq_status batq_debug_wait_timeout(int64_t limit_ns, void* stream);
 batq_status batq_debug_mma_peak(int32_t pair, int32_t bn, int32_t iters, int32_t sf_copies,
                                 double* flops_out, void* stream);
 
+/* Measurement: the same loop with a load stream beside it.  While warp 1 of every CTA issues the
+ * MMAs of batq_debug_mma_peak (scale copies repeated every K-step) on its resident operands,
+ * warp 0 loads `load_iters` stages of 32 KiB (two TMA boxes of 128 rows x 128 bytes of w's codes,
+ * the size of a GEMM stage) into a ring of four stages (batq_debug_mma_peak_load_stages: 1..5)
+ * that nobody reads; neither waits for the other.
+ * iters = 0: the loads alone; load_iters = 0: the MMAs alone.  w (m, n >= 256; may be NULL when
+ * load_iters = 0) is only read; 58 MB or less keeps it in L2.  store_iters > 0: warps 2-3 write
+ * that many 32 KiB stages into the same ring with ordinary st.shared instructions (no global
+ * memory traffic), to tell a shared-memory bandwidth limit from one of the path from L2.
+ * *flops_out and *bytes_out (host, may be NULL) receive the launch's floating-point operations and
+ * loaded plus stored bytes.  What the numbers show: whether the tensor cores and a stream into
+ * shared memory slow one another down when no barrier couples them. */
+void batq_debug_mma_peak_load_stages(int32_t stages);   /* ring depth of the load stream, 1..5 (default 4) */
+batq_status batq_debug_mma_peak_with_loads(const batq_weight* w, int32_t pair, int32_t bn, int32_t iters,
+                                           int32_t load_iters, int32_t store_iters, double* flops_out,
+                                           double* bytes_out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -60,6 +60,9 @@ SIGNATURES = {
     "batq_last_device_status": (C.c_int, [_P]),
     "batq_debug_wait_timeout": (C.c_int, [_I64, _P]),
     "batq_debug_mma_peak": (C.c_int, [_I32, _I32, _I32, _I32, C.POINTER(C.c_double), _P]),
+    "batq_debug_mma_peak_load_stages": (None, [_I32]),
+    "batq_debug_mma_peak_with_loads": (C.c_int, [_P, _I32, _I32, _I32, _I32, _I32, C.POINTER(C.c_double),
+                                                 C.POINTER(C.c_double), _P]),
 }
 
 
@@ -353,6 +356,20 @@ def batq_debug_mma_peak(pair: bool, bn: int, iters: int, sf_copies: bool = False
     _check(load().batq_debug_mma_peak(1 if pair else 0, bn, iters, 1 if sf_copies else 0, C.byref(flops), _stream()),
            "batq_debug_mma_peak")
     return flops.value
+
+
+def batq_debug_mma_peak_load_stages(stages: int) -> None:
+    load().batq_debug_mma_peak_load_stages(stages)
+
+
+def batq_debug_mma_peak_with_loads(w, pair: bool, bn: int, iters: int, load_iters: int, store_iters: int = 0):
+    """Launches the MMA loop with an unsynchronised TMA load stream (and/or a stream of ordinary
+    shared-memory stores) beside it on the current stream; returns (flops, loaded + stored bytes)."""
+    flops, nbytes = C.c_double(0.0), C.c_double(0.0)
+    _check(load().batq_debug_mma_peak_with_loads(w.handle if w is not None else None, 1 if pair else 0, bn, iters,
+                                                 load_iters, store_iters, C.byref(flops),
+                                                 C.byref(nbytes), _stream()), "batq_debug_mma_peak_with_loads")
+    return flops.value, nbytes.value
 
 
 def bits_to_cuda_bf16(bits: np.ndarray) -> torch.Tensor:

@@ -135,8 +135,8 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(gemm_w4a8_kernel<128, true>, W4A8Cfg<128>::kSmemBytes);
     e = e ? e : set_smem(gemm_w4a8_kernel<256, false>, W4A8Cfg<256>::kSmemBytes);
     e = e ? e : set_smem(gemm_w4a8_kernel<256, true>, W4A8Cfg<256>::kSmemBytes);
-    e = e ? e : set_smem(mma_peak_kernel<false>, kPeakSmemBytes);
-    e = e ? e : set_smem(mma_peak_kernel<true>, kPeakSmemBytes);
+    e = e ? e : set_smem(mma_peak_kernel<false>, kPeakSmemBytesLoads);
+    e = e ? e : set_smem(mma_peak_kernel<true>, kPeakSmemBytesLoads);
     e = e ? e : set_smem(gemm_mxfp4_pair_kernel<false>, PairCfg::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_pair_kernel<true>, PairCfg::kSmemBytes);
     e = e ? e : set_smem(linear_prefill_fused_kernel<false, false>, kPfSmemBytes);
@@ -1631,19 +1631,38 @@ batq_status batq_debug_wait_timeout(int64_t limit_ns, void* stream) {
   return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
 }
 
-batq_status batq_debug_mma_peak(int32_t pair, int32_t bn, int32_t iters, int32_t sf_copies, double* flops_out, void* stream) {
+std::atomic<int> g_peak_load_stages{4};
+
+static batq_status launch_mma_peak(const batq_weight* w, int32_t pair, int32_t bn, int32_t iters, int32_t sf_copies,
+                                   int32_t load_iters, int32_t store_iters, double* flops_out, double* bytes_out,
+                                   cudaStream_t stream) {
   if (bn != 64 && bn != 128 && bn != 192 && bn != 256) return BATQ_ERR_SHAPE;
-  if (iters <= 0 || iters > (1 << 24)) return BATQ_ERR_SHAPE;
+  if (iters < 0 || iters > (1 << 24) || load_iters < 0 || load_iters > (1 << 24) || store_iters < 0 ||
+      store_iters > (1 << 24) || iters + load_iters + store_iters == 0)
+    return BATQ_ERR_SHAPE;
+  if (load_iters > 0 && (w == nullptr || w->m < 256 || w->n < 256)) return BATQ_ERR_SHAPE;
+  int dev;
   const DeviceInfo* info;
-  batq_status st = device_setup(nullptr, &info);
+  batq_status st = device_setup(&dev, &info);
   if (st != BATQ_OK) return st;
-  PeakParams p{iters, bn, sf_copies ? 1 : 0};
+  if (w != nullptr && w->device != dev) return BATQ_ERR_CUDA;
+  PeakParams p{};
+  p.iters = iters;
+  p.bn = bn;
+  p.sf_copies = sf_copies ? 1 : 0;
+  p.load_iters = load_iters;
+  p.store_iters = store_iters;
+  p.load_stages = g_peak_load_stages.load(std::memory_order_relaxed);
+  p.w_row_tiles = load_iters > 0 ? static_cast<int32_t>(w->m / 128) : 1;   // whole boxes only
+  p.w_k_steps = load_iters > 0 ? static_cast<int32_t>(w->n / 256) : 1;
+  CUtensorMap none{};
+  const CUtensorMap& map = load_iters > 0 ? w->tmap_b128 : none;
   const int ctas = pair ? (info->sm_count / 2) * 2 : info->sm_count;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(static_cast<unsigned>(ctas));
   cfg.blockDim = dim3(kPeakThreads);
-  cfg.dynamicSmemBytes = kPeakSmemBytes;
-  cfg.stream = static_cast<cudaStream_t>(stream);
+  cfg.dynamicSmemBytes = load_iters + store_iters > 0 ? kPeakSmemBytesLoads : kPeakSmemBytes;
+  cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
@@ -1651,11 +1670,29 @@ batq_status batq_debug_mma_peak(int32_t pair, int32_t bn, int32_t iters, int32_t
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pair ? 1 : 0;
-  const cudaError_t e = pair ? cudaLaunchKernelEx(&cfg, mma_peak_kernel<true>, p) : cudaLaunchKernelEx(&cfg, mma_peak_kernel<false>, p);
+  const cudaError_t e = pair ? cudaLaunchKernelEx(&cfg, mma_peak_kernel<true>, map, p)
+                             : cudaLaunchKernelEx(&cfg, mma_peak_kernel<false>, map, p);
   if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
   if (flops_out != nullptr)
     *flops_out = 2.0 * (pair ? 256.0 : 128.0) * bn * 256.0 * iters * (pair ? ctas / 2 : ctas);
+  if (bytes_out != nullptr) *bytes_out = static_cast<double>(kPeakLoadStageBytes) * (load_iters + store_iters) * ctas;
   return BATQ_OK;
+}
+
+void batq_debug_mma_peak_load_stages(int32_t stages) {
+  g_peak_load_stages.store(stages < 1 ? 1 : (stages > kPeakLoadStages ? kPeakLoadStages : stages), std::memory_order_relaxed);
+}
+
+batq_status batq_debug_mma_peak(int32_t pair, int32_t bn, int32_t iters, int32_t sf_copies, double* flops_out, void* stream) {
+  if (iters <= 0) return BATQ_ERR_SHAPE;
+  return launch_mma_peak(nullptr, pair, bn, iters, sf_copies, 0, 0, flops_out, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+batq_status batq_debug_mma_peak_with_loads(const batq_weight* w, int32_t pair, int32_t bn, int32_t iters,
+                                           int32_t load_iters, int32_t store_iters, double* flops_out,
+                                           double* bytes_out, void* stream) {
+  return launch_mma_peak(w, pair, bn, iters, 1, load_iters, store_iters, flops_out, bytes_out,
+                         static_cast<cudaStream_t>(stream));
 }
 
 size_t batq_static_workspace_capacity(void) { return BATQ_STATIC_WORKSPACE_BYTES - 1024; }

@@ -15,22 +15,40 @@ constexpr int kPeakSfbAtoms = 2;         // 256 weight rows
 constexpr int kPeakABytes = 128 * kBKBytes;
 constexpr int kPeakBBytes = 256 * kBKBytes;
 constexpr int kPeakSfBytes = 1024 + kPeakSfbAtoms * 1024;
-constexpr int kPeakSmemBytes = kPeakABytes + kPeakBBytes + kPeakSfBytes + 1024;
+constexpr int kPeakOperandBytes = kPeakABytes + kPeakBBytes + kPeakSfBytes;
+constexpr int kPeakSmemBytes = kPeakOperandBytes + 1024;
 constexpr int kPeakSfCols = 8 + 2 * 4 * kPeakSfbAtoms;
+// The optional load stream: a ring of stages the size of a GEMM stage (two boxes of 128 rows x 128
+// bytes), filled by TMA from a prepared weight and read by nobody.
+constexpr int kPeakLoadStages = 5;   // at most; PeakParams::load_stages of them are used
+constexpr int kPeakLoadBoxBytes = 128 * kBKBytes;
+constexpr int kPeakLoadStageBytes = 2 * kPeakLoadBoxBytes;
+constexpr int kPeakSmemBytesLoads = (kPeakOperandBytes + 1023) / 1024 * 1024 + kPeakLoadStages * kPeakLoadStageBytes + 1024;
 
 struct PeakParams {
-  int32_t iters;      // K-steps (four MMAs of K = 64 each)
+  int32_t iters;      // K-steps (four MMAs of K = 64 each); 0 = no MMAs
   int32_t bn;         // tile width
   int32_t sf_copies;  // 0: scale factors copied to tensor memory once; 1: again before every K-step, as a GEMM must
+  int32_t load_iters; // stages (32 KiB) every CTA loads next to the MMAs, unsynchronised with them; 0 = none
+  int32_t w_row_tiles;  // the weight the loads walk over: 128-row tiles and 128-byte K steps
+  int32_t w_k_steps;
+  int32_t load_stages;  // 1..kPeakLoadStages: copies in flight per CTA
+  int32_t store_iters;  // stages (32 KiB) warps 2-3 of every CTA write into the ring with ordinary stores; 0 = none
 };
 
 // PAIR = false: every CTA issues tcgen05.mma.cta_group::1 on a 128 x bn tile.
 // PAIR = true:  clusters of two; the leader issues cta_group::2 on a 256 x bn tile whose A rows and
 //               B rows are split over the two CTAs' shared memories, as in the CTA-pair GEMM.
+// With load_iters > 0 warp 0 of every CTA streams boxes of a prepared weight into a ring of its own
+// while warp 1 issues the MMAs on the resident operands: the two share the shared memory and the
+// path from L2 but never wait for one another, which separates what the hardware sustains from what
+// a GEMM's barrier hand-shakes cost.
 template <bool PAIR>
-__global__ void __launch_bounds__(kPeakThreads, 1) mma_peak_kernel(const PeakParams p) {
+__global__ void __launch_bounds__(kPeakThreads, 1)
+mma_peak_kernel(const __grid_constant__ CUtensorMap tmap_w, const PeakParams p) {
   extern __shared__ uint8_t peak_smem_raw[];
   __shared__ __align__(8) uint64_t batch_bar[2];
+  __shared__ __align__(8) uint64_t load_bar[kPeakLoadStages];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   const int tid = threadIdx.x;
@@ -51,6 +69,7 @@ __global__ void __launch_bounds__(kPeakThreads, 1) mma_peak_kernel(const PeakPar
   if (tid == 0) {
     mbar_init(smem_u32(&batch_bar[0]), 1);
     mbar_init(smem_u32(&batch_bar[1]), 1);
+    for (int i = 0; i < kPeakLoadStages; ++i) mbar_init(smem_u32(&load_bar[i]), 1);
     abort_flag = 0;
     mbar_fence_init();
   }
@@ -65,7 +84,64 @@ __global__ void __launch_bounds__(kPeakThreads, 1) mma_peak_kernel(const PeakPar
   tc_fence_after_sync();
   const uint32_t tmem_base = tmem_base_slot;
 
-  if (warp == 1 && rank == 0) {
+  if (warp == 0 && p.load_iters > 0) {
+    // ------------------------------------------------------------ load stream (every CTA its own)
+    const uint32_t ring = smem_u32(smem) + (kPeakOperandBytes + 1023) / 1024 * 1024;
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    int issued = 0;
+    for (int i = 0; i < p.load_iters; ++i) {
+      // a stage is refilled as soon as the copy that filled it last has landed
+      if (i >= p.load_stages) {
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&load_bar[stage]), phase ^ 1u, &abort_flag));
+        if (!ok) break;
+      }
+      if (elect_one()) {
+        const int rt = static_cast<int>((static_cast<int64_t>(blockIdx.x) * 13 + i / p.w_k_steps) % p.w_row_tiles);
+        const int rt2 = (rt + p.w_row_tiles / 2) % p.w_row_tiles;
+        const int kt = i % p.w_k_steps;
+        const uint32_t dst = ring + stage * kPeakLoadStageBytes;
+        const uint32_t bar = smem_u32(&load_bar[stage]);
+        mbar_arrive_expect_tx(bar, kPeakLoadStageBytes);
+        tma_load_2d(dst, &tmap_w, kt * kBKBytes, rt * 128, bar);
+        tma_load_2d(dst + kPeakLoadBoxBytes, &tmap_w, kt * kBKBytes, rt2 * 128, bar);
+      }
+      ++issued;
+      if (++stage == p.load_stages) { stage = 0; phase ^= 1u; }
+    }
+    // drain: every copy issued has landed before the CTA exits (also after a wait that gave up)
+    if ((tid & 31) == 0) {
+      const int pending = min(issued, p.load_stages);
+      for (int i = 0; i < pending; ++i) {
+        if (--stage < 0) { stage = p.load_stages - 1; phase ^= 1u; }
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(smem_u32(&load_bar[stage]), phase) && global_timer_ns() - t0 < 100000000ull) {}
+      }
+    }
+    __syncwarp();
+  }
+
+  if (warp >= 2 && p.store_iters > 0) {
+    // ------------------------------------------------------------ ordinary shared-memory stores
+    // 64 threads x 16 bytes = 1 KiB per instruction, 32 instructions per stage; the ring is only
+    // written (with load_iters > 0 as well, both write the same bytes: nobody reads them).
+    uint8_t* ring = smem + (kPeakOperandBytes + 1023) / 1024 * 1024;
+    const int t64 = tid - 64;
+    uint4 val = make_uint4(tid, 2u, 3u, 4u);
+    for (int i = 0; i < p.store_iters; ++i) {
+      uint8_t* st = ring + (i % p.load_stages) * kPeakLoadStageBytes + t64 * 16;
+#pragma unroll 8
+      for (int j = 0; j < kPeakLoadStageBytes / 1024; ++j) {
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(st + j * 1024)), "r"(val.x), "r"(val.y),
+                     "r"(val.z), "r"(val.w)
+                     : "memory");
+      }
+      val.x += 1u;
+    }
+  }
+
+  if (warp == 1 && rank == 0 && p.iters > 0) {
     const uint32_t smem_base = smem_u32(smem);
     const uint64_t adesc = make_smem_desc(smem_base, 16, 1024, 2);
     const uint64_t bdesc = adesc + (kPeakABytes >> 4);

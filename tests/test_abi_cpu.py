@@ -89,6 +89,10 @@ def test_host_validation_without_a_device(lib):
     assert lib.batq_transform_set_bf16_intermediates(None, 1) == 1
     assert lib.batq_debug_mma_peak(0, 100, 10, 0, None, None) == 2
     assert lib.batq_debug_mma_peak(0, 256, 0, 0, None, None) == 2
+    # the loop with a load stream: a weight is needed as soon as something is loaded
+    assert lib.batq_debug_mma_peak_with_loads(None, 1, 256, 10, 10, 0, None, None, None) == 2
+    assert lib.batq_debug_mma_peak_with_loads(None, 1, 256, 0, 0, 0, None, None, None) == 2
+    assert lib.batq_debug_mma_peak_with_loads(None, 1, 100, 10, 0, 0, None, None, None) == 2
 
 
 def test_debug_hooks_are_not_in_the_public_header():

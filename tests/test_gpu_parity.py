@@ -301,6 +301,31 @@ def test_quantizer_is_independent_of_the_row_order(batq, qmode, S):
     assert torch.equal(y0[torch.from_numpy(perm).cuda()], y1)
 
 
+def test_measurement_loops_leave_the_device_clean(batq):
+    """The MMA-only loop and its variants with a TMA load stream or ordinary shared-memory stores
+    beside it (the roofline denominators of the GEMM): every combination runs to the end, reports
+    the work it did and leaves no device status behind; a weight is only read."""
+    M, N = 1024, 1024
+    wb = synth.make_weight(M, N, 77)
+    w = batq.batq_prepare_weight(None, batq.bits_to_cuda_bf16(wb))
+    codes0, sf0 = batq.batq_weight_export(w)
+    for pair in (False, True):
+        ctas = 148 if not pair else 74
+        for it, lit, sit in ((40, 0, 0), (0, 37, 0), (0, 0, 9), (40, 37, 0), (33, 0, 9), (16, 5, 3)):
+            flops, nbytes = batq.batq_debug_mma_peak_with_loads(w, pair, 256, it, lit, sit)
+            torch.cuda.synchronize()
+            assert batq.batq_last_device_status() == 0
+            assert flops > 0 if it else flops == 0
+            assert nbytes % 32768 == 0 and nbytes >= (lit + sit) * 32768 * ctas * 0.9
+    for stages in (1, 5, 4):
+        batq.batq_debug_mma_peak_load_stages(stages)
+        batq.batq_debug_mma_peak_with_loads(w, True, 128, 20, 23, 0)
+        torch.cuda.synchronize()
+        assert batq.batq_last_device_status() == 0
+    codes1, sf1 = batq.batq_weight_export(w)
+    assert torch.equal(codes0, codes1) and torch.equal(sf0, sf1)
+
+
 # ---------------------------------------------------------------------------- other factorisations of the block
 FACTOR_SIZES = [(1, 32), (2, 16), (8, 4), (16, 2), (32, 1)]
 
