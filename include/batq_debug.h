@@ -102,6 +102,9 @@ batq_status batq_debug_mma_peak(int32_t pair, int32_t bn, int32_t iters, int32_t
  * loaded plus stored bytes.  What the numbers show: whether the tensor cores and a stream into
  * shared memory slow one another down when no barrier couples them. */
 void batq_debug_mma_peak_load_stages(int32_t stages);   /* ring depth of the load stream, 1..5 (default 4) */
+/* How many CTAs (consecutive block indices) load the same boxes at the same time, as the tiles of a
+ * GEMM that share a row or column block do; 1 (default) = every CTA its own boxes. */
+void batq_debug_mma_peak_load_sharing(int32_t ctas);
 batq_status batq_debug_mma_peak_with_loads(const batq_weight* w, int32_t pair, int32_t bn, int32_t iters,
                                            int32_t load_iters, int32_t store_iters, double* flops_out,
                                            double* bytes_out, void* stream);

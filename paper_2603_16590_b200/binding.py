@@ -61,6 +61,7 @@ SIGNATURES = {
     "batq_debug_wait_timeout": (C.c_int, [_I64, _P]),
     "batq_debug_mma_peak": (C.c_int, [_I32, _I32, _I32, _I32, C.POINTER(C.c_double), _P]),
     "batq_debug_mma_peak_load_stages": (None, [_I32]),
+    "batq_debug_mma_peak_load_sharing": (None, [_I32]),
     "batq_debug_mma_peak_with_loads": (C.c_int, [_P, _I32, _I32, _I32, _I32, _I32, C.POINTER(C.c_double),
                                                  C.POINTER(C.c_double), _P]),
 }
@@ -360,6 +361,10 @@ def batq_debug_mma_peak(pair: bool, bn: int, iters: int, sf_copies: bool = False
 
 def batq_debug_mma_peak_load_stages(stages: int) -> None:
     load().batq_debug_mma_peak_load_stages(stages)
+
+
+def batq_debug_mma_peak_load_sharing(ctas: int) -> None:
+    load().batq_debug_mma_peak_load_sharing(ctas)
 
 
 def batq_debug_mma_peak_with_loads(w, pair: bool, bn: int, iters: int, load_iters: int, store_iters: int = 0):

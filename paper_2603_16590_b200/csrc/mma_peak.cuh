@@ -33,6 +33,7 @@ struct PeakParams {
   int32_t w_row_tiles;  // the weight the loads walk over: 128-row tiles and 128-byte K steps
   int32_t w_k_steps;
   int32_t load_stages;  // 1..kPeakLoadStages: copies in flight per CTA
+  int32_t load_sharing; // >= 1: this many CTAs (blockIdx.x / load_sharing equal) load the same boxes at the same time
   int32_t store_iters;  // stages (32 KiB) warps 2-3 of every CTA write into the ring with ordinary stores; 0 = none
 };
 
@@ -98,7 +99,7 @@ mma_peak_kernel(const __grid_constant__ CUtensorMap tmap_w, const PeakParams p) 
         if (!ok) break;
       }
       if (elect_one()) {
-        const int rt = static_cast<int>((static_cast<int64_t>(blockIdx.x) * 13 + i / p.w_k_steps) % p.w_row_tiles);
+        const int rt = static_cast<int>((static_cast<int64_t>(blockIdx.x / p.load_sharing) * 13 + i / p.w_k_steps) % p.w_row_tiles);
         const int rt2 = (rt + p.w_row_tiles / 2) % p.w_row_tiles;
         const int kt = i % p.w_k_steps;
         const uint32_t dst = ring + stage * kPeakLoadStageBytes;
