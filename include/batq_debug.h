@@ -105,6 +105,10 @@ void batq_debug_mma_peak_load_stages(int32_t stages);   /* ring depth of the loa
 /* How many CTAs (consecutive block indices) load the same boxes at the same time, as the tiles of a
  * GEMM that share a row or column block do; 1 (default) = every CTA its own boxes. */
 void batq_debug_mma_peak_load_sharing(int32_t ctas);
+/* on != 0, pairs only: half of every stage (16 KiB) is not loaded from L2 but copied by the other
+ * CTA of the pair from its shared memory (cp.async.bulk shared::cta -> shared::cluster, no
+ * multicast), as a GEMM would forward an operand tile that two CTAs need. */
+void batq_debug_mma_peak_load_from_peer(int32_t on);
 batq_status batq_debug_mma_peak_with_loads(const batq_weight* w, int32_t pair, int32_t bn, int32_t iters,
                                            int32_t load_iters, int32_t store_iters, double* flops_out,
                                            double* bytes_out, void* stream);

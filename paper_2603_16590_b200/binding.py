@@ -62,6 +62,7 @@ SIGNATURES = {
     "batq_debug_mma_peak": (C.c_int, [_I32, _I32, _I32, _I32, C.POINTER(C.c_double), _P]),
     "batq_debug_mma_peak_load_stages": (None, [_I32]),
     "batq_debug_mma_peak_load_sharing": (None, [_I32]),
+    "batq_debug_mma_peak_load_from_peer": (None, [_I32]),
     "batq_debug_mma_peak_with_loads": (C.c_int, [_P, _I32, _I32, _I32, _I32, _I32, C.POINTER(C.c_double),
                                                  C.POINTER(C.c_double), _P]),
 }
@@ -365,6 +366,10 @@ def batq_debug_mma_peak_load_stages(stages: int) -> None:
 
 def batq_debug_mma_peak_load_sharing(ctas: int) -> None:
     load().batq_debug_mma_peak_load_sharing(ctas)
+
+
+def batq_debug_mma_peak_load_from_peer(on: bool) -> None:
+    load().batq_debug_mma_peak_load_from_peer(1 if on else 0)
 
 
 def batq_debug_mma_peak_with_loads(w, pair: bool, bn: int, iters: int, load_iters: int, store_iters: int = 0):

@@ -1633,6 +1633,7 @@ batq_status batq_debug_wait_timeout(int64_t limit_ns, void* stream) {
 
 std::atomic<int> g_peak_load_stages{4};
 std::atomic<int> g_peak_load_sharing{1};
+std::atomic<int> g_peak_load_from_peer{0};
 
 static batq_status launch_mma_peak(const batq_weight* w, int32_t pair, int32_t bn, int32_t iters, int32_t sf_copies,
                                    int32_t load_iters, int32_t store_iters, double* flops_out, double* bytes_out,
@@ -1655,6 +1656,7 @@ static batq_status launch_mma_peak(const batq_weight* w, int32_t pair, int32_t b
   p.store_iters = store_iters;
   p.load_stages = g_peak_load_stages.load(std::memory_order_relaxed);
   p.load_sharing = g_peak_load_sharing.load(std::memory_order_relaxed);
+  p.load_from_peer = pair ? g_peak_load_from_peer.load(std::memory_order_relaxed) : 0;
   p.w_row_tiles = load_iters > 0 ? static_cast<int32_t>(w->m / 128) : 1;   // whole boxes only
   p.w_k_steps = load_iters > 0 ? static_cast<int32_t>(w->n / 256) : 1;
   CUtensorMap none{};
@@ -1684,6 +1686,7 @@ static batq_status launch_mma_peak(const batq_weight* w, int32_t pair, int32_t b
 void batq_debug_mma_peak_load_stages(int32_t stages) {
   g_peak_load_stages.store(stages < 1 ? 1 : (stages > kPeakLoadStages ? kPeakLoadStages : stages), std::memory_order_relaxed);
 }
+void batq_debug_mma_peak_load_from_peer(int32_t on) { g_peak_load_from_peer.store(on != 0, std::memory_order_relaxed); }
 void batq_debug_mma_peak_load_sharing(int32_t ctas) {
   g_peak_load_sharing.store(ctas < 1 ? 1 : (ctas > 1024 ? 1024 : ctas), std::memory_order_relaxed);
 }

@@ -34,6 +34,8 @@ struct PeakParams {
   int32_t w_k_steps;
   int32_t load_stages;  // 1..kPeakLoadStages: copies in flight per CTA
   int32_t load_sharing; // >= 1: this many CTAs (blockIdx.x / load_sharing equal) load the same boxes at the same time
+  int32_t load_from_peer;  // pairs only, != 0: the second box of every stage is not loaded from L2 but copied from
+                           // the other CTA of the pair, shared memory to shared memory
   int32_t store_iters;  // stages (32 KiB) warps 2-3 of every CTA write into the ring with ordinary stores; 0 = none
 };
 
@@ -44,6 +46,16 @@ struct PeakParams {
 // while warp 1 issues the MMAs on the resident operands: the two share the shared memory and the
 // path from L2 but never wait for one another, which separates what the hardware sustains from what
 // a GEMM's barrier hand-shakes cost.
+// Shared memory of this CTA -> shared memory of another CTA of the cluster; the bytes are counted
+// on a barrier of the destination CTA.  Both addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_s2s_cluster(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes,
+                                                 uint32_t bar_cluster) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   dst_cluster),
+               "r"(src_cta), "r"(bytes), "r"(bar_cluster)
+               : "memory");
+}
+
 template <bool PAIR>
 __global__ void __launch_bounds__(kPeakThreads, 1)
 mma_peak_kernel(const __grid_constant__ CUtensorMap tmap_w, const PeakParams p) {
@@ -106,7 +118,15 @@ mma_peak_kernel(const __grid_constant__ CUtensorMap tmap_w, const PeakParams p) 
         const uint32_t bar = smem_u32(&load_bar[stage]);
         mbar_arrive_expect_tx(bar, kPeakLoadStageBytes);
         tma_load_2d(dst, &tmap_w, kt * kBKBytes, rt * 128, bar);
-        tma_load_2d(dst + kPeakLoadBoxBytes, &tmap_w, kt * kBKBytes, rt2 * 128, bar);
+        if (PAIR && p.load_from_peer) {
+          // this CTA fills the second half of the PEER's stage (from its own resident operands) and
+          // the peer fills this CTA's: 16 KiB of every stage arrive over the cluster's network
+          const uint32_t peer = rank ^ 1u;
+          bulk_s2s_cluster(map_to_cta(dst + kPeakLoadBoxBytes, peer), smem_u32(smem), kPeakLoadBoxBytes,
+                           map_to_cta(bar, peer));
+        } else {
+          tma_load_2d(dst + kPeakLoadBoxBytes, &tmap_w, kt * kBKBytes, rt2 * 128, bar);
+        }
       }
       ++issued;
       if (++stage == p.load_stages) { stage = 0; phase ^= 1u; }

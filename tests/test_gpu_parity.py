@@ -317,11 +317,20 @@ def test_measurement_loops_leave_the_device_clean(batq):
             assert batq.batq_last_device_status() == 0
             assert flops > 0 if it else flops == 0
             assert nbytes % 32768 == 0 and nbytes >= (lit + sit) * 32768 * ctas * 0.9
-    for stages in (1, 5, 4):
-        batq.batq_debug_mma_peak_load_stages(stages)
-        batq.batq_debug_mma_peak_with_loads(w, True, 128, 20, 23, 0)
-        torch.cuda.synchronize()
-        assert batq.batq_last_device_status() == 0
+    try:
+        for stages, sharing, peer in ((1, 1, 0), (5, 8, 0), (2, 1, 1), (4, 148, 1), (4, 1, 0)):
+            batq.batq_debug_mma_peak_load_stages(stages)
+            batq.batq_debug_mma_peak_load_sharing(sharing)
+            batq.batq_debug_mma_peak_load_from_peer(peer)
+            for pair in (True, False):   # copies between the CTAs of a pair: ignored without pairs
+                batq.batq_debug_mma_peak_with_loads(w, pair, 128, 20, 23, 0)
+                batq.batq_debug_mma_peak_with_loads(w, pair, 256, 0, 11, 0)
+                torch.cuda.synchronize()
+                assert batq.batq_last_device_status() == 0
+    finally:
+        batq.batq_debug_mma_peak_load_stages(4)
+        batq.batq_debug_mma_peak_load_sharing(1)
+        batq.batq_debug_mma_peak_load_from_peer(0)
     codes1, sf1 = batq.batq_weight_export(w)
     assert torch.equal(codes0, codes1) and torch.equal(sf0, sf1)
 
