@@ -35,9 +35,16 @@ void batq_debug_force_tile_width(int32_t bn);
 int32_t batq_debug_pair_schedule(int64_t s, int64_t m, int64_t n, int32_t sm_count, int32_t pair,
                                  int32_t* tiles, int32_t max_tiles);
 
+/* The same for the wide-tile CTA-pair GEMM (tiles of up to 448 features, one accumulator). */
+int32_t batq_debug_wide_schedule(int64_t s, int64_t m, int64_t n, int32_t sm_count, int32_t pair,
+                                 int32_t* tiles, int32_t max_tiles);
+
 /* Which prefill GEMM kernel later calls use.  0 = automatic (CTA pairs sharing a 256-token tile
- * for s > 128, one CTA per 128-token tile otherwise), 1 = always one CTA per tile, 2 = always CTA
- * pairs. */
+ * for s > 128 -- with tiles of up to 256 features and two accumulators, or tiles of up to 448
+ * features and one, whichever the cost model expects to finish first --, one CTA per 128-token
+ * tile otherwise), 1 = always one CTA per tile, 2 = always CTA pairs with two accumulators,
+ * 3 = always CTA pairs with wide tiles (batq_debug_force_tile_width then takes any multiple of 64
+ * up to 448 and makes every column that wide). */
 void batq_debug_force_gemm_kernel(int32_t which);
 
 /* Which activation quantiser later calls use.  0 = automatic (up to 128 tokens the per-block ALU

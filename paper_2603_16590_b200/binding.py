@@ -53,6 +53,7 @@ SIGNATURES = {
     "batq_linear_workspace_bytes": (_SZ, [_P, _I64]),
     "batq_linear_kernel_launches": (C.c_int32, [_P, _P, _I64]),
     "batq_debug_pair_schedule": (C.c_int32, [_I64, _I64, _I64, _I32, _I32, _P, _I32]),
+    "batq_debug_wide_schedule": (C.c_int32, [_I64, _I64, _I64, _I32, _I32, _P, _I32]),
     "batq_linear_w4a4": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P, _SZ, _P]),
     "batq_linear_w4a4_host": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _P, _P, _P, _SZ, _P]),
     "batq_static_workspace_capacity": (_SZ, []),
@@ -289,19 +290,27 @@ def batq_linear_workspace_bytes(w: Weight, s) -> int:
     return load().batq_linear_workspace_bytes(w.handle, s)
 
 
-def batq_debug_pair_schedule(s, m, n, sm_count=148):
-    """[[(row block, first feature, width), ...] per CTA pair] of the CTA-pair GEMM (host only)."""
-    lib = load()
-    pairs = lib.batq_debug_pair_schedule(s, m, n, sm_count, -1, None, 0)
+def _schedule(fn, s, m, n, sm_count):
+    pairs = fn(s, m, n, sm_count, -1, None, 0)
     if pairs < 0:
         raise ValueError("bad shape")
     out = []
     for p in range(pairs):
-        cnt = lib.batq_debug_pair_schedule(s, m, n, sm_count, p, None, 0)
+        cnt = fn(s, m, n, sm_count, p, None, 0)
         buf = (C.c_int32 * (3 * max(cnt, 1)))()
-        lib.batq_debug_pair_schedule(s, m, n, sm_count, p, buf, cnt)
+        fn(s, m, n, sm_count, p, buf, cnt)
         out.append([(buf[3 * i], buf[3 * i + 1], buf[3 * i + 2]) for i in range(cnt)])
     return out
+
+
+def batq_debug_pair_schedule(s, m, n, sm_count=148):
+    """[[(row block, first feature, width), ...] per CTA pair] of the CTA-pair GEMM (host only)."""
+    return _schedule(load().batq_debug_pair_schedule, s, m, n, sm_count)
+
+
+def batq_debug_wide_schedule(s, m, n, sm_count=148):
+    """The same for the wide-tile CTA-pair GEMM (host only)."""
+    return _schedule(load().batq_debug_wide_schedule, s, m, n, sm_count)
 
 
 def batq_linear_kernel_launches(t, w: Weight, s) -> int:

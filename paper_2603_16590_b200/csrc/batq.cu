@@ -16,6 +16,7 @@
 
 #include "gemm_mxfp4.cuh"
 #include "gemm_mxfp4_pair.cuh"
+#include "gemm_mxfp4_wide.cuh"
 #include "gemm_small_s.cuh"
 #include "gemm_w4a8.cuh"
 #include "linear_prefill_fused.cuh"
@@ -59,7 +60,7 @@ struct batq_weight {
   CUtensorMap tmap_b32;   // boxes of 32 weight rows: the CTA-pair kernel composes its half tiles from them
   CUtensorMap tmap_sf;    // scale atoms: [row tiles x KA] rows of 512 bytes, boxes of two atoms
   // CTA-pair schedules already worked out for this weight, by token count (host only)
-  struct SchedEntry { int64_t s; int force_bn; int32_t n_cols, n_segs, pairs; batq::PairSeg seg[batq::kPairMaxSegs]; };
+  struct SchedEntry { int64_t s; int force_bn; bool wide; double cost; int32_t n_cols, n_segs, pairs; batq::PairSeg seg[batq::kPairMaxSegs]; };
   mutable std::mutex sched_mutex;
   mutable std::vector<SchedEntry> sched_cache;
   bool has_u4;            // n % 128 == 0: the maps below exist (W4A8 GEMM)
@@ -139,6 +140,8 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(mma_peak_kernel<true>, kPeakSmemBytesLoads);
     e = e ? e : set_smem(gemm_mxfp4_pair_kernel<false>, PairCfg::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_pair_kernel<true>, PairCfg::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_wide_kernel<false>, WideCfg::kSmemBytes);
+    e = e ? e : set_smem(gemm_mxfp4_wide_kernel<true>, WideCfg::kSmemBytes);
     e = e ? e : set_smem(linear_prefill_fused_kernel<false, false>, kPfSmemBytes);
     e = e ? e : set_smem(linear_prefill_fused_kernel<false, true>, kPfSmemBytes);
     e = e ? e : set_smem(linear_prefill_fused_kernel<true, false>, kPfSmemBytes);
@@ -479,17 +482,19 @@ batq_status launch_quantize(const batq_transform* t, const void* x, int64_t s, i
   return cudaGetLastError() == cudaSuccess ? BATQ_OK : BATQ_ERR_CUDA;
 }
 
-// Tensor map over a row-major output [rows x cols], box = 128 bytes x 32 rows, 128-byte swizzle.
-batq_status make_y_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, bool bf16) {
+// Tensor map over a row-major output [rows x cols], box = 128 (or 64) bytes x 32 rows with the
+// swizzle of that width.
+batq_status make_y_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, bool bf16,
+                        int row_bytes = 128) {
   const int esz = bf16 ? 2 : 4;
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
   const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld * esz)};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / esz), 32};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(row_bytes / esz), 32};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = g_encode_tiled(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
                                     const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                                    row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                                    CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? BATQ_OK : BATQ_ERR_CUDA;
 }
 
@@ -517,7 +522,7 @@ int pick_bn(int64_t s, int64_t m, int64_t n, int sm_count) {
   return c256 <= c128 ? 256 : 128;
 }
 
-std::atomic<int> g_force_gemm_kernel{0};  // tuning hook: 0 = automatic, 1 = one CTA per tile, 2 = CTA pairs
+std::atomic<int> g_force_gemm_kernel{0};  // tuning hook: 0 = automatic, 1 = one CTA per tile, 2 = CTA pairs (two accumulators), 3 = CTA pairs (wide tiles)
 
 // The schedule of the CTA-pair kernel for an s x m output with k_steps K-steps: the segments of
 // column widths and the number of pairs.  Candidates: columns all 128, 192 or 256 wide; 256 and
@@ -663,14 +668,123 @@ bool pair_schedule(int64_t s, int64_t m, int64_t k_steps, int sm_count, PairPara
   return true;
 }
 
+// ---- the wide-tile pair kernel: one accumulator of up to 448 columns per tile ---------------------
+// Cost of a pair's tiles in microseconds, fitted to measured layers (2048 tokens, K = 4096 and
+// 14336, every column 256 / 320 / 384 / 448 wide): a K-step of a tile up to 384 wide takes
+// 0.17 + 0.0009 bn us (0.40 at 256, 0.52 at 384: the bytes the SM pulls from L2), one of a 448-wide
+// tile 0.66 us (four stages of 49 KiB turn over at the latency of a load from L2); about 1.4 us
+// per tile pass between the last MMA of one tile and the first of the next.
+double wide_tile_us(int bn, int64_t k_steps) {
+  const double step = bn > 384 ? 0.66 : 0.17 + 0.0009 * bn;
+  return static_cast<double>(k_steps) * step + 1.4;
+}
+// The same for the two-accumulator kernel: bound by its loads (36 KiB per K-step at 256 columns),
+// the epilogue hidden unless two tiles in a row need the same accumulator.
+double pair_tile_us(int bn, int64_t k_steps, bool same_slot) {
+  return static_cast<double>(k_steps) * 0.383 * (32.0 + bn / 8.0) / 64.0 + (same_slot ? 1.7 : 1.1);
+}
+
+double wide_cost(const PairSched& c, PairParams* p, int64_t k_steps, int max_pairs, int* pairs_out) {
+  p->n_cols = c.n_cols;
+  p->n_segs = c.n_segs;
+  for (int i = 0; i < kPairMaxSegs; ++i) p->seg[i] = c.seg[i];
+  const int np = static_cast<int>(std::min<int64_t>(max_pairs, static_cast<int64_t>(p->m_pairs) * c.n_cols));
+  *pairs_out = np;
+  double worst = 0.0;
+  for (int pr = 0; pr < np; ++pr) {
+    PairWalk walk(*p, pr, np);
+    PairTile t;
+    double cost = 0.0;
+    while (walk.next(t)) cost += wide_tile_us(t.bn, k_steps);
+    worst = std::max(worst, cost);
+  }
+  return worst + 5.5;   // launch, first loads, the last tile's stores
+}
+
+// The two-accumulator schedule's cost in the same unit, for the choice between the kernels.
+double pair_cost_us(PairParams* p, int64_t k_steps, int np) {
+  double worst = 0.0;
+  for (int pr = 0; pr < np; ++pr) {
+    PairWalk walk(*p, pr, np);
+    PairSlots slots;
+    PairTile t;
+    int last = -1;
+    double cost = 0.0;
+    while (walk.next(t)) {
+      int slot;
+      uint32_t phase;
+      slots.take(t.bn, slot, phase);
+      cost += pair_tile_us(t.bn, k_steps, slot == last);
+      last = slot;
+    }
+    worst = std::max(worst, cost);
+  }
+  return worst + 1.5;   // the last tile's epilogue
+}
+
+bool wide_schedule(int64_t s, int64_t m, int64_t k_steps, int sm_count, int force_w, PairParams* p, int* pairs,
+                   double* cost_us) {
+  const int64_t m_pairs = (s + 255) / 256;
+  const int max_pairs = std::max(1, sm_count / 2);
+  if (m_pairs * ((m + 63) / 64) > INT32_MAX) return false;
+  p->s = static_cast<int32_t>(s);
+  p->m = static_cast<int32_t>(m);
+  p->m_pairs = static_cast<int32_t>(m_pairs);
+  PairSched best{};
+  double best_cost = 1e30;
+  auto consider = [&](const PairSched& c) {
+    const PairSeg& l = c.seg[c.n_segs - 1];
+    const int64_t end = l.n0 + seg_span(l.wa, l.wb, l.cols);
+    if (end < m || end - l.wb >= m) return;
+    int np;
+    const double cost = wide_cost(c, p, k_steps, max_pairs, &np);
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = c; best.pairs = np; }
+  };
+  const int widths[6] = {448, 384, 320, 256, 192, 128};
+  if (force_w > 0) {   // tuning hook: every column this wide
+    PairSched c{};
+    sched_add(&c, force_w, force_w, (m + force_w - 1) / force_w);
+    consider(c);
+  }
+  for (int i = 0; i < 6 && force_w <= 0; ++i) {
+    const int w1 = widths[i];
+    {
+      PairSched c{};
+      sched_add(&c, w1, w1, (m + w1 - 1) / w1);
+      consider(c);
+    }
+    // x columns of w1, then columns of w2 to the edge, and the other way round
+    const int64_t x_max = m / w1;
+    const int64_t x_step = std::max<int64_t>(1, x_max * m_pairs / (32 * max_pairs));
+    for (int j = 0; j < 6; ++j) {
+      const int w2 = widths[j];
+      if (w2 == w1) continue;
+      for (int64_t x = 1; x <= x_max; x += x_step) {
+        const int64_t rest = m - x * w1;
+        if (rest <= 0) break;
+        PairSched c{};
+        if (sched_add(&c, w1, w1, x) && sched_add(&c, w2, w2, (rest + w2 - 1) / w2)) consider(c);
+      }
+    }
+  }
+  if (best_cost >= 1e30) return false;
+  p->n_cols = best.n_cols;
+  p->n_segs = best.n_segs;
+  for (int i = 0; i < kPairMaxSegs; ++i) p->seg[i] = best.seg[i];
+  *pairs = best.pairs;
+  *cost_us = best_cost;
+  return true;
+}
+
 // The same, remembered per prepared weight and token count (the search walks a few hundred
 // candidates; a layer is called with few distinct token counts).
-bool pair_schedule_cached(const batq_weight* w, int64_t s, int sm_count, PairParams* p, int* pairs) {
+bool pair_schedule_cached(const batq_weight* w, int64_t s, int sm_count, bool wide, PairParams* p, int* pairs,
+                          double* cost_us) {
   const int force_bn = g_force_bn.load(std::memory_order_relaxed);
   {
     std::lock_guard<std::mutex> lock(w->sched_mutex);
     for (const auto& e : w->sched_cache)
-      if (e.s == s && e.force_bn == force_bn) {
+      if (e.s == s && e.force_bn == force_bn && e.wide == wide) {
         p->s = static_cast<int32_t>(s);
         p->m = static_cast<int32_t>(w->m);
         p->m_pairs = static_cast<int32_t>((s + 255) / 256);
@@ -678,12 +792,21 @@ bool pair_schedule_cached(const batq_weight* w, int64_t s, int sm_count, PairPar
         p->n_segs = e.n_segs;
         for (int i = 0; i < kPairMaxSegs; ++i) p->seg[i] = e.seg[i];
         *pairs = e.pairs;
+        *cost_us = e.cost;
         return true;
       }
   }
-  if (!pair_schedule(s, w->m, (w->n + 255) / 256, sm_count, p, pairs)) return false;
+  const int64_t k_steps = (w->n + 255) / 256;
+  if (wide) {
+    const bool fw = force_bn >= 64 && force_bn <= kWideMaxBn && force_bn % 64 == 0;
+    if (!wide_schedule(s, w->m, k_steps, sm_count, fw ? force_bn : 0, p, pairs, cost_us)) return false;
+  } else {
+    if (!pair_schedule(s, w->m, k_steps, sm_count, p, pairs)) return false;
+    *cost_us = pair_cost_us(p, k_steps, *pairs);
+  }
   batq_weight::SchedEntry e{};
-  e.s = s; e.force_bn = force_bn; e.n_cols = p->n_cols; e.n_segs = p->n_segs; e.pairs = *pairs;
+  e.s = s; e.force_bn = force_bn; e.wide = wide; e.cost = *cost_us;
+  e.n_cols = p->n_cols; e.n_segs = p->n_segs; e.pairs = *pairs;
   for (int i = 0; i < kPairMaxSegs; ++i) e.seg[i] = p->seg[i];
   std::lock_guard<std::mutex> lock(w->sched_mutex);
   if (w->sched_cache.size() >= 16) w->sched_cache.erase(w->sched_cache.begin());
@@ -691,14 +814,14 @@ bool pair_schedule_cached(const batq_weight* w, int64_t s, int sm_count, PairPar
   return true;
 }
 
-template <bool BF>
+template <bool BF, bool WIDE>
 cudaError_t launch_pair_kernel(int grid, cudaStream_t stream, bool dependent, const CUtensorMap& ta, const CUtensorMap& tb,
                                const CUtensorMap& tsfa, const CUtensorMap& tsfb, const CUtensorMap& ty,
                                const PairParams& p) {
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(static_cast<unsigned>(grid));
-  cfg.blockDim = dim3(kPairThreads);
-  cfg.dynamicSmemBytes = PairCfg::kSmemBytes;
+  cfg.blockDim = dim3(WIDE ? kWideThreads : kPairThreads);
+  cfg.dynamicSmemBytes = WIDE ? WideCfg::kSmemBytes : PairCfg::kSmemBytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -709,6 +832,7 @@ cudaError_t launch_pair_kernel(int grid, cudaStream_t stream, bool dependent, co
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = dependent ? 2 : 1;
+  if (WIDE) return cudaLaunchKernelEx(&cfg, gemm_mxfp4_wide_kernel<BF>, ta, tb, tsfa, tsfb, ty, p);
   return cudaLaunchKernelEx(&cfg, gemm_mxfp4_pair_kernel<BF>, ta, tb, tsfa, tsfb, ty, p);
 }
 
@@ -719,17 +843,46 @@ batq_status launch_gemm_pair(const void* x_codes, const void* x_sf, const batq_w
   CUtensorMap tmap_sfa;
   batq_status st = make_sf_tmap(&tmap_sfa, x_sf, (s + 127) / 128, w->katoms);
   if (st != BATQ_OK) return st;
-  PairParams p{};
-  int pairs = 0;
-  if (!pair_schedule_cached(w, s, sm_count, &p, &pairs)) return BATQ_ERR_SHAPE;
+  // Two kernels share this launcher: tiles of up to 256 features with two accumulators, or tiles of
+  // up to 448 with one; each comes with its own schedule and an estimate of its time.
+  const int force_gemm = g_force_gemm_kernel.load(std::memory_order_relaxed);
+  const int force_bn = g_force_bn.load(std::memory_order_relaxed);
+  const bool may_wide = force_gemm == 3 ? (force_bn == 0 || (force_bn >= 64 && force_bn <= kWideMaxBn && force_bn % 64 == 0))
+                                        : (w->m >= 320 && force_bn == 0);
+  PairParams p{}, pw{};
+  int pairs = 0, pairs_w = 0;
+  double us = 0.0, us_w = 0.0;
+  bool wide = false;
+  if (force_gemm == 3 && may_wide) {
+    if (!pair_schedule_cached(w, s, sm_count, true, &pw, &pairs_w, &us_w)) return BATQ_ERR_SHAPE;
+    wide = true;
+  } else {
+    if (!pair_schedule_cached(w, s, sm_count, false, &p, &pairs, &us)) return BATQ_ERR_SHAPE;
+    if (force_gemm == 0 && may_wide &&
+        pair_schedule_cached(w, s, sm_count, true, &pw, &pairs_w, &us_w))
+      wide = us_w < us;
+  }
+  CUtensorMap tmap_y64;
+  std::memset(&tmap_y64, 0, sizeof(tmap_y64));
+  if (wide) {
+    p = pw;
+    pairs = pairs_w;
+    if (m16 > 0) {   // the wide kernel stages its output in boxes of 64-byte rows
+      st = make_y_tmap(&tmap_y64, y, s, m16, ldy, bf, 64);
+      if (st != BATQ_OK) return st;
+    }
+  }
   p.katoms = w->katoms;
   p.k_steps = static_cast<int32_t>((w->n + 255) / 256);
   p.m16 = static_cast<int32_t>(m16);
   p.y = y;
   p.ldy = ldy;
   const int grid = 2 * pairs;
-  const cudaError_t e = bf ? launch_pair_kernel<true>(grid, stream, dependent, tmap_a, w->tmap_b32, tmap_sfa, w->tmap_sf, tmap_y, p)
-                           : launch_pair_kernel<false>(grid, stream, dependent, tmap_a, w->tmap_b32, tmap_sfa, w->tmap_sf, tmap_y, p);
+  cudaError_t e;
+  if (wide) e = bf ? launch_pair_kernel<true, true>(grid, stream, dependent, tmap_a, w->tmap_b32, tmap_sfa, w->tmap_sf, tmap_y64, p)
+                   : launch_pair_kernel<false, true>(grid, stream, dependent, tmap_a, w->tmap_b32, tmap_sfa, w->tmap_sf, tmap_y64, p);
+  else      e = bf ? launch_pair_kernel<true, false>(grid, stream, dependent, tmap_a, w->tmap_b32, tmap_sfa, w->tmap_sf, tmap_y, p)
+                   : launch_pair_kernel<false, false>(grid, stream, dependent, tmap_a, w->tmap_b32, tmap_sfa, w->tmap_sf, tmap_y, p);
   if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
   return BATQ_OK;
 }
@@ -752,7 +905,7 @@ batq_status launch_gemm(const void* x_codes, const void* x_sf, const batq_weight
   if (st != BATQ_OK) return st;
   // CTA pairs need at least two 128-token tiles to pay, and wide enough a layer for their tiles.
   const int force_gemm = g_force_gemm_kernel.load(std::memory_order_relaxed);
-  const bool use_pair = force_gemm == 2 || (force_gemm == 0 && s > 128 && w->m >= 192);
+  const bool use_pair = force_gemm == 2 || force_gemm == 3 || (force_gemm == 0 && s > 128 && w->m >= 192);
   if (use_pair) return launch_gemm_pair(x_codes, x_sf, w, s, y, bf, ldy, stream, info->sm_count, tmap_a, tmap_y, m16, dependent);
   const int bn = pick_bn(s, w->m, w->n, info->sm_count);
   GemmParams p{};
@@ -1052,7 +1205,8 @@ batq_status launch_linear_prefill_fused(const batq_transform* t, const batq_weig
   if (st != BATQ_OK) return st;
   PrefillFusedParams q{};
   int pairs = 0;
-  if (!pair_schedule_cached(w, s, info->sm_count, &q.g, &pairs)) return BATQ_ERR_SHAPE;
+  double sched_us = 0.0;
+  if (!pair_schedule_cached(w, s, info->sm_count, false, &q.g, &pairs, &sched_us)) return BATQ_ERR_SHAPE;
   q.g.katoms = w->katoms;
   q.g.k_steps = static_cast<int32_t>((n + 255) / 256);
   q.g.m16 = static_cast<int32_t>(m16);
@@ -1601,6 +1755,30 @@ int32_t batq_debug_pair_schedule(int64_t s, int64_t m, int64_t n, int32_t sm_cou
   PairParams p{};
   int pairs = 0;
   if (!pair_schedule(s, m, (n + 255) / 256, sm_count, &p, &pairs)) return -1;
+  if (pair < 0) return pairs;
+  if (pair >= pairs) return 0;
+  PairWalk w(p, pair, pairs);
+  PairTile t;
+  int32_t cnt = 0;
+  while (w.next(t)) {
+    if (tiles != nullptr && cnt < max_tiles) {
+      tiles[3 * cnt] = t.mp;
+      tiles[3 * cnt + 1] = t.n0;
+      tiles[3 * cnt + 2] = t.bn;
+    }
+    ++cnt;
+  }
+  return cnt;
+}
+int32_t batq_debug_wide_schedule(int64_t s, int64_t m, int64_t n, int32_t sm_count, int32_t pair, int32_t* tiles,
+                                 int32_t max_tiles) {
+  if (s <= 0 || m <= 0 || n <= 0 || sm_count < 2) return -1;
+  PairParams p{};
+  int pairs = 0;
+  double us = 0.0;
+  const int force_bn = g_force_bn.load(std::memory_order_relaxed);
+  const bool fw = force_bn >= 64 && force_bn <= kWideMaxBn && force_bn % 64 == 0;
+  if (!wide_schedule(s, m, (n + 255) / 256, sm_count, fw ? force_bn : 0, &p, &pairs, &us)) return -1;
   if (pair < 0) return pairs;
   if (pair >= pairs) return 0;
   PairWalk w(p, pair, pairs);

@@ -31,9 +31,10 @@ def qmode(request, batq):
     batq.batq_debug_force_quantizer(0)
 
 
-@pytest.fixture(params=[1, 2], ids=["cta", "ctapair"])
+@pytest.fixture(params=[1, 2, 3], ids=["cta", "ctapair", "widepair"])
 def gkernel(request, batq):
-    """Runs a test once per prefill GEMM kernel (one CTA per tile / CTA pairs)."""
+    """Runs a test once per prefill GEMM kernel (one CTA per tile / CTA pairs with two accumulators
+    / CTA pairs with tiles of up to 448 features)."""
     batq.batq_debug_force_gemm_kernel(request.param)
     yield request.param
     batq.batq_debug_force_gemm_kernel(0)
@@ -596,9 +597,11 @@ def test_gemm_vs_oracle_same_codes(batq, gkernel, S, M, N):
     assert np.max(np.abs(got - Y) / (Sabs + 1e-30)) < 1e-5
 
 
-@pytest.mark.parametrize("bn", [64, 128, 192, 256, 448])
+@pytest.mark.parametrize("bn", [64, 128, 192, 256, 320, 384, 448])
 @pytest.mark.parametrize("S,M,N", [(300, 520, 3584), (129, 257, 2048 + 32), (260, 1000, 512), (600, 2300, 768)])
 def test_gemm_every_tile_width(batq, gkernel, bn, S, M, N):
+    if bn in (320, 384) and gkernel != 3:
+        pytest.skip("only the wide-tile kernel has these widths")
     batq.batq_debug_force_tile_width(bn)
     try:
         got, Y, Sabs = _gemm_case(batq, S, M, N, 700 + S)
@@ -610,8 +613,10 @@ def test_gemm_every_tile_width(batq, gkernel, bn, S, M, N):
     assert np.array_equal(got16.astype(np.float32), want16)
 
 
-@pytest.mark.parametrize("bn", [64, 128, 192, 256, 448])
+@pytest.mark.parametrize("bn", [64, 128, 192, 256, 320, 384, 448])
 def test_gemm_scale_layout_localising_case_every_tile_width(batq, gkernel, bn):
+    if bn in (320, 384) and gkernel != 3:
+        pytest.skip("only the wide-tile kernel has these widths")
     batq.batq_debug_force_tile_width(bn)
     try:
         test_gemm_scale_layout_localising_case(batq)

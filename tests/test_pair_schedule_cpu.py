@@ -94,3 +94,56 @@ def test_schedule_ends_the_pairs_together():
     for tiles in sched:
         assert all(not (a[2] == 256 and b[2] == 256) for a, b in zip(tiles, tiles[1:]))
     assert sum(t[2] for tiles in sched for t in tiles) == 8 * 6144
+
+
+# ---------------------------------------------------------------------------- wide tiles (one accumulator of up to 448 columns)
+def _check_wide(sched, s, m):
+    rows = -(-s // 256)
+    cover = np.zeros((rows, -(-m // 64)), dtype=np.int32)
+    cols = {}
+    for p, tiles in enumerate(sched):
+        for i, (mp, n0, bn) in enumerate(tiles):
+            assert n0 % 64 == 0 and bn % 64 == 0 and 64 <= bn <= 448 and 0 <= mp < rows
+            cols.setdefault(n0, set()).add(bn)
+            cover[mp, n0 // 64:(n0 + bn) // 64] += 1
+    assert np.all(cover == 1)
+    starts = sorted(cols)
+    assert all(len(v) == 1 for v in cols.values())
+    widths = [next(iter(cols[c])) for c in starts]
+    index = {c: k for k, c in enumerate(starts)}
+    for p, tiles in enumerate(sched):
+        for i, (mp, n0, bn) in enumerate(tiles):
+            assert index[n0] * rows + mp == p + i * len(sched)
+    # at most two widths before the ragged last column
+    assert len(set(widths[:-1])) <= 2
+    assert starts[-1] + widths[-1] >= m > starts[-1] + widths[-1] - 64
+    counts = [len(t) for t in sched]
+    assert max(counts) - min(counts) <= 1
+    return widths
+
+
+@pytest.mark.parametrize("s,m,n", SHAPES)
+@pytest.mark.parametrize("sm_count", [148, 132, 2])
+def test_wide_tiles_cover_the_output_once(s, m, n, sm_count):
+    sched = B.batq_debug_wide_schedule(s, m, n, sm_count)
+    assert 1 <= len(sched) <= max(1, sm_count // 2)
+    _check_wide(sched, s, m)
+
+
+@pytest.mark.parametrize("bn", [64, 128, 192, 256, 320, 384, 448])
+def test_wide_forced_widths(bn):
+    for s, m, n in SHAPES[:8]:
+        B.batq_debug_force_tile_width(bn)
+        try:
+            sched = B.batq_debug_wide_schedule(s, m, n)
+        finally:
+            B.batq_debug_force_tile_width(0)
+        widths = _check_wide(sched, s, m)
+        assert all(w == bn for w in widths[:-1])
+
+
+def test_wide_schedule_of_the_gate_up_projection():
+    """28672 features at 2048 tokens on 74 pairs: 64 columns of 448 give every pair 6 or 7 tiles."""
+    sched = B.batq_debug_wide_schedule(2048, 28672, 4096)
+    cols = [sum(t[2] for t in tiles) for tiles in sched]
+    assert max(cols) <= 3200 and len(sched) == 74
