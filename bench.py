@@ -58,12 +58,12 @@ FP8_OVER_BF16 = 2.0       # nominal dense peak ratio 4.5 / 2.25 PFLOP/s
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, MB per step = the four GEMM launches of
 # cfg1_llama8b_prefill) from the ncu capture summarised under profiles/, valid for the kernel source
 # with this hash only.
-GEMM_TRAFFIC = {"workload": "cfg1_llama8b_prefill", "mb_per_step": 213.4, "source_sha256": "9a42d26cc1a1a606"}
+GEMM_TRAFFIC = {"workload": "cfg1_llama8b_prefill", "mb_per_step": 214.5, "source_sha256": "86454977d11cfd34"}
 
 
 def kernel_source_hash():
     h = hashlib.sha256()
-    for f in ("gemm_mxfp4.cuh", "gemm_mxfp4_pair.cuh", "ptx.cuh"):
+    for f in ("gemm_mxfp4.cuh", "gemm_mxfp4_pair.cuh", "gemm_mxfp4_wide.cuh", "ptx.cuh"):
         with open(os.path.join(ROOT, "paper_2603_16590_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -638,7 +638,8 @@ def run_ours(args):
         nominal_at_clock = (NOMINAL_FP4_TFLOPS / 2 if a8 else NOMINAL_FP4_TFLOPS) * mhz / mhz_max if mhz and mhz_max else None
         nominal_peak = NOMINAL_FP4_TFLOPS / 2 if a8 else NOMINAL_FP4_TFLOPS
         b2b_peak = peaks["bf16_tflops"] * (FP8_OVER_BF16 if a8 else FP4_OVER_BF16)
-        roof = {"bound": "tensor", "kernel": "gemm_w4a8_kernel" if a8 else ("gemm_mxfp4_pair_kernel" if S > 128 else "gemm_mxfp4_kernel"),
+        roof = {"bound": "tensor", "kernel": "gemm_w4a8_kernel" if a8 else ("gemm_mxfp4_wide_kernel / gemm_mxfp4_pair_kernel (per layer, by the "
+                                                                "library's cost model)" if S > 128 else "gemm_mxfp4_kernel"),
                 "achieved": gemm_achieved, "peak": fp4_peak,
                 "events": "around every launch in every %dth step of the timed region (%d steps) and in %d more steps "
                           "right after it" % (EVENT_EVERY, len(sampled), extra),
