@@ -357,11 +357,11 @@ def measure_mma_peak(B, torch, iters):
 
 
 def measure_mma_with_loads(B, torch, w, iters=8192):
-    """What a streaming GEMM can reach at most with 256 x 256 tiles per CTA pair: the MMA-only loop
-    with, beside it in every CTA, a TMA load stream of the GEMM's volume (32 KiB of a prepared
-    weight, L2-resident, per K-step) into a ring nobody reads.  No barrier couples the two, so the
-    result is what the tensor cores and the path from L2 to shared memory sustain together; a GEMM
-    adds its hand-shakes on top.  Also the two alone, and the MMAs with half the loads."""
+    """A probe of how the tensor cores and the path from L2 into shared memory get along: the MMA-only
+    loop with, beside it in every CTA, a TMA load stream of a 256 x 256 pair tile's volume (32 KiB
+    of a prepared weight, L2-resident, per K-step) into a ring nobody reads.  No barrier couples
+    the two.  Also the two alone, and the MMAs with fewer loads.  Context for the GEMM's fraction,
+    not a ceiling: the GEMM's own access pattern takes in more bytes per second than this stream."""
     def timed(it, lit):
         B.batq_debug_mma_peak_with_loads(w, True, 256, min(it, 256), min(lit, 256))
         torch.cuda.synchronize()
