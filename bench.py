@@ -333,13 +333,14 @@ def timed_region(h, step, steps, warmup):
     return h.max_over_ranks(e0.elapsed_time(e1)), clocks
 
 
-def measure_mma_peak(B, torch, iters):
-    """The block-scaled FP4 tensor-core rate with operands resident in shared memory (MMA-only loop,
-    every SM busy, nothing loaded or stored): CTA pairs on 256 x 256 tiles and single CTAs on
-    128 x 256 tiles, one timed launch each after a short warm-up launch."""
-    out = {}
-    for name, pair, sfc in (("pair_256x256", True, False), ("cta_128x256", False, False),
-                            ("pair_256x256_with_scale_copies", True, True), ("cta_128x256_with_scale_copies", False, True)):
+def measure_mma_peak(B, torch, iters, a8=False):
+    """The block-scaled tensor-core rate with operands resident in shared memory (MMA-only loop, every
+    SM busy, nothing loaded or stored): CTA pairs on 256 x 256 tiles and single CTAs on 128 x 256
+    tiles, one timed launch each after a short warm-up launch.  a8: kind::mxf8f6f4 (the W4A8 GEMM's
+    instruction) instead of kind::mxf4.  For kind::mxf4 also: the CTA-pair GEMM's own issue loop on
+    the same resident operands, and the wide-tile GEMM's issue pattern (a second MMA of width 192
+    into a second accumulator after every MMA)."""
+    def timed(pair, sfc):
         B.batq_debug_mma_peak(pair, 256, max(64, iters // 50), sfc)
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -348,12 +349,29 @@ def measure_mma_peak(B, torch, iters):
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1)
-        out[name] = {"tflops": flops / (ms * 1e-3) / 1e12, "ms": ms}
+        return {"tflops": flops / (ms * 1e-3) / 1e12, "ms": ms}
+    out = {}
+    B.batq_debug_mma_peak_kind(a8)
+    try:
+        for name, pair, sfc in (("pair_256x256", True, False), ("cta_128x256", False, False),
+                                ("pair_256x256_with_scale_copies", True, True), ("cta_128x256_with_scale_copies", False, True)):
+            out[name] = timed(pair, sfc)
+        if not a8:
+            B.batq_debug_mma_peak_gemm_loop(True)
+            out["pair_256x256_issued_by_the_gemm_loop"] = timed(True, True)
+            B.batq_debug_mma_peak_gemm_loop(False)
+            B.batq_debug_mma_peak_second_width(192)
+            out["pair_256x448_two_accumulators"] = timed(True, True)
+    finally:
+        B.batq_debug_mma_peak_kind(False)
+        B.batq_debug_mma_peak_gemm_loop(False)
+        B.batq_debug_mma_peak_second_width(0)
     if B.batq_last_device_status() != 0:
         raise SystemExit("device status after the MMA-only loop")
-    best = max((k for k in out if "scale_copies" not in k), key=lambda k: out[k]["tflops"])
+    best = max((k for k in ("pair_256x256", "cta_128x256")), key=lambda k: out[k]["tflops"])
     return {"tflops": out[best]["tflops"], "shape": best, "variants": out,
-            "how": "tcgen05.mma kind::mxf4.block_scale only, %d K-steps per CTA (pair), CUDA events" % iters}
+            "how": "tcgen05.mma kind::%s.block_scale only, %d K-steps per CTA (pair), CUDA events"
+                   % ("mxf8f6f4" if a8 else "mxf4", iters)}
 
 
 def measure_mma_with_loads(B, torch, w, iters=8192):
@@ -445,6 +463,7 @@ def run_peak(args, h, B, peaks):
     (launches back to back for about a second, under the power cap), with the clocks sampled."""
     import torch
     burst = measure_mma_peak(B, torch, 20000)
+    burst_a8 = measure_mma_peak(B, torch, 10000, a8=True)
     pair = burst["shape"].startswith("pair")
     wq = B.batq_prepare_weight(None, B.bits_to_cuda_bf16(synth.make_weight(8192, 4096, synth.BASE_SEED + 77)))
     with_loads = measure_mma_with_loads(B, torch, wq)
@@ -470,7 +489,8 @@ def run_peak(args, h, B, peaks):
             "warmup": 1, "ms_per_step": ms / n, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "mxfp4", "data": "synthetic",
             "config": {"workload": "peak_mxf4", "shape": burst["shape"], "k_steps_per_launch": 20000},
-            "burst": burst, "sustained": {"tflops": sustained, "ms": ms}, "with_loads": with_loads,
+            "burst": burst, "burst_mxf8f6f4": burst_a8, "sustained": {"tflops": sustained, "ms": ms},
+            "with_loads": with_loads,
             "context": {"cublas_bf16_x4_burst": peaks["bf16_tflops"] * FP4_OVER_BF16,
                         "cublas_bf16_x4_sustained": peaks["bf16_tflops_sustained"] * FP4_OVER_BF16,
                         "nominal": NOMINAL_FP4_TFLOPS, "source": peaks["source"]},
@@ -592,7 +612,7 @@ def run_ours(args):
             gg, r = graph_of(lambda L=L: f_gemm(L["codes"], L["sf"], L["w"], S, L["y"]))
             gq, _ = graph_of(lambda L=L: f_quant(L["tr"], L["x"], L["codes"], L["sf"], B.SF_MMA))
             b2b.append((time_graph(gq, r), time_graph(gg, r)))
-        mma_only = measure_mma_peak(B, torch, 20000) if (S > 128 and not a8) else None
+        mma_only = measure_mma_peak(B, torch, 20000, a8) if S > 128 else None
         big_w = max(layers, key=lambda L: L["m"] * L["n"])["w"]
         mma_loads = measure_mma_with_loads(B, torch, big_w) if (S > 128 and not a8) else None
         big_quant = measure_big_quantizer(B, torch, seed) if (S > 128 and h.rank == 0 and not a8) else None
@@ -638,7 +658,7 @@ def run_ours(args):
         nominal_at_clock = (NOMINAL_FP4_TFLOPS / 2 if a8 else NOMINAL_FP4_TFLOPS) * mhz / mhz_max if mhz and mhz_max else None
         nominal_peak = NOMINAL_FP4_TFLOPS / 2 if a8 else NOMINAL_FP4_TFLOPS
         b2b_peak = peaks["bf16_tflops"] * (FP8_OVER_BF16 if a8 else FP4_OVER_BF16)
-        roof = {"bound": "tensor", "kernel": "gemm_w4a8_kernel" if a8 else ("gemm_mxfp4_wide_kernel / gemm_mxfp4_pair_kernel (per layer, by the "
+        roof = {"bound": "tensor", "kernel": "gemm_w4a8_wide_kernel / gemm_w4a8_pair_kernel (per layer)" if a8 else ("gemm_mxfp4_wide_kernel / gemm_mxfp4_pair_kernel (per layer, by the "
                                                                 "library's cost model)" if S > 128 else "gemm_mxfp4_kernel"),
                 "achieved": gemm_achieved, "peak": fp4_peak,
                 "events": "around every launch in every %dth step of the timed region (%d steps) and in %d more steps "

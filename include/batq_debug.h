@@ -108,6 +108,23 @@ batq_status batq_debug_mma_peak(int32_t pair, int32_t bn, int32_t iters, int32_t
  * *flops_out and *bytes_out (host, may be NULL) receive the launch's floating-point operations and
  * loaded plus stored bytes.  What the numbers show: whether the tensor cores and a stream into
  * shared memory slow one another down when no barrier couples them. */
+/* a8 != 0: the loops below issue tcgen05.mma kind::mxf8f6f4 (E4M3 x E2M1 in 8-bit containers, K = 32
+ * per MMA, 128 elements per K-step: the W4A8 GEMM's instruction) instead of kind::mxf4; the flops
+ * reported follow. */
+void batq_debug_mma_peak_kind(int32_t a8);
+/* bn2 in {64, 128, 192} (kind::mxf4 only; anything else switches it off): every MMA of the loops
+ * below is followed by one of width bn2 on the same operands into a second accumulator (tensor
+ * memory columns 256..), the issue pattern of the wide-tile GEMM. */
+void batq_debug_mma_peak_second_width(int32_t bn2);
+/* on != 0 (kind::mxf4, one accumulator): the MMAs are issued by the CTA-pair GEMM's own loop, statement
+ * for statement (a wait on a completed barrier phase, a fence, the scale copies into alternating
+ * slots, four MMAs from descriptors that depend on a run-time stage index and a commit per K-step),
+ * on the same resident operands: what that loop costs with the operand stream taken away. */
+void batq_debug_mma_peak_gemm_loop(int32_t on);
+/* Tensor-memory column at which the loops below keep their scale factors: a multiple of 4 behind
+ * the accumulators (from 256, from 448 with a second accumulator) up to 488; anything else = right
+ * behind the accumulators. */
+void batq_debug_mma_peak_sf_column(int32_t col);
 void batq_debug_mma_peak_load_stages(int32_t stages);   /* ring depth of the load stream, 1..5 (default 4) */
 /* How many CTAs (consecutive block indices) load the same boxes at the same time, as the tiles of a
  * GEMM that share a row or column block do; 1 (default) = every CTA its own boxes. */

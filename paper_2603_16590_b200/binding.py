@@ -61,6 +61,10 @@ SIGNATURES = {
     "batq_last_device_status": (C.c_int, [_P]),
     "batq_debug_wait_timeout": (C.c_int, [_I64, _P]),
     "batq_debug_mma_peak": (C.c_int, [_I32, _I32, _I32, _I32, C.POINTER(C.c_double), _P]),
+    "batq_debug_mma_peak_kind": (None, [_I32]),
+    "batq_debug_mma_peak_second_width": (None, [_I32]),
+    "batq_debug_mma_peak_gemm_loop": (None, [_I32]),
+    "batq_debug_mma_peak_sf_column": (None, [_I32]),
     "batq_debug_mma_peak_load_stages": (None, [_I32]),
     "batq_debug_mma_peak_load_sharing": (None, [_I32]),
     "batq_debug_mma_peak_load_from_peer": (None, [_I32]),
@@ -367,6 +371,22 @@ def batq_debug_mma_peak(pair: bool, bn: int, iters: int, sf_copies: bool = False
     _check(load().batq_debug_mma_peak(1 if pair else 0, bn, iters, 1 if sf_copies else 0, C.byref(flops), _stream()),
            "batq_debug_mma_peak")
     return flops.value
+
+
+def batq_debug_mma_peak_kind(a8: bool) -> None:
+    load().batq_debug_mma_peak_kind(1 if a8 else 0)
+
+
+def batq_debug_mma_peak_second_width(bn2: int) -> None:
+    load().batq_debug_mma_peak_second_width(bn2)
+
+
+def batq_debug_mma_peak_gemm_loop(on: bool) -> None:
+    load().batq_debug_mma_peak_gemm_loop(1 if on else 0)
+
+
+def batq_debug_mma_peak_sf_column(col: int) -> None:
+    load().batq_debug_mma_peak_sf_column(col)
 
 
 def batq_debug_mma_peak_load_stages(stages: int) -> None:

@@ -19,6 +19,8 @@
 #include "gemm_mxfp4_wide.cuh"
 #include "gemm_small_s.cuh"
 #include "gemm_w4a8.cuh"
+#include "gemm_w4a8_pair.cuh"
+#include "gemm_w4a8_wide.cuh"
 #include "linear_prefill_fused.cuh"
 #include "linear_small_s_fused.cuh"
 #include "mma_peak.cuh"
@@ -60,12 +62,14 @@ struct batq_weight {
   CUtensorMap tmap_b32;   // boxes of 32 weight rows: the CTA-pair kernel composes its half tiles from them
   CUtensorMap tmap_sf;    // scale atoms: [row tiles x KA] rows of 512 bytes, boxes of two atoms
   // CTA-pair schedules already worked out for this weight, by token count (host only)
-  struct SchedEntry { int64_t s; int force_bn; bool wide; double cost; int32_t n_cols, n_segs, pairs; batq::PairSeg seg[batq::kPairMaxSegs]; };
+  struct SchedEntry { int64_t s; int force_bn; bool wide, a8; double cost; int32_t n_cols, n_segs, pairs; batq::PairSeg seg[batq::kPairMaxSegs]; };
   mutable std::mutex sched_mutex;
   mutable std::vector<SchedEntry> sched_cache;
   bool has_u4;            // n % 128 == 0: the maps below exist (W4A8 GEMM)
   CUtensorMap tmap_u4_128;  // packed 4-bit codes widened to 8-bit containers by the TMA unit: boxes of
   CUtensorMap tmap_u4_256;  // 128 elements x 128 / 256 weight rows
+  CUtensorMap tmap_u4_32;   // 128 elements x 32 weight rows: the W4A8 CTA-pair kernel composes its half tiles from them
+  CUtensorMap tmap_sf1;     // scale atoms, boxes of one atom = the 4 blocks of one 128-element K step
 };
 
 // Scratch for batq_linear_w4a4_noalloc: part of the library image, one copy per GPU.
@@ -136,8 +140,18 @@ batq_status device_setup(int* device_out, const DeviceInfo** info_out) {
     e = e ? e : set_smem(gemm_w4a8_kernel<128, true>, W4A8Cfg<128>::kSmemBytes);
     e = e ? e : set_smem(gemm_w4a8_kernel<256, false>, W4A8Cfg<256>::kSmemBytes);
     e = e ? e : set_smem(gemm_w4a8_kernel<256, true>, W4A8Cfg<256>::kSmemBytes);
-    e = e ? e : set_smem(mma_peak_kernel<false>, kPeakSmemBytesLoads);
-    e = e ? e : set_smem(mma_peak_kernel<true>, kPeakSmemBytesLoads);
+    e = e ? e : set_smem(gemm_w4a8_pair_kernel<false>, A8PairCfg::kSmemBytes);
+    e = e ? e : set_smem(gemm_w4a8_pair_kernel<true>, A8PairCfg::kSmemBytes);
+    e = e ? e : set_smem(gemm_w4a8_wide_kernel<false>, A8WideCfg::kSmemBytes);
+    e = e ? e : set_smem(gemm_w4a8_wide_kernel<true>, A8WideCfg::kSmemBytes);
+    e = e ? e : set_smem(mma_peak_kernel<false, 0>, kPeakSmemBytesLoads);
+    e = e ? e : set_smem(mma_peak_kernel<true, 0>, kPeakSmemBytesLoads);
+    e = e ? e : set_smem(mma_peak_kernel<false, 1>, kPeakSmemBytesLoads);
+    e = e ? e : set_smem(mma_peak_kernel<true, 1>, kPeakSmemBytesLoads);
+    e = e ? e : set_smem(mma_peak_kernel<false, 2>, kPeakSmemBytesLoads);
+    e = e ? e : set_smem(mma_peak_kernel<true, 2>, kPeakSmemBytesLoads);
+    e = e ? e : set_smem(mma_peak_kernel<false, 3>, kPeakSmemBytesLoads);
+    e = e ? e : set_smem(mma_peak_kernel<true, 3>, kPeakSmemBytesLoads);
     e = e ? e : set_smem(gemm_mxfp4_pair_kernel<false>, PairCfg::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_pair_kernel<true>, PairCfg::kSmemBytes);
     e = e ? e : set_smem(gemm_mxfp4_wide_kernel<false>, WideCfg::kSmemBytes);
@@ -218,8 +232,8 @@ batq_status make_tmap_2d(CUtensorMap* map, CUtensorMapDataType dt, int esz, cons
 
 // Tensor map over scale bytes in the BATQ_SF_MMA layout: one row per 512-byte atom (128 uint32),
 // boxes of two consecutive atoms = the 8 blocks of one K step; rows past the buffer read as zero.
-batq_status make_sf_tmap(CUtensorMap* map, const void* base, int64_t row_tiles, int64_t katoms) {
-  return make_tmap_2d(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, base, 128, row_tiles * katoms, 512, 128, 2,
+batq_status make_sf_tmap(CUtensorMap* map, const void* base, int64_t row_tiles, int64_t katoms, int box_atoms = 2) {
+  return make_tmap_2d(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, base, 128, row_tiles * katoms, 512, 128, box_atoms,
                       CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 
@@ -674,8 +688,10 @@ bool pair_schedule(int64_t s, int64_t m, int64_t k_steps, int sm_count, PairPara
 // 0.17 + 0.0009 bn us (0.40 at 256, 0.52 at 384: the bytes the SM pulls from L2), one of a 448-wide
 // tile 0.66 us (four stages of 49 KiB turn over at the latency of a load from L2); about 1.4 us
 // per tile pass between the last MMA of one tile and the first of the next.
-double wide_tile_us(int bn, int64_t k_steps) {
-  const double step = bn > 384 ? 0.66 : 0.17 + 0.0009 * bn;
+// With MXFP8 activations (a8) the tensor cores run at half the rate and are the only limit:
+// 0.60 us per 256 elements of K at 256 columns, in proportion to the width.
+double wide_tile_us(int bn, int64_t k_steps, bool a8 = false) {
+  const double step = a8 ? 0.60 * bn / 256.0 : (bn > 384 ? 0.66 : 0.17 + 0.0009 * bn);
   return static_cast<double>(k_steps) * step + 1.4;
 }
 // The same for the two-accumulator kernel: bound by its loads (36 KiB per K-step at 256 columns),
@@ -684,7 +700,7 @@ double pair_tile_us(int bn, int64_t k_steps, bool same_slot) {
   return static_cast<double>(k_steps) * 0.383 * (32.0 + bn / 8.0) / 64.0 + (same_slot ? 1.7 : 1.1);
 }
 
-double wide_cost(const PairSched& c, PairParams* p, int64_t k_steps, int max_pairs, int* pairs_out) {
+double wide_cost(const PairSched& c, PairParams* p, int64_t k_steps, int max_pairs, bool a8, int* pairs_out) {
   p->n_cols = c.n_cols;
   p->n_segs = c.n_segs;
   for (int i = 0; i < kPairMaxSegs; ++i) p->seg[i] = c.seg[i];
@@ -695,7 +711,7 @@ double wide_cost(const PairSched& c, PairParams* p, int64_t k_steps, int max_pai
     PairWalk walk(*p, pr, np);
     PairTile t;
     double cost = 0.0;
-    while (walk.next(t)) cost += wide_tile_us(t.bn, k_steps);
+    while (walk.next(t)) cost += wide_tile_us(t.bn, k_steps, a8);
     worst = std::max(worst, cost);
   }
   return worst + 5.5;   // launch, first loads, the last tile's stores
@@ -722,7 +738,7 @@ double pair_cost_us(PairParams* p, int64_t k_steps, int np) {
   return worst + 1.5;   // the last tile's epilogue
 }
 
-bool wide_schedule(int64_t s, int64_t m, int64_t k_steps, int sm_count, int force_w, PairParams* p, int* pairs,
+bool wide_schedule(int64_t s, int64_t m, int64_t k_steps, int sm_count, int force_w, bool a8, PairParams* p, int* pairs,
                    double* cost_us) {
   const int64_t m_pairs = (s + 255) / 256;
   const int max_pairs = std::max(1, sm_count / 2);
@@ -737,7 +753,7 @@ bool wide_schedule(int64_t s, int64_t m, int64_t k_steps, int sm_count, int forc
     const int64_t end = l.n0 + seg_span(l.wa, l.wb, l.cols);
     if (end < m || end - l.wb >= m) return;
     int np;
-    const double cost = wide_cost(c, p, k_steps, max_pairs, &np);
+    const double cost = wide_cost(c, p, k_steps, max_pairs, a8, &np);
     if (cost < best_cost - 1e-9) { best_cost = cost; best = c; best.pairs = np; }
   };
   const int widths[6] = {448, 384, 320, 256, 192, 128};
@@ -779,12 +795,13 @@ bool wide_schedule(int64_t s, int64_t m, int64_t k_steps, int sm_count, int forc
 // The same, remembered per prepared weight and token count (the search walks a few hundred
 // candidates; a layer is called with few distinct token counts).
 bool pair_schedule_cached(const batq_weight* w, int64_t s, int sm_count, bool wide, PairParams* p, int* pairs,
-                          double* cost_us) {
+                          double* cost_us, bool a8 = false) {
+  a8 = a8 && wide;   // the activations' format only enters the wide tiles' cost
   const int force_bn = g_force_bn.load(std::memory_order_relaxed);
   {
     std::lock_guard<std::mutex> lock(w->sched_mutex);
     for (const auto& e : w->sched_cache)
-      if (e.s == s && e.force_bn == force_bn && e.wide == wide) {
+      if (e.s == s && e.force_bn == force_bn && e.wide == wide && e.a8 == a8) {
         p->s = static_cast<int32_t>(s);
         p->m = static_cast<int32_t>(w->m);
         p->m_pairs = static_cast<int32_t>((s + 255) / 256);
@@ -799,13 +816,13 @@ bool pair_schedule_cached(const batq_weight* w, int64_t s, int sm_count, bool wi
   const int64_t k_steps = (w->n + 255) / 256;
   if (wide) {
     const bool fw = force_bn >= 64 && force_bn <= kWideMaxBn && force_bn % 64 == 0;
-    if (!wide_schedule(s, w->m, k_steps, sm_count, fw ? force_bn : 0, p, pairs, cost_us)) return false;
+    if (!wide_schedule(s, w->m, k_steps, sm_count, fw ? force_bn : 0, a8, p, pairs, cost_us)) return false;
   } else {
     if (!pair_schedule(s, w->m, k_steps, sm_count, p, pairs)) return false;
     *cost_us = pair_cost_us(p, k_steps, *pairs);
   }
   batq_weight::SchedEntry e{};
-  e.s = s; e.force_bn = force_bn; e.wide = wide; e.cost = *cost_us;
+  e.s = s; e.force_bn = force_bn; e.wide = wide; e.a8 = a8; e.cost = *cost_us;
   e.n_cols = p->n_cols; e.n_segs = p->n_segs; e.pairs = *pairs;
   for (int i = 0; i < kPairMaxSegs; ++i) e.seg[i] = p->seg[i];
   std::lock_guard<std::mutex> lock(w->sched_mutex);
@@ -1269,7 +1286,82 @@ batq_status launch_gemm_w4a8(const void* x_codes8, const void* x_sf, const batq_
   const int64_t m16 = w->m / (bf ? 8 : 4) * (bf ? 8 : 4);
   if (st == BATQ_OK && m16 > 0) st = make_y_tmap(&tmap_y, y, s, m16, ldy, bf);
   if (st != BATQ_OK) return st;
-  // Tile width: 256 (half the operand bytes per flop of a 128-wide tile; measured 16 % faster on
+  // CTA pairs above 128 tokens (two 128-token tiles to share a weight tile), as in the W4A4 GEMM:
+  // tiles of up to 256 features on two accumulators, or tiles of up to 448 on one.  kind::mxf8f6f4
+  // runs at half the rate of kind::mxf4, so the wide tile (fewer bytes per flop, tensor-bound) is
+  // the rule here; the two-accumulator kernel keeps the layers where a pair has at most two tiles
+  // whichever way the features are cut.
+  const int force_gemm = g_force_gemm_kernel.load(std::memory_order_relaxed);
+  if (force_gemm == 2 || force_gemm == 3 || (force_gemm == 0 && s > 128 && w->m >= 192)) {
+    CUtensorMap tmap_sfa, tmap_y64;
+    std::memset(&tmap_y64, 0, sizeof(tmap_y64));
+    st = make_sf_tmap(&tmap_sfa, x_sf, (s + 127) / 128, w->katoms, 1);
+    if (st != BATQ_OK) return st;
+    const int force_bn = g_force_bn.load(std::memory_order_relaxed);
+    const bool forced_w = force_bn >= 64 && force_bn <= kWideMaxBn && force_bn % 64 == 0;
+    PairParams p{}, pw{};
+    int pairs = 0, pairs_w = 0;
+    double us = 0.0, us_w = 0.0;
+    bool wide = false;
+    if (force_gemm == 3) {
+      if (force_bn != 0 && !forced_w) return BATQ_ERR_SHAPE;
+      if (!pair_schedule_cached(w, s, info->sm_count, true, &pw, &pairs_w, &us_w, true)) return BATQ_ERR_SHAPE;
+      wide = true;
+    } else {
+      if (!pair_schedule_cached(w, s, info->sm_count, false, &p, &pairs, &us)) return BATQ_ERR_SHAPE;
+      if (force_gemm == 0 && force_bn == 0 && w->m >= 320 &&
+          pair_schedule_cached(w, s, info->sm_count, true, &pw, &pairs_w, &us_w, true)) {
+        // four or more tiles for some pair in the two-accumulator schedule: take the wide tiles
+        // (measured at 2048 tokens: gate/up, 14 tiles, 158 against 172 us; qkv, 3 tiles, 39.5 against 37.3)
+        int max_tiles = 0;
+        for (int pr = 0; pr < pairs; ++pr) {
+          PairWalk walk(p, pr, pairs);
+          PairTile t;
+          int cnt = 0;
+          while (walk.next(t)) ++cnt;
+          max_tiles = std::max(max_tiles, cnt);
+        }
+        wide = max_tiles >= 4;
+      }
+    }
+    if (wide) {
+      p = pw;
+      pairs = pairs_w;
+      if (m16 > 0) {
+        st = make_y_tmap(&tmap_y64, y, s, m16, ldy, bf, 64);
+        if (st != BATQ_OK) return st;
+      }
+    }
+    p.katoms = w->katoms;
+    p.k_steps = static_cast<int32_t>(w->n / kW4A8KElems);
+    p.m16 = static_cast<int32_t>(m16);
+    p.y = y;
+    p.ldy = ldy;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs));
+    cfg.blockDim = dim3(wide ? kWideThreads : kPairThreads);
+    cfg.dynamicSmemBytes = wide ? A8WideCfg::kSmemBytes : A8PairCfg::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 2 : 1;
+    cudaError_t e;
+    if (wide)
+      e = bf ? cudaLaunchKernelEx(&cfg, gemm_w4a8_wide_kernel<true>, tmap_a, w->tmap_u4_32, tmap_sfa, w->tmap_sf1, tmap_y64, p)
+             : cudaLaunchKernelEx(&cfg, gemm_w4a8_wide_kernel<false>, tmap_a, w->tmap_u4_32, tmap_sfa, w->tmap_sf1, tmap_y64, p);
+    else
+      e = bf ? cudaLaunchKernelEx(&cfg, gemm_w4a8_pair_kernel<true>, tmap_a, w->tmap_u4_32, tmap_sfa, w->tmap_sf1, tmap_y, p)
+             : cudaLaunchKernelEx(&cfg, gemm_w4a8_pair_kernel<false>, tmap_a, w->tmap_u4_32, tmap_sfa, w->tmap_sf1, tmap_y, p);
+    if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+    return BATQ_OK;
+  }
+  // One CTA per tile.  Tile width: 256 (half the operand bytes per flop of a 128-wide tile; measured 16 % faster on
   // the config-1 shapes at equal wave counts) unless 128-wide tiles need clearly fewer waves' worth
   // of time (a layer too small to fill the SMs with 256-wide tiles).
   const int64_t mt = (s + kBM - 1) / kBM;
@@ -1563,6 +1655,8 @@ batq_status batq_prepare_weight(const batq_transform* t, const void* w_bf16, int
   w->has_u4 = n % 128 == 0;
   if (st == BATQ_OK && w->has_u4) st = make_u4_unpack_tmap(&w->tmap_u4_128, w->codes, m, n, 128);
   if (st == BATQ_OK && w->has_u4) st = make_u4_unpack_tmap(&w->tmap_u4_256, w->codes, m, n, 256);
+  if (st == BATQ_OK && w->has_u4) st = make_u4_unpack_tmap(&w->tmap_u4_32, w->codes, m, n, 32);
+  if (st == BATQ_OK && w->has_u4) st = make_sf_tmap(&w->tmap_sf1, w->scales, (m + 127) / 128, w->katoms, 1);
   if (st != BATQ_OK) { delete w; return st; }
   *out = w;
   return BATQ_OK;
@@ -1778,7 +1872,7 @@ int32_t batq_debug_wide_schedule(int64_t s, int64_t m, int64_t n, int32_t sm_cou
   double us = 0.0;
   const int force_bn = g_force_bn.load(std::memory_order_relaxed);
   const bool fw = force_bn >= 64 && force_bn <= kWideMaxBn && force_bn % 64 == 0;
-  if (!wide_schedule(s, m, (n + 255) / 256, sm_count, fw ? force_bn : 0, &p, &pairs, &us)) return -1;
+  if (!wide_schedule(s, m, (n + 255) / 256, sm_count, fw ? force_bn : 0, false, &p, &pairs, &us)) return -1;
   if (pair < 0) return pairs;
   if (pair >= pairs) return 0;
   PairWalk w(p, pair, pairs);
@@ -1812,6 +1906,10 @@ batq_status batq_debug_wait_timeout(int64_t limit_ns, void* stream) {
 std::atomic<int> g_peak_load_stages{4};
 std::atomic<int> g_peak_load_sharing{1};
 std::atomic<int> g_peak_load_from_peer{0};
+std::atomic<int> g_peak_a8{0};
+std::atomic<int> g_peak_bn2{0};
+std::atomic<int> g_peak_gemm_loop{0};
+std::atomic<int> g_peak_sf_col{0};
 
 static batq_status launch_mma_peak(const batq_weight* w, int32_t pair, int32_t bn, int32_t iters, int32_t sf_copies,
                                    int32_t load_iters, int32_t store_iters, double* flops_out, double* bytes_out,
@@ -1835,6 +1933,14 @@ static batq_status launch_mma_peak(const batq_weight* w, int32_t pair, int32_t b
   p.load_stages = g_peak_load_stages.load(std::memory_order_relaxed);
   p.load_sharing = g_peak_load_sharing.load(std::memory_order_relaxed);
   p.load_from_peer = pair ? g_peak_load_from_peer.load(std::memory_order_relaxed) : 0;
+  const bool a8 = g_peak_a8.load(std::memory_order_relaxed) != 0;
+  p.bn2 = a8 ? 0 : g_peak_bn2.load(std::memory_order_relaxed);
+  const int kind = a8 ? 2 : (p.bn2 > 0 ? 1 : (g_peak_gemm_loop.load(std::memory_order_relaxed) != 0 ? 3 : 0));
+  {
+    const int want = g_peak_sf_col.load(std::memory_order_relaxed);
+    const int lowest = p.bn2 > 0 ? 448 : 256;
+    p.sf_col = (want >= lowest && want <= 512 - kPeakSfCols && want % 4 == 0) ? want : lowest;
+  }
   p.w_row_tiles = load_iters > 0 ? static_cast<int32_t>(w->m / 128) : 1;   // whole boxes only
   p.w_k_steps = load_iters > 0 ? static_cast<int32_t>(w->n / 256) : 1;
   CUtensorMap none{};
@@ -1852,11 +1958,14 @@ static batq_status launch_mma_peak(const batq_weight* w, int32_t pair, int32_t b
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pair ? 1 : 0;
-  const cudaError_t e = pair ? cudaLaunchKernelEx(&cfg, mma_peak_kernel<true>, map, p)
-                             : cudaLaunchKernelEx(&cfg, mma_peak_kernel<false>, map, p);
+  cudaError_t e;
+  if (kind == 0)      e = pair ? cudaLaunchKernelEx(&cfg, mma_peak_kernel<true, 0>, map, p) : cudaLaunchKernelEx(&cfg, mma_peak_kernel<false, 0>, map, p);
+  else if (kind == 1) e = pair ? cudaLaunchKernelEx(&cfg, mma_peak_kernel<true, 1>, map, p) : cudaLaunchKernelEx(&cfg, mma_peak_kernel<false, 1>, map, p);
+  else if (kind == 3) e = pair ? cudaLaunchKernelEx(&cfg, mma_peak_kernel<true, 3>, map, p) : cudaLaunchKernelEx(&cfg, mma_peak_kernel<false, 3>, map, p);
+  else                e = pair ? cudaLaunchKernelEx(&cfg, mma_peak_kernel<true, 2>, map, p) : cudaLaunchKernelEx(&cfg, mma_peak_kernel<false, 2>, map, p);
   if (e != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
   if (flops_out != nullptr)
-    *flops_out = 2.0 * (pair ? 256.0 : 128.0) * bn * 256.0 * iters * (pair ? ctas / 2 : ctas);
+    *flops_out = 2.0 * (pair ? 256.0 : 128.0) * (bn + p.bn2) * (a8 ? 128.0 : 256.0) * iters * (pair ? ctas / 2 : ctas);
   if (bytes_out != nullptr) *bytes_out = static_cast<double>(kPeakLoadStageBytes) * (load_iters + store_iters) * ctas;
   return BATQ_OK;
 }
@@ -1864,6 +1973,12 @@ static batq_status launch_mma_peak(const batq_weight* w, int32_t pair, int32_t b
 void batq_debug_mma_peak_load_stages(int32_t stages) {
   g_peak_load_stages.store(stages < 1 ? 1 : (stages > kPeakLoadStages ? kPeakLoadStages : stages), std::memory_order_relaxed);
 }
+void batq_debug_mma_peak_gemm_loop(int32_t on) { g_peak_gemm_loop.store(on != 0, std::memory_order_relaxed); }
+void batq_debug_mma_peak_sf_column(int32_t col) { g_peak_sf_col.store(col, std::memory_order_relaxed); }
+void batq_debug_mma_peak_second_width(int32_t bn2) {
+  g_peak_bn2.store((bn2 == 64 || bn2 == 128 || bn2 == 192) ? bn2 : 0, std::memory_order_relaxed);
+}
+void batq_debug_mma_peak_kind(int32_t a8) { g_peak_a8.store(a8 != 0, std::memory_order_relaxed); }
 void batq_debug_mma_peak_load_from_peer(int32_t on) { g_peak_load_from_peer.store(on != 0, std::memory_order_relaxed); }
 void batq_debug_mma_peak_load_sharing(int32_t ctas) {
   g_peak_load_sharing.store(ctas < 1 ? 1 : (ctas > 1024 ? 1024 : ctas), std::memory_order_relaxed);

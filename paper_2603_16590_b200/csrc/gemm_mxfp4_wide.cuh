@@ -29,6 +29,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "gemm_mxfp4_pair.cuh"
 #include "ptx.cuh"
 
@@ -221,9 +223,14 @@ gemm_mxfp4_wide_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
         ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&acc_empty_bar[0]), (n_tile & 1u) ^ 1u, &abort_flag));
         if (!ok) break;
         tc_fence_after_sync();
-        for (int kt = 0; kt < p.k_steps; ++kt) {
+        // One K-step.  FIRST (the tile's first: the accumulators start from zero, and part b's MMAs
+        // wait for part b of the accumulator) and TWO (the tile has a part b) are compile-time: the
+        // elected lane's instruction stream between two MMAs holds no run-time branch.
+        auto k_step = [&](auto first_c, auto two_c) {
+          constexpr bool FIRST = decltype(first_c)::value;
+          constexpr bool TWO = decltype(two_c)::value;
           ok = __all_sync(0xFFFFFFFFu, mbar_wait(full0 + 8u * stage, phase, &abort_flag));
-          if (!ok) break;
+          if (!ok) return;
           tc_fence_after_sync();
           const uint32_t soff = static_cast<uint32_t>(stage * (Cfg::kStageBytes >> 4));
           const uint64_t adesc = ab_desc0 + soff;
@@ -246,16 +253,16 @@ gemm_mxfp4_wide_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
               const uint32_t sfid = (kb & 1) * 2;
               const uint32_t sa = (sfa_col + 4 * c) | (sfid << 30);
               const uint32_t sb = (sfb_col + c * 4 * Cfg::kSfbAtoms) | (sfid << 30);
-              const uint32_t accum = (kt | kb) != 0 ? 1u : 0u;
-              tc_mma_mxf4_pair(tmem_base, adesc + 2 * kb, bdesc + 2 * kb, (kb & 1) ? ia1 : ia0, sa, sb, accum);
-              if (bnb > 0 && kt != 0)   // weight rows 256.. of the tile: eight scale columns (256 rows) further on
+              tc_mma_mxf4_pair(tmem_base, adesc + 2 * kb, bdesc + 2 * kb, (kb & 1) ? ia1 : ia0, sa, sb,
+                               (FIRST && kb == 0) ? 0u : 1u);
+              if (TWO && !FIRST)   // weight rows 256.. of the tile: eight scale columns (256 rows) further on
                 tc_mma_mxf4_pair(tmem_base + 256, adesc + 2 * kb, bdesc + b_part_b + 2 * kb, (kb & 1) ? ib1 : ib0, sa,
-                                 sb + 8, accum);
+                                 sb + 8, 1u);
             }
           }
-          if (bnb > 0 && kt == 0) {   // the first K-step: part a's MMAs are under way, now part b
+          if (TWO && FIRST) {   // part a's MMAs are under way, now part b
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&acc_empty_bar[1]), (n_tile & 1u) ^ 1u, &abort_flag));
-            if (!ok) break;
+            if (!ok) return;
             tc_fence_after_sync();
             if (elect_one()) {
 #pragma unroll
@@ -271,6 +278,15 @@ gemm_mxfp4_wide_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
           if (elect_one()) tc_commit_pair(empty0 + 8u * stage, 3);  // frees the stage in both CTAs
           __syncwarp();
           if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+        };
+        using yes = std::integral_constant<bool, true>;
+        using no = std::integral_constant<bool, false>;
+        if (bnb > 0) {
+          k_step(yes{}, yes{});
+          for (int kt = 1; kt < p.k_steps && ok; ++kt) k_step(no{}, yes{});
+        } else {
+          k_step(yes{}, no{});
+          for (int kt = 1; kt < p.k_steps && ok; ++kt) k_step(no{}, no{});
         }
         if (!ok) break;
         if (bnb == 0) {   // part b unused by this tile: take its barrier's phase along

@@ -1,0 +1,341 @@
+// MXFP8 (E4M3) activations x MXFP4 (E2M1) weights on CTA pairs (stage 3 of the W4A8
+// configurations of Sec. 4, prefill shapes):
+//
+//   Y[s, m] = sum_j 2^(ex[s,j] + ew[m,j]) * sum_{i<32} q8x[s,j,i] * q4w[m,j,i]
+//
+// The pipeline, work distribution, accumulator slots and barriers are those of
+// gemm_mxfp4_pair.cuh (two CTAs share a 256-token tile of up to 256 features; PairParams,
+// PairWalk, PairSlots); the operands are those of gemm_w4a8.cuh: tcgen05.mma kind::mxf8f6f4 takes
+// both element types in 8-bit containers, the packed 4-bit weight codes are widened on the way
+// into shared memory by the TMA unit (tensor-map type 16U4_ALIGN16B), and a K-step is 128
+// elements = one 128-byte swizzle row of either operand = four MMAs of K = 32, each with one scale
+// byte per row (one 512-byte atom per 128 rows and K-step).  Against one CTA per tile, a CTA
+// stages only half of the tile's weight rows: 16 + 8 KiB come from L2 per K-step instead of
+// 16 + 16, the stage shrinks from 50 to 34 KiB (five stages and two accumulators fit), and the
+// epilogue of a tile runs under the MMAs of the next.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "gemm_mxfp4_pair.cuh"
+#include "gemm_w4a8.cuh"
+#include "ptx.cuh"
+
+namespace batq {
+
+struct A8PairCfg {
+  static constexpr int kABytes = kBM * 128;               // 16 KiB: this CTA's 128 token rows, 128 E4M3 codes each
+  static constexpr int kBBytes = 128 * 128;               // this CTA's half of the widest tile, 8-bit containers
+  static constexpr int kSfaBytes = 512;                   // 128 rows x 4 blocks
+  static constexpr int kSfbAtoms = 3;                     // 128-row scale tiles a tile can touch (256 columns from row 64)
+  static constexpr int kSfbBytes = kSfbAtoms * 512;
+  static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;   // 34 KiB
+  static constexpr int kStages = 5;
+  static constexpr int kSlot1Col = 256;                   // accumulator slot 0: [0, 256), slot 1: [256, 448)
+  static constexpr int kSlot1Width = 192;
+  static constexpr int kAccCols = 448;
+  static constexpr int kSfCols = 4 + 4 * kSfbAtoms;       // scale columns of one K-step
+  static constexpr int kSfSlots = 2;
+  static constexpr int kTmemCols = 512;
+  static constexpr int kStagingBufs = 2;
+  static constexpr int kStagingBytes = 4 * kStagingBufs * 4096;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kStagingBytes + 1024;
+  static constexpr int kBRowTxBytes = 64;                 // what the TMA unit counts per widened weight row of a K-step
+  static_assert(kAccCols + kSfSlots * kSfCols <= kTmemCols, "tensor memory budget");
+  static_assert(kSmemBytes <= 232448, "shared memory budget");
+  static_assert(kStageBytes % 1024 == 0, "stage alignment");
+  static_assert(kSlot1Col == PairCfg::kSlot1Col && kSlot1Width == PairCfg::kSlot1Width, "PairSlots is shared");
+};
+
+__device__ __forceinline__ void tc_mma_mxf8f6f4_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                     uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale.scale_vec::1X [%0], %1, %2, %3, [%4], [%5], p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
+      : "memory");
+}
+
+template <bool OUT_BF16>
+__global__ void __launch_bounds__(kPairThreads, 1)
+gemm_w4a8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b32,
+                       const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfb,
+                       const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ PairParams p) {
+  using Cfg = A8PairCfg;
+  extern __shared__ uint8_t a8pair_smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[Cfg::kStages];   // used in the leader only
+  __shared__ __align__(8) uint64_t empty_bar[Cfg::kStages];  // one set per CTA
+  __shared__ __align__(8) uint64_t acc_full_bar[2];          // one set per CTA
+  __shared__ __align__(8) uint64_t acc_empty_bar[2];         // used in the leader only
+  __shared__ __align__(8) uint64_t drain_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  // A kernel launched as a programmatic dependent of this one may be scheduled on every SM this
+  // grid has left; it must still wait for this grid before it touches memory.
+  grid_launch_dependents();
+  const int tid = threadIdx.x;
+  const int warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0);
+  const int lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();          // 0 = leader
+  const int pair = blockIdx.x >> 1;
+  const int n_pairs = gridDim.x >> 1;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(a8pair_smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* staging = smem + Cfg::kStages * Cfg::kStageBytes;
+
+  if (tid == 0) {
+    for (int i = 0; i < Cfg::kStages; ++i) {
+      mbar_init(smem_u32(&full_bar[i]), 1);
+      mbar_init(smem_u32(&empty_bar[i]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&acc_full_bar[i]), 1);
+      mbar_init(smem_u32(&acc_empty_bar[i]), 8);  // 4 epilogue warps of each CTA
+    }
+    mbar_init(smem_u32(&drain_bar), 1);
+    abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmap_a);
+    tma_prefetch_desc(&tmap_b32);
+    tma_prefetch_desc(&tmap_sfa);
+    tma_prefetch_desc(&tmap_sfb);
+    tma_prefetch_desc(&tmap_y);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(&tmem_base_slot), Cfg::kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();  // the other CTA's barriers are initialised before anything signals them
+  tc_fence_after_sync();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  const PairWalk walk0(p, pair, n_pairs);
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer (both CTAs)
+    bool ok = true;
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t full0_leader = map_to_cta(smem_u32(&full_bar[0]), 0);
+    int my_steps = 0;
+    {
+      PairWalk w = walk0;
+      PairTile t;
+      while (w.next(t)) my_steps += p.k_steps;
+    }
+    // K-step kt of tile t into ring stage `stage`.  `what`: 1 = the weight side (this CTA's half of
+    // the B tile in boxes of 32 rows, weight scales; the leader also arms the barrier with the
+    // bytes of both CTAs), 2 = the activation side (A tile, activation scales), 3 = both.
+    auto issue = [&](const PairTile& t, int kt, int stage, int what) {
+      const int m0 = t.mp * 256 + static_cast<int>(rank) * kBM;
+      const int half = t.bn >> 1;
+      const uint32_t st = smem_base + stage * Cfg::kStageBytes;
+      const uint32_t bar = full0_leader + 8u * stage;
+      if (what & 1) {
+        if (rank == 0)
+          mbar_arrive_expect_tx(smem_u32(&full_bar[stage]),
+                                2u * static_cast<uint32_t>(Cfg::kABytes + half * Cfg::kBRowTxBytes + Cfg::kSfaBytes + Cfg::kSfbBytes));
+        const int b0 = t.n0 + static_cast<int>(rank) * half;
+        for (int r = 0; r < half; r += 32)   // x in elements: the map widens 64 packed bytes to a 128-byte row
+          tma_load_2d_pair(st + Cfg::kABytes + r * 128, &tmap_b32, kt * kW4A8KElems, b0 + r, bar);
+#pragma unroll
+        for (int rt = 0; rt < Cfg::kSfbAtoms; ++rt)
+          tma_load_2d_pair(st + Cfg::kABytes + Cfg::kBBytes + Cfg::kSfaBytes + rt * 512, &tmap_sfb, 0,
+                           ((t.n0 >> 7) + rt) * p.katoms + kt, bar);
+      }
+      if (what & 2) {
+        tma_load_2d_pair(st, &tmap_a, kt * 128, m0, bar);
+        tma_load_2d_pair(st + Cfg::kABytes + Cfg::kBBytes, &tmap_sfa, 0, (m0 >> 7) * p.katoms + kt, bar);
+      }
+    };
+    // The first `prefill` steps of the pair, side `what`, into stages 0, 1, ...
+    const int prefill = min(my_steps, Cfg::kStages);
+    auto issue_prefill = [&](int what) {
+      PairWalk w = walk0;
+      PairTile t;
+      int g = 0;
+      while (g < prefill && w.next(t))
+        for (int kt = 0; kt < p.k_steps && g < prefill; ++kt, ++g) issue(t, kt, g, what);
+    };
+    // The weights do not depend on the kernel that quantises the activations: fill the ring's
+    // weight side first, then wait for that kernel (programmatic dependent launch; an ordinary
+    // launch does not wait here), then add the activation side.
+    if (elect_one()) issue_prefill(1);
+    __syncwarp();
+    grid_dependency_wait();
+    if (elect_one()) issue_prefill(2);
+    __syncwarp();
+    int stage = prefill % Cfg::kStages;
+    uint32_t phase = (prefill == Cfg::kStages) ? 1u : 0u;
+    {
+      PairWalk w = walk0;
+      PairTile t;
+      int g = 0;
+      while (ok && w.next(t)) {
+        for (int kt = 0; kt < p.k_steps; ++kt, ++g) {
+          if (g < prefill) continue;
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag));
+          if (!ok) break;
+          if (elect_one()) issue(t, kt, stage, 3);
+          if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+    if (!ok && lane == 0) {
+      // Given up: the loads of both CTAs are counted on the leader's barriers, so neither CTA can
+      // wait for its own; give the copies already in flight ample time to land instead.
+      const uint64_t t0 = global_timer_ns();
+      while (global_timer_ns() - t0 < 1000000ull) {}
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer (leader CTA only)
+    if (rank == 0) {
+      const uint32_t smem_base = smem_u32(smem);
+      const uint64_t ab_desc0 = make_smem_desc(smem_base, 16, 1024, 2);
+      const uint64_t sf_desc0 = make_smem_desc(smem_base + Cfg::kABytes + Cfg::kBBytes, 0, 128, 0);
+      const uint32_t sf_tmem0 = tmem_base + Cfg::kAccCols;
+      const uint32_t full0 = smem_u32(&full_bar[0]);
+      const uint32_t empty0 = smem_u32(&empty_bar[0]);
+
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t g = 0;  // K-steps issued so far: the scale slot alternates with it
+      bool ok = true;
+      PairWalk w = walk0;
+      PairTile t;
+      PairSlots slots;
+      while (ok && w.next(t)) {
+        const uint32_t idesc0 = mxf8f6f4_idesc_e4m3_e2m1(256, t.bn);
+        const uint32_t sfb_sub = static_cast<uint32_t>(t.n0 & 127) >> 5;
+        int acc;
+        uint32_t acc_phase;
+        slots.take(t.bn, acc, acc_phase);
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&acc_empty_bar[acc]), acc_phase ^ 1u, &abort_flag));
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * Cfg::kSlot1Col;
+        for (int kt = 0; kt < p.k_steps; ++kt, ++g) {
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(full0 + 8u * stage, phase, &abort_flag));
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t soff = static_cast<uint32_t>(stage * (Cfg::kStageBytes >> 4));
+          const uint64_t adesc = ab_desc0 + soff;
+          const uint64_t bdesc = adesc + (Cfg::kABytes >> 4);
+          const uint64_t sfd = sf_desc0 + soff;
+          const uint32_t sfa_col = sf_tmem0 + (g & 1u) * Cfg::kSfCols;
+          const uint32_t sfb_col = sfa_col + 4 + sfb_sub;
+          if (elect_one()) {
+            tc_cp_32x128b_warpx4_pair(sfa_col, sfd);
+#pragma unroll
+            for (int rt = 0; rt < Cfg::kSfbAtoms; ++rt)
+              tc_cp_32x128b_warpx4_pair(sfa_col + 4 + 4 * rt, sfd + ((Cfg::kSfaBytes + rt * 512) >> 4));
+#pragma unroll
+            for (uint32_t kb = 0; kb < 4; ++kb)   // block kb of the K-step: byte kb of every scale column
+              tc_mma_mxf8f6f4_pair(d_tmem, adesc + 2 * kb, bdesc + 2 * kb, idesc0 | (kb << 29) | (kb << 4),
+                                   sfa_col | (kb << 30), sfb_col | (kb << 30), (kt | static_cast<int>(kb)) != 0 ? 1u : 0u);
+            tc_commit_pair(empty0 + 8u * stage, 3);  // frees the stage in both CTAs
+          }
+          if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        if (elect_one()) tc_commit_pair(smem_u32(&acc_full_bar[acc]), 3);
+      }
+      if (lane == 0) {
+        tc_commit_pair_local(smem_u32(&drain_bar));
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(smem_u32(&drain_bar), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
+      }
+      __syncwarp();
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue warps (both CTAs)
+    const int quad = warp & 3;
+    uint8_t* my_staging = staging + quad * (Cfg::kStagingBufs * 4096);
+    constexpr int kChunkCols = OUT_BF16 ? 64 : 32;
+    const uint32_t acc_empty0_leader = map_to_cta(smem_u32(&acc_empty_bar[0]), 0);
+    int buf = 0;
+    PairWalk wk = walk0;
+    PairTile t;
+    PairSlots slots;
+    while (wk.next(t)) {
+      int acc;
+      uint32_t acc_phase;
+      slots.take(t.bn, acc, acc_phase);
+      bool ok = mbar_wait(smem_u32(&acc_full_bar[acc]), acc_phase, &abort_flag);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const int row0 = t.mp * 256 + static_cast<int>(rank) * kBM + quad * 32;
+      const uint32_t taddr = tmem_base + acc * Cfg::kSlot1Col + (static_cast<uint32_t>(quad * 32) << 16);
+#pragma unroll 1
+      for (int c0 = 0; c0 < t.bn; c0 += kChunkCols) {
+        uint32_t w[32];
+        if (OUT_BF16) {
+          uint32_t r0[32], r1[32];
+          tmem_ld_32x32b_x32(taddr + c0, r0);
+          tmem_ld_32x32b_x32(taddr + c0 + 32, r1);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const __nv_bfloat162 a = __floats2bfloat162_rn(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]));
+            const __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(r1[2 * i]), __uint_as_float(r1[2 * i + 1]));
+            w[i] = *reinterpret_cast<const uint32_t*>(&a);
+            w[16 + i] = *reinterpret_cast<const uint32_t*>(&b);
+          }
+        } else {
+          tmem_ld_32x32b_x32(taddr + c0, w);
+          tmem_ld_wait();
+        }
+        const int col0 = t.n0 + c0;
+        if (p.m16 < p.m && col0 < p.m && col0 + kChunkCols > p.m16 && row0 + lane < p.s) {
+          if (OUT_BF16) {
+            __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(p.y) + static_cast<int64_t>(row0 + lane) * p.ldy + col0;
+#pragma unroll
+            for (int i = 0; i < kChunkCols; ++i)
+              if (col0 + i >= p.m16 && col0 + i < p.m) {
+                const uint32_t word = w[((i >> 5) << 4) + ((i & 31) >> 1)];
+                const uint16_t hv = static_cast<uint16_t>((i & 1) ? (word >> 16) : (word & 0xFFFFu));
+                yp[i] = *reinterpret_cast<const __nv_bfloat16*>(&hv);
+              }
+          } else {
+            float* yp = reinterpret_cast<float*>(p.y) + static_cast<int64_t>(row0 + lane) * p.ldy + col0;
+#pragma unroll
+            for (int i = 0; i < kChunkCols; ++i)
+              if (col0 + i >= p.m16 && col0 + i < p.m) yp[i] = __uint_as_float(w[i]);
+          }
+        }
+        if (lane == 0) bulk_wait_group_read<Cfg::kStagingBufs - 1>();
+        __syncwarp();
+        uint8_t* sb = my_staging + buf * 4096 + lane * 128;
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          *reinterpret_cast<uint4*>(sb + ((q ^ (lane & 7)) << 4)) = make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          if (row0 < p.s && col0 < p.m16) tma_store_2d(&tmap_y, col0, row0, smem_u32(my_staging + buf * 4096));
+          bulk_commit_group();
+        }
+        buf = (buf + 1) % Cfg::kStagingBufs;
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(acc_empty0_leader + 8u * acc);
+    }
+    if (lane == 0) bulk_wait_group<0>();
+  }
+
+  // Neither CTA may leave (or release tensor memory) while the other can still read its shared
+  // memory or signal its barriers.
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, Cfg::kTmemCols);
+  }
+}
+
+}  // namespace batq

@@ -5,6 +5,7 @@
 #include <cuda.h>
 
 #include "gemm_mxfp4.cuh"
+#include "gemm_w4a8_pair.cuh"
 #include "ptx.cuh"
 
 namespace batq {
@@ -36,6 +37,9 @@ struct PeakParams {
   int32_t load_sharing; // >= 1: this many CTAs (blockIdx.x / load_sharing equal) load the same boxes at the same time
   int32_t load_from_peer;  // pairs only, != 0: the second box of every stage is not loaded from L2 but copied from
                            // the other CTA of the pair, shared memory to shared memory
+  int32_t sf_col;       // tensor-memory column of the scale factors (behind the accumulators: 256, or 448 with bn2)
+  int32_t bn2;          // KIND 1: width of the second MMA (into columns 256.. on the same operands: the issue
+                        // pattern of the wide-tile GEMM)
   int32_t store_iters;  // stages (32 KiB) warps 2-3 of every CTA write into the ring with ordinary stores; 0 = none
 };
 
@@ -56,7 +60,13 @@ __device__ __forceinline__ void bulk_s2s_cluster(uint32_t dst_cluster, uint32_t 
                : "memory");
 }
 
-template <bool PAIR>
+// KIND 0: kind::mxf4 on one accumulator; 1: kind::mxf4, every MMA followed by one of width bn2 into
+// a second accumulator; 2: kind::mxf8f6f4; 3: kind::mxf4 issued by the CTA-pair GEMM's own loop
+// (a wait, a fence, eight scale copies into alternating slots, four MMAs from stage-dependent
+// descriptors and a commit per K-step, the whole warp around one elected lane).  A template parameter, not a field of PeakParams: the
+// issue loop must stay free of run-time branches (with two of them per MMA the same loop measured
+// 6.4 instead of 8.1 PFLOP/s: the rate at which one thread can issue is part of what is measured).
+template <bool PAIR, int KIND>
 __global__ void __launch_bounds__(kPeakThreads, 1)
 mma_peak_kernel(const __grid_constant__ CUtensorMap tmap_w, const PeakParams p) {
   extern __shared__ uint8_t peak_smem_raw[];
@@ -73,7 +83,8 @@ mma_peak_kernel(const __grid_constant__ CUtensorMap tmap_w, const PeakParams p) 
   uint32_t h = 0x9E3779B9u * (blockIdx.x * kPeakThreads + tid + 1u);
   for (int i = tid; i < (kPeakABytes + kPeakBBytes) / 4; i += kPeakThreads) {
     h = h * 1664525u + 1013904223u;
-    reinterpret_cast<uint32_t*>(smem)[i] = h ^ (h >> 15);
+    // (8-bit containers: the top two bits of every byte clear, so that no E4M3 code is a NaN)
+    reinterpret_cast<uint32_t*>(smem)[i] = KIND == 2 ? ((h ^ (h >> 15)) & 0x3F3F3F3Fu) : (h ^ (h >> 15));
   }
   for (int i = tid; i < kPeakSfBytes; i += kPeakThreads) {
     h = h * 1664525u + 1013904223u;
@@ -167,10 +178,12 @@ mma_peak_kernel(const __grid_constant__ CUtensorMap tmap_w, const PeakParams p) 
     const uint64_t adesc = make_smem_desc(smem_base, 16, 1024, 2);
     const uint64_t bdesc = adesc + (kPeakABytes >> 4);
     const uint64_t sfd = make_smem_desc(smem_base + kPeakABytes + kPeakBBytes, 0, 128, 0);
-    const uint32_t sfa_col = tmem_base + 256;
+    const uint32_t sfa_col = tmem_base + static_cast<uint32_t>(p.sf_col);
     const uint32_t sfb_col = sfa_col + 8;
     const uint32_t idesc0 = mxf4_idesc(PAIR ? 256 : 128, p.bn);
     const uint32_t idesc1 = idesc0 | (2u << 29) | (2u << 4);
+    const uint32_t idesc8 = mxf8f6f4_idesc_e4m3_e2m1(PAIR ? 256 : 128, p.bn);
+    const uint32_t idesc2 = mxf4_idesc(PAIR ? 256 : 128, p.bn2 > 0 ? p.bn2 : 64);
     bool ok = true;
     if (elect_one()) {
       // scale factors once: shared -> tensor memory, the layout of the GEMM kernels
@@ -191,7 +204,61 @@ mma_peak_kernel(const __grid_constant__ CUtensorMap tmap_w, const PeakParams p) 
         }
     }
     __syncwarp();
-    const int n_batches = (p.iters + kPeakBatch - 1) / kPeakBatch;
+    if (KIND == 3) {
+      // The issue loop of the CTA-pair GEMM, statement for statement: the whole warp waits for a stage
+      // (here a barrier phase that is complete from the start), one elected lane copies the scales of
+      // the K-step into one of two slots and issues its four MMAs from descriptors that depend on the
+      // run-time stage index, then commits.  All five "stages" are the same resident operands.
+      const uint32_t zero = static_cast<uint32_t>(p.w_k_steps - 1);   // 0 at run time (no load stream)
+      const uint64_t ab_desc0 = adesc;
+      const uint32_t sf_tmem0 = sfa_col;
+      const uint32_t full0 = smem_u32(&load_bar[0]);
+      int stage = 0;
+      uint32_t phase = 1;
+      uint32_t g = 0;
+      for (int kt = 0; kt < p.iters && ok; ++kt, ++g) {
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(full0 + 8u * stage * zero, phase, &abort_flag));
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t soff = static_cast<uint32_t>(stage * (36864 >> 4)) * zero;
+        const uint64_t a_k = ab_desc0 + soff;
+        const uint64_t b_k = a_k + (kPeakABytes >> 4);
+        const uint64_t sfd_k = sfd + soff;
+        const uint32_t sfa_k = sf_tmem0 + (g & 1u) * 24u;
+        const uint32_t sfb_k = sfa_k + 8;
+        if (elect_one()) {
+          if (PAIR) { tc_cp_32x128b_warpx4_pair(sfa_k, sfd_k); tc_cp_32x128b_warpx4_pair(sfa_k + 4, sfd_k + 32); }
+          else      { tc_cp_32x128b_warpx4(sfa_k, sfd_k); tc_cp_32x128b_warpx4(sfa_k + 4, sfd_k + 32); }
+#pragma unroll
+          for (int rt = 0; rt < kPeakSfbAtoms; ++rt)
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+              const uint32_t col = sfa_k + 8 + c * 4 * kPeakSfbAtoms + 4 * rt;
+              const uint64_t src = sfd_k + ((1024 + rt * 1024 + c * 512) >> 4);
+              if (PAIR) tc_cp_32x128b_warpx4_pair(col, src); else tc_cp_32x128b_warpx4(col, src);
+            }
+#pragma unroll
+          for (int kb = 0; kb < 4; ++kb) {
+            const uint32_t c = kb >> 1;
+            const uint32_t sfid = (kb & 1) * 2;
+            const uint32_t sa = (sfa_k + 4 * c) | (sfid << 30);
+            const uint32_t sb = (sfb_k + c * 4 * kPeakSfbAtoms) | (sfid << 30);
+            const uint32_t acc = (kt | kb) != 0 ? 1u : 0u;
+            if (PAIR) tc_mma_mxf4_pair(tmem_base, a_k + 2 * kb, b_k + 2 * kb, (kb & 1) ? idesc1 : idesc0, sa, sb, acc);
+            else      tc_mma_mxf4(tmem_base, a_k + 2 * kb, b_k + 2 * kb, (kb & 1) ? idesc1 : idesc0, sa, sb, acc);
+          }
+          if (PAIR) tc_commit_pair_local(smem_u32(&load_bar[1])); else tc_commit(smem_u32(&load_bar[1]));
+        }
+        if (++stage == 5) { stage = 0; phase ^= zero; }
+      }
+      if (elect_one()) {
+        if (PAIR) tc_commit_pair_local(smem_u32(&batch_bar[0])); else tc_commit(smem_u32(&batch_bar[0]));
+      }
+      __syncwarp();
+      mbar_wait(smem_u32(&batch_bar[0]), 0, &abort_flag);
+      __syncwarp();
+    }
+    const int n_batches = KIND == 3 ? 0 : (p.iters + kPeakBatch - 1) / kPeakBatch;
     for (int b = 0; b < n_batches && ok; ++b) {
       // at most two batches in flight, like a ring of stages
       if (b >= 2) {
@@ -218,15 +285,30 @@ mma_peak_kernel(const __grid_constant__ CUtensorMap tmap_w, const PeakParams p) 
                 if (PAIR) tc_cp_32x128b_warpx4_pair(col, src); else tc_cp_32x128b_warpx4(col, src);
               }
           }
+          if (KIND == 2) {
 #pragma unroll
-          for (int kb = 0; kb < 4; ++kb) {
-            const uint32_t c = kb >> 1;
-            const uint32_t sfid = (kb & 1) * 2;
-            const uint32_t sa = (sfa_col + 4 * c) | (sfid << 30);
-            const uint32_t sb = (sfb_col + c * 4 * kPeakSfbAtoms) | (sfid << 30);
-            const uint32_t acc = (kt | kb) != 0 ? 1u : 0u;
-            if (PAIR) tc_mma_mxf4_pair(tmem_base, adesc + 2 * kb, bdesc + 2 * kb, (kb & 1) ? idesc1 : idesc0, sa, sb, acc);
-            else      tc_mma_mxf4(tmem_base, adesc + 2 * kb, bdesc + 2 * kb, (kb & 1) ? idesc1 : idesc0, sa, sb, acc);
+            for (uint32_t kb = 0; kb < 4; ++kb) {   // byte kb of one scale column per 32 rows
+              const uint32_t id = idesc8 | (kb << 29) | (kb << 4);
+              const uint32_t acc = (kt | static_cast<int>(kb)) != 0 ? 1u : 0u;
+              if (PAIR) tc_mma_mxf8f6f4_pair(tmem_base, adesc + 2 * kb, bdesc + 2 * kb, id, sfa_col | (kb << 30), sfb_col | (kb << 30), acc);
+              else      tc_mma_mxf8f6f4(tmem_base, adesc + 2 * kb, bdesc + 2 * kb, id, sfa_col | (kb << 30), sfb_col | (kb << 30), acc);
+            }
+          } else {
+#pragma unroll
+            for (int kb = 0; kb < 4; ++kb) {
+              const uint32_t c = kb >> 1;
+              const uint32_t sfid = (kb & 1) * 2;
+              const uint32_t sa = (sfa_col + 4 * c) | (sfid << 30);
+              const uint32_t sb = (sfb_col + c * 4 * kPeakSfbAtoms) | (sfid << 30);
+              const uint32_t acc = (kt | kb) != 0 ? 1u : 0u;
+              if (PAIR) tc_mma_mxf4_pair(tmem_base, adesc + 2 * kb, bdesc + 2 * kb, (kb & 1) ? idesc1 : idesc0, sa, sb, acc);
+              else      tc_mma_mxf4(tmem_base, adesc + 2 * kb, bdesc + 2 * kb, (kb & 1) ? idesc1 : idesc0, sa, sb, acc);
+              if (KIND == 1) {
+                const uint32_t i2 = idesc2 | ((kb & 1) ? ((2u << 29) | (2u << 4)) : 0u);
+                if (PAIR) tc_mma_mxf4_pair(tmem_base + 256, adesc + 2 * kb, bdesc + 2 * kb, i2, sa, sb, acc);
+                else      tc_mma_mxf4(tmem_base + 256, adesc + 2 * kb, bdesc + 2 * kb, i2, sa, sb, acc);
+              }
+            }
           }
         }
         if (PAIR) tc_commit_pair_local(smem_u32(&batch_bar[b & 1])); else tc_commit(smem_u32(&batch_bar[b & 1]));

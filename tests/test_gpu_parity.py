@@ -319,6 +319,23 @@ def test_measurement_loops_leave_the_device_clean(batq):
             assert flops > 0 if it else flops == 0
             assert nbytes % 32768 == 0 and nbytes >= (lit + sit) * 32768 * ctas * 0.9
     try:
+        for a8, gemm_loop, bn2, col in ((True, False, 0, 0), (False, True, 0, 0), (False, False, 192, 0),
+                                        (False, False, 128, 480), (False, False, 0, 320)):
+            batq.batq_debug_mma_peak_kind(a8)
+            batq.batq_debug_mma_peak_gemm_loop(gemm_loop)
+            batq.batq_debug_mma_peak_second_width(bn2)
+            batq.batq_debug_mma_peak_sf_column(col)
+            for pair in (True, False):
+                flops = batq.batq_debug_mma_peak(pair, 256, 50, True)
+                assert flops == 2.0 * (256 if pair else 128) * (256 + bn2) * (128 if a8 else 256) * 50 * (74 if pair else 148)
+                torch.cuda.synchronize()
+                assert batq.batq_last_device_status() == 0
+    finally:
+        batq.batq_debug_mma_peak_kind(False)
+        batq.batq_debug_mma_peak_gemm_loop(False)
+        batq.batq_debug_mma_peak_second_width(0)
+        batq.batq_debug_mma_peak_sf_column(0)
+    try:
         for stages, sharing, peer in ((1, 1, 0), (5, 8, 0), (2, 1, 1), (4, 148, 1), (4, 1, 0)):
             batq.batq_debug_mma_peak_load_stages(stages)
             batq.batq_debug_mma_peak_load_sharing(sharing)

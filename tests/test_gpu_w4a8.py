@@ -40,13 +40,26 @@ def _gemm_case(batq, S, M, N, seed, xb=None, wb=None, out_dtype=torch.float32):
     return yh[:S, :M].astype(np.float64), Y, Sabs
 
 
+@pytest.fixture(params=[1, 2, 3], ids=["cta", "ctapair", "widepair"])
+def gkernel(request, batq):
+    """Runs a test once per W4A8 GEMM kernel (one CTA per tile / CTA pairs sharing a 256-token tile
+    with two accumulators / CTA pairs with tiles of up to 448 features)."""
+    batq.batq_debug_force_gemm_kernel(request.param)
+    yield request.param
+    batq.batq_debug_force_gemm_kernel(0)
+
+
 SHAPES = [(128, 128, 256), (128, 1024, 1024), (1, 8, 128), (77, 200, 384), (300, 520, 3584), (260, 384, 512),
           (129, 257, 2048 + 128), (1000, 1100, 768)]
 
 
-@pytest.mark.parametrize("bn", [0, 128, 256])
+@pytest.mark.parametrize("bn", [0, 64, 128, 192, 256, 320, 384, 448])
 @pytest.mark.parametrize("S,M,N", SHAPES)
-def test_w4a8_gemm_vs_oracle_same_codes(batq, S, M, N, bn):
+def test_w4a8_gemm_vs_oracle_same_codes(batq, gkernel, S, M, N, bn):
+    if gkernel == 1 and bn not in (0, 128, 256):
+        pytest.skip("the one-CTA kernel has tiles of 128 and 256 features")
+    if gkernel == 2 and bn in (320, 384):
+        pytest.skip("only the wide-tile kernel has these widths")
     batq.batq_debug_force_tile_width(bn)
     try:
         got, Y, Sabs = _gemm_case(batq, S, M, N, 1600 + S)
@@ -58,8 +71,8 @@ def test_w4a8_gemm_vs_oracle_same_codes(batq, S, M, N, bn):
     assert np.max(np.abs(got - Y) / (Sabs + 1e-30)) < 1e-5
 
 
-@pytest.mark.parametrize("bn", [128, 256])
-def test_w4a8_scale_layout_localising_case(batq, bn):
+@pytest.mark.parametrize("bn", [64, 128, 192, 256, 320, 384, 448])
+def test_w4a8_scale_layout_localising_case(batq, gkernel, bn):
     """Constant codes and a distinct power-of-two scale per (row, block) on both sides: a mistake in
     the scale layout, in the byte of the scale column an MMA takes, or in the operand pairing shows
     up as a wrong power of two in a specific output."""
@@ -69,6 +82,10 @@ def test_w4a8_scale_layout_localising_case(batq, bn):
     ew = ((np.arange(M)[:, None] * 5 + np.arange(k)[None, :] * 11) % 21) - 10
     X = np.repeat(256.0 * np.exp2(ex), 32, axis=1).astype(np.float32)     # amax 2^8 * 2^ex: element code 1.0 * 2^8
     W = np.repeat(4.0 * np.exp2(ew), 32, axis=1).astype(np.float32)
+    if gkernel == 1 and bn not in (128, 256):
+        pytest.skip("the one-CTA kernel has tiles of 128 and 256 features")
+    if gkernel == 2 and bn in (320, 384):
+        pytest.skip("only the wide-tile kernel has these widths")
     batq.batq_debug_force_tile_width(bn)
     try:
         got, Y, Sabs = _gemm_case(batq, S, M, N, 0, synth.f32_to_bf16_bits(X), synth.f32_to_bf16_bits(W))
@@ -80,7 +97,7 @@ def test_w4a8_scale_layout_localising_case(batq, bn):
     assert np.all(np.abs(got - want) <= k * 2.0 ** -23 * want)
 
 
-def test_w4a8_distinct_codes_in_every_position(batq):
+def test_w4a8_distinct_codes_in_every_position(batq, gkernel):
     """Every K position of a block carries a different weight code and a different activation code,
     rows differ too: a permutation of elements inside a 16-code container, a swapped nibble or a
     shifted K sub-block changes the exact result."""
@@ -92,7 +109,7 @@ def test_w4a8_distinct_codes_in_every_position(batq):
     assert np.array_equal(got, Y)          # small integers and halves: fp32 accumulation is exact
 
 
-def test_w4a8_bf16_output_is_rounded_fp32(batq):
+def test_w4a8_bf16_output_is_rounded_fp32(batq, gkernel):
     a, _, _ = _gemm_case(batq, 130, 264, 1024, 42, out_dtype=torch.float32)
     b, _, _ = _gemm_case(batq, 130, 264, 1024, 42, out_dtype=torch.bfloat16)
     want = torch.from_numpy(a.astype(np.float32)).bfloat16().float().numpy()
