@@ -142,10 +142,12 @@ def test_linear_w4a8_vs_oracle(batq, S, M, N, geometry):
     assert np.linalg.norm(got - ref) < np.linalg.norm(y4.cpu().numpy().astype(np.float64) - ref)
 
 
-def test_w4a8_full_size_sampled(batq):
-    """Config 1's qkv projection (2048 x 4096 -> 6144) through the W4A8 layer, bf16 output, checked
-    on sampled rows and columns from the codes the GPU itself produced."""
-    S, N, M = 2048, 4096, 6144
+@pytest.mark.parametrize("N,M", [(4096, 6144), (4096, 28672)])
+def test_w4a8_full_size_sampled(batq, N, M):
+    """Config 1's qkv (2048 x 4096 -> 6144: CTA pairs with two accumulators) and gate/up (-> 28672:
+    wide tiles) projections through the W4A8 layer in the launch configuration the benchmark times,
+    bf16 output, checked on sampled rows and columns from the codes the GPU itself produced."""
+    S = 2048
     rng = np.random.default_rng(11)
     xb = synth.make_activations(S, N, synth.BASE_SEED)
     wb = synth.make_weight(M, N, synth.BASE_SEED + 2)
@@ -161,7 +163,8 @@ def test_w4a8_full_size_sampled(batq):
     sf = torch.empty(batq.batq_sf_bytes(S, N, 1), dtype=torch.uint8, device="cuda")
     batq.batq_quantize_act_mxfp8(tr, x, codes, sf, 1)
     rows = np.sort(rng.choice(S, size=48, replace=False))
-    cols = np.sort(rng.choice(M, size=384, replace=False))
+    cols = np.sort(np.concatenate([rng.choice(M, size=376, replace=False), [0, 255, 256, 447, 448, M - 449, M - 257, M - 1]]))
+    cols = np.unique(cols)
     gc = codes[torch.from_numpy(rows).cuda()].cpu().numpy()
     gs = sf_mma_to_rowmajor(sf.cpu().numpy(), S, N // 32)[rows]
     wc_d, wsc_d = batq.batq_weight_export(w)
