@@ -214,13 +214,31 @@ batq_status batq_linear_w4a4(const batq_transform* t, const batq_weight* w, cons
 
 /* Same layer with HOST input and output: copies x_host (pinned or pageable host
  * memory, [s x n] bf16 dense) to x_stage_dev, runs batq_linear_w4a4, copies the
- * result from y_stage_dev to y_host, all on `stream`; returns after the stream
- * has drained.  x_stage_dev (s*n*2 bytes) and y_stage_dev (s*m*{4,2} bytes) are
- * caller-provided device staging buffers. */
+ * result from y_stage_dev to y_host; returns after everything has drained.
+ * The copies run on two streams the library keeps per device; from 512 tokens
+ * on the rows go through in up to four chunks, so that with pinned host memory
+ * the copy-in of one chunk, the kernels of the one before and the copy-out of
+ * the one before that overlap (token rows are independent: the result is that
+ * of one call on all rows).  x_stage_dev (s*n*2 bytes) and y_stage_dev
+ * (s*m*{4,2} bytes) are caller-provided device staging buffers; workspace as
+ * for batq_linear_w4a4 with s rows. */
 batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w, const void* x_host,
                                   int64_t s, void* y_host, int32_t y_dtype, void* x_stage_dev,
                                   void* y_stage_dev, void* workspace, size_t workspace_bytes,
                                   void* stream);
+/* The same, enqueued only: returns without waiting, so that the copies of several
+ * layers (each with staging buffers and a workspace of its own) overlap one
+ * another and the kernels.  y_host, and the right to reuse x_host, the staging
+ * buffers and the workspace, are the caller's again after batq_host_drain(stream)
+ * on the same device has returned BATQ_OK.  An error found while enqueueing is
+ * returned at once; what was enqueued before it still runs. */
+batq_status batq_linear_w4a4_host_async(const batq_transform* t, const batq_weight* w,
+                                        const void* x_host, int64_t s, void* y_host, int32_t y_dtype,
+                                        void* x_stage_dev, void* y_stage_dev, void* workspace,
+                                        size_t workspace_bytes, void* stream);
+/* Waits for everything the host entry points have enqueued on the current device:
+ * the library's copy streams and `stream`. */
+batq_status batq_host_drain(void* stream);
 
 /* The same layer for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is a deployment convenience of this library.)  Some hosts of

@@ -56,6 +56,8 @@ SIGNATURES = {
     "batq_debug_wide_schedule": (C.c_int32, [_I64, _I64, _I64, _I32, _I32, _P, _I32]),
     "batq_linear_w4a4": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P, _SZ, _P]),
     "batq_linear_w4a4_host": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _P, _P, _P, _SZ, _P]),
+    "batq_linear_w4a4_host_async": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _P, _P, _P, _SZ, _P]),
+    "batq_host_drain": (C.c_int, [_P]),
     "batq_static_workspace_capacity": (_SZ, []),
     "batq_linear_w4a4_noalloc": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P]),
     "batq_last_device_status": (C.c_int, [_P]),
@@ -340,6 +342,19 @@ def batq_linear_w4a4_host(t, w: Weight, x_host, y_host, x_stage, y_stage, worksp
     st = load().batq_linear_w4a4_host(t.handle if t else None, w.handle, _ptr(x_host), x_host.shape[0], _ptr(y_host),
                                       dt, _ptr(x_stage), _ptr(y_stage), _ptr(workspace), workspace.numel(), _stream())
     _check(st, "batq_linear_w4a4_host")
+
+
+def batq_linear_w4a4_host_async(t, w: Weight, x_host, y_host, x_stage, y_stage, workspace):
+    """Enqueues copy-in, layer and copy-out and returns; batq_host_drain() waits for them."""
+    dt = F32 if y_host.dtype == torch.float32 else BF16
+    st = load().batq_linear_w4a4_host_async(t.handle if t else None, w.handle, _ptr(x_host), x_host.shape[0],
+                                            _ptr(y_host), dt, _ptr(x_stage), _ptr(y_stage), _ptr(workspace),
+                                            workspace.numel(), _stream())
+    _check(st, "batq_linear_w4a4_host_async")
+
+
+def batq_host_drain():
+    _check(load().batq_host_drain(_stream()), "batq_host_drain")
 
 
 def batq_static_workspace_capacity() -> int:

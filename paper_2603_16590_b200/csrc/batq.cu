@@ -1819,26 +1819,127 @@ batq_status batq_linear_w4a4(const batq_transform* t, const batq_weight* w, cons
   return launch_gemm(codes, sf, w, s, y, y_dtype, ldy, cs, true);
 }
 
-batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w, const void* x_host, int64_t s,
-                                  void* y_host, int32_t y_dtype, void* x_stage_dev, void* y_stage_dev, void* workspace,
-                                  size_t workspace_bytes, void* stream) {
+// Streams of the host entry points' copy pipeline, one pair per device, made on first use and kept
+// for the life of the process.
+constexpr int kHostChunks = 4;
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t in = nullptr, out = nullptr;
+};
+static std::mutex g_host_pipe_mutex;
+static HostPipe g_host_pipe[kMaxDevices];
+
+static batq_status host_pipe(int dev, HostPipe** out) {   // caller holds g_host_pipe_mutex
+  if (dev < 0 || dev >= kMaxDevices) return BATQ_ERR_CUDA;
+  HostPipe& hp = g_host_pipe[dev];
+  if (!hp.ready) {
+    if (cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) != cudaSuccess) {
+      cudaGetLastError();
+      return BATQ_ERR_CUDA;
+    }
+    hp.ready = true;
+  }
+  *out = &hp;
+  return BATQ_OK;
+}
+
+// src_stream has reached this point before dst_stream goes on.  The event is destroyed at once:
+// the runtime keeps it alive until the wait has been served.
+static bool stream_follows(cudaStream_t dst_stream, cudaStream_t src_stream) {
+  cudaEvent_t ev;
+  if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return false;
+  const bool ok = cudaEventRecord(ev, src_stream) == cudaSuccess && cudaStreamWaitEvent(dst_stream, ev, 0) == cudaSuccess;
+  cudaEventDestroy(ev);
+  return ok;
+}
+
+// Enqueues copy-in, layer and copy-out; nothing is waited for.
+static batq_status host_enqueue(const batq_transform* t, const batq_weight* w, const void* x_host, int64_t s, void* y_host,
+                                int32_t y_dtype, void* x_stage_dev, void* y_stage_dev, void* workspace,
+                                size_t workspace_bytes, void* stream) {
   if (w == nullptr) return BATQ_ERR_NULL;
   if (s < 0) return BATQ_ERR_SHAPE;
   if (s == 0) return BATQ_OK;
   if (x_host == nullptr || y_host == nullptr || x_stage_dev == nullptr || y_stage_dev == nullptr) return BATQ_ERR_NULL;
   if (y_dtype != BATQ_F32 && y_dtype != BATQ_BF16) return BATQ_ERR_UNSUPPORTED;
+  if (workspace_bytes < batq_linear_workspace_bytes(w, s)) return BATQ_ERR_WORKSPACE;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  const size_t xb = static_cast<size_t>(s * w->n) * 2;
-  const size_t yb = static_cast<size_t>(s * w->m) * (y_dtype == BATQ_F32 ? 4 : 2);
-  if (cudaMemcpyAsync(x_stage_dev, x_host, xb, cudaMemcpyHostToDevice, cs) != cudaSuccess) { cudaGetLastError(); return BATQ_ERR_CUDA; }
-  batq_status st = batq_linear_w4a4(t, w, x_stage_dev, s, w->n, y_stage_dev, y_dtype, w->m, workspace, workspace_bytes, stream);
-  if (st != BATQ_OK) return st;
-  if (cudaMemcpyAsync(y_host, y_stage_dev, yb, cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
-      cudaStreamSynchronize(cs) != cudaSuccess) {
-    cudaGetLastError();
-    return BATQ_ERR_CUDA;
+  const size_t ysz = y_dtype == BATQ_F32 ? 4 : 2;
+  // Token rows are independent, so a large batch goes through in up to four chunks of rows: the
+  // copy-in of chunk i + 1 and the copy-out of chunk i - 1 run on streams of their own beside
+  // the kernels of chunk i (PCIe carries both directions at once).  A small batch is one chunk.
+  int64_t rows_per_chunk = s >= 512 ? ((s + kHostChunks - 1) / kHostChunks + 127) / 128 * 128 : s;
+  int n_chunks = static_cast<int>((s + rows_per_chunk - 1) / rows_per_chunk);
+  if (n_chunks > 1) {   // the workspace was sized for s rows at once: every chunk must fit it too
+    const int64_t last = s - (n_chunks - 1) * rows_per_chunk;
+    if (batq_linear_workspace_bytes(w, rows_per_chunk) > workspace_bytes || batq_linear_workspace_bytes(w, last) > workspace_bytes) {
+      rows_per_chunk = s;
+      n_chunks = 1;
+    }
   }
+  int dev;
+  const DeviceInfo* info;
+  batq_status st = device_setup(&dev, &info);
+  if (st != BATQ_OK) return st;
+  std::lock_guard<std::mutex> lock(g_host_pipe_mutex);
+  HostPipe* hp;
+  st = host_pipe(dev, &hp);
+  if (st != BATQ_OK) return st;
+  // earlier work on the caller's stream may still use the staging buffers and the workspace
+  bool ok = stream_follows(hp->in, cs);
+  for (int c = 0; c < n_chunks && ok && st == BATQ_OK; ++c) {
+    const int64_t r0 = c * rows_per_chunk;
+    const int64_t rows = std::min<int64_t>(rows_per_chunk, s - r0);
+    const uint8_t* xh = static_cast<const uint8_t*>(x_host) + static_cast<size_t>(r0 * w->n) * 2;
+    uint8_t* xd = static_cast<uint8_t*>(x_stage_dev) + static_cast<size_t>(r0 * w->n) * 2;
+    uint8_t* yd = static_cast<uint8_t*>(y_stage_dev) + static_cast<size_t>(r0 * w->m) * ysz;
+    uint8_t* yh = static_cast<uint8_t*>(y_host) + static_cast<size_t>(r0 * w->m) * ysz;
+    ok = cudaMemcpyAsync(xd, xh, static_cast<size_t>(rows * w->n) * 2, cudaMemcpyHostToDevice, hp->in) == cudaSuccess &&
+         stream_follows(cs, hp->in);
+    if (!ok) break;
+    st = batq_linear_w4a4(t, w, xd, rows, w->n, yd, y_dtype, w->m, workspace, workspace_bytes, stream);
+    if (st != BATQ_OK) break;
+    ok = stream_follows(hp->out, cs) &&
+         cudaMemcpyAsync(yh, yd, static_cast<size_t>(rows * w->m) * ysz, cudaMemcpyDeviceToHost, hp->out) == cudaSuccess;
+  }
+  if (st != BATQ_OK) return st;
+  if (!ok) { cudaGetLastError(); return BATQ_ERR_CUDA; }
   return BATQ_OK;
+}
+
+batq_status batq_host_drain(void* stream) {
+  int dev;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BATQ_ERR_CUDA;
+  cudaStream_t in = nullptr, out = nullptr;
+  bool have = false;
+  {
+    std::lock_guard<std::mutex> lock(g_host_pipe_mutex);
+    have = g_host_pipe[dev].ready;
+    in = g_host_pipe[dev].in;
+    out = g_host_pipe[dev].out;
+  }
+  bool ok = !have || cudaStreamSynchronize(in) == cudaSuccess;
+  ok = (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) == cudaSuccess) && ok;
+  ok = (!have || cudaStreamSynchronize(out) == cudaSuccess) && ok;
+  if (!ok) { cudaGetLastError(); return BATQ_ERR_CUDA; }
+  return BATQ_OK;
+}
+
+batq_status batq_linear_w4a4_host_async(const batq_transform* t, const batq_weight* w, const void* x_host, int64_t s,
+                                        void* y_host, int32_t y_dtype, void* x_stage_dev, void* y_stage_dev,
+                                        void* workspace, size_t workspace_bytes, void* stream) {
+  return host_enqueue(t, w, x_host, s, y_host, y_dtype, x_stage_dev, y_stage_dev, workspace, workspace_bytes, stream);
+}
+
+batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w, const void* x_host, int64_t s,
+                                  void* y_host, int32_t y_dtype, void* x_stage_dev, void* y_stage_dev, void* workspace,
+                                  size_t workspace_bytes, void* stream) {
+  const batq_status st = host_enqueue(t, w, x_host, s, y_host, y_dtype, x_stage_dev, y_stage_dev, workspace,
+                                      workspace_bytes, stream);
+  // whatever happened above: nothing of this call is left in flight when it returns
+  const batq_status dr = (w != nullptr && s > 0) ? batq_host_drain(stream) : BATQ_OK;
+  return st != BATQ_OK ? st : dr;
 }
 
 void batq_debug_force_tile_width(int32_t bn) { g_force_bn.store(bn, std::memory_order_relaxed); }

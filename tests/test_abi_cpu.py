@@ -85,6 +85,9 @@ def test_host_validation_without_a_device(lib):
     assert lib.batq_weight_destroy(None) == 0 and lib.batq_transform_destroy(None) == 0
     assert lib.batq_gemm_mxfp8_mxfp4(16, 16, None, 4, 16, 0, 128, None) == 1
     assert lib.batq_linear_w4a8(None, None, 16, 4, 128, 16, 0, 128, 1024, 0, None) == 1
+    # host entry points: a NULL weight is refused before anything touches a device
+    assert lib.batq_linear_w4a4_host(None, None, 16, 4, 16, 0, 16, 16, 1024, 0, None) == 1
+    assert lib.batq_linear_w4a4_host_async(None, None, 16, 4, 16, 0, 16, 16, 1024, 0, None) == 1
     assert lib.batq_linear_w4a8_workspace_bytes(None, 4) == 0
     assert lib.batq_transform_set_bf16_intermediates(None, 1) == 1
     assert lib.batq_debug_mma_peak(0, 100, 10, 0, None, None) == 2

@@ -865,8 +865,12 @@ def test_linear_kernel_launches_reports_the_dispatch(batq):
         batq.batq_debug_force_small_s_path(0)
 
 
-def test_linear_host_entry_point_matches_device_entry_point(batq):
-    S, M, N = 96, 256, 512
+@pytest.mark.parametrize("S,M,N,pinned", [(96, 256, 512, True), (2048, 520, 1024, True), (640, 264, 2048, True),
+                                          (1000, 1104, 768, False)])
+def test_linear_host_entry_point_matches_device_entry_point(batq, S, M, N, pinned):
+    """Host buffers in and out.  From 512 tokens on the rows go through in chunks whose copies and
+    kernels overlap; token rows are independent, so the result is bit for bit that of one device
+    call on all rows, also when a second call follows at once and when the host memory is pageable."""
     xb = synth.make_activations(S, N, 5)
     t = synth.make_transform(N, 5, "baseline")
     tr = _mk_transform(batq, t)
@@ -874,12 +878,36 @@ def test_linear_host_entry_point_matches_device_entry_point(batq):
     ws = batq.aligned_workspace(batq.batq_linear_workspace_bytes(w, S))
     y = torch.empty((S, M), dtype=torch.float32, device="cuda")
     batq.batq_linear_w4a4(tr, w, batq.bits_to_cuda_bf16(xb), y, ws)
-    xh = torch.from_numpy(xb.view(np.int16)).pin_memory()
-    yh = torch.empty((S, M), dtype=torch.float32).pin_memory()
+    xh = torch.from_numpy(xb.view(np.int16))
+    yh = torch.full((S, M), float("nan"), dtype=torch.float32)
+    if pinned:
+        xh, yh = xh.pin_memory(), yh.pin_memory()
     xs = torch.empty((S, N), dtype=torch.bfloat16, device="cuda")
     ys = torch.empty((S, M), dtype=torch.float32, device="cuda")
-    batq.batq_linear_w4a4_host(tr, w, xh, yh, xs, ys, ws)
-    assert torch.equal(yh, y.cpu())
+    for _ in range(2):
+        yh.fill_(float("nan"))
+        batq.batq_linear_w4a4_host(tr, w, xh, yh, xs, ys, ws)
+        assert batq.batq_last_device_status() == 0
+        assert torch.equal(yh, y.cpu())
+    yb = torch.empty((S, M), dtype=torch.bfloat16)
+    ysb = torch.empty((S, M), dtype=torch.bfloat16, device="cuda")
+    batq.batq_linear_w4a4_host(tr, w, xh, yb, xs, ysb, ws)
+    assert torch.equal(yb, y.cpu().bfloat16())
+    # enqueued only: two layers' copies and kernels in flight together, one wait
+    w2 = batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(synth.make_weight(M + 8, N, 6)))
+    ws2 = batq.aligned_workspace(batq.batq_linear_workspace_bytes(w2, S))
+    y2 = torch.empty((S, M + 8), dtype=torch.float32, device="cuda")
+    batq.batq_linear_w4a4(tr, w2, batq.bits_to_cuda_bf16(xb), y2, ws2)
+    yh.fill_(float("nan"))
+    yh2 = torch.full((S, M + 8), float("nan"), dtype=torch.float32)
+    yh2 = yh2.pin_memory() if pinned else yh2
+    xs2 = torch.empty((S, N), dtype=torch.bfloat16, device="cuda")
+    ys2 = torch.empty((S, M + 8), dtype=torch.float32, device="cuda")
+    batq.batq_linear_w4a4_host_async(tr, w, xh, yh, xs, ys, ws)
+    batq.batq_linear_w4a4_host_async(tr, w2, xh, yh2, xs2, ys2, ws2)
+    batq.batq_host_drain()
+    assert batq.batq_last_device_status() == 0
+    assert torch.equal(yh, y.cpu()) and torch.equal(yh2, y2.cpu())
 
 
 def test_empty_input_is_a_noop(batq):
