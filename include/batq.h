@@ -147,6 +147,14 @@ batq_status batq_weight_destroy(batq_weight* w);
  * scale bytes [m x k] (dev buffers), for inspection and tests. */
 batq_status batq_weight_export(const batq_weight* w, void* codes_rowmajor, void* scales_rowmajor,
                                void* stream);
+/* The way back: a prepared weight from stored codes and scales (what batq_weight_export
+ * wrote: dev buffers, packed codes [m x n/2] and scale bytes [m x n/32], both
+ * row-major), so that the offline fusion runs once per checkpoint and a server
+ * only loads its result.  weight_buf as for batq_prepare_weight.  Codes and
+ * scales are taken as they are (a scale byte of 255 is a NaN to the tensor
+ * cores).  Synchronises the stream. */
+batq_status batq_weight_import(const void* codes_rowmajor, const void* scales_rowmajor, int64_t m,
+                               int64_t n, void* weight_buf, batq_weight** out, void* stream);
 
 /* Stage 3 alone: Y[s, m] = sum_j 2^(ex[s,j] + ew[m,j]) * sum_{i<32} qx[s,j,i] * qw[m,j,i]
  * (the low-bit matrix multiplication of Sec. 3.2) on the block-scaled FP4

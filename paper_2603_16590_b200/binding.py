@@ -37,6 +37,7 @@ SIGNATURES = {
     "batq_prepare_weight": (C.c_int, [_P, _P, _I64, _I64, _I64, _P, _P, _P, C.POINTER(_P), _P]),
     "batq_weight_destroy": (C.c_int, [_P]),
     "batq_weight_export": (C.c_int, [_P, _P, _P, _P]),
+    "batq_weight_import": (C.c_int, [_P, _P, _I64, _I64, _P, C.POINTER(_P), _P]),
     "batq_gemm_mxfp4": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _I64, _P]),
     "batq_gemm_mxfp8_mxfp4": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _I64, _P]),
     "batq_linear_w4a8_workspace_bytes": (_SZ, [_P, _I64]),
@@ -193,16 +194,28 @@ def batq_debug_transform_clip_f32(t, x, out):
 class Weight:
     """Owns a batq_weight handle and the device buffer behind it."""
 
-    def __init__(self, t, w, clip_lo=None, clip_hi=None):
-        m, n = w.shape
+    def __init__(self, t, w, clip_lo=None, clip_hi=None, stored=None):
+        """From a bf16 weight w (offline fusion with the transform t), or from stored = (codes, scales)
+        as batq_weight_export wrote them."""
+        if stored is not None:
+            codes, scales = stored
+            m, n = codes.shape[0], codes.shape[1] * 2
+            device = codes.device
+        else:
+            m, n = w.shape
+            device = w.device
         self.m, self.n = m, n
-        self.buf = torch.empty(batq_weight_bytes(m, n) + 1024, dtype=torch.uint8, device=w.device)
+        self.buf = torch.empty(batq_weight_bytes(m, n) + 1024, dtype=torch.uint8, device=device)
         off = (-self.buf.data_ptr()) % 1024
         self._base = self.buf.data_ptr() + off
         h = _P()
-        st = load().batq_prepare_weight(t.handle if t else None, _ptr(w), m, n, w.stride(0), _ptr(clip_lo),
-                                        _ptr(clip_hi), self._base, C.byref(h), _stream())
-        _check(st, "batq_prepare_weight")
+        if stored is not None:
+            st = load().batq_weight_import(_ptr(codes), _ptr(scales), m, n, self._base, C.byref(h), _stream())
+            _check(st, "batq_weight_import")
+        else:
+            st = load().batq_prepare_weight(t.handle if t else None, _ptr(w), m, n, w.stride(0), _ptr(clip_lo),
+                                            _ptr(clip_hi), self._base, C.byref(h), _stream())
+            _check(st, "batq_prepare_weight")
         self.handle = h
 
     def close(self):
@@ -219,6 +232,11 @@ class Weight:
 
 def batq_prepare_weight(t, w, clip_lo=None, clip_hi=None) -> Weight:
     return Weight(t, w, clip_lo, clip_hi)
+
+
+def batq_weight_import(codes, scales) -> Weight:
+    """A prepared weight from stored row-major codes [m x n/2] and scale bytes [m x n/32] (CUDA uint8)."""
+    return Weight(None, None, stored=(codes.contiguous(), scales.contiguous()))
 
 
 def batq_weight_export(w: Weight):

@@ -1568,6 +1568,23 @@ batq_status batq_debug_transform_clip_f32(const batq_transform* t, const void* x
   return launch_quantize(t, x_bf16, s, n, ld, nullptr, nullptr, BATQ_SF_ROWMAJOR, out, static_cast<cudaStream_t>(stream));
 }
 
+// The tensor maps every GEMM kernel takes over a prepared weight's codes and scales.
+static batq_status weight_tensor_maps(batq_weight* w) {
+  const int64_t m = w->m, n = w->n;
+  batq_status st = make_codes_tmap(&w->tmap_b256, w->codes, m, n / 2, 256);
+  if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b192, w->codes, m, n / 2, 192);
+  if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b128, w->codes, m, n / 2, 128);
+  if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b64, w->codes, m, n / 2, 64);
+  if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b32, w->codes, m, n / 2, 32);
+  if (st == BATQ_OK) st = make_sf_tmap(&w->tmap_sf, w->scales, (m + 127) / 128, w->katoms);
+  w->has_u4 = n % 128 == 0;
+  if (st == BATQ_OK && w->has_u4) st = make_u4_unpack_tmap(&w->tmap_u4_128, w->codes, m, n, 128);
+  if (st == BATQ_OK && w->has_u4) st = make_u4_unpack_tmap(&w->tmap_u4_256, w->codes, m, n, 256);
+  if (st == BATQ_OK && w->has_u4) st = make_u4_unpack_tmap(&w->tmap_u4_32, w->codes, m, n, 32);
+  if (st == BATQ_OK && w->has_u4) st = make_sf_tmap(&w->tmap_sf1, w->scales, (m + 127) / 128, w->katoms, 1);
+  return st;
+}
+
 size_t batq_weight_bytes(int64_t m, int64_t n) {
   if (m <= 0 || n <= 0 || n % 32 != 0) return 0;
   return round_up(static_cast<size_t>(m * (n / 2)), 1024) + batq_sf_bytes(m, n, BATQ_SF_MMA);
@@ -1646,17 +1663,44 @@ batq_status batq_prepare_weight(const batq_transform* t, const void* w_bf16, int
   e = e ? e : cudaStreamSynchronize(cs);
   cudaFree(d_fac);
   if (e != cudaSuccess) { cudaGetLastError(); delete w; return BATQ_ERR_CUDA; }
-  st = make_codes_tmap(&w->tmap_b256, w->codes, m, n / 2, 256);
-  if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b192, w->codes, m, n / 2, 192);
-  if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b128, w->codes, m, n / 2, 128);
-  if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b64, w->codes, m, n / 2, 64);
-  if (st == BATQ_OK) st = make_codes_tmap(&w->tmap_b32, w->codes, m, n / 2, 32);
-  if (st == BATQ_OK) st = make_sf_tmap(&w->tmap_sf, w->scales, (m + 127) / 128, w->katoms);
-  w->has_u4 = n % 128 == 0;
-  if (st == BATQ_OK && w->has_u4) st = make_u4_unpack_tmap(&w->tmap_u4_128, w->codes, m, n, 128);
-  if (st == BATQ_OK && w->has_u4) st = make_u4_unpack_tmap(&w->tmap_u4_256, w->codes, m, n, 256);
-  if (st == BATQ_OK && w->has_u4) st = make_u4_unpack_tmap(&w->tmap_u4_32, w->codes, m, n, 32);
-  if (st == BATQ_OK && w->has_u4) st = make_sf_tmap(&w->tmap_sf1, w->scales, (m + 127) / 128, w->katoms, 1);
+  st = weight_tensor_maps(w);
+  if (st != BATQ_OK) { delete w; return st; }
+  *out = w;
+  return BATQ_OK;
+}
+
+batq_status batq_weight_import(const void* codes_rowmajor, const void* scales_rowmajor, int64_t m, int64_t n,
+                               void* weight_buf, batq_weight** out, void* stream) {
+  if (out == nullptr) return BATQ_ERR_NULL;
+  *out = nullptr;
+  if (m <= 0 || m > (int64_t(1) << 24) || n <= 0 || n % 32 != 0 || n > (int64_t(1) << 24)) return BATQ_ERR_SHAPE;
+  if (codes_rowmajor == nullptr || scales_rowmajor == nullptr || weight_buf == nullptr) return BATQ_ERR_NULL;
+  if (!aligned(weight_buf, 1024)) return BATQ_ERR_ALIGN;
+  int dev;
+  const DeviceInfo* dinfo;
+  batq_status st = device_setup(&dev, &dinfo);
+  if (st != BATQ_OK) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  batq_weight* w = new (std::nothrow) batq_weight();
+  if (w == nullptr) return BATQ_ERR_CUDA;
+  w->device = dev;
+  w->m = m; w->n = n; w->k = static_cast<int32_t>(n / 32); w->katoms = katoms_of(w->k);
+  w->sm_count = dinfo->sm_count;
+  w->codes = static_cast<uint8_t*>(weight_buf);
+  const size_t code_bytes = static_cast<size_t>(m * (n / 2));
+  w->scales = w->codes + round_up(code_bytes, 1024);
+  const int64_t items = m * w->k;
+  // padded rows and blocks of the scale layout must hold finite scales: zero everything first
+  cudaError_t e = cudaMemsetAsync(w->codes + code_bytes, 0, batq_weight_bytes(m, n) - code_bytes, cs);
+  e = e ? e : cudaMemcpyAsync(w->codes, codes_rowmajor, code_bytes, cudaMemcpyDeviceToDevice, cs);
+  if (e == cudaSuccess) {
+    import_scales_kernel<<<static_cast<unsigned>((items + 255) / 256), 256, 0, cs>>>(
+        static_cast<const uint8_t*>(scales_rowmajor), w->scales, m, w->k, w->katoms);
+    e = cudaGetLastError();
+  }
+  e = e ? e : cudaStreamSynchronize(cs);
+  if (e != cudaSuccess) { cudaGetLastError(); delete w; return BATQ_ERR_CUDA; }
+  st = weight_tensor_maps(w);
   if (st != BATQ_OK) { delete w; return st; }
   *out = w;
   return BATQ_OK;

@@ -109,4 +109,13 @@ __global__ void export_scales_kernel(const uint8_t* sf_mma, uint8_t* out, int64_
   out[item] = sf_mma[sf_mma_offset(row, j, katoms)];
 }
 
+// Row-major scale bytes -> the layout of a prepared weight (the padding was zeroed before).
+__global__ void import_scales_kernel(const uint8_t* in, uint8_t* sf_mma, int64_t m, int32_t k, int32_t katoms) {
+  const int64_t item = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (item >= m * k) return;
+  const int64_t row = item / k;
+  const int j = static_cast<int>(item - row * k);
+  sf_mma[sf_mma_offset(row, j, katoms)] = in[item];
+}
+
 }  // namespace batq

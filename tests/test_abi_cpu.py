@@ -85,6 +85,10 @@ def test_host_validation_without_a_device(lib):
     assert lib.batq_weight_destroy(None) == 0 and lib.batq_transform_destroy(None) == 0
     assert lib.batq_gemm_mxfp8_mxfp4(16, 16, None, 4, 16, 0, 128, None) == 1
     assert lib.batq_linear_w4a8(None, None, 16, 4, 128, 16, 0, 128, 1024, 0, None) == 1
+    h2 = C.c_void_p()
+    assert lib.batq_weight_import(16, 16, 0, 64, 1024, C.byref(h2), None) == 2      # shape before anything else
+    assert lib.batq_weight_import(None, 16, 8, 64, 1024, C.byref(h2), None) == 1
+    assert lib.batq_weight_import(16, 16, 8, 64, 1000, C.byref(h2), None) == 3      # weight_buf not 1024-byte aligned
     # host entry points: a NULL weight is refused before anything touches a device
     assert lib.batq_linear_w4a4_host(None, None, 16, 4, 16, 0, 16, 16, 1024, 0, None) == 1
     assert lib.batq_linear_w4a4_host_async(None, None, 16, 4, 16, 0, 16, 16, 1024, 0, None) == 1

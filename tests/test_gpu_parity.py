@@ -566,6 +566,50 @@ def test_prepare_weight_with_clip(batq):
     _weight_mismatch_ok(gc, gs, oc, os_, Wt)
 
 
+@pytest.mark.parametrize("S,M,N", [(300, 520, 1024), (16, 264, 2048), (77, 200, 96), (2048, 1100, 768)])
+def test_weight_import_reproduces_the_prepared_weight(batq, S, M, N):
+    """Export -> import gives a weight that exports the same bytes and computes the same layer, bit
+    for bit, on every path (prefill GEMMs, small-s GEMM, fused small-s kernel), W4A8 included; the
+    scale layout's padding (rows past m, blocks past k) is finite whatever the buffer held before."""
+    t = synth.make_transform(N, 21, "baseline")
+    tr = _mk_transform(batq, t)
+    w = batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(synth.make_weight(M, N, 21)))
+    codes, scales = batq.batq_weight_export(w)
+    junk = torch.full((1 << 22,), 0xFF, dtype=torch.uint8, device="cuda")   # what a recycled buffer may hold
+    del junk
+    w2 = batq.batq_weight_import(codes, scales)
+    c2, s2 = batq.batq_weight_export(w2)
+    assert torch.equal(codes, c2) and torch.equal(scales, s2)
+    x = batq.bits_to_cuda_bf16(synth.make_activations(S, N, 22))
+    for ww in (w, w2):
+        ws = batq.aligned_workspace(batq.batq_linear_workspace_bytes(ww, S))
+        y = torch.full((S, M + (-M) % 8), float("nan"), dtype=torch.float32, device="cuda")
+        batq.batq_linear_w4a4(tr, ww, x, y[:, :M], ws)
+        if ww is w:
+            y_ref = y.clone()
+    assert batq.batq_last_device_status() == 0
+    assert torch.equal(y[:, :M], y_ref[:, :M]) and torch.isfinite(y[:, :M]).all()
+    if N % 128 == 0:
+        outs = []
+        for ww in (w, w2):
+            ws = batq.aligned_workspace(batq.batq_linear_w4a8_workspace_bytes(ww, S))
+            y8 = torch.empty((S, M + (-M) % 8), dtype=torch.float32, device="cuda")
+            batq.batq_linear_w4a8(tr, ww, x, y8[:, :M], ws)
+            outs.append(y8[:, :M].clone())
+        assert torch.equal(outs[0], outs[1])
+
+
+def test_weight_import_checks_its_arguments(batq):
+    z = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    for args, status in (((z, z, 0, 64), 2), ((z, z, 8, 48), 2), ((None, z, 8, 64), 1), ((z, None, 8, 64), 1)):
+        h = batq.C.c_void_p()
+        buf = batq.aligned_workspace(4096)
+        st = batq.load().batq_weight_import(args[0].data_ptr() if args[0] is not None else None,
+                                            args[1].data_ptr() if args[1] is not None else None, args[2], args[3],
+                                            buf.data_ptr(), batq.C.byref(h), None)
+        assert st == status
+
+
 def test_singular_factor_is_reported(batq):
     N = 64
     t = synth.make_transform(N, 3, "baseline", clip=False)
