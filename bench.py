@@ -620,15 +620,10 @@ def run_ours(args):
         # end to end: host buffers in and out through the C-ABI host entry point
         def step_host():
             for L in layers:
-                if a8:   # no host entry point for the 8-bit format: the same copies around the device call
-                    L["x"].copy_(L["x_host"].view(torch.bfloat16), non_blocking=True)
-                    f_linear(L["tr"], L["w"], L["x"], L["y"], L["ws"])
-                    L["y_host"].copy_(L["y"], non_blocking=True)
-                    torch.cuda.synchronize()
-                else:   # every layer has staging buffers and a workspace of its own: enqueue all, wait once
-                    B.batq_linear_w4a4_host_async(L["tr"], L["w"], L["x_host"], L["y_host"], L["x"], L["y"], L["ws"])
-            if not a8:
-                B.batq_host_drain()
+                # every layer has staging buffers and a workspace of its own: enqueue all, wait once
+                (B.batq_linear_w4a8_host_async if a8 else B.batq_linear_w4a4_host_async)(
+                    L["tr"], L["w"], L["x_host"], L["y_host"], L["x"], L["y"], L["ws"])
+            B.batq_host_drain()
 
         e2e_steps = max(1, min(steps, 5))
         for _ in range(2):

@@ -244,6 +244,12 @@ batq_status batq_linear_w4a4_host_async(const batq_transform* t, const batq_weig
                                         const void* x_host, int64_t s, void* y_host, int32_t y_dtype,
                                         void* x_stage_dev, void* y_stage_dev, void* workspace,
                                         size_t workspace_bytes, void* stream);
+/* The W4A8 layer (batq_linear_w4a8) with host input and output, enqueued only; the rest as for
+ * batq_linear_w4a4_host_async, with a workspace of batq_linear_w4a8_workspace_bytes(w, s). */
+batq_status batq_linear_w4a8_host_async(const batq_transform* t, const batq_weight* w,
+                                        const void* x_host, int64_t s, void* y_host, int32_t y_dtype,
+                                        void* x_stage_dev, void* y_stage_dev, void* workspace,
+                                        size_t workspace_bytes, void* stream);
 /* Waits for everything the host entry points have enqueued on the current device:
  * the library's copy streams and `stream`. */
 batq_status batq_host_drain(void* stream);

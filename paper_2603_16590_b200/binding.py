@@ -58,6 +58,7 @@ SIGNATURES = {
     "batq_linear_w4a4": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P, _SZ, _P]),
     "batq_linear_w4a4_host": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _P, _P, _P, _SZ, _P]),
     "batq_linear_w4a4_host_async": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _P, _P, _P, _SZ, _P]),
+    "batq_linear_w4a8_host_async": (C.c_int, [_P, _P, _P, _I64, _P, _I32, _P, _P, _P, _SZ, _P]),
     "batq_host_drain": (C.c_int, [_P]),
     "batq_static_workspace_capacity": (_SZ, []),
     "batq_linear_w4a4_noalloc": (C.c_int, [_P, _P, _P, _I64, _I64, _P, _I32, _I64, _P]),
@@ -369,6 +370,15 @@ def batq_linear_w4a4_host_async(t, w: Weight, x_host, y_host, x_stage, y_stage, 
                                             _ptr(y_host), dt, _ptr(x_stage), _ptr(y_stage), _ptr(workspace),
                                             workspace.numel(), _stream())
     _check(st, "batq_linear_w4a4_host_async")
+
+
+def batq_linear_w4a8_host_async(t, w: Weight, x_host, y_host, x_stage, y_stage, workspace):
+    """The W4A8 layer with host buffers, enqueued only; batq_host_drain() waits."""
+    dt = F32 if y_host.dtype == torch.float32 else BF16
+    st = load().batq_linear_w4a8_host_async(t.handle if t else None, w.handle, _ptr(x_host), x_host.shape[0],
+                                            _ptr(y_host), dt, _ptr(x_stage), _ptr(y_stage), _ptr(workspace),
+                                            workspace.numel(), _stream())
+    _check(st, "batq_linear_w4a8_host_async")
 
 
 def batq_host_drain():

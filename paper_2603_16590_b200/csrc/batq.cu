@@ -1901,13 +1901,14 @@ static bool stream_follows(cudaStream_t dst_stream, cudaStream_t src_stream) {
 // Enqueues copy-in, layer and copy-out; nothing is waited for.
 static batq_status host_enqueue(const batq_transform* t, const batq_weight* w, const void* x_host, int64_t s, void* y_host,
                                 int32_t y_dtype, void* x_stage_dev, void* y_stage_dev, void* workspace,
-                                size_t workspace_bytes, void* stream) {
-  if (w == nullptr) return BATQ_ERR_NULL;
+                                size_t workspace_bytes, void* stream, bool a8) {
+  if (w == nullptr || (a8 && t == nullptr)) return BATQ_ERR_NULL;
+  auto ws_bytes = [&](int64_t rows) { return a8 ? batq_linear_w4a8_workspace_bytes(w, rows) : batq_linear_workspace_bytes(w, rows); };
   if (s < 0) return BATQ_ERR_SHAPE;
   if (s == 0) return BATQ_OK;
   if (x_host == nullptr || y_host == nullptr || x_stage_dev == nullptr || y_stage_dev == nullptr) return BATQ_ERR_NULL;
   if (y_dtype != BATQ_F32 && y_dtype != BATQ_BF16) return BATQ_ERR_UNSUPPORTED;
-  if (workspace_bytes < batq_linear_workspace_bytes(w, s)) return BATQ_ERR_WORKSPACE;
+  if (workspace_bytes < ws_bytes(s)) return BATQ_ERR_WORKSPACE;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   const size_t ysz = y_dtype == BATQ_F32 ? 4 : 2;
   // Token rows are independent, so a large batch goes through in up to four chunks of rows: the
@@ -1917,7 +1918,7 @@ static batq_status host_enqueue(const batq_transform* t, const batq_weight* w, c
   int n_chunks = static_cast<int>((s + rows_per_chunk - 1) / rows_per_chunk);
   if (n_chunks > 1) {   // the workspace was sized for s rows at once: every chunk must fit it too
     const int64_t last = s - (n_chunks - 1) * rows_per_chunk;
-    if (batq_linear_workspace_bytes(w, rows_per_chunk) > workspace_bytes || batq_linear_workspace_bytes(w, last) > workspace_bytes) {
+    if (ws_bytes(rows_per_chunk) > workspace_bytes || ws_bytes(last) > workspace_bytes) {
       rows_per_chunk = s;
       n_chunks = 1;
     }
@@ -1942,7 +1943,8 @@ static batq_status host_enqueue(const batq_transform* t, const batq_weight* w, c
     ok = cudaMemcpyAsync(xd, xh, static_cast<size_t>(rows * w->n) * 2, cudaMemcpyHostToDevice, hp->in) == cudaSuccess &&
          stream_follows(cs, hp->in);
     if (!ok) break;
-    st = batq_linear_w4a4(t, w, xd, rows, w->n, yd, y_dtype, w->m, workspace, workspace_bytes, stream);
+    st = a8 ? batq_linear_w4a8(t, w, xd, rows, w->n, yd, y_dtype, w->m, workspace, workspace_bytes, stream)
+            : batq_linear_w4a4(t, w, xd, rows, w->n, yd, y_dtype, w->m, workspace, workspace_bytes, stream);
     if (st != BATQ_OK) break;
     ok = stream_follows(hp->out, cs) &&
          cudaMemcpyAsync(yh, yd, static_cast<size_t>(rows * w->m) * ysz, cudaMemcpyDeviceToHost, hp->out) == cudaSuccess;
@@ -1973,14 +1975,20 @@ batq_status batq_host_drain(void* stream) {
 batq_status batq_linear_w4a4_host_async(const batq_transform* t, const batq_weight* w, const void* x_host, int64_t s,
                                         void* y_host, int32_t y_dtype, void* x_stage_dev, void* y_stage_dev,
                                         void* workspace, size_t workspace_bytes, void* stream) {
-  return host_enqueue(t, w, x_host, s, y_host, y_dtype, x_stage_dev, y_stage_dev, workspace, workspace_bytes, stream);
+  return host_enqueue(t, w, x_host, s, y_host, y_dtype, x_stage_dev, y_stage_dev, workspace, workspace_bytes, stream, false);
+}
+
+batq_status batq_linear_w4a8_host_async(const batq_transform* t, const batq_weight* w, const void* x_host, int64_t s,
+                                        void* y_host, int32_t y_dtype, void* x_stage_dev, void* y_stage_dev,
+                                        void* workspace, size_t workspace_bytes, void* stream) {
+  return host_enqueue(t, w, x_host, s, y_host, y_dtype, x_stage_dev, y_stage_dev, workspace, workspace_bytes, stream, true);
 }
 
 batq_status batq_linear_w4a4_host(const batq_transform* t, const batq_weight* w, const void* x_host, int64_t s,
                                   void* y_host, int32_t y_dtype, void* x_stage_dev, void* y_stage_dev, void* workspace,
                                   size_t workspace_bytes, void* stream) {
   const batq_status st = host_enqueue(t, w, x_host, s, y_host, y_dtype, x_stage_dev, y_stage_dev, workspace,
-                                      workspace_bytes, stream);
+                                      workspace_bytes, stream, false);
   // whatever happened above: nothing of this call is left in flight when it returns
   const batq_status dr = (w != nullptr && s > 0) ? batq_host_drain(stream) : BATQ_OK;
   return st != BATQ_OK ? st : dr;

@@ -92,6 +92,7 @@ def test_host_validation_without_a_device(lib):
     # host entry points: a NULL weight is refused before anything touches a device
     assert lib.batq_linear_w4a4_host(None, None, 16, 4, 16, 0, 16, 16, 1024, 0, None) == 1
     assert lib.batq_linear_w4a4_host_async(None, None, 16, 4, 16, 0, 16, 16, 1024, 0, None) == 1
+    assert lib.batq_linear_w4a8_host_async(None, None, 16, 4, 16, 0, 16, 16, 1024, 0, None) == 1
     assert lib.batq_linear_w4a8_workspace_bytes(None, 4) == 0
     assert lib.batq_transform_set_bf16_intermediates(None, 1) == 1
     assert lib.batq_debug_mma_peak(0, 100, 10, 0, None, None) == 2

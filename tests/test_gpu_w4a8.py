@@ -201,3 +201,25 @@ def test_linear_w4a8_with_row_strides_and_bf16_output(batq):
     batq.batq_linear_w4a8(tr, w, xp[:, :N], yp[:, :M], ws)
     assert batq.batq_last_device_status() == 0
     assert torch.equal(yp[:, :M], y32.bfloat16()) and (yp[:, M:] == 3.0).all()
+
+
+@pytest.mark.parametrize("S", [96, 2048])
+def test_linear_w4a8_host_entry_point_matches_device_entry_point(batq, S):
+    """Host buffers in and out for the W4A8 layer (row chunks from 512 tokens on): bit for bit the
+    device entry point's result."""
+    M, N = 520, 1024
+    xb = synth.make_activations(S, N, 31)
+    t = synth.make_transform(N, 31, "baseline")
+    tr = _mk(batq, t)
+    w = batq.batq_prepare_weight(tr, batq.bits_to_cuda_bf16(synth.make_weight(M, N, 31)))
+    ws = batq.aligned_workspace(batq.batq_linear_w4a8_workspace_bytes(w, S))
+    y = torch.empty((S, M), dtype=torch.float32, device="cuda")
+    batq.batq_linear_w4a8(tr, w, batq.bits_to_cuda_bf16(xb), y, ws)
+    xh = torch.from_numpy(xb.view(np.int16)).pin_memory()
+    yh = torch.full((S, M), float("nan"), dtype=torch.float32).pin_memory()
+    xs = torch.empty((S, N), dtype=torch.bfloat16, device="cuda")
+    ys = torch.empty((S, M), dtype=torch.float32, device="cuda")
+    batq.batq_linear_w4a8_host_async(tr, w, xh, yh, xs, ys, ws)
+    batq.batq_host_drain()
+    assert batq.batq_last_device_status() == 0
+    assert torch.equal(yh, y.cpu())
