@@ -355,26 +355,8 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
       tc_fence_after_sync();
       const int row0 = t.mp * 256 + static_cast<int>(rank) * kBM + quad * 32;
       const uint32_t taddr = tmem_base + acc * Cfg::kSlot1Col + (static_cast<uint32_t>(quad * 32) << 16);
-#pragma unroll 1
-      for (int c0 = 0; c0 < t.bn; c0 += kChunkCols) {
-        uint32_t w[32];
-        if (OUT_BF16) {
-          uint32_t r0[32], r1[32];
-          tmem_ld_32x32b_x32(taddr + c0, r0);
-          tmem_ld_32x32b_x32(taddr + c0 + 32, r1);
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const __nv_bfloat162 a = __floats2bfloat162_rn(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]));
-            const __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(r1[2 * i]), __uint_as_float(r1[2 * i + 1]));
-            w[i] = *reinterpret_cast<const uint32_t*>(&a);
-            w[16 + i] = *reinterpret_cast<const uint32_t*>(&b);
-          }
-        } else {
-          tmem_ld_32x32b_x32(taddr + c0, w);
-          tmem_ld_wait();
-        }
-        const int col0 = t.n0 + c0;
+      // Rows [row0, row0 + 32) x columns [col0, col0 + kChunkCols) of y from w (one row per lane).
+      auto write_chunk = [&](const uint32_t (&w)[32], int col0) {
         if (p.m16 < p.m && col0 < p.m && col0 + kChunkCols > p.m16 && row0 + lane < p.s) {
           if (OUT_BF16) {
             __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(p.y) + static_cast<int64_t>(row0 + lane) * p.ldy + col0;
@@ -405,10 +387,48 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
           bulk_commit_group();
         }
         buf = (buf + 1) % Cfg::kStagingBufs;
+      };
+      if (OUT_BF16) {
+        // All columns of the tile into registers first (rounded and packed: 32 words per 64 columns,
+        // at most four such chunks), then the accumulator goes back -- a tile that needs the same
+        // slot next waits for these loads only -- and the stores follow.
+        uint32_t w[4][32];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          if (64 * i < t.bn) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              uint32_t r[32];
+              tmem_ld_32x32b_x32(taddr + 64 * i + 32 * h, r);
+              tmem_ld_wait();
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const __nv_bfloat162 a = __floats2bfloat162_rn(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+                w[i][16 * h + j] = *reinterpret_cast<const uint32_t*>(&a);
+              }
+            }
+          }
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(acc_empty0_leader + 8u * acc);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (64 * i < t.bn) write_chunk(w[i], t.n0 + 64 * i);
+      } else {
+#pragma unroll 1
+        for (int c0 = 0; c0 < t.bn; c0 += kChunkCols) {
+          uint32_t w[32];
+          tmem_ld_32x32b_x32(taddr + c0, w);
+          tmem_ld_wait();
+          if (c0 + kChunkCols >= t.bn) {   // the last columns sit in registers: hand the accumulator back
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(acc_empty0_leader + 8u * acc);
+          }
+          write_chunk(w, t.n0 + c0);
+        }
       }
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(acc_empty0_leader + 8u * acc);
     }
     if (lane == 0) bulk_wait_group<0>();
   }

@@ -3,6 +3,8 @@ one.  It is meant for callers that may not call cudaMalloc when they run a layer
 (the device already belongs to their own pool, or an allocation's device-wide
 synchronisation is not acceptable there), so its scratch is an array inside the
 library.  Collected last on purpose: a failure here stops nothing else."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -32,6 +34,7 @@ def test_noalloc_entry_point_matches_regular_one_twice_in_a_row(batq):
     # one call first: it resolves the array's address on this device (documented set-up step)
     batq.batq_linear_w4a4_noalloc(*layers[0][:3], torch.empty_like(layers[0][3]))
     torch.cuda.synchronize()
+    gc.collect()   # tensors of earlier tests that are still waiting for the collector go now, not between the readings
     # what the driver itself hands out (torch's own counter would not see a cudaMalloc inside the library)
     free_before = torch.cuda.mem_get_info()[0]
     torch_before = torch.cuda.memory_allocated()
